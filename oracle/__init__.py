@@ -1,0 +1,16 @@
+"""CPU oracle (test infrastructure): the plain fp64 definition the CUDA library is checked against.
+
+Not part of the product.  Imported only by tests/, the smoke check and the benchmark's CPU-baseline leg.
+"""
+from .exit_head import (  # noqa: F401
+    bf16_decode,
+    bf16_rne,
+    layer_norm,
+    logits,
+    softmax_stats,
+    exit_decision,
+    exit_head,
+    compact,
+    dssd_accept,
+    decisive_rows,
+)
