@@ -1,0 +1,143 @@
+/*
+ * eexit -- early-exit head decision and DSSD verify step for sm_100a (B200).
+ *
+ * C ABI.  Unless a parameter says otherwise every pointer is a DEVICE pointer owned by the caller.
+ * Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream), never
+ * allocate, never synchronise and never take ownership.  Outputs are fully overwritten.  Argument
+ * errors are detected on the host before anything is launched and reported through the return code;
+ * there is no CPU fallback: a device that is not compute capability 10.x yields EE_ERR_ARCH.
+ * Identical inputs give bit-identical outputs (all reductions run in a fixed order).
+ *
+ * Notation follows the paper: a head h_k maps the hidden features of a transformer block to a
+ * distribution p_k over the vocabulary V (section 3.1 "Early exit heads", section 3.2); the confidence
+ * is the entropy of p_k (section 3.4.1); tau_k is the calibrated threshold of head k (section 3.4.1);
+ * a row exits when H(p_k) < tau_k (section 3.4.2 and the drafting paragraph of section 4.3.1).
+ */
+#ifndef EEXIT_H_
+#define EEXIT_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EE_OK = 0,
+    EE_ERR_NULL = 1,       /* a required pointer is NULL                                    */
+    EE_ERR_SHAPE = 2,      /* a size is out of range (see each call)                        */
+    EE_ERR_ALIGN = 3,      /* a pointer or stride breaks the stated alignment               */
+    EE_ERR_WORKSPACE = 4,  /* workspace smaller than ee_exit_head_workspace_bytes()         */
+    EE_ERR_ARCH = 5,       /* current device is not sm_100                                  */
+    EE_ERR_CUDA = 6,       /* a CUDA runtime/driver call failed                             */
+    EE_ERR_TIMEOUT = 7     /* a bounded device-side wait gave up (see ee_query_async_error) */
+} ee_status;
+
+/* Kernel selection for ee_exit_head_path(). */
+typedef enum {
+    EE_PATH_AUTO = 0,      /* by M: streaming kernel for decode-sized M, tensor-core kernel above   */
+    EE_PATH_STREAM = 1,    /* fused LayerNorm + split-V streaming kernel (any M, in slabs of rows)  */
+    EE_PATH_TCGEN05 = 2    /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics     */
+} ee_path;
+
+/* Static, human-readable name of a status code. */
+const char* ee_status_string(ee_status status);
+
+/*
+ * Bytes of device scratch ee_exit_head needs for these sizes (host-only, pure; 0 if a size is invalid).
+ * The scratch holds the per-(row, vocabulary-slice) partial softmax states, the bf16 LayerNorm output
+ * on the tensor-core path, and a 256-byte control block (completion ticket, error word).
+ */
+size_t ee_exit_head_workspace_bytes(int M, int d, int V);
+
+/*
+ * Zeroes the control block at the start of `workspace`.  Must run once after the workspace is
+ * allocated (and after ee_query_async_error reported EE_ERR_TIMEOUT); every ee_exit_head call leaves
+ * the block ready for the next one.  The workspace must be 256-byte aligned.  One workspace serves one
+ * call at a time: calls sharing a workspace must be ordered on one stream.
+ */
+ee_status ee_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The exit decision of one head for M hidden-state rows (sections 3.2, 3.4.1, 3.4.2):
+ *   y      = bf16( LayerNorm(h; gamma, beta, ln_eps) )       biased variance, eps under the root
+ *   z[v]   = sum_j W[v, j] * y[j]                            fp32 accumulation, logits never stored
+ *   argmax = lowest v attaining max z   (the head's prediction, as in Eq. 2)
+ *   entropy= ln sum exp(z - max) - sum exp(z - max)(z - max) / sum exp(z - max)      (nats)
+ *   maxprob= 1 / sum exp(z - max)                            (the max-probability metric of 3.4.1)
+ *   exit   = entropy < tau                                   (strict; NaN entropy never exits)
+ *
+ * h      bf16 [M, d], row stride ld_h elements (ld_h >= d, ld_h % 8 == 0), 16-byte aligned
+ * gamma, beta  fp32 [d], 16-byte aligned
+ * W      bf16 [V, d] row-major contiguous, 16-byte aligned;  d % 8 == 0, 8 <= d <= 8192, V >= 1
+ * tau_per_row  fp32 [M] thresholds in nats, or NULL to use the scalar `tau` for every row
+ * argmax int32 [M]; entropy fp32 [M]; maxprob fp32 [M]; exit_mask uint8 [M] (1 = exit)
+ * workspace    >= ee_exit_head_workspace_bytes(M, d, V) bytes, 256-byte aligned, initialised once
+ * M = 0 is a no-op returning EE_OK.
+ */
+ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                       const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                       int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same operation with the kernel chosen by the caller (`path` is an ee_path); used to cross-check the
+ * kernels against each other and to time them separately. */
+ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                            int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask,
+                            void* workspace, size_t workspace_bytes, void* stream, int path);
+
+/*
+ * ee_exit_head for a caller whose activations and results live in HOST memory (pinned memory makes
+ * the copies asynchronous).  Copies h_host -> h_dev on `stream`, runs the head, copies the four outputs
+ * to the *_host arrays.  The device arrays are caller-provided staging of the same shapes as in
+ * ee_exit_head; weights, thresholds and workspace stay device pointers.  Returns without synchronising:
+ * the host arrays are valid after the caller synchronises `stream`.
+ * h_host is dense [M, d] (row stride d); h_dev receives it with row stride d.
+ */
+ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                            int* argmax_host, float* entropy_host, float* maxprob_host, unsigned char* exit_mask_host,
+                            int* argmax_dev, float* entropy_dev, float* maxprob_dev, unsigned char* exit_mask_dev,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Continuation of the rows that did not exit (section 3.4.2: an input keeps going through the model's
+ * layers until a head is confident).  Order-preserving stream compaction:
+ *   kept_idx   int32 [M]: ascending indices i with exit_mask[i] == 0 (first *kept_count entries valid)
+ *   kept_count int32 [1] on the device
+ *   h_out      bf16 [M, d] capacity (row stride d): h_out[r, :] = h[kept_idx[r], :] bit for bit;
+ *              may be NULL to skip the gather.  Rows at and beyond *kept_count are left untouched.
+ * h is the head's INPUT (pre-LayerNorm) rows: bf16 [M, d], row stride ld_h, d % 8 == 0, 16-byte
+ * aligned (h may be NULL iff h_out is NULL).  Any non-zero mask byte counts as "exited".  M = 0 writes
+ * kept_count = 0.
+ */
+ee_status ee_compact(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
+                     int* kept_idx, int* kept_count, void* h_out, void* stream);
+
+/*
+ * DSSD drafting stop and verification (section 4.3.1).  For each of S sequences with k draft slots:
+ *   draft_len[s]  = number of leading slots with draft_exit_mask[s, j] != 0, at most k  (drafting stops
+ *                   at the buffer limit or at the first position where the head is not confident)
+ *   accept_len[s] = number of leading j < draft_len[s] with draft_tok[s, j] == verify_tok[s, j]
+ *                   (the accepted prefix)
+ *   next_tok[s]   = verify_tok[s, accept_len[s]] if accept_len[s] < kv, else -1  (the full model's token
+ *                   that rewrites the first mismatch, or follows a fully accepted draft)
+ * draft_tok int32 [S, k]; draft_exit_mask uint8 [S, k] or NULL (all confident); verify_tok int32
+ * [S, kv], kv >= k >= 1; outputs int32 [S].  S = 0 is a no-op.
+ */
+ee_status dssd_accept(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok,
+                      int S, int k, int kv, int* draft_len, int* accept_len, int* next_tok, void* stream);
+
+/*
+ * Synchronises `stream`, then reads and clears the error word of the workspace's control block.
+ * Every device-side wait in the tensor-core kernel is bounded; one that gives up records itself there
+ * and the kernel drains and returns.  EE_OK if nothing was recorded, EE_ERR_TIMEOUT otherwise (outputs
+ * of that call are then undefined; call ee_workspace_init before reusing the workspace).
+ */
+ee_status ee_query_async_error(void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EEXIT_H_ */

@@ -1,0 +1,171 @@
+// Shared device helpers: the mergeable softmax state, workspace layout, small load/pack wrappers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <math_constants.h>
+
+#include "eexit.h"
+
+namespace ee {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ---------------------------------------------------------------------------------------------
+// Softmax state of a subset of the vocabulary.  For logits z_v over the subset:
+//   m = max z_v,  s = sum e^(z_v - m),  t = sum e^(z_v - m) (z_v - m)  (<= 0),  idx = lowest v with z_v = m.
+// Entropy of the full softmax = ln s - t / s, max probability = 1 / s.  States of disjoint subsets
+// merge exactly (up to rounding), so the reduction can be split across threads, warps and CTAs.
+// ---------------------------------------------------------------------------------------------
+struct __align__(16) State {
+    float m, s, t;
+    int idx;
+};
+
+__device__ __forceinline__ State state_empty() { return State{-CUDART_INF_F, 0.f, 0.f, 0x7fffffff}; }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Fold one logit into a state.  Indices arrive in increasing order within a thread, so a strict
+// comparison keeps the lowest index among equal maxima.
+__device__ __forceinline__ void state_push(State& a, float z, int idx) {
+    if (z > a.m) {
+        const float dl = a.m - z;                                  // <= 0, -inf for an empty state
+        const bool was_empty = (a.s == 0.f);
+        const float al = was_empty ? 0.f : ex2(dl * kLog2e);
+        a.t = was_empty ? 0.f : al * fmaf(dl, a.s, a.t);
+        a.s = fmaf(al, a.s, 1.f);
+        a.m = z;
+        a.idx = idx;
+    } else {
+        const float dz = z - a.m;                                  // <= 0 (NaN propagates into s, t)
+        const float e = ex2(dz * kLog2e);
+        a.s += e;
+        a.t = fmaf(e, dz, a.t);
+    }
+}
+
+// a <- merge(a, b).  Ties on the maximum keep the lower index.  Bitwise symmetric in (a, b).
+__device__ __forceinline__ void state_merge(State& a, const State& b) {
+    if (b.s == 0.f) return;                                        // b empty (a non-empty state has s >= 1)
+    if (a.s == 0.f) { a = b; return; }                             // a empty
+    const float m = fmaxf(a.m, b.m);
+    const float da = a.m - m, db = b.m - m;                        // <= 0
+    const float ea = ex2(da * kLog2e), eb = ex2(db * kLog2e);
+    const float s = ea * a.s + eb * b.s;
+    const float t = ea * fmaf(da, a.s, a.t) + eb * fmaf(db, b.s, b.t);
+    const bool take_a = (a.m > b.m) || (a.m == b.m && a.idx < b.idx);
+    a.idx = take_a ? a.idx : b.idx;
+    a.m = (a.m != a.m || b.m != b.m) ? CUDART_NAN_F : m;
+    a.s = s;
+    a.t = t;
+}
+
+__device__ __forceinline__ State state_shfl_xor(const State& a, int mask) {
+    State b;
+    b.m = __shfl_xor_sync(0xffffffffu, a.m, mask);
+    b.s = __shfl_xor_sync(0xffffffffu, a.s, mask);
+    b.t = __shfl_xor_sync(0xffffffffu, a.t, mask);
+    b.idx = __shfl_xor_sync(0xffffffffu, a.idx, mask);
+    return b;
+}
+
+__device__ __forceinline__ State state_load_cg(const State* p) {
+    const int4 raw = __ldcg(reinterpret_cast<const int4*>(p));
+    State o;
+    o.m = __int_as_float(raw.x);
+    o.s = __int_as_float(raw.y);
+    o.t = __int_as_float(raw.z);
+    o.idx = raw.w;
+    return o;
+}
+
+// Final statistics of a full-vocabulary state, and the exit decision.
+__device__ __forceinline__ void state_finish(const State& a, float tau, int* argmax, float* entropy,
+                                             float* maxprob, unsigned char* exit_mask, int row) {
+    const float H = logf(a.s) - a.t / a.s;
+    argmax[row] = a.idx;
+    entropy[row] = H;
+    maxprob[row] = 1.f / a.s;
+    exit_mask[row] = (H < tau) ? 1 : 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Workspace layout.  [0, 256): control block.  Then the partial states, then (tensor-core path) y.
+// ---------------------------------------------------------------------------------------------
+struct Control {
+    unsigned int ticket;      // completion counter of the streaming kernel; returns to 0 after every call
+    unsigned int error;       // 0, or a code recorded by a bounded wait that gave up
+    unsigned int error_info;  // where it gave up (role << 24 | stage << 16 | low bits of the tile index)
+    unsigned int pad[61];
+};
+static_assert(sizeof(Control) == 256, "control block is 256 bytes");
+
+constexpr int kCtrlBytes = 256;
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// Loads, packing, warp reductions
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&p);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// LayerNorm of eight consecutive elements (one 16-byte vector of bf16) -> eight bf16, given the row's
+// mean and reciprocal standard deviation.  c is the vector index within the row.
+__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, const float* gamma,
+                                                 const float* beta, int c) {
+    const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+    const float4 g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+    const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+    const float4 b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+    uint4 o;
+    o.x = pack_bf16(fmaf((bf16_lo(v.x) - mu) * rstd, g0.x, b0.x), fmaf((bf16_hi(v.x) - mu) * rstd, g0.y, b0.y));
+    o.y = pack_bf16(fmaf((bf16_lo(v.y) - mu) * rstd, g0.z, b0.z), fmaf((bf16_hi(v.y) - mu) * rstd, g0.w, b0.w));
+    o.z = pack_bf16(fmaf((bf16_lo(v.z) - mu) * rstd, g1.x, b1.x), fmaf((bf16_hi(v.z) - mu) * rstd, g1.y, b1.y));
+    o.w = pack_bf16(fmaf((bf16_lo(v.w) - mu) * rstd, g1.z, b1.z), fmaf((bf16_hi(v.w) - mu) * rstd, g1.w, b1.w));
+    return o;
+}
+
+__device__ __forceinline__ float vec8_sum(uint4 v) {
+    return ((bf16_lo(v.x) + bf16_hi(v.x)) + (bf16_lo(v.y) + bf16_hi(v.y))) +
+           ((bf16_lo(v.z) + bf16_hi(v.z)) + (bf16_lo(v.w) + bf16_hi(v.w)));
+}
+
+__device__ __forceinline__ float vec8_sqdev(uint4 v, float mu, float acc) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float a = bf16_lo(w[i]) - mu, b = bf16_hi(w[i]) - mu;
+        acc = fmaf(a, a, acc);
+        acc = fmaf(b, b, acc);
+    }
+    return acc;
+}
+
+}  // namespace ee

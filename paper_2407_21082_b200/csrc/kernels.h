@@ -1,0 +1,53 @@
+// Internal launch interface between the C-ABI layer (api.cu) and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "eexit.h"
+
+namespace ee {
+
+constexpr int kMaxDevices = 64;
+
+struct HeadArgs {
+    const void* h;
+    long long ld_h;
+    const float* gamma;
+    const float* beta;
+    float ln_eps;
+    const void* W;
+    int M, d, V;
+    const float* tau_per_row;
+    float tau;
+    int* argmax;
+    float* entropy;
+    float* maxprob;
+    unsigned char* exit_mask;
+    void* workspace;
+    size_t workspace_bytes;
+    cudaStream_t stream;
+    int device;       // current device ordinal
+    int num_sms;      // its multiprocessor count
+};
+
+// ---- streaming kernel (fused LayerNorm + split-V mma.sync GEMV + last-CTA merge) ----
+constexpr int kStreamMaxCtas = 256;        // upper bound on the grid, used for workspace sizing
+constexpr int kStreamMaxRows = 32;         // rows per launch (slab)
+int stream_slab_rows(int d);               // rows one launch can take for this d (0 if d does not fit)
+size_t stream_workspace_bytes(int M, int d, int V);
+ee_status stream_launch(const HeadArgs& a);
+
+// ---- tensor-core kernel (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge) ----
+int gemm_tile_n(int M);                    // vocabulary tile width used for M rows
+size_t gemm_workspace_bytes(int M, int d, int V);
+ee_status gemm_launch(const HeadArgs& a);
+
+// ---- compaction and DSSD accept ----
+ee_status compact_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
+                         int* kept_idx, int* kept_count, void* h_out, cudaStream_t stream);
+ee_status accept_launch(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok,
+                        int S, int k, int kv, int* draft_len, int* accept_len, int* next_tok,
+                        cudaStream_t stream);
+
+}  // namespace ee
