@@ -1,0 +1,46 @@
+"""Loads libeexit.so and declares the C prototypes of include/eexit.h for ctypes."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+from . import build as _build
+
+_LIB = None
+
+_p = C.c_void_p
+PROTOTYPES = {
+    "ee_status_string": (C.c_char_p, [C.c_int]),
+    "ee_exit_head_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
+    "ee_workspace_init": (C.c_int, [_p, C.c_size_t, _p]),
+    "ee_exit_head": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
+                               _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_exit_head_path": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
+                                    _p, _p, _p, _p, _p, C.c_size_t, _p, C.c_int]),
+    "ee_exit_head_host": (C.c_int, [_p, _p, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
+                                    _p, _p, _p, _p, _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),
+    "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
+    "ee_query_async_error": (C.c_int, [_p, _p]),
+}
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Returns the loaded library.  Raises if it has not been built: there is no fallback path."""
+    global _LIB
+    if _LIB is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2407_21082_b200.build` "
+                               "(needs nvcc); this package has no other implementation")
+        lib = C.CDLL(path)
+        for name, (res, args) in PROTOTYPES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _LIB = lib
+    return _LIB

@@ -1,0 +1,146 @@
+"""Python binding of the C ABI in include/eexit.h: argument marshalling only.
+
+Tensors are torch CUDA tensors (torch supplies device memory and the current stream); bf16 tensors may be
+passed as torch.bfloat16 or as int16/uint16 bit patterns.  Every function launches on torch's current
+stream and returns without synchronising, exactly like the C calls underneath.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import _lib
+
+EE_PATH_AUTO, EE_PATH_STREAM, EE_PATH_TCGEN05 = 0, 1, 2
+
+
+class EExitError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        msg = _lib.load().ee_status_string(int(code)).decode()
+        super().__init__(f"{where}: {msg} (ee_status {int(code)})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise EExitError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _bf16(t: torch.Tensor) -> torch.Tensor:
+    if t.dtype in (torch.int16, torch.uint16):
+        t = t.view(torch.bfloat16)
+    if t.dtype != torch.bfloat16:
+        raise TypeError(f"expected bf16 (or its 16-bit patterns), got {t.dtype}")
+    return t
+
+
+def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    return t
+
+
+def ee_exit_head_workspace_bytes(M: int, d: int, V: int) -> int:
+    return int(_lib.load().ee_exit_head_workspace_bytes(int(M), int(d), int(V)))
+
+
+def ee_workspace_init(workspace: torch.Tensor) -> None:
+    _check(_lib.load().ee_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+           "ee_workspace_init")
+
+
+def new_workspace(M: int, d: int, V: int, device="cuda") -> torch.Tensor:
+    """Allocates (through torch) and initialises a workspace for ee_exit_head at these sizes."""
+    nbytes = ee_exit_head_workspace_bytes(M, d, V)
+    if nbytes == 0:
+        raise EExitError(2, "ee_exit_head_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    ee_workspace_init(ws)
+    return ws
+
+
+def new_outputs(M: int, device="cuda") -> dict:
+    return dict(argmax=torch.empty(M, dtype=torch.int32, device=device),
+                entropy=torch.empty(M, dtype=torch.float32, device=device),
+                maxprob=torch.empty(M, dtype=torch.float32, device=device),
+                exit_mask=torch.empty(M, dtype=torch.uint8, device=device))
+
+
+def ee_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> dict:
+    """LayerNorm + exit-head projection + entropy / argmax / max-prob + exit decision for the rows of h.
+
+    tau is a float (nats) or a float32 CUDA tensor [M] of per-row thresholds.  `out` (see new_outputs) and
+    `workspace` (see new_workspace) are allocated when not given.
+    """
+    h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
+    M, d = h.shape
+    V = W.shape[0]
+    if W.shape[1] != d or not W.is_contiguous() or h.stride(1) != 1:
+        raise ValueError("W must be contiguous [V, d] and h row-major [M, d]")
+    out = out if out is not None else new_outputs(M, h.device)
+    workspace = workspace if workspace is not None else new_workspace(M, d, V, h.device)
+    tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+    _check(_lib.load().ee_exit_head_path(
+        _ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W),
+        M, d, V, _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
+        _ptr(out["exit_mask"]), _ptr(workspace), workspace.numel(), _stream(), int(path)), "ee_exit_head")
+    return out
+
+
+def ee_exit_head_host(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host: dict, out_dev: dict, workspace) -> None:
+    """Host-buffer variant: copies h_host (pinned CPU tensor) in, runs the head, copies the outputs to out_host."""
+    W = _bf16(W)
+    M, d = h_host.shape
+    tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+    _check(_lib.load().ee_exit_head_host(
+        _ptr(h_host), _ptr(h_dev), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W), M, d, W.shape[0], _ptr(tau_t), tau_f,
+        _ptr(out_host["argmax"]), _ptr(out_host["entropy"]), _ptr(out_host["maxprob"]), _ptr(out_host["exit_mask"]),
+        _ptr(out_dev["argmax"]), _ptr(out_dev["entropy"]), _ptr(out_dev["maxprob"]), _ptr(out_dev["exit_mask"]),
+        _ptr(workspace), workspace.numel(), _stream()), "ee_exit_head_host")
+
+
+def ee_compact(exit_mask, h=None, *, gather=True, out=None) -> dict:
+    """Indices (ascending) and count of the rows with exit_mask == 0, and a dense copy of their rows of h."""
+    M = exit_mask.numel()
+    dev = exit_mask.device
+    gather = gather and h is not None
+    if gather:
+        h = _bf16(_dev(h, "h"))
+    d = h.shape[1] if h is not None else 0
+    if out is None:
+        out = dict(kept_idx=torch.empty(M, dtype=torch.int32, device=dev),
+                   kept_count=torch.empty(1, dtype=torch.int32, device=dev))
+        if gather:
+            out["h_out"] = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
+    ld = (h.stride(0) if M > 1 else max(h.stride(0), d)) if gather else 0
+    _check(_lib.load().ee_compact(_ptr(exit_mask), _ptr(h) if gather else None, ld, M, d, _ptr(out["kept_idx"]),
+                                  _ptr(out["kept_count"]), _ptr(out.get("h_out")) if gather else None, _stream()),
+           "ee_compact")
+    return out
+
+
+def dssd_accept(draft_tok, draft_exit_mask, verify_tok, *, out=None) -> dict:
+    """Draft length, accepted prefix length and next token per sequence (see include/eexit.h)."""
+    S, k = draft_tok.shape
+    kv = verify_tok.shape[1]
+    dev = draft_tok.device
+    if not (draft_tok.is_contiguous() and verify_tok.is_contiguous()):
+        raise ValueError("token arrays must be contiguous")
+    if out is None:
+        out = {n: torch.empty(S, dtype=torch.int32, device=dev) for n in ("draft_len", "accept_len", "next_tok")}
+    _check(_lib.load().dssd_accept(_ptr(draft_tok), _ptr(draft_exit_mask), _ptr(verify_tok), S, k, kv,
+                                   _ptr(out["draft_len"]), _ptr(out["accept_len"]), _ptr(out["next_tok"]), _stream()),
+           "dssd_accept")
+    return out
+
+
+def ee_query_async_error(workspace) -> int:
+    """Synchronises the current stream; 0 if no bounded wait gave up since the last query, else EE_ERR_TIMEOUT."""
+    return int(_lib.load().ee_query_async_error(_ptr(workspace), _stream()))

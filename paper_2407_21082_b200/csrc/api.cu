@@ -1,0 +1,183 @@
+// The C ABI: argument validation, device checks, kernel selection.  No compute happens here.
+#include <stdint.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ee {
+namespace {
+
+struct DeviceInfo {
+    bool known = false;
+    bool sm100 = false;
+    int num_sms = 0;
+};
+
+// Properties of the current device (cached per ordinal).
+ee_status current_device(int* device, int* num_sms) {
+    static DeviceInfo info[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return EE_ERR_CUDA;
+    if (!info[dev].known) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return EE_ERR_CUDA;
+        info[dev].sm100 = (major == 10);
+        info[dev].num_sms = sms;
+        info[dev].known = true;
+    }
+    if (!info[dev].sm100) return EE_ERR_ARCH;
+    *device = dev;
+    *num_sms = info[dev].num_sms;
+    return EE_OK;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool sizes_ok(int M, int d, int V) { return M >= 0 && V >= 1 && d >= 8 && d <= 8192 && (d % 8) == 0; }
+
+// Kernel used for M rows when the caller does not choose.
+int auto_path(int M, int d) {
+    const int slab = stream_slab_rows(d);
+    return (slab > 0 && M <= slab) ? EE_PATH_STREAM : EE_PATH_TCGEN05;
+}
+
+size_t workspace_bytes(int M, int d, int V) {
+    size_t need = gemm_workspace_bytes(M, d, V);
+    const size_t s = stream_workspace_bytes(M, d, V);
+    if (s > need) need = s;
+    return kCtrlBytes + need;
+}
+
+}  // namespace
+}  // namespace ee
+
+using namespace ee;
+
+extern "C" {
+
+const char* ee_status_string(ee_status status) {
+    switch (status) {
+        case EE_OK: return "ok";
+        case EE_ERR_NULL: return "a required pointer is NULL";
+        case EE_ERR_SHAPE: return "a size is out of range";
+        case EE_ERR_ALIGN: return "a pointer or stride is misaligned";
+        case EE_ERR_WORKSPACE: return "workspace too small";
+        case EE_ERR_ARCH: return "device is not sm_100";
+        case EE_ERR_CUDA: return "a CUDA call failed";
+        case EE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    }
+    return "unknown status";
+}
+
+size_t ee_exit_head_workspace_bytes(int M, int d, int V) {
+    if (!sizes_ok(M, d, V)) return 0;
+    return workspace_bytes(M, d, V);
+}
+
+ee_status ee_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!workspace) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < (size_t)kCtrlBytes) return EE_ERR_WORKSPACE;
+    return cudaMemsetAsync(workspace, 0, kCtrlBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? EE_OK
+                                                                                                       : EE_ERR_CUDA;
+}
+
+ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau, int* argmax,
+                            float* entropy, float* maxprob, unsigned char* exit_mask, void* workspace,
+                            size_t workspace_bytes_, void* stream, int path) {
+    if (!sizes_ok(M, d, V)) return EE_ERR_SHAPE;
+    if (path != EE_PATH_AUTO && path != EE_PATH_STREAM && path != EE_PATH_TCGEN05) return EE_ERR_SHAPE;
+    if (M == 0) return EE_OK;
+    if (!h || !gamma || !beta || !W || !argmax || !entropy || !maxprob || !exit_mask || !workspace) return EE_ERR_NULL;
+    if (ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
+    if (!aligned(h, 16) || !aligned(W, 16) || !aligned(gamma, 16) || !aligned(beta, 16) || !aligned(workspace, 256))
+        return EE_ERR_ALIGN;
+    if (workspace_bytes_ < workspace_bytes(M, d, V)) return EE_ERR_WORKSPACE;
+
+    HeadArgs a;
+    const ee_status dev = current_device(&a.device, &a.num_sms);
+    if (dev != EE_OK) return dev;
+    a.h = h; a.ld_h = ld_h; a.gamma = gamma; a.beta = beta; a.ln_eps = ln_eps; a.W = W;
+    a.M = M; a.d = d; a.V = V; a.tau_per_row = tau_per_row; a.tau = tau;
+    a.argmax = argmax; a.entropy = entropy; a.maxprob = maxprob; a.exit_mask = exit_mask;
+    a.workspace = workspace; a.workspace_bytes = workspace_bytes_;
+    a.stream = static_cast<cudaStream_t>(stream);
+
+    if (path == EE_PATH_AUTO) path = auto_path(M, d);
+    if (path == EE_PATH_STREAM) return stream_launch(a);
+    return gemm_launch(a);
+}
+
+ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                       const void* W, int M, int d, int V, const float* tau_per_row, float tau, int* argmax,
+                       float* entropy, float* maxprob, unsigned char* exit_mask, void* workspace,
+                       size_t workspace_bytes_, void* stream) {
+    return ee_exit_head_path(h, ld_h, gamma, beta, ln_eps, W, M, d, V, tau_per_row, tau, argmax, entropy, maxprob,
+                             exit_mask, workspace, workspace_bytes_, stream, EE_PATH_AUTO);
+}
+
+ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                            int* argmax_host, float* entropy_host, float* maxprob_host, unsigned char* exit_mask_host,
+                            int* argmax_dev, float* entropy_dev, float* maxprob_dev, unsigned char* exit_mask_dev,
+                            void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!sizes_ok(M, d, V)) return EE_ERR_SHAPE;
+    if (M == 0) return EE_OK;
+    if (!h_host || !h_dev || !argmax_host || !entropy_host || !maxprob_host || !exit_mask_host) return EE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(h_dev, h_host, (size_t)M * d * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return EE_ERR_CUDA;
+    const ee_status st = ee_exit_head(h_dev, d, gamma, beta, ln_eps, W, M, d, V, tau_per_row, tau, argmax_dev,
+                                      entropy_dev, maxprob_dev, exit_mask_dev, workspace, workspace_bytes_, stream);
+    if (st != EE_OK) return st;
+    if (cudaMemcpyAsync(argmax_host, argmax_dev, (size_t)M * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(entropy_host, entropy_dev, (size_t)M * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(maxprob_host, maxprob_dev, (size_t)M * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(exit_mask_host, exit_mask_dev, (size_t)M, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return EE_ERR_CUDA;
+    return EE_OK;
+}
+
+ee_status ee_compact(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d, int* kept_idx,
+                     int* kept_count, void* h_out, void* stream) {
+    if (M < 0) return EE_ERR_SHAPE;
+    if (!kept_count) return EE_ERR_NULL;
+    if (M > 0 && (!exit_mask || !kept_idx)) return EE_ERR_NULL;
+    if (h_out) {
+        if (M > 0 && !h) return EE_ERR_NULL;
+        if (d < 8 || (d % 8) != 0 || ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
+        if (!aligned(h, 16) || !aligned(h_out, 16)) return EE_ERR_ALIGN;
+    }
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return compact_launch(exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out, static_cast<cudaStream_t>(stream));
+}
+
+ee_status dssd_accept(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k,
+                      int kv, int* draft_len, int* accept_len, int* next_tok, void* stream) {
+    if (S < 0 || k < 1 || kv < k) return EE_ERR_SHAPE;
+    if (S == 0) return EE_OK;
+    if (!draft_tok || !verify_tok || !draft_len || !accept_len || !next_tok) return EE_ERR_NULL;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return accept_launch(draft_tok, draft_exit_mask, verify_tok, S, k, kv, draft_len, accept_len, next_tok,
+                         static_cast<cudaStream_t>(stream));
+}
+
+ee_status ee_query_async_error(void* workspace, void* stream) {
+    if (!workspace) return EE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned int words[3] = {0, 0, 0};
+    if (cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, s) != cudaSuccess) return EE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EE_ERR_CUDA;
+    if (words[1] == 0) return EE_OK;
+    if (cudaMemsetAsync(static_cast<unsigned char*>(workspace) + 4, 0, 8, s) != cudaSuccess) return EE_ERR_CUDA;
+    return EE_ERR_TIMEOUT;
+}
+
+}  // extern "C"

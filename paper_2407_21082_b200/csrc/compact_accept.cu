@@ -1,0 +1,108 @@
+// Order-preserving compaction of the rows that did not exit (with the gather of their hidden states),
+// and the DSSD draft-length / accepted-prefix count.  Integer work: ballots, popcounts, first-set-bit.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ee {
+
+namespace {
+
+constexpr int kCompactThreads = 256;
+constexpr int kRowsPerCta = 32;           // one ballot's worth of rows per CTA
+
+// CTA b owns rows [32b, 32b + 32).  Its output offset is the number of surviving rows before 32b, which it
+// counts itself from the mask (M bytes at most, L2-resident), so no CTA waits for another.
+__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned char* __restrict__ exit_mask,
+                                                                  const __nv_bfloat16* __restrict__ h, long long ld_h,
+                                                                  int M, int d, int* __restrict__ kept_idx,
+                                                                  int* __restrict__ kept_count,
+                                                                  __nv_bfloat16* __restrict__ h_out) {
+    __shared__ int s_warp_cnt[kCompactThreads / 32];
+    __shared__ int s_src[kRowsPerCta];
+    __shared__ int s_base, s_n;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = blockIdx.x * kRowsPerCta;
+
+    int cnt = 0;
+    for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (exit_mask[i] == 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0) s_warp_cnt[warp] = cnt;
+    __syncthreads();
+    if (warp == 0) {
+        int base = 0;
+#pragma unroll
+        for (int w = 0; w < kCompactThreads / 32; ++w) base += s_warp_cnt[w];
+        const int row = row0 + lane;
+        const bool keep = (row < M) && (exit_mask[row] == 0);
+        const unsigned int ballot = __ballot_sync(0xffffffffu, keep);
+        const int rank = __popc(ballot & ((1u << lane) - 1u));
+        if (keep) {
+            kept_idx[base + rank] = row;
+            s_src[rank] = row;
+        }
+        if (lane == 0) {
+            s_base = base;
+            s_n = __popc(ballot);
+            if (row0 + kRowsPerCta >= M) *kept_count = base + __popc(ballot);     // the last CTA knows the total
+        }
+    }
+    __syncthreads();
+    if (h_out == nullptr) return;
+    const int nvec = d >> 3;
+    for (int r = warp; r < s_n; r += kCompactThreads / 32) {
+        const uint4* src = reinterpret_cast<const uint4*>(h + (size_t)s_src[r] * ld_h);
+        uint4* dst = reinterpret_cast<uint4*>(h_out + (size_t)(s_base + r) * d);
+        for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(src + c);
+    }
+}
+
+// One warp per sequence; lane j looks at draft slot j (slots beyond 32 in further rounds).
+__global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ draft_tok,
+                                                     const unsigned char* __restrict__ draft_exit_mask,
+                                                     const int* __restrict__ verify_tok, int S, int k, int kv,
+                                                     int* __restrict__ draft_len, int* __restrict__ accept_len,
+                                                     int* __restrict__ next_tok) {
+    const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (s >= S) return;
+    int n = k;             // first slot that is not confident (draft length)
+    int first_mis = k;     // first slot whose drafted token differs from the verifier's
+    for (int base = 0; base < k; base += 32) {
+        const int j = base + lane;
+        const bool in = j < k;
+        const bool conf = in && (draft_exit_mask == nullptr || draft_exit_mask[(size_t)s * k + j] != 0);
+        const bool same = in && (draft_tok[(size_t)s * k + j] == verify_tok[(size_t)s * kv + j]);
+        const unsigned int stop_b = __ballot_sync(0xffffffffu, in && !conf);
+        const unsigned int mis_b = __ballot_sync(0xffffffffu, in && !same);
+        if (first_mis == k && mis_b) first_mis = base + __ffs(mis_b) - 1;
+        if (stop_b) { n = base + __ffs(stop_b) - 1; break; }     // slots after the stop are never drafted
+    }
+    const int a = first_mis < n ? first_mis : n;
+    if (lane == 0) {
+        draft_len[s] = n;
+        accept_len[s] = a;
+        next_tok[s] = (a < kv) ? verify_tok[(size_t)s * kv + a] : -1;
+    }
+}
+
+}  // namespace
+
+ee_status compact_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d, int* kept_idx,
+                         int* kept_count, void* h_out, cudaStream_t stream) {
+    if (M == 0) return cudaMemsetAsync(kept_count, 0, sizeof(int), stream) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    const int grid = (M + kRowsPerCta - 1) / kRowsPerCta;
+    compact_kernel<<<grid, kCompactThreads, 0, stream>>>(exit_mask, static_cast<const __nv_bfloat16*>(h), ld_h, M, d,
+                                                         kept_idx, kept_count, static_cast<__nv_bfloat16*>(h_out));
+    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+ee_status accept_launch(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k,
+                        int kv, int* draft_len, int* accept_len, int* next_tok, cudaStream_t stream) {
+    if (S == 0) return EE_OK;
+    accept_kernel<<<(S + 3) / 4, 128, 0, stream>>>(draft_tok, draft_exit_mask, verify_tok, S, k, kv, draft_len,
+                                                   accept_len, next_tok);
+    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+}  // namespace ee

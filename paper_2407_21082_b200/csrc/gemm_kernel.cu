@@ -1,0 +1,400 @@
+// Verify/prefill-sized exit head: LayerNorm kernel -> persistent TMA + tcgen05 GEMM whose epilogue reduces
+// every 128 x BN block of logits to per-row softmax states straight out of tensor memory -> merge kernel.
+// The M x V logits are never written anywhere.
+//
+// GEMM kernel, one CTA per SM, 192 threads:
+//   warp 0 (one lane)  TMA producer: y tile [128 x 64] and W tile [BN x 64] per k-block into a smem ring
+//   warp 1 (one lane)  tcgen05.mma issuer; accumulators [128 x BN] fp32 double-buffered in TMEM
+//   warps 2..5         epilogue: tcgen05.ld 32 columns at a time, thread = row, online softmax state,
+//                      one 16-byte partial state per (row, vocabulary tile)
+// All mbarrier waits are bounded; a wait that gives up records an error word, raises the CTA's abort
+// flag, and every role drains to the common exit where TMEM is released.
+#include "common.cuh"
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace ee {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kGemmThreads = 192;
+constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile order
+constexpr int kATileBytes = BM * BK * 2;    // 16 KB
+
+template <int BN>
+struct Cfg {
+    static constexpr int kStages = (BN >= 256) ? 4 : 6;
+    static constexpr int kBTileBytes = BN * BK * 2;
+    static constexpr int kStageBytes = kATileBytes + kBTileBytes;
+    static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;       // power of two for BN in {16..256}
+    static constexpr int kBarBytes = 256;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;   // + slack to align to 1024
+};
+
+struct GemmParams {
+    int M, V, d;
+    int m_tiles, n_tiles, k_blocks;
+    State* partials;       // [M][n_tiles]
+    Control* ctrl;
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
+    const int per_group = kGroupM * n_tiles;
+    const int grp = tile / per_group;
+    const int within = tile - grp * per_group;
+    const int rows_in_group = min(kGroupM, m_tiles - grp * kGroupM);
+    n_tile = within / rows_in_group;
+    m_tile = grp * kGroupM + (within - n_tile * rows_in_group);
+}
+
+__device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abort_flag, unsigned role, unsigned stage,
+                                               unsigned tile) {
+    if (atomicCAS(&ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
+        ctrl->error_info = (role << 24) | ((stage & 0xffu) << 16) | (tile & 0xffffu);
+    *abort_flag = 1;
+    __threadfence_block();
+}
+
+// Fold 32 consecutive logits of one row (columns col0 .. col0+31, the first `nvalid` of them real).
+template <bool kFull>
+__device__ __forceinline__ void fold_chunk(State& st, const float (&v)[32], int col0, int nvalid) {
+    float cm = v[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j)
+        if (kFull || j < nvalid) cm = fmaxf(cm, v[j]);
+    if (cm > st.m) {
+        int j0 = 0;
+#pragma unroll
+        for (int j = 31; j >= 0; --j)
+            if ((kFull || j < nvalid) && v[j] == cm) j0 = j;
+        const float dl = st.m - cm;
+        const bool was_empty = (st.s == 0.f);
+        const float al = was_empty ? 0.f : ex2(dl * kLog2e);
+        st.t = was_empty ? 0.f : al * fmaf(dl, st.s, st.t);
+        st.s = al * st.s;
+        st.m = cm;
+        st.idx = col0 + j0;
+    }
+    const float neg_m2 = -st.m * kLog2e;
+    float s = 0.f, t2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (kFull || j < nvalid) {
+            const float a = fmaf(v[j], kLog2e, neg_m2);      // (z - m) * log2(e)
+            const float e = ex2(a);
+            s += e;
+            t2 = fmaf(e, a, t2);
+        }
+    }
+    st.s += s;
+    st.t = fmaf(t2, kLn2, st.t);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
+                      const GemmParams p) {
+    using C = Cfg<BN>;
+    constexpr int S = C::kStages;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+    const uint32_t a_base = ptx::smem_addr(smem);
+    const uint32_t b_base = a_base + S * kATileBytes;
+    unsigned char* bar_mem = smem + S * C::kStageBytes;
+    const uint32_t bar_base = ptx::smem_addr(bar_mem);
+    // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * S + 4);
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_mem + 8 * (2 * S + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 5) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull_bar(b), 1);
+            ptx::mbar_init(tempty_bar(b), 4);
+        }
+        ptx::mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tm_y);
+        ptx::prefetch_tensormap(&tm_w);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), C::kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, armed = 0, armed_parity = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                int m_tile, n_tile;
+                tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                        record_failure(p.ctrl, abort_flag, 1, stage, tile);
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
+                    ptx::tma_load_2d(a_base + stage * kATileBytes, &tm_y, kb * BK, m_tile * BM, full_bar(stage));
+                    ptx::tma_load_2d(b_base + stage * C::kBTileBytes, &tm_w, kb * BK, n_tile * BN, full_bar(stage));
+                    armed |= 1u << stage;
+                    armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (*abort_flag) {
+                // Let the copies still in flight land before the CTA gives its shared memory back.
+                for (int s = 0; s < S; ++s)
+                    if (armed & (1u << s)) {
+                        const uint32_t par = (armed_parity >> s) & 1u;
+                        for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
+                    }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+                const int buf = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1u;
+                if (!ptx::mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag)) {
+                    record_failure(p.ctrl, abort_flag, 2, 0x80 | buf, tile);
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
+                        record_failure(p.ctrl, abort_flag, 2, stage, tile);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
+                    const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * C::kBTileBytes);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units per step
+                        ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    ptx::mma_commit(empty_bar(stage));    // frees the smem stage when these MMAs are done
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) ptx::mma_commit(tfull_bar(buf));  // accumulator complete
+            }
+            if (*abort_flag) {
+                // Make sure no MMA is still writing TMEM when it is released.
+                ptx::mma_commit(drain_bar);
+                for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int row_in_tile = quarter * 32 + lane;
+        int local = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+            int m_tile, n_tile;
+            tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+            const int buf = local & 1;
+            const uint32_t acc_phase = (local >> 1) & 1u;
+            const bool landed = ptx::mbar_wait(tfull_bar(buf), acc_phase, abort_flag);
+            if (!__all_sync(0xffffffffu, landed)) {       // also reconverges the warp for the aligned TMEM loads
+                if (lane == 0) record_failure(p.ctrl, abort_flag, 3, buf, tile);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int n0 = n_tile * BN;
+            const int ncols = min(BN, p.V - n0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+            State st = state_empty();
+            for (int c = 0; c * 32 < ncols; ++c) {
+                float v[32];
+                ptx::tmem_ld_32x32(taddr + c * 32, v);
+                ptx::tmem_ld_wait();
+                const int nvalid = ncols - c * 32;
+                if (nvalid >= 32) fold_chunk<true>(st, v, n0 + c * 32, 32);
+                else fold_chunk<false>(st, v, n0 + c * 32, nvalid);
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
+            const int row = m_tile * BM + row_in_tile;
+            if (row < p.M) p.partials[(size_t)row * p.n_tiles + n_tile] = st;
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm: h [M, d] (row stride ld_h) -> y [M, d] bf16, one warp per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat16* __restrict__ h, long long ld_h,
+                                                              const float* __restrict__ gamma,
+                                                              const float* __restrict__ beta, float ln_eps,
+                                                              __nv_bfloat16* __restrict__ y, int M, int d) {
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    const int nvec = d >> 3;
+    const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)row * ld_h);
+    uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
+    const float inv_d = 1.f / (float)d;
+    float sum = 0.f;
+    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
+    const float mu = warp_sum(sum) * inv_d;
+    float sq = 0.f;
+    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
+    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
+    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials, int n_tiles, int M,
+                                                         const float* __restrict__ tau_per_row, float tau,
+                                                         int* argmax, float* entropy, float* maxprob,
+                                                         unsigned char* exit_mask) {
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    State a = state_empty();
+    for (int n = lane; n < n_tiles; n += 32) {
+        const State o = state_load_cg(partials + (size_t)row * n_tiles + n);
+        state_merge(a, o);
+    }
+#pragma unroll
+    for (int msk = 1; msk <= 16; msk <<= 1) {
+        const State o = state_shfl_xor(a, msk);
+        state_merge(a, o);
+    }
+    if (lane == 0) state_finish(a, tau_per_row ? tau_per_row[row] : tau, argmax, entropy, maxprob, exit_mask, row);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major (row stride = cols), box = [box_rows x 64 columns], 128-byte swizzle.
+bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+ee_status launch_gemm(const CUtensorMap& tm_y, const CUtensorMap& tm_w, const GemmParams& p, int grid, int device,
+                      cudaStream_t stream) {
+    static bool configured[kMaxDevices] = {};
+    if (!configured[device]) {
+        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg<BN>::kSmemBytes) != cudaSuccess)
+            return EE_ERR_CUDA;
+        configured[device] = true;
+    }
+    exit_head_gemm_kernel<BN><<<grid, kGemmThreads, Cfg<BN>::kSmemBytes, stream>>>(tm_y, tm_w, p);
+    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+size_t partials_bytes(int M, int V) {
+    const int bn = gemm_tile_n(M);
+    return align_up((size_t)M * ((V + bn - 1) / bn) * sizeof(State), 256);
+}
+
+}  // namespace
+
+int gemm_tile_n(int M) { return M > 1024 ? 256 : 128; }
+
+size_t gemm_workspace_bytes(int M, int d, int V) {
+    return partials_bytes(M, V) + align_up((size_t)M * d * sizeof(__nv_bfloat16), 256);
+}
+
+ee_status gemm_launch(const HeadArgs& a) {
+    unsigned char* ws = static_cast<unsigned char*>(a.workspace);
+    State* partials = reinterpret_cast<State*>(ws + kCtrlBytes);
+    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + partials_bytes(a.M, a.V));
+    const int bn = gemm_tile_n(a.M);
+
+    layer_norm_rows_kernel<<<(a.M + 7) / 8, 256, 0, a.stream>>>(static_cast<const __nv_bfloat16*>(a.h), a.ld_h, a.gamma,
+                                                                a.beta, a.ln_eps, y, a.M, a.d);
+    if (cudaGetLastError() != cudaSuccess) return EE_ERR_CUDA;
+
+    CUtensorMap tm_y, tm_w;
+    if (!make_tile_map(&tm_y, y, a.M, a.d, BM) || !make_tile_map(&tm_w, a.W, a.V, a.d, bn)) return EE_ERR_CUDA;
+
+    GemmParams p;
+    p.M = a.M;
+    p.V = a.V;
+    p.d = a.d;
+    p.m_tiles = (a.M + BM - 1) / BM;
+    p.n_tiles = (a.V + bn - 1) / bn;
+    p.k_blocks = (a.d + BK - 1) / BK;
+    p.partials = partials;
+    p.ctrl = reinterpret_cast<Control*>(ws);
+    const long long total = (long long)p.m_tiles * p.n_tiles;
+    const int grid = (int)(total < a.num_sms ? total : a.num_sms);
+    const ee_status st = (bn == 256) ? launch_gemm<256>(tm_y, tm_w, p, grid, a.device, a.stream)
+                                     : launch_gemm<128>(tm_y, tm_w, p, grid, a.device, a.stream);
+    if (st != EE_OK) return st;
+
+    merge_rows_kernel<<<(a.M + 7) / 8, 256, 0, a.stream>>>(partials, p.n_tiles, a.M, a.tau_per_row, a.tau, a.argmax,
+                                                           a.entropy, a.maxprob, a.exit_mask);
+    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+}  // namespace ee

@@ -1,0 +1,187 @@
+"""Parity of ee_exit_head (both kernels) with the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from _util import assert_head_matches, dev, dev_bf16, head_to_dev, oracle_head
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ee():
+    import paper_2407_21082_b200 as ee
+    assert torch.cuda.is_available()
+    return ee
+
+
+def _run(ee, cfg, head_id, tau, path, h_key="h"):
+    hd = head_to_dev(cfg["heads"][head_id])
+    tau_arg = dev(tau) if isinstance(tau, np.ndarray) else tau
+    out = ee.ee_exit_head(dev_bf16(cfg[h_key]), hd["gamma"], hd["beta"], hd["ln_eps"], hd["W"], tau_arg, path=path)
+    torch.cuda.synchronize()
+    return out
+
+
+# Reduced shapes: several vocabulary tiles with a ragged last one, K tails (d % 64 != 0, d % 32 != 0),
+# partial row tiles, degenerate V = 1, and row counts around the slab (32) and tile (128) sizes.
+SMALL = [
+    # name, M, d, V
+    ("v1", 3, 64, 1), ("tiny", 1, 8, 5), ("ragged", 5, 72, 257), ("k_tail", 8, 520, 1000),
+    ("two_ntiles", 16, 128, 300), ("slab_edge", 32, 256, 2049), ("slab_over", 33, 264, 1031),
+    ("mtile_edge", 128, 64, 700), ("mtile_over", 129, 320, 515), ("wide_d", 4, 4096, 600),
+]
+
+
+@pytest.mark.parametrize("path_name", ["stream", "tcgen05"])
+@pytest.mark.parametrize("name,M,d,V", SMALL)
+def test_small_shapes_match_oracle(ee, path_name, name, M, d, V):
+    path = ee.EE_PATH_STREAM if path_name == "stream" else ee.EE_PATH_TCGEN05
+    for planted in (False, True):
+        cfg = gen.make_config("c0", seed=11, planted=planted, M=M, d=d, V=V)
+        tau = 1.0 if planted else float(np.log(V) - 0.05) if V > 1 else 1.0
+        ref = oracle_head(cfg["h"], cfg["heads"][0], tau)
+        out = _run(ee, cfg, 0, tau, path)
+        assert_head_matches(out, ref, label=f"{name}/{path_name}/planted={planted}")
+
+
+def test_exact_small_integer_case(ee):
+    """Alternating +-1 rows normalise to exactly +-1; dyadic W makes every logit exact in fp32."""
+    d, V, M = 64, 40, 2
+    x = np.tile([1.0, -1.0], d // 2)[None, :].repeat(M, 0)
+    x[1] *= -1
+    Wv = ((np.arange(V * d).reshape(V, d) * 7) % 13 - 6) / 8.0
+    head = dict(gamma=np.ones(d, np.float32), beta=np.zeros(d, np.float32), ln_eps=1e-5,
+                W=gen.bf16_bits_from_f32(Wv.astype(np.float32)))
+    h = gen.bf16_bits_from_f32(x.astype(np.float32))
+    ref = oracle.exit_head(h, head["gamma"], head["beta"], 1e-5, head["W"], 1.0)
+    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+        hd = head_to_dev(head)
+        out = ee.ee_exit_head(dev_bf16(h), hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, path=path)
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        assert np.array_equal(got["argmax"], ref["argmax"])
+        assert np.allclose(got["entropy"], ref["entropy"], atol=1e-5)
+        assert np.allclose(got["maxprob"], ref["maxprob"], atol=1e-6)
+
+
+def test_uniform_logits_give_ln_V_and_lowest_index(ee):
+    """W = 0 makes all logits equal: H = ln V, p_max = 1/V, argmax = 0 (lowest index wins ties)."""
+    d, V, M = 128, 50304, 4
+    cfg = gen.make_config("c0", seed=1, M=M, d=d, V=8)
+    Wz = torch.zeros((V, d), dtype=torch.bfloat16, device="cuda")
+    hd = head_to_dev(cfg["heads"][0])
+    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+        out = ee.ee_exit_head(dev_bf16(cfg["h"]), hd["gamma"], hd["beta"], 1e-5, Wz, 11.0, path=path)
+        assert torch.all(out["argmax"] == 0)
+        assert np.allclose(out["entropy"].cpu().numpy(), 10.825839875788878, atol=2e-4)
+        assert np.allclose(out["maxprob"].cpu().numpy(), 1 / V, rtol=1e-4)
+        assert torch.all(out["exit_mask"] == 1)
+
+
+@pytest.mark.parametrize("planted", [False, True])
+def test_c0_full_size(ee, planted):
+    cfg = gen.make_config("c0", seed=0, planted=planted)
+    for tau in cfg["taus"]:
+        ref = oracle_head(cfg["h"], cfg["heads"][0], tau)
+        for path in (ee.EE_PATH_AUTO, ee.EE_PATH_TCGEN05):
+            assert_head_matches(_run(ee, cfg, 0, tau, path), ref, label=f"c0 tau={tau} path={path}")
+
+
+@pytest.mark.parametrize("planted", [False, True])
+def test_c1_three_heads_full_size(ee, planted):
+    cfg = gen.make_config("c1", seed=0, planted=planted)
+    exits = 0
+    for hid in range(3):
+        ref64 = oracle_head(cfg["h"], cfg["heads"][hid], cfg["tau"])
+        exits += int(ref64["exit_mask"].sum())
+        for M in gen.CONFIGS["c1"]["Ms"]:
+            sub = dict(cfg, h=cfg["h"][:M])
+            ref = {k: v[:M] for k, v in ref64.items()}
+            for path in (ee.EE_PATH_AUTO, ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+                assert_head_matches(_run(ee, sub, hid, cfg["tau"], path), ref, label=f"c1 head{hid} M={M} path={path}")
+    if planted:
+        assert 0 < exits < 3 * 64          # the planted inputs exercise both outcomes
+
+
+@pytest.mark.parametrize("planted", [False, True])
+def test_c2_per_row_thresholds_full_size(ee, planted):
+    cfg = gen.make_config("c2", seed=0, planted=planted)
+    ref = oracle_head(cfg["h"], cfg["heads"][0], cfg["tau_per_row"])
+    for path in (ee.EE_PATH_AUTO, ee.EE_PATH_STREAM):
+        assert_head_matches(_run(ee, cfg, 0, cfg["tau_per_row"], path), ref, label=f"c2 path={path}")
+
+
+def test_c4_full_size_on_a_stratified_row_sample(ee):
+    """M = 16384: the oracle checks >= 4 rows of every 128-row tile, every row residue mod 128 covered."""
+    cfg = gen.make_config("c4", seed=0, planted=True)
+    out = _run(ee, cfg, 0, cfg["tau"], ee.EE_PATH_AUTO)
+    assert ee.ee_query_async_error is not None
+    rows = np.array([t * 128 + (t + 32 * i) % 128 for t in range(128) for i in range(4)])
+    rows = np.unique(np.concatenate([rows, [0, 127, 128, 16383]]))
+    ref = oracle_head(cfg["h"], cfg["heads"][0], cfg["tau"], rows=rows)
+    info = assert_head_matches(out, ref, rows=rows, label="c4 sample")
+    assert len(set(rows // 128)) == 128 and len(set(rows % 128)) == 128
+    # properties that hold for every row
+    H = out["entropy"].cpu().numpy(); P = out["maxprob"].cpu().numpy(); A = out["argmax"].cpu().numpy()
+    assert np.all((H >= -1e-4) & (H <= np.log(50304) + 1e-3)) and np.all((P > 0) & (P <= 1 + 1e-6))
+    assert np.all((A >= 0) & (A < 50304))
+    assert np.array_equal(out["exit_mask"].cpu().numpy(), (H < cfg["tau"]).astype(np.uint8))
+    assert np.all(H >= -np.log(np.minimum(P, 1.0)) - 1e-3)        # H >= -ln p_max for any distribution
+    assert info["max_dH"] <= 2e-3
+
+
+def test_both_kernels_agree_and_runs_are_bit_identical(ee):
+    cfg = gen.make_config("c1", seed=5, planted=True, M=32, V=20000)
+    a = _run(ee, cfg, 0, 1.0, ee.EE_PATH_STREAM)
+    b = _run(ee, cfg, 0, 1.0, ee.EE_PATH_STREAM)
+    c = _run(ee, cfg, 0, 1.0, ee.EE_PATH_TCGEN05)
+    e = _run(ee, cfg, 0, 1.0, ee.EE_PATH_TCGEN05)
+    for k in a:
+        assert torch.equal(a[k], b[k]) and torch.equal(c[k], e[k]), k
+    assert torch.allclose(a["entropy"], c["entropy"], atol=1e-3) and torch.equal(a["argmax"], c["argmax"])
+
+
+def test_row_stride_and_workspace_reuse(ee):
+    cfg = gen.make_config("c0", seed=2, planted=True, M=9, d=128, V=3000)
+    hd = head_to_dev(cfg["heads"][0])
+    wide = torch.zeros((9, 256), dtype=torch.bfloat16, device="cuda")
+    wide[:, :128] = dev_bf16(cfg["h"])
+    ref = oracle_head(cfg["h"], cfg["heads"][0], 1.0)
+    ws = ee.new_workspace(9, 128, 3000)
+    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05, ee.EE_PATH_STREAM):
+        out = ee.ee_exit_head(wide[:, :128], hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, workspace=ws, path=path)
+        assert_head_matches(out, ref, label=f"strided path={path}")
+    assert ee.ee_query_async_error(ws) == 0
+
+
+def test_host_buffer_variant(ee):
+    cfg = gen.make_config("c0", seed=4, planted=True, M=8, d=256, V=5000)
+    hd = head_to_dev(cfg["heads"][0])
+    h_host = torch.from_numpy(cfg["h"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    out_host = {k: v.cpu().pin_memory() for k, v in ee.new_outputs(8).items()}
+    out_dev = ee.new_outputs(8)
+    h_dev = torch.empty((8, 256), dtype=torch.bfloat16, device="cuda")
+    ws = ee.new_workspace(8, 256, 5000)
+    ee.ee_exit_head_host(h_host, h_dev, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, out_host, out_dev, ws)
+    torch.cuda.synchronize()
+    ref = oracle_head(cfg["h"], cfg["heads"][0], 1.0)
+    assert_head_matches({k: v.cuda() for k, v in out_host.items()}, ref, label="host variant")
+
+
+def test_device_side_argument_errors(ee):
+    cfg = gen.make_config("c0", seed=2, M=4, d=64, V=100)
+    hd = head_to_dev(cfg["heads"][0])
+    h = dev_bf16(cfg["h"])
+    small_ws = torch.zeros(512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_exit_head(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, workspace=small_ws)
+    assert e.value.code == 4
+    ws = ee.new_workspace(4, 64, 100)
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_exit_head(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, workspace=ws[8:])
+    assert e.value.code in (3, 4)
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_exit_head(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, workspace=ws, path=7)
+    assert e.value.code == 2
