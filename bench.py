@@ -1,0 +1,392 @@
+"""Benchmark of the exit-head hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c1] [--no-extra]
+
+A step is one pass of the whole hot path over one batch: LayerNorm + head projection + entropy / argmax /
+max-prob + exit decision for every head of the workload, compaction of the rows that did not exit, and
+the DSSD draft-length / accepted-prefix count.  The headline workload is the Pythia-410M-shaped decode
+batch (d = 1024, V = 50304, three heads, M = 64 rows).  `value` counts head evaluations of a row per
+second (a row through three heads counts three times), which is what the HBM roofline of one head call
+bounds: M / (bytes of W / bandwidth).
+
+Prints one JSON line.  With --impl reference the same metric is measured for the fp64 CPU oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "exit-head tokens/s (LN+head+entropy+exit)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons), samples=len(sm))
+
+
+# --------------------------------------------------------------------------------------------- workloads
+
+
+def _algorithmic(M, d, V):
+    """Bytes and flops one head call must move / do: W once, h once, 13 bytes of output per row."""
+    return 2.0 * V * d + 2.0 * M * d + 13.0 * M, 2.0 * M * V * d
+
+
+class Workload:
+    """Device tensors of one workload and a `step()` that runs the whole hot path once."""
+
+    def __init__(self, name: str, M: int | None, seed: int, n_copies: int):
+        import torch
+        import paper_2407_21082_b200 as ee
+        self.torch, self.ee = torch, ee
+        cfg = gen.make_config(name, seed=seed, planted=False, M=M)
+        self.name, self.cfg = name, cfg
+        self.M, self.d, self.V = cfg["M"], cfg["d"], cfg["V"]
+
+        def bf16(bits):
+            return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+        self.heads = []
+        for hd in cfg["heads"]:
+            dev = dict(gamma=torch.from_numpy(hd["gamma"]).cuda(), beta=torch.from_numpy(hd["beta"]).cuda(), W=[bf16(hd["W"])])
+            for _ in range(n_copies - 1):          # distinct copies of W so that consecutive calls miss in L2
+                dev["W"].append(dev["W"][0].clone())
+            self.heads.append(dev)
+        if name == "c3":
+            self.h = [bf16(cfg["h_draft"]), bf16(cfg["h_verify"])]
+            self.S, self.k = cfg["S"], cfg["k"]
+        else:
+            self.h = [bf16(cfg["h"])] * len(self.heads)
+            self.k = 8
+            self.S = self.M // self.k
+        self.tau = torch.from_numpy(cfg["tau_per_row"]).cuda() if "tau_per_row" in cfg else float(cfg["tau"])
+        self.ws = ee.new_workspace(self.M, self.d, self.V)
+        self.outs = [ee.new_outputs(self.M) for _ in self.heads]
+        self.comp = dict(kept_idx=torch.empty(self.M, dtype=torch.int32, device="cuda"),
+                         kept_count=torch.zeros(1, dtype=torch.int32, device="cuda"),
+                         h_out=torch.empty((self.M, self.d), dtype=torch.bfloat16, device="cuda"))
+        self.acc = {n: torch.empty(max(self.S, 1), dtype=torch.int32, device="cuda") for n in ("draft_len", "accept_len", "next_tok")}
+        self.calls = 0
+        self.n_copies = n_copies
+        self.head_launches = ee.ee_exit_head_launches(self.M, self.d, self.V)
+        self.launches_per_step = len(self.heads) * self.head_launches + 1 + (1 if self.S > 0 else 0)
+        self.bytes_per_call, self.flops_per_call = _algorithmic(self.M, self.d, self.V)
+        self.w_bytes_total = sum(w.numel() * 2 for hd in self.heads for w in hd["W"])
+
+    def run_heads(self):
+        ee = self.ee
+        c = self.calls % self.n_copies
+        for i, hd in enumerate(self.heads):
+            ee.ee_exit_head(self.h[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], self.tau, out=self.outs[i], workspace=self.ws)
+        self.calls += 1
+
+    def run_tail(self):
+        ee = self.ee
+        ee.ee_compact(self.outs[0]["exit_mask"], self.h[0], out=self.comp)
+        if self.S > 0:
+            n = self.S * self.k
+            ee.dssd_accept(self.outs[0]["argmax"][:n].view(self.S, self.k), self.outs[0]["exit_mask"][:n].view(self.S, self.k),
+                           self.outs[-1]["argmax"][:n].view(self.S, self.k), out=self.acc)
+
+    def step(self):
+        self.run_heads()
+        self.run_tail()
+
+
+def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSampler | None = None) -> dict:
+    """Times `steps` steps with CUDA events on the launching stream; also the head calls alone inside them."""
+    torch = wl.torch
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for a, b in ev:
+        a.record()
+        wl.run_heads()
+        b.record()
+        wl.run_tail()
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    total_ms = t0.elapsed_time(t1)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    heads_ms = sum(a.elapsed_time(b) for a, b in ev)
+    n_heads = len(wl.heads)
+    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, head_call_us=1e3 * heads_ms / (steps * n_heads),
+                tail_us=1e3 * (total_ms - heads_ms) / steps, clocks=clocks)
+
+
+def roofline(wl: Workload, head_call_us: float, peaks: dict, src: str) -> dict:
+    gbs = wl.bytes_per_call / (head_call_us * 1e-6) / 1e9
+    tfs = wl.flops_per_call / (head_call_us * 1e-6) / 1e12
+    t_hbm = wl.bytes_per_call / (peaks["hbm_gbs"] * 1e9)
+    t_tc = wl.flops_per_call / (peaks["bf16_tflops"] * 1e12)
+    if t_hbm >= t_tc:
+        return dict(bound="hbm", achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s", frac=round(gbs / peaks["hbm_gbs"], 4),
+                    traffic=None, peak_source=f"of {src}", tensor_frac=round(tfs / peaks["bf16_tflops"], 4))
+    return dict(bound="tensor", achieved=round(tfs, 1), peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                frac=round(tfs / peaks["bf16_tflops"], 4), traffic=None, peak_source=f"of {src} (burst)",
+                frac_of_sustained=round(tfs / peaks["bf16_tflops_sustained"], 4), hbm_frac=round(gbs / peaks["hbm_gbs"], 4))
+
+
+# --------------------------------------------------------------------------------------------- e2e and CPU baseline
+
+
+def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
+    """Same step driven through ee_exit_head_host: h comes from pinned host memory and the results go back to it."""
+    torch, ee = wl.torch, wl.ee
+    h_host = [h.cpu().pin_memory() for h in wl.h]
+    h_dev = [torch.empty_like(h) for h in wl.h]
+    out_host = [{k: v.cpu().pin_memory() for k, v in o.items()} for o in wl.outs]
+    small_host = {k: v.cpu().pin_memory() for k, v in {**wl.acc, "kept_count": wl.comp["kept_count"]}.items()}
+
+    def step():
+        c = wl.calls % wl.n_copies
+        for i, hd in enumerate(wl.heads):
+            ee.ee_exit_head_host(h_host[i], h_dev[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], wl.tau, out_host[i], wl.outs[i], wl.ws)
+        wl.calls += 1
+        ee.ee_compact(wl.outs[0]["exit_mask"], h_dev[0], out=wl.comp)
+        if wl.S > 0:
+            n = wl.S * wl.k
+            ee.dssd_accept(wl.outs[0]["argmax"][:n].view(wl.S, wl.k), wl.outs[0]["exit_mask"][:n].view(wl.S, wl.k),
+                           wl.outs[-1]["argmax"][:n].view(wl.S, wl.k), out=wl.acc)
+        small_host["kept_count"].copy_(wl.comp["kept_count"], non_blocking=True)
+        for k in wl.acc:
+            small_host[k].copy_(wl.acc[k], non_blocking=True)
+        torch.cuda.synchronize()          # the caller reads its results every step
+
+    for _ in range(warmup):
+        step()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    n_heads = len(wl.heads)
+    h2d = n_heads * wl.M * wl.d * 2
+    d2h = n_heads * wl.M * 13 + 4 + 3 * 4 * max(wl.S, 1)
+    return dict(value=n_heads * wl.M * steps / wall, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                ms_per_step=1e3 * wall / steps, device_ms_per_step=t0.elapsed_time(t1) / steps)
+
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_step(cfg: dict, rows: int, heads: int):
+    """The oracle's version of a step on the first `rows` rows and `heads` heads.  Returns rows*heads."""
+    import oracle
+    hb = cfg["h_draft" if "h_draft" in cfg else "h"][:rows]
+    tau = cfg["tau_per_row"][:rows] if "tau_per_row" in cfg else cfg["tau"]
+    outs = []
+    for hd in cfg["heads"][:heads]:
+        outs.append(oracle.exit_head(hb, hd["gamma"], hd["beta"], hd["ln_eps"], hd["W"], tau))
+    oracle.compact(outs[0]["exit_mask"], hb)
+    S = rows // 8
+    if S:
+        oracle.dssd_accept(outs[0]["argmax"][:S * 8].reshape(S, 8), outs[0]["exit_mask"][:S * 8].reshape(S, 8),
+                           outs[-1]["argmax"][:S * 8].reshape(S, 8))
+    return rows * heads
+
+
+def cpu_baseline(cfg: dict, steps: int = 1, warmup: int = 0) -> dict:
+    """Times the oracle, as it stands, on the host cores on a bounded sample of the headline workload."""
+    rows, heads = min(cfg["M"], 64), len(cfg["heads"])
+    for _ in range(warmup):
+        oracle_step(cfg, rows, heads)
+    t0 = time.perf_counter()
+    done = 0
+    for _ in range(steps):
+        done += oracle_step(cfg, rows, heads)
+    dt = time.perf_counter() - t0
+    return dict(value=done / dt, unit=UNIT, cores=oracle_threads(), kind="oracle", seconds=round(dt, 2),
+                sample=f"{steps} step(s) of all {rows} rows x {heads} heads of the workload (fp64 numpy, weights decoded per call)")
+
+
+# --------------------------------------------------------------------------------------------- main
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c1")
+    ap.add_argument("--rows", type=int, default=None, help="override M of the workload")
+    ap.add_argument("--no-extra", action="store_true", help="skip the per-config table and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    spec = gen.CONFIGS[args.workload]
+    M = args.rows if args.rows is not None else spec["M"]
+    config = dict(workload=f"{args.workload}: Pythia-shaped exit heads d={spec['d']} V={spec['V']} M={M} heads={spec['heads']}",
+                  rows_per_gpu=M, heads=spec["heads"], d=spec["d"], V=spec["V"], seed=0,
+                  step="all heads on the batch, ee_compact of head 0's survivors, dssd_accept(head 0 vs last head, k=8)")
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        cfg = gen.make_config(args.workload, seed=0, planted=False, M=M)
+        steps = max(1, min(args.steps, 3))
+        base = cpu_baseline(cfg, steps=steps, warmup=min(args.warmup, 1))
+        config["l2"] = "n/a (CPU)"
+        line = dict(metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus, steps=steps, warmup=min(args.warmup, 1),
+                    ms_per_step=1e3 * base["seconds"] / steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="f64", data="synthetic", config=config, impl="reference", cpu_baseline=base,
+                    e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+        print(json.dumps(line))
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks, peak_src = load_peaks()
+
+    n_copies = {"c0": 8, "c1": 2}.get(args.workload, 2)
+    wl = Workload(args.workload, M, seed=rank, n_copies=n_copies)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    res = measure(wl, args.steps, args.warmup, dist, sampler)
+    n_heads = len(wl.heads)
+    value = world * n_heads * wl.M / (res["ms_per_step"] * 1e-3)
+    config["l2"] = (f"inputs larger than L2: the step cycles through {wl.w_bytes_total / 1e6:.0f} MB of head weights "
+                    f"({n_heads} heads x {n_copies} copies) against a 126 MB L2")
+    config["parallelism"] = f"replicas x{world} (independent batches, no collective)"
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic", config=config, clocks=res["clocks"], gpu_launches=wl.launches_per_step * args.steps,
+                head_call_us=res["head_call_us"], tail_us=res["tail_us"])
+    line["roofline"] = roofline(wl, res["head_call_us"], peaks, peak_src)
+    line["roofline"]["kernel"] = ("one ee_exit_head call (%d launch(es)); duration = CUDA events around the %d head calls of "
+                                  "each step, averaged" % (wl.head_launches, n_heads))
+    if rank == 0:
+        line["e2e"] = measure_e2e(wl, max(10, args.steps // 4), 3)
+        if world > 1:
+            line["e2e"]["note"] = "rank 0 only"
+    if not args.no_extra and rank == 0 and world == 1:
+        extra = {}
+        del wl
+        torch.cuda.empty_cache()
+        table = [("c0", None, 8, 200), ("c1", 1, 2, 200), ("c1", 4, 2, 200), ("c1", 16, 2, 200), ("c1", 64, 2, 200),
+                 ("c2", None, 2, 100), ("c3", None, 2, 100), ("c4", None, 2, 10)]
+        for name, rows, copies, steps in table:
+            w = Workload(name, rows, seed=0, n_copies=copies)
+            r = measure(w, steps, 5)
+            key = name if rows is None else f"{name}_M{rows}"
+            extra[key] = dict(M=w.M, d=w.d, heads=len(w.heads), head_call_us=round(r["head_call_us"], 2),
+                              tail_us=round(r["tail_us"], 2), tokens_per_s=w.M / (r["head_call_us"] * 1e-6),
+                              roofline=roofline(w, r["head_call_us"], peaks, peak_src), launches_per_head=w.head_launches)
+            del w
+            torch.cuda.empty_cache()
+        line["configs"] = extra
+        cfg = gen.make_config(args.workload, seed=0, planted=False, M=M)
+        line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

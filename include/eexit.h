@@ -51,6 +51,12 @@ const char* ee_status_string(ee_status status);
 size_t ee_exit_head_workspace_bytes(int M, int d, int V);
 
 /*
+ * Number of kernels one ee_exit_head_path call launches for these sizes and `path` (host-only, pure;
+ * 0 if a size is invalid).  For callers that account for launches, e.g. when sizing a CUDA graph.
+ */
+int ee_exit_head_launches(int M, int d, int V, int path);
+
+/*
  * Zeroes the control block at the start of `workspace`.  Must run once after the workspace is
  * allocated (and after ee_query_async_error reported EE_ERR_TIMEOUT); every ee_exit_head call leaves
  * the block ready for the next one.  The workspace must be 256-byte aligned.  One workspace serves one

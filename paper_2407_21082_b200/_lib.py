@@ -12,6 +12,7 @@ _p = C.c_void_p
 PROTOTYPES = {
     "ee_status_string": (C.c_char_p, [C.c_int]),
     "ee_exit_head_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
+    "ee_exit_head_launches": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "ee_workspace_init": (C.c_int, [_p, C.c_size_t, _p]),
     "ee_exit_head": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                _p, _p, _p, _p, _p, C.c_size_t, _p]),

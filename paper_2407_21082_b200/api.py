@@ -51,6 +51,10 @@ def ee_exit_head_workspace_bytes(M: int, d: int, V: int) -> int:
     return int(_lib.load().ee_exit_head_workspace_bytes(int(M), int(d), int(V)))
 
 
+def ee_exit_head_launches(M: int, d: int, V: int, path: int = EE_PATH_AUTO) -> int:
+    return int(_lib.load().ee_exit_head_launches(int(M), int(d), int(V), int(path)))
+
+
 def ee_workspace_init(workspace: torch.Tensor) -> None:
     _check(_lib.load().ee_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
            "ee_workspace_init")

@@ -77,6 +77,16 @@ size_t ee_exit_head_workspace_bytes(int M, int d, int V) {
     return workspace_bytes(M, d, V);
 }
 
+int ee_exit_head_launches(int M, int d, int V, int path) {
+    if (!sizes_ok(M, d, V) || M == 0) return 0;
+    if (path == EE_PATH_AUTO) path = auto_path(M, d);
+    if (path == EE_PATH_STREAM) {
+        const int slab = stream_slab_rows(d);
+        return slab > 0 ? (M + slab - 1) / slab : 0;
+    }
+    return path == EE_PATH_TCGEN05 ? 3 : 0;      // LayerNorm, GEMM with fused statistics, merge
+}
+
 ee_status ee_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     if (!aligned(workspace, 256)) return EE_ERR_ALIGN;

@@ -253,6 +253,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
+        __syncwarp();
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, C::kTmemCols);
     }

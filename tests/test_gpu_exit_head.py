@@ -125,7 +125,7 @@ def test_c4_full_size_on_a_stratified_row_sample(ee):
     assert len(set(rows // 128)) == 128 and len(set(rows % 128)) == 128
     # properties that hold for every row
     H = out["entropy"].cpu().numpy(); P = out["maxprob"].cpu().numpy(); A = out["argmax"].cpu().numpy()
-    assert np.all((H >= -1e-4) & (H <= np.log(50304) + 1e-3)) and np.all((P > 0) & (P <= 1 + 1e-6))
+    assert np.all((H >= -1e-4) & (H <= np.log(50304) + 1e-3)) and np.all((P > 0) & (P <= 1 + 1e-4))
     assert np.all((A >= 0) & (A < 50304))
     assert np.array_equal(out["exit_mask"].cpu().numpy(), (H < cfg["tau"]).astype(np.uint8))
     assert np.all(H >= -np.log(np.minimum(P, 1.0)) - 1e-3)        # H >= -ln p_max for any distribution
