@@ -108,6 +108,33 @@ ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * ee_exit_head without a workspace argument, for callers that have no way to provide scratch memory.
+ * (The paper has no counterpart for this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs after a serving process has handed all device memory to its own pool
+ * and banned cudaMalloc (which stalls the whole device and can fail on a fragmented heap), plug-ins
+ * and callbacks hosted by a runtime whose allocator they may not call, and latency-critical loops
+ * where no allocator of any kind is permitted.  This entry point calls no cudaMalloc, no cudaFree and no
+ * allocating library routine.  Its scratch is a fixed ~128 KB array inside the library's device image;
+ * every GPU that loads the library carries that array until the process exits.
+ *
+ * Same arguments, results and error codes as ee_exit_head, minus workspace, with these limits:
+ *   - M <= EE_STATIC_MAX_ROWS (decode-sized batches; the fused streaming kernel is always used) and the
+ *     rows must fit one launch of that kernel (any d <= 2048 does for 32 rows).  Larger sizes return
+ *     EE_ERR_SHAPE and launch nothing: use ee_exit_head with a workspace for them.
+ *   - The first call on each device looks up the array's device address and zeroes its control block
+ *     (on `stream`, ahead of the kernel).  Make that first call during start-up, before any stream
+ *     capture, with the device it is meant for current.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the kernel
+ *     rewrites what it reads and leaves the control block zeroed.  Calls that overlap on the GPU (two
+ *     streams, two host threads) therefore race: order them on one stream or with events.
+ */
+#define EE_STATIC_MAX_ROWS 32
+ee_status ee_exit_head_static(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                              const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                              int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask, void* stream);
+
+/*
  * Continuation of the rows that did not exit (section 3.4.2: an input keeps going through the model's
  * layers until a head is confident).  Order-preserving stream compaction:
  *   kept_idx   int32 [M]: ascending indices i with exit_mask[i] == 0 (first *kept_count entries valid)

@@ -9,6 +9,8 @@ from .api import (  # noqa: F401
     ee_exit_head,
     ee_exit_head_host,
     ee_exit_head_launches,
+    ee_exit_head_static,
+    EE_STATIC_MAX_ROWS,
     ee_exit_head_workspace_bytes,
     ee_query_async_error,
     ee_workspace_init,

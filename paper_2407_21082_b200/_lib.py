@@ -20,6 +20,8 @@ PROTOTYPES = {
                                     _p, _p, _p, _p, _p, C.c_size_t, _p, C.c_int]),
     "ee_exit_head_host": (C.c_int, [_p, _p, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                     _p, _p, _p, _p, _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_exit_head_static": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
+                                      _p, _p, _p, _p, _p]),
     "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_query_async_error": (C.c_int, [_p, _p]),

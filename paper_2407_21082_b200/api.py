@@ -98,6 +98,25 @@ def ee_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, pa
     return out
 
 
+EE_STATIC_MAX_ROWS = 32
+
+
+def ee_exit_head_static(h, gamma, beta, ln_eps, W, tau, *, out: dict) -> dict:
+    """ee_exit_head for callers that may not allocate: no workspace argument, at most EE_STATIC_MAX_ROWS rows.
+
+    The library's built-in scratch array is used, so nothing is allocated by the call.  `out` must be given
+    (see new_outputs) -- this wrapper creates no tensors either.  Calls sharing a GPU must not overlap.
+    """
+    h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
+    M, d = h.shape
+    tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+    _check(_lib.load().ee_exit_head_static(
+        _ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W),
+        M, d, W.shape[0], _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
+        _ptr(out["exit_mask"]), _stream()), "ee_exit_head_static")
+    return out
+
+
 def ee_exit_head_host(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host: dict, out_dev: dict, workspace) -> None:
     """Host-buffer variant: copies h_host (pinned CPU tensor) in, runs the head, copies the outputs to out_host."""
     W = _bf16(W)
