@@ -164,13 +164,19 @@ class Workload:
         self.run_heads()
         self.run_tail()
 
+    def check(self):
+        """Synchronises and raises if a bounded device-side wait gave up (results would be meaningless)."""
+        code = self.ee.ee_query_async_error(self.ws)
+        if code != 0:
+            raise RuntimeError(f"device-side wait timed out in workload {self.name} (ee_status {code})")
+
 
 def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSampler | None = None) -> dict:
     """Times `steps` steps with CUDA events on the launching stream; also the head calls alone inside them."""
     torch = wl.torch
     for _ in range(warmup):
         wl.step()
-    torch.cuda.synchronize()
+    wl.check()
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
@@ -190,6 +196,7 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
         dist.barrier()
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
+    wl.check()
     total_ms = t0.elapsed_time(t1)
     if dist is not None:
         t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")

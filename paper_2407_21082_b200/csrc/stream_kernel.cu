@@ -1,24 +1,29 @@
 // Decode-sized exit head: one launch does LayerNorm, the V x d projection and the softmax statistics.
 //
-// The kernel is bound by the single read of W from HBM.  The vocabulary is split evenly over all warps
-// of the grid; a warp streams its rows with 128-bit loads that land directly in mma.sync A-fragment
-// layout (the K permutation this implies is applied to the activations as well, which is legal because
-// a dot product does not care about the order of its terms).  The M <= 32 normalised rows live in shared
-// memory as bf16 and serve as the B operand.  Each thread folds the logits it owns into an online
-// (max, sum exp, sum exp*(z-max), argmax) state; states merge by warp shuffles, through shared memory
-// across warps, and the last CTA to finish (atomic ticket, no spinning) merges the per-CTA partials and
-// writes argmax / entropy / max-prob / exit mask.
+// The kernel is bound by the single read of W from HBM, so W is read the way HBM likes it: every CTA owns
+// one contiguous range of vocabulary rows and walks it front to back with bulk asynchronous copies
+// (cp.async.bulk, one per row segment of up to 2 KB, 16 rows per stage) into a shared-memory ring guarded
+// by mbarriers.  A producer warp keeps the ring full; eight consumer warps take the stages in turn.  A
+// consumer reads its 16 x 32 sub-blocks of W straight into mma.sync m16n8k16 A-fragments (the K permutation
+// this implies is applied to the activations too, which a dot product does not notice) and multiplies them
+// with the M <= 32 LayerNorm'ed rows that sit in shared memory as bf16.  Each thread folds the logits it
+// owns into an online (max, sum exp, sum exp*(z-max), argmax) state; states merge by warp shuffles, through
+// shared memory across warps, and the last CTA to finish (atomic ticket, no spinning) merges the per-CTA
+// partials and writes argmax / entropy / max-prob / exit mask.
 #include "common.cuh"
 #include "kernels.h"
+#include "sm100_ptx.cuh"
 
 namespace ee {
 
 namespace {
 
-constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
-constexpr int kDepth = 4;                  // k-chunks of W in flight per thread (2 x 16 B each)
-constexpr size_t kSmemBudget = 200 * 1024;
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
+constexpr int kStageRows = 16;                        // one m16 row group per stage
+constexpr int kSegMax = 1024;                         // columns of W per stage (2 KB per row)
+constexpr int kMaxStages = 12;
+constexpr size_t kSmemBudget = 216 * 1024;
 
 struct StreamParams {
     const __nv_bfloat16* h;
@@ -37,6 +42,12 @@ struct StreamParams {
     State* partials;                       // [gridDim.x][8 * NT]
     Control* ctrl;
     int y_stride;                          // bf16 elements between rows of y in shared memory
+    int seg_cols;                          // columns of W per stage (multiple of 64)
+    int n_segs;                            // stages per 16-row group = ceil(d / seg_cols)
+    int stage_row_bytes;                   // bytes between rows of a stage: 2 * seg_cols + 64
+    int n_stages;                          // ring slots in total = n_consumers * slots_per_warp
+    int n_consumers;                       // consumer warps that take row groups (<= kConsumerWarps)
+    int slots_per_warp;                    // each consumer warp owns this many ring slots
 };
 
 // Row stride (in bf16 elements) of y in shared memory: d rounded up to the 32-wide k-chunk, padded so
@@ -55,14 +66,23 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// LayerNorm of the slab's rows into shared memory (bf16), one warp per row.  Rows >= M and the k padding
-// are zero-filled so that they contribute nothing and stay finite.
-__device__ void layer_norm_to_smem(const StreamParams& p, __nv_bfloat16* y_s, int m_pad) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void consumer_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
+// LayerNorm of the slab's rows into shared memory (bf16), one consumer warp per row.  Rows >= M and the k
+// padding are zero-filled so that they contribute nothing and stay finite.
+__device__ void layer_norm_to_smem(const StreamParams& p, __nv_bfloat16* y_s, int m_pad, int warp, int lane) {
     const int nvec = p.d >> 3;                                   // 16-byte vectors per row
     const int svec = p.y_stride >> 3;
     const float inv_d = 1.f / (float)p.d;
-    for (int r = warp; r < m_pad; r += kWarps) {
+    for (int r = warp; r < m_pad; r += kConsumerWarps) {
         uint4* yrow = reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride);
         if (r >= p.M) {
             for (int c = lane; c < svec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
@@ -87,111 +107,195 @@ __device__ void layer_norm_to_smem(const StreamParams& p, __nv_bfloat16* y_s, in
 template <int NT>
 __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const StreamParams p) {
     constexpr int MPAD = 8 * NT;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    __nv_bfloat16* y_s = reinterpret_cast<__nv_bfloat16*>(smem_raw);
-    State* wpart = reinterpret_cast<State*>(smem_raw + (size_t)MPAD * p.y_stride * sizeof(__nv_bfloat16));
+    constexpr int CH = (NT >= 4) ? 1 : 4 / NT;                    // independent accumulator chains per n-tile
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // layout: ring stages | y | per-warp partial states | barriers
+    const int stage_bytes = kStageRows * p.stage_row_bytes;
+    unsigned char* ring = smem_raw;
+    __nv_bfloat16* y_s = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_stages * stage_bytes);
+    State* wpart = reinterpret_cast<State*>(reinterpret_cast<unsigned char*>(y_s) +
+                                            (size_t)MPAD * p.y_stride * sizeof(__nv_bfloat16));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + kConsumerWarps * MPAD);
     __shared__ int s_is_last;
+    __shared__ int s_abort;
+    const uint32_t bar_base = ptx::smem_addr(bars);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (p.n_stages + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, t = lane & 3;
 
-    // This warp's slice of the vocabulary.
-    const long long nw = (long long)gridDim.x * kWarps;
-    const long long gw = (long long)blockIdx.x * kWarps + warp;
-    const int r_begin = (int)(((long long)p.V * gw) / nw);
-    const int r_end = (int)(((long long)p.V * (gw + 1)) / nw);
-    const int ngroups = (r_end - r_begin + 15) >> 4;
-    const int nchunks = (p.d + 31) >> 5;
-    const int total = ngroups * nchunks;
-
-    // Prefetch cursor (group, chunk) and the loader.
-    int pg = 0, pc = 0;
-    auto load_next = [&](uint4& lo, uint4& hi) {
-        lo = make_uint4(0, 0, 0, 0);
-        hi = make_uint4(0, 0, 0, 0);
-        if (pg < ngroups) {
-            const int k = pc * 32 + t * 8;
-            const int row0 = r_begin + pg * 16 + g;
-            if (k < p.d) {
-                if (row0 < r_end) lo = ld_stream_v4(p.W + (size_t)row0 * p.d + k);
-                if (row0 + 8 < r_end) hi = ld_stream_v4(p.W + (size_t)(row0 + 8) * p.d + k);
-            }
-            if (++pc == nchunks) { pc = 0; ++pg; }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.n_stages; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
         }
-    };
-
-    uint4 lo[kDepth], hi[kDepth];
-#pragma unroll
-    for (int u = 0; u < kDepth; ++u) load_next(lo[u], hi[u]);     // W is in flight while LayerNorm runs
-
-    layer_norm_to_smem(p, y_s, MPAD);
+        s_abort = 0;
+        ptx::fence_mbar_init();
+    }
     __syncthreads();
 
-    float acc[NT][4];
+    // This CTA's contiguous slice of the vocabulary, in 16-row groups.
+    const int r_begin = (int)(((long long)p.V * blockIdx.x) / gridDim.x);
+    const int r_end = (int)(((long long)p.V * (blockIdx.x + 1)) / gridDim.x);
+    const int ngroups = (r_end - r_begin + kStageRows - 1) / kStageRows;
+    const int total_stages = ngroups * p.n_segs;
+    const uint32_t ring_addr = ptx::smem_addr(ring);
+
     State st[NT][2];
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
-        acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
         st[n][0] = state_empty();
         st[n][1] = state_empty();
     }
 
-    // y for n-tile n, row g, elements [cc*32 + t*8, +8): one 16-byte vector.
-    const uint4* y_lane = reinterpret_cast<const uint4*>(y_s + (size_t)g * p.y_stride + t * 8);
-    const int y_tile_vecs = p.y_stride;                           // 8 rows * y_stride elements / 8 per vector
-    int cg = 0, cc = 0;
-    for (int it = 0; it < total; it += kDepth) {
-#pragma unroll
-        for (int u = 0; u < kDepth; ++u) {
-            if (it + u < total) {
-                const uint4 a_lo = lo[u], a_hi = hi[u];
-                load_next(lo[u], hi[u]);
-#pragma unroll
-                for (int n = 0; n < NT; ++n) {
-                    const uint4 yv = y_lane[(size_t)n * y_tile_vecs + cc * 4];
-                    mma_bf16_16816(acc[n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, yv.x, yv.y);
-                    mma_bf16_16816(acc[n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, yv.z, yv.w);
-                }
-                if (++cc == nchunks) {
-                    // The 16 x MPAD logits of this row group are complete.
-                    const int rowA = r_begin + cg * 16 + g, rowB = rowA + 8;
-#pragma unroll
-                    for (int n = 0; n < NT; ++n) {
-                        if (rowA < r_end) {
-                            state_push(st[n][0], acc[n][0], rowA);
-                            state_push(st[n][1], acc[n][1], rowA);
-                        }
-                        if (rowB < r_end) {
-                            state_push(st[n][0], acc[n][2], rowB);
-                            state_push(st[n][1], acc[n][3], rowB);
-                        }
-                        acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-                    }
-                    cc = 0;
-                    ++cg;
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer warp
+        // Lane r copies row r of the stage; lane 0 first announces the stage's byte count.
+        // Row group grp belongs to consumer warp grp % n_consumers, which owns a private ring of
+        // slots_per_warp slots and uses them in the order its stages arrive.  A slot therefore has one
+        // producer and one consumer that both see every phase of its barriers, so parity waits are exact.
+        int armed = 0;                                            // stages armed so far (for the abort drain)
+        for (int i = 0; i < total_stages; ++i) {
+            const int grp = i / p.n_segs, seg = i - grp * p.n_segs;
+            const int cw = grp % p.n_consumers;
+            const int j = (grp / p.n_consumers) * p.n_segs + seg; // index of this stage in cw's private sequence
+            const int slot = cw * p.slots_per_warp + j % p.slots_per_warp;
+            const uint32_t phase = (uint32_t)(j / p.slots_per_warp) & 1u;
+            const int row0 = r_begin + grp * kStageRows;
+            const int nrows = min(kStageRows, r_end - row0);
+            const int k0 = seg * p.seg_cols;
+            const uint32_t seg_bytes = (uint32_t)(min(p.seg_cols, p.d - k0) * 2);
+            bool ok = true;
+            if (lane == 0) {
+                ok = ptx::mbar_wait(empty_bar(slot), phase ^ 1u, &s_abort);
+                if (ok) ptx::mbar_arrive_expect_tx(full_bar(slot), seg_bytes * nrows);
+                else {
+                    if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
+                        p.ctrl->error_info = (1u << 24) | ((unsigned)slot << 16) | ((unsigned)i & 0xffffu);
+                    s_abort = 1;
                 }
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            if (lane < nrows)
+                bulk_copy_g2s(ring_addr + slot * stage_bytes + lane * p.stage_row_bytes,
+                              p.W + (size_t)(row0 + lane) * p.d + k0, seg_bytes, full_bar(slot));
+            ++armed;
         }
-    }
+        if (s_abort && lane == 0) {
+            // Let copies that are still in flight land before the CTA gives its shared memory back: re-derive
+            // the slot and phase of every stage armed in the last round of each slot and wait (bounded) for it.
+            for (int i = max(0, armed - p.n_stages * p.n_segs * 2); i < armed; ++i) {
+                const int grp = i / p.n_segs, seg = i - grp * p.n_segs;
+                const int cw = grp % p.n_consumers;
+                const int j = (grp / p.n_consumers) * p.n_segs + seg;
+                const int slot = cw * p.slots_per_warp + j % p.slots_per_warp;
+                const uint32_t par = (uint32_t)(j / p.slots_per_warp) & 1u;
+                for (uint32_t n = 0; n < (1u << 12) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        layer_norm_to_smem(p, y_s, MPAD, warp, lane);
+        consumer_barrier();
 
-    // Merge over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then own tokens 2t, 2t+1.
+        const int g = lane >> 2, t = lane & 3;
+        const uint4* y_lane = reinterpret_cast<const uint4*>(y_s + (size_t)g * p.y_stride + t * 8);
+        const int y_tile_vecs = p.y_stride;                       // 8 rows * y_stride elements / 8 per vector
+        const bool k_ragged = (p.d & 31) != 0;
+        bool ok = true;
+        int j = 0;                                                // this warp's private stage counter
+        for (int grp = warp; ok && warp < p.n_consumers && grp < ngroups; grp += p.n_consumers) {
+            float acc[NT][CH][4];
 #pragma unroll
-    for (int n = 0; n < NT; ++n)
+            for (int n = 0; n < NT; ++n)
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
+                for (int u = 0; u < CH; ++u) acc[n][u][0] = acc[n][u][1] = acc[n][u][2] = acc[n][u][3] = 0.f;
+
+            for (int seg = 0; seg < p.n_segs; ++seg, ++j) {
+                const int i = grp * p.n_segs + seg;
+                const int slot = warp * p.slots_per_warp + j % p.slots_per_warp;
+                const uint32_t phase = (uint32_t)(j / p.slots_per_warp) & 1u;
+                const bool landed = ptx::mbar_wait(full_bar(slot), phase, &s_abort);
+                if (!__all_sync(0xffffffffu, landed)) {
+                    if (lane == 0) {
+                        if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
+                            p.ctrl->error_info = (2u << 24) | ((unsigned)slot << 16) | ((unsigned)i & 0xffffu);
+                        s_abort = 1;
+                    }
+                    ok = false;
+                    break;
+                }
+                const int k0 = seg * p.seg_cols;
+                const int nch = (min(p.seg_cols, p.d - k0) + 31) >> 5;
+                const unsigned char* a_lo = ring + (size_t)slot * stage_bytes + g * p.stage_row_bytes + t * 16;
+                const unsigned char* a_hi = a_lo + 8 * p.stage_row_bytes;
+                const uint4* yk = y_lane + (k0 >> 3);
+                for (int c0 = 0; c0 < nch; c0 += CH) {
 #pragma unroll
-            for (int msk = 4; msk <= 16; msk <<= 1) {
-                const State o = state_shfl_xor(st[n][e], msk);
-                state_merge(st[n][e], o);
+                    for (int u = 0; u < CH; ++u) {
+                        const int c = c0 + u;
+                        if (c < nch) {
+                            uint4 lo = *reinterpret_cast<const uint4*>(a_lo + c * 64);
+                            uint4 hi = *reinterpret_cast<const uint4*>(a_hi + c * 64);
+                            if (k_ragged && k0 + c * 32 + t * 8 >= p.d) {      // beyond d: whatever the ring holds
+                                lo = make_uint4(0, 0, 0, 0);
+                                hi = make_uint4(0, 0, 0, 0);
+                            }
+#pragma unroll
+                            for (int n = 0; n < NT; ++n) {
+                                const uint4 yv = yk[(size_t)n * y_tile_vecs + c * 4];
+                                mma_bf16_16816(acc[n][u], lo.x, hi.x, lo.y, hi.y, yv.x, yv.y);
+                                mma_bf16_16816(acc[n][u], lo.z, hi.z, lo.w, hi.w, yv.z, yv.w);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(empty_bar(slot));  // the stage may be refilled
             }
-            if (g == 0) wpart[warp * MPAD + n * 8 + t * 2 + e] = st[n][e];
+            if (!ok) break;
+            // The 16 x MPAD logits of this row group are complete.
+            const int rowA = r_begin + grp * kStageRows + g, rowB = rowA + 8;
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                float z[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    z[q] = acc[n][0][q];
+#pragma unroll
+                    for (int u = 1; u < CH; ++u) z[q] += acc[n][u][q];
+                }
+                if (rowA < r_end) {
+                    state_push(st[n][0], z[0], rowA);
+                    state_push(st[n][1], z[1], rowA);
+                }
+                if (rowB < r_end) {
+                    state_push(st[n][0], z[2], rowB);
+                    state_push(st[n][1], z[3], rowB);
+                }
+            }
         }
+
+        // Merge over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then own tokens 2t, 2t+1.
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+#pragma unroll
+                for (int msk = 4; msk <= 16; msk <<= 1) {
+                    const State o = state_shfl_xor(st[n][e], msk);
+                    state_merge(st[n][e], o);
+                }
+                if (g == 0) wpart[warp * MPAD + n * 8 + t * 2 + e] = st[n][e];
+            }
+    }
     __syncthreads();
 
-    // Merge over the CTA's warps in vocabulary order; publish the CTA partial.
+    // Merge over the CTA's consumer warps; publish the CTA partial.
     if (threadIdx.x < MPAD) {
         State a = wpart[threadIdx.x];
-        for (int w = 1; w < kWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
+        for (int w = 1; w < kConsumerWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
         p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = a;
         __threadfence();
     }
@@ -205,7 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
 
     // Last CTA: merge the partials of all CTAs, one warp per token, and decide.
     __threadfence();
-    for (int tok = warp; tok < p.M; tok += kWarps) {
+    for (int tok = warp; tok < p.M; tok += kThreads / 32) {
         State a = state_empty();
         for (int b = lane; b < (int)gridDim.x; b += 32) {
             const State o = state_load_cg(p.partials + (size_t)b * MPAD + tok);
@@ -224,13 +328,59 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     if (threadIdx.x == 0) p.ctrl->ticket = 0;                     // ready for the next call
 }
 
-size_t stream_smem_bytes(int d, int nt) {
-    return (size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) + (size_t)kWarps * 8 * nt * sizeof(State);
+// ---------------------------------------------------------------------------------------------
+// Host side: shared-memory plan and launch
+// ---------------------------------------------------------------------------------------------
+struct SmemPlan {
+    int seg_cols, n_segs, stage_row_bytes, n_stages, n_consumers, slots_per_warp;
+    size_t bytes;
+};
+
+// Ring geometry for hidden size d with 8*nt rows of y resident; n_stages = 0 if it does not fit.
+// Stages hold up to 1024 columns (2 KB per row); narrower stages are chosen when y leaves little room,
+// so that at least four stages are in flight.
+SmemPlan plan_smem(int d, int nt) {
+    SmemPlan best;
+    best.n_stages = 0;
+    best.bytes = 0;
+    const int d64 = (d + 63) / 64 * 64;
+    const size_t fixed = (size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
+                         (size_t)kConsumerWarps * 8 * nt * sizeof(State) + 2 * kMaxStages * sizeof(uint64_t);
+    const long long room = (long long)kSmemBudget - (long long)fixed;
+    for (int seg = kSegMax; seg >= 256; seg >>= 1) {
+        SmemPlan s;
+        s.seg_cols = d64 < seg ? d64 : seg;
+        s.n_segs = (d + s.seg_cols - 1) / s.seg_cols;
+        s.stage_row_bytes = 2 * s.seg_cols + 64;
+        const long long stage = (long long)kStageRows * s.stage_row_bytes;
+        long long n = room > 0 ? room / stage : 0;
+        if (n > kMaxStages) n = kMaxStages;
+        // Split the slots into private rings: n_consumers warps x slots_per_warp, as many slots as fit.
+        s.n_consumers = 0;
+        s.slots_per_warp = 0;
+        for (int c = kConsumerWarps; c >= 1; --c) {
+            if (c < 4 && c < n) continue;                       // keep at least four warps busy when slots allow
+            const int b = (int)(n / c);
+            if (b >= 1 && c * b > s.n_consumers * s.slots_per_warp) { s.n_consumers = c; s.slots_per_warp = b; }
+        }
+        s.n_stages = s.n_consumers * s.slots_per_warp;
+        s.bytes = fixed + (size_t)s.n_stages * (size_t)stage;
+        if (s.n_stages >= 4 || (seg == 256 && s.n_stages >= 2)) return s;
+        if (d64 <= seg / 2) break;          // a narrower cap would not change the stage
+    }
+    return best;
 }
 
 template <int NT>
-ee_status launch_one(const StreamParams& p, int grid, int device, cudaStream_t stream) {
-    const size_t smem = stream_smem_bytes(p.d, NT);
+ee_status launch_one(StreamParams& p, int grid, int device, cudaStream_t stream) {
+    const SmemPlan plan = plan_smem(p.d, NT);
+    if (plan.n_stages == 0) return EE_ERR_SHAPE;
+    p.seg_cols = plan.seg_cols;
+    p.n_segs = plan.n_segs;
+    p.stage_row_bytes = plan.stage_row_bytes;
+    p.n_stages = plan.n_stages;
+    p.n_consumers = plan.n_consumers;
+    p.slots_per_warp = plan.slots_per_warp;
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
         if (cudaFuncSetAttribute(exit_head_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -238,7 +388,7 @@ ee_status launch_one(const StreamParams& p, int grid, int device, cudaStream_t s
             return EE_ERR_CUDA;
         configured[device] = true;
     }
-    exit_head_stream_kernel<NT><<<grid, kThreads, smem, stream>>>(p);
+    exit_head_stream_kernel<NT><<<grid, kThreads, plan.bytes, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
@@ -246,7 +396,7 @@ ee_status launch_one(const StreamParams& p, int grid, int device, cudaStream_t s
 
 int stream_slab_rows(int d) {
     for (int nt = kStreamMaxRows / 8; nt >= 1; nt >>= 1)
-        if (stream_smem_bytes(d, nt) <= kSmemBudget) return 8 * nt;
+        if (plan_smem(d, nt).n_stages > 0) return 8 * nt;
     return 0;
 }
 
