@@ -77,12 +77,7 @@ def new_outputs(M: int, device="cuda") -> dict:
                 exit_mask=torch.empty(M, dtype=torch.uint8, device=device))
 
 
-def ee_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> dict:
-    """LayerNorm + exit-head projection + entropy / argmax / max-prob + exit decision for the rows of h.
-
-    tau is a float (nats) or a float32 CUDA tensor [M] of per-row thresholds.  `out` (see new_outputs) and
-    `workspace` (see new_workspace) are allocated when not given.
-    """
+def _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path):
     h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
     M, d = h.shape
     V = W.shape[0]
@@ -91,11 +86,48 @@ def ee_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, pa
     out = out if out is not None else new_outputs(M, h.device)
     workspace = workspace if workspace is not None else new_workspace(M, d, V, h.device)
     tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
-    _check(_lib.load().ee_exit_head_path(
-        _ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W),
-        M, d, V, _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
-        _ptr(out["exit_mask"]), _ptr(workspace), workspace.numel(), _stream(), int(path)), "ee_exit_head")
+    args = (_ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W),
+            M, d, V, _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
+            _ptr(out["exit_mask"]), _ptr(workspace), workspace.numel(), _stream(), int(path))
+    return args, out, (h, gamma, beta, W, tau_t, out, workspace)
+
+
+def ee_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> dict:
+    """LayerNorm + exit-head projection + entropy / argmax / max-prob + exit decision for the rows of h.
+
+    tau is a float (nats) or a float32 CUDA tensor [M] of per-row thresholds.  `out` (see new_outputs) and
+    `workspace` (see new_workspace) are allocated when not given.
+    """
+    args, out, _ = _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path)
+    _check(_lib.load().ee_exit_head_path(*args), "ee_exit_head")
     return out
+
+
+class PreparedCall:
+    """A C-ABI call with its arguments marshalled once, for loops that repeat the same call.
+
+    Holds references to the tensors so that their memory stays alive; the stream is the one that was current
+    at preparation time.  Calling it launches and returns, like the function it wraps.
+    """
+    __slots__ = ("_fn", "_args", "_where", "_keep", "out")
+
+    def __init__(self, fn, args, where, keep, out):
+        import ctypes as C
+        self._fn = fn
+        self._args = tuple(C.c_void_p(a) if (t is C.c_void_p) else t(a) for a, t in zip(args, fn.argtypes))
+        self._where, self._keep, self.out = where, keep, out
+
+    def __call__(self):
+        code = self._fn(*self._args)
+        if code:
+            raise EExitError(code, self._where)
+        return self.out
+
+
+def prepare_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> PreparedCall:
+    """ee_exit_head with the arguments marshalled once; see PreparedCall."""
+    args, out, keep = _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path)
+    return PreparedCall(_lib.load().ee_exit_head_path, args, "ee_exit_head", keep, out)
 
 
 EE_STATIC_MAX_ROWS = 32
@@ -117,20 +149,41 @@ def ee_exit_head_static(h, gamma, beta, ln_eps, W, tau, *, out: dict) -> dict:
     return out
 
 
-def ee_exit_head_host(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host: dict, out_dev: dict, workspace) -> None:
-    """Host-buffer variant: copies h_host (pinned CPU tensor) in, runs the head, copies the outputs to out_host."""
+def _exit_head_host_args(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host, out_dev, workspace):
     W = _bf16(W)
     M, d = h_host.shape
     tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
-    _check(_lib.load().ee_exit_head_host(
-        _ptr(h_host), _ptr(h_dev), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W), M, d, W.shape[0], _ptr(tau_t), tau_f,
-        _ptr(out_host["argmax"]), _ptr(out_host["entropy"]), _ptr(out_host["maxprob"]), _ptr(out_host["exit_mask"]),
-        _ptr(out_dev["argmax"]), _ptr(out_dev["entropy"]), _ptr(out_dev["maxprob"]), _ptr(out_dev["exit_mask"]),
-        _ptr(workspace), workspace.numel(), _stream()), "ee_exit_head_host")
+    args = (_ptr(h_host), _ptr(h_dev), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W), M, d, W.shape[0], _ptr(tau_t), tau_f,
+            _ptr(out_host["argmax"]), _ptr(out_host["entropy"]), _ptr(out_host["maxprob"]), _ptr(out_host["exit_mask"]),
+            _ptr(out_dev["argmax"]), _ptr(out_dev["entropy"]), _ptr(out_dev["maxprob"]), _ptr(out_dev["exit_mask"]),
+            _ptr(workspace), workspace.numel(), _stream())
+    return args, (h_host, h_dev, gamma, beta, W, tau_t, out_host, out_dev, workspace)
+
+
+def ee_exit_head_host(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host: dict, out_dev: dict, workspace) -> None:
+    """Host-buffer variant: copies h_host (pinned CPU tensor) in, runs the head, copies the outputs to out_host."""
+    args, _ = _exit_head_host_args(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host, out_dev, workspace)
+    _check(_lib.load().ee_exit_head_host(*args), "ee_exit_head_host")
+
+
+def prepare_exit_head_host(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host, out_dev, workspace) -> PreparedCall:
+    args, keep = _exit_head_host_args(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host, out_dev, workspace)
+    return PreparedCall(_lib.load().ee_exit_head_host, args, "ee_exit_head_host", keep, out_host)
 
 
 def ee_compact(exit_mask, h=None, *, gather=True, out=None) -> dict:
     """Indices (ascending) and count of the rows with exit_mask == 0, and a dense copy of their rows of h."""
+    args, out, _ = _compact_args(exit_mask, h, gather, out)
+    _check(_lib.load().ee_compact(*args), "ee_compact")
+    return out
+
+
+def prepare_compact(exit_mask, h=None, *, gather=True, out=None) -> PreparedCall:
+    args, out, keep = _compact_args(exit_mask, h, gather, out)
+    return PreparedCall(_lib.load().ee_compact, args, "ee_compact", keep, out)
+
+
+def _compact_args(exit_mask, h, gather, out):
     M = exit_mask.numel()
     dev = exit_mask.device
     gather = gather and h is not None
@@ -143,14 +196,24 @@ def ee_compact(exit_mask, h=None, *, gather=True, out=None) -> dict:
         if gather:
             out["h_out"] = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
     ld = (h.stride(0) if M > 1 else max(h.stride(0), d)) if gather else 0
-    _check(_lib.load().ee_compact(_ptr(exit_mask), _ptr(h) if gather else None, ld, M, d, _ptr(out["kept_idx"]),
-                                  _ptr(out["kept_count"]), _ptr(out.get("h_out")) if gather else None, _stream()),
-           "ee_compact")
-    return out
+    args = (_ptr(exit_mask), _ptr(h) if gather else None, ld, M, d, _ptr(out["kept_idx"]),
+            _ptr(out["kept_count"]), _ptr(out.get("h_out")) if gather else None, _stream())
+    return args, out, (exit_mask, h, out)
 
 
 def dssd_accept(draft_tok, draft_exit_mask, verify_tok, *, out=None) -> dict:
     """Draft length, accepted prefix length and next token per sequence (see include/eexit.h)."""
+    args, out, _ = _accept_args(draft_tok, draft_exit_mask, verify_tok, out)
+    _check(_lib.load().dssd_accept(*args), "dssd_accept")
+    return out
+
+
+def prepare_accept(draft_tok, draft_exit_mask, verify_tok, *, out=None) -> PreparedCall:
+    args, out, keep = _accept_args(draft_tok, draft_exit_mask, verify_tok, out)
+    return PreparedCall(_lib.load().dssd_accept, args, "dssd_accept", keep, out)
+
+
+def _accept_args(draft_tok, draft_exit_mask, verify_tok, out):
     S, k = draft_tok.shape
     kv = verify_tok.shape[1]
     dev = draft_tok.device
@@ -158,10 +221,9 @@ def dssd_accept(draft_tok, draft_exit_mask, verify_tok, *, out=None) -> dict:
         raise ValueError("token arrays must be contiguous")
     if out is None:
         out = {n: torch.empty(S, dtype=torch.int32, device=dev) for n in ("draft_len", "accept_len", "next_tok")}
-    _check(_lib.load().dssd_accept(_ptr(draft_tok), _ptr(draft_exit_mask), _ptr(verify_tok), S, k, kv,
-                                   _ptr(out["draft_len"]), _ptr(out["accept_len"]), _ptr(out["next_tok"]), _stream()),
-           "dssd_accept")
-    return out
+    args = (_ptr(draft_tok), _ptr(draft_exit_mask), _ptr(verify_tok), S, k, kv,
+            _ptr(out["draft_len"]), _ptr(out["accept_len"]), _ptr(out["next_tok"]), _stream())
+    return args, out, (draft_tok, draft_exit_mask, verify_tok, out)
 
 
 def ee_query_async_error(workspace) -> int:
