@@ -137,19 +137,25 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // LayerNorm of eight consecutive elements (one 16-byte vector of bf16) -> eight bf16, given the row's
-// mean and reciprocal standard deviation.  c is the vector index within the row.
-__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, const float* gamma,
-                                                 const float* beta, int c) {
-    const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
-    const float4 g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
-    const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
-    const float4 b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+// mean and reciprocal standard deviation and the eight gammas / betas of these columns.
+__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, float4 g0, float4 g1, float4 b0,
+                                                 float4 b1) {
     uint4 o;
     o.x = pack_bf16(fmaf((bf16_lo(v.x) - mu) * rstd, g0.x, b0.x), fmaf((bf16_hi(v.x) - mu) * rstd, g0.y, b0.y));
     o.y = pack_bf16(fmaf((bf16_lo(v.y) - mu) * rstd, g0.z, b0.z), fmaf((bf16_hi(v.y) - mu) * rstd, g0.w, b0.w));
     o.z = pack_bf16(fmaf((bf16_lo(v.z) - mu) * rstd, g1.x, b1.x), fmaf((bf16_hi(v.z) - mu) * rstd, g1.y, b1.y));
     o.w = pack_bf16(fmaf((bf16_lo(v.w) - mu) * rstd, g1.z, b1.z), fmaf((bf16_hi(v.w) - mu) * rstd, g1.w, b1.w));
     return o;
+}
+
+// Same, reading gamma and beta of vector c (columns 8c .. 8c+7) from global memory.
+__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, const float* gamma,
+                                                 const float* beta, int c) {
+    const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+    const float4 g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+    const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+    const float4 b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+    return layer_norm_vec8(v, mu, rstd, g0, g1, b0, b1);
 }
 
 __device__ __forceinline__ float vec8_sum(uint4 v) {

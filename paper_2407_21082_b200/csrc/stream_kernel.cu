@@ -1,15 +1,17 @@
 // Decode-sized exit head: one launch does LayerNorm, the V x d projection and the softmax statistics.
 //
 // The kernel is bound by the single read of W from HBM, so W is read the way HBM likes it: every CTA owns
-// one contiguous range of vocabulary rows and walks it front to back with bulk asynchronous copies
-// (cp.async.bulk, one per row segment of up to 2 KB, 16 rows per stage) into a shared-memory ring guarded
-// by mbarriers.  A producer warp keeps the ring full; eight consumer warps take the stages in turn.  A
-// consumer reads its 16 x 32 sub-blocks of W straight into mma.sync m16n8k16 A-fragments (the K permutation
-// this implies is applied to the activations too, which a dot product does not notice) and multiplies them
-// with the M <= 32 LayerNorm'ed rows that sit in shared memory as bf16.  Each thread folds the logits it
-// owns into an online (max, sum exp, sum exp*(z-max), argmax) state; states merge by warp shuffles, through
-// shared memory across warps, and the last CTA to finish (atomic ticket, no spinning) merges the per-CTA
-// partials and writes argmax / entropy / max-prob / exit mask.
+// one contiguous range of vocabulary rows and walks it front to back in 16-row stages that are fetched by
+// bulk asynchronous copies (cp.async.bulk) into a shared-memory ring guarded by mbarriers.  For rows of up
+// to 2 KB a stage is one contiguous 16-row block fetched by a single copy; wider rows are cut into column
+// segments fetched row by row.  Every worker warp owns a private set of ring slots and a share of the row
+// groups: it issues the copies for its own stages, waits for them, consumes them and re-arms the slot, so no
+// barrier is shared between warps.  A worker reads its 16 x 32 sub-blocks of W straight into mma.sync
+// m16n8k16 A-fragments (the K permutation this implies is applied to the activations too, which a dot
+// product does not notice) and multiplies them with the M <= 32 LayerNorm'ed rows that sit in shared memory
+// as bf16.  Each thread folds the logits it owns into an online (max, sum exp, sum exp*(z-max), argmax)
+// state; states merge by warp shuffles, through shared memory across warps, and the last CTA to finish
+// (atomic ticket, no spinning) merges the per-CTA partials and writes argmax / entropy / max-prob / exit mask.
 #include "common.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -18,12 +20,12 @@ namespace ee {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
 constexpr int kStageRows = 16;                        // one m16 row group per stage
 constexpr int kSegMax = 1024;                         // columns of W per stage (2 KB per row)
-constexpr int kMaxStages = 12;
-constexpr size_t kSmemBudget = 216 * 1024;
+constexpr int kMaxStages = 32;
+constexpr size_t kSmemBudget = 226 * 1024;
 
 struct StreamParams {
     const __nv_bfloat16* h;
@@ -42,12 +44,13 @@ struct StreamParams {
     State* partials;                       // [gridDim.x][8 * NT]
     Control* ctrl;
     int y_stride;                          // bf16 elements between rows of y in shared memory
-    int seg_cols;                          // columns of W per stage (multiple of 64)
+    int seg_cols;                          // columns of W per stage
     int n_segs;                            // stages per 16-row group = ceil(d / seg_cols)
-    int stage_row_bytes;                   // bytes between rows of a stage: 2 * seg_cols + 64
-    int n_stages;                          // ring slots in total = n_consumers * slots_per_warp
-    int n_consumers;                       // consumer warps that take row groups (<= kConsumerWarps)
-    int slots_per_warp;                    // each consumer warp owns this many ring slots
+    int stage_row_bytes;                   // bytes between rows of a stage
+    int n_stages;                          // ring slots in total = n_workers * slots_per_warp
+    int n_workers;                         // warps that take row groups (<= kWarps)
+    int slots_per_warp;                    // each worker owns this many ring slots
+    int contiguous;                        // 1: a stage is 16 whole rows fetched by one copy (rows unpadded)
 };
 
 // Row stride (in bf16 elements) of y in shared memory: d rounded up to the 32-wide k-chunk, padded so
@@ -72,35 +75,66 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
                  : "memory");
 }
 
-__device__ __forceinline__ void consumer_barrier() {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+// Programmatic dependent launch: the next kernel in the stream may start its preamble once every CTA of this
+// one has passed launch_dependents(); a kernel must call grid_dependency_wait() before it touches anything an
+// earlier kernel in the stream produces (here: h, the workspace and the outputs -- not the weights).
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void cp_async_16(void* dst_smem, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_addr(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
-// LayerNorm of the slab's rows into shared memory (bf16), one consumer warp per row.  Rows >= M and the k
-// padding are zero-filled so that they contribute nothing and stay finite.
-__device__ void layer_norm_to_smem(const StreamParams& p, __nv_bfloat16* y_s, int m_pad, int warp, int lane) {
+// Starts the asynchronous copies of everything LayerNorm reads -- the slab's rows of h (into their rows of
+// y), gamma and beta -- 16 bytes per thread and step.
+__device__ void stage_layer_norm_inputs(const StreamParams& p, __nv_bfloat16* y_s, float* gamma_s, float* beta_s) {
+    const int nvec = p.d >> 3;
+    for (int i = threadIdx.x; i < p.M * nvec; i += kThreads) {
+        const int r = i / nvec, c = i - r * nvec;
+        cp_async_16(reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c,
+                    reinterpret_cast<const uint4*>(p.h + (size_t)r * p.ld_h) + c);
+    }
+    for (int i = threadIdx.x; i < (p.d >> 2); i += kThreads) {
+        cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(p.gamma) + i);
+        cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(p.beta) + i);
+    }
+}
+
+// LayerNorm in shared memory: the rows of y hold raw h on entry and the normalised bf16 rows on exit.
+// Warp w owns rows w, w + 8, ...  Rows >= M and the k padding are zero-filled so that they contribute nothing
+// and stay finite.
+template <int NT>
+__device__ void layer_norm_in_smem(const StreamParams& p, __nv_bfloat16* y_s, const float* gamma_s,
+                                   const float* beta_s, int warp, int lane) {
     const int nvec = p.d >> 3;                                   // 16-byte vectors per row
     const int svec = p.y_stride >> 3;
     const float inv_d = 1.f / (float)p.d;
-    for (int r = warp; r < m_pad; r += kConsumerWarps) {
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+        const int r = warp + i * kWarps;
         uint4* yrow = reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride);
         if (r >= p.M) {
             for (int c = lane; c < svec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
             continue;
         }
-        const uint4* hrow = reinterpret_cast<const uint4*>(p.h + (size_t)r * p.ld_h);
         float sum = 0.f;
-        for (int c = lane; c < nvec; c += 32) {
-            const uint4 v = __ldg(hrow + c);
-            yrow[c] = v;
-            sum += vec8_sum(v);
-        }
+        for (int c = lane; c < nvec; c += 32) sum += vec8_sum(yrow[c]);
         const float mu = warp_sum(sum) * inv_d;
         float sq = 0.f;
         for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(yrow[c], mu, sq);
         const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
-        for (int c = lane; c < svec; c += 32)
-            yrow[c] = (c < nvec) ? layer_norm_vec8(yrow[c], mu, rstd, p.gamma, p.beta, c) : make_uint4(0, 0, 0, 0);
+        for (int c = lane; c < svec; c += 32) {
+            if (c < nvec) {
+                const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
+                const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
+                yrow[c] = layer_norm_vec8(yrow[c], mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+            } else {
+                yrow[c] = make_uint4(0, 0, 0, 0);
+            }
+        }
     }
 }
 
@@ -109,26 +143,25 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     constexpr int MPAD = 8 * NT;
     constexpr int CH = (NT >= 4) ? 1 : 4 / NT;                    // independent accumulator chains per n-tile
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // layout: ring stages | y | per-warp partial states | barriers
+    // layout: ring stages | y | per-warp partial states | gamma, beta (fp32) | barriers
     const int stage_bytes = kStageRows * p.stage_row_bytes;
     unsigned char* ring = smem_raw;
     __nv_bfloat16* y_s = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_stages * stage_bytes);
     State* wpart = reinterpret_cast<State*>(reinterpret_cast<unsigned char*>(y_s) +
                                             (size_t)MPAD * p.y_stride * sizeof(__nv_bfloat16));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(wpart + kConsumerWarps * MPAD);
+    float* gamma_s = reinterpret_cast<float*>(wpart + kWarps * MPAD);
+    float* beta_s = gamma_s + p.d;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(beta_s + p.d);
     __shared__ int s_is_last;
     __shared__ int s_abort;
     const uint32_t bar_base = ptx::smem_addr(bars);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (p.n_stages + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.n_stages; ++s) {
-            ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(empty_bar(s), 1);
-        }
+        for (int s = 0; s < p.n_stages; ++s) ptx::mbar_init(full_bar(s), 1);
         s_abort = 0;
         ptx::fence_mbar_init();
     }
@@ -138,7 +171,6 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     const int r_begin = (int)(((long long)p.V * blockIdx.x) / gridDim.x);
     const int r_end = (int)(((long long)p.V * (blockIdx.x + 1)) / gridDim.x);
     const int ngroups = (r_end - r_begin + kStageRows - 1) / kStageRows;
-    const int total_stages = ngroups * p.n_segs;
     const uint32_t ring_addr = ptx::smem_addr(ring);
 
     State st[NT][2];
@@ -148,64 +180,51 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         st[n][1] = state_empty();
     }
 
-    if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------------ producer warp
-        // Lane r copies row r of the stage; lane 0 first announces the stage's byte count.
-        // Row group grp belongs to consumer warp grp % n_consumers, which owns a private ring of
-        // slots_per_warp slots and uses them in the order its stages arrive.  A slot therefore has one
-        // producer and one consumer that both see every phase of its barriers, so parity waits are exact.
-        int armed = 0;                                            // stages armed so far (for the abort drain)
-        for (int i = 0; i < total_stages; ++i) {
-            const int grp = i / p.n_segs, seg = i - grp * p.n_segs;
-            const int cw = grp % p.n_consumers;
-            const int j = (grp / p.n_consumers) * p.n_segs + seg; // index of this stage in cw's private sequence
-            const int slot = cw * p.slots_per_warp + j % p.slots_per_warp;
-            const uint32_t phase = (uint32_t)(j / p.slots_per_warp) & 1u;
-            const int row0 = r_begin + grp * kStageRows;
-            const int nrows = min(kStageRows, r_end - row0);
-            const int k0 = seg * p.seg_cols;
-            const uint32_t seg_bytes = (uint32_t)(min(p.seg_cols, p.d - k0) * 2);
-            bool ok = true;
+    // Row group grp belongs to worker warp grp % n_workers.  The warp's stages, in order, are the column
+    // segments of its groups; stage j of the warp uses its private slot j % slots_per_warp, phase
+    // (j / slots_per_warp) & 1.  One warp arms, waits for, reads and re-arms a slot, so parity waits are exact.
+    const bool worker = warp < p.n_workers;
+    const int my_groups = worker ? (ngroups - warp + p.n_workers - 1) / p.n_workers : 0;
+    const int my_stages = my_groups * p.n_segs;
+    auto issue_stage = [&](int j) {
+        const int grp = warp + (j / p.n_segs) * p.n_workers;
+        const int seg = j % p.n_segs;
+        const int slot = warp * p.slots_per_warp + j % p.slots_per_warp;
+        const int row0 = r_begin + grp * kStageRows;
+        const int nrows = min(kStageRows, r_end - row0);
+        const int k0 = seg * p.seg_cols;
+        const uint32_t seg_bytes = (uint32_t)(min(p.seg_cols, p.d - k0) * 2);
+        if (p.contiguous) {
             if (lane == 0) {
-                ok = ptx::mbar_wait(empty_bar(slot), phase ^ 1u, &s_abort);
-                if (ok) ptx::mbar_arrive_expect_tx(full_bar(slot), seg_bytes * nrows);
-                else {
-                    if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
-                        p.ctrl->error_info = (1u << 24) | ((unsigned)slot << 16) | ((unsigned)i & 0xffffu);
-                    s_abort = 1;
-                }
+                ptx::mbar_arrive_expect_tx(full_bar(slot), seg_bytes * nrows);
+                bulk_copy_g2s(ring_addr + slot * stage_bytes, p.W + (size_t)row0 * p.d, seg_bytes * nrows, full_bar(slot));
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            if (lane < nrows)
-                bulk_copy_g2s(ring_addr + slot * stage_bytes + lane * p.stage_row_bytes,
-                              p.W + (size_t)(row0 + lane) * p.d + k0, seg_bytes, full_bar(slot));
-            ++armed;
+            return;
         }
-        if (s_abort && lane == 0) {
-            // Let copies that are still in flight land before the CTA gives its shared memory back: re-derive
-            // the slot and phase of every stage armed in the last round of each slot and wait (bounded) for it.
-            for (int i = max(0, armed - p.n_stages * p.n_segs * 2); i < armed; ++i) {
-                const int grp = i / p.n_segs, seg = i - grp * p.n_segs;
-                const int cw = grp % p.n_consumers;
-                const int j = (grp / p.n_consumers) * p.n_segs + seg;
-                const int slot = cw * p.slots_per_warp + j % p.slots_per_warp;
-                const uint32_t par = (uint32_t)(j / p.slots_per_warp) & 1u;
-                for (uint32_t n = 0; n < (1u << 12) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ consumer warps
-        layer_norm_to_smem(p, y_s, MPAD, warp, lane);
-        consumer_barrier();
+        if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar(slot), seg_bytes * nrows);
+        __syncwarp();
+        if (lane < nrows)
+            bulk_copy_g2s(ring_addr + slot * stage_bytes + lane * p.stage_row_bytes,
+                          p.W + (size_t)(row0 + lane) * p.d + k0, seg_bytes, full_bar(slot));
+    };
+    int issued = 0;
+    for (; issued < my_stages && issued < p.slots_per_warp; ++issued) issue_stage(issued);   // W is in flight ...
 
+    grid_dependency_wait();                                       // h and the workspace may come from earlier kernels
+    stage_layer_norm_inputs(p, y_s, gamma_s, beta_s);
+    cp_async_wait_all();
+    __syncthreads();
+    layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, warp, lane);  // ... while LayerNorm runs
+    __syncthreads();
+
+    if (worker) {
         const int g = lane >> 2, t = lane & 3;
         const uint4* y_lane = reinterpret_cast<const uint4*>(y_s + (size_t)g * p.y_stride + t * 8);
         const int y_tile_vecs = p.y_stride;                       // 8 rows * y_stride elements / 8 per vector
         const bool k_ragged = (p.d & 31) != 0;
         bool ok = true;
-        int j = 0;                                                // this warp's private stage counter
-        for (int grp = warp; ok && warp < p.n_consumers && grp < ngroups; grp += p.n_consumers) {
+        int j = 0;                                                // this warp's stage counter
+        for (int grp = warp; ok && grp < ngroups; grp += p.n_workers) {
             float acc[NT][CH][4];
 #pragma unroll
             for (int n = 0; n < NT; ++n)
@@ -213,14 +232,13 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
                 for (int u = 0; u < CH; ++u) acc[n][u][0] = acc[n][u][1] = acc[n][u][2] = acc[n][u][3] = 0.f;
 
             for (int seg = 0; seg < p.n_segs; ++seg, ++j) {
-                const int i = grp * p.n_segs + seg;
                 const int slot = warp * p.slots_per_warp + j % p.slots_per_warp;
                 const uint32_t phase = (uint32_t)(j / p.slots_per_warp) & 1u;
                 const bool landed = ptx::mbar_wait(full_bar(slot), phase, &s_abort);
                 if (!__all_sync(0xffffffffu, landed)) {
                     if (lane == 0) {
                         if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
-                            p.ctrl->error_info = (2u << 24) | ((unsigned)slot << 16) | ((unsigned)i & 0xffffu);
+                            p.ctrl->error_info = (2u << 24) | ((unsigned)slot << 16) | ((unsigned)j & 0xffffu);
                         s_abort = 1;
                     }
                     ok = false;
@@ -231,28 +249,50 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
                 const unsigned char* a_lo = ring + (size_t)slot * stage_bytes + g * p.stage_row_bytes + t * 16;
                 const unsigned char* a_hi = a_lo + 8 * p.stage_row_bytes;
                 const uint4* yk = y_lane + (k0 >> 3);
-                for (int c0 = 0; c0 < nch; c0 += CH) {
+                // Four 32-column chunks per step: all operand loads first, then the MMAs ordered so that
+                // consecutive ones are independent (chains of different chunks).
+                int c = 0;
+                for (; c + 4 <= nch && !(k_ragged && c + 4 == nch); c += 4) {
+                    uint4 lo[4], hi[4];
 #pragma unroll
-                    for (int u = 0; u < CH; ++u) {
-                        const int c = c0 + u;
-                        if (c < nch) {
-                            uint4 lo = *reinterpret_cast<const uint4*>(a_lo + c * 64);
-                            uint4 hi = *reinterpret_cast<const uint4*>(a_hi + c * 64);
-                            if (k_ragged && k0 + c * 32 + t * 8 >= p.d) {      // beyond d: whatever the ring holds
-                                lo = make_uint4(0, 0, 0, 0);
-                                hi = make_uint4(0, 0, 0, 0);
-                            }
+                    for (int u = 0; u < 4; ++u) {
+                        lo[u] = *reinterpret_cast<const uint4*>(a_lo + (c + u) * 64);
+                        hi[u] = *reinterpret_cast<const uint4*>(a_hi + (c + u) * 64);
+                    }
 #pragma unroll
-                            for (int n = 0; n < NT; ++n) {
-                                const uint4 yv = yk[(size_t)n * y_tile_vecs + c * 4];
-                                mma_bf16_16816(acc[n][u], lo.x, hi.x, lo.y, hi.y, yv.x, yv.y);
-                                mma_bf16_16816(acc[n][u], lo.z, hi.z, lo.w, hi.w, yv.z, yv.w);
-                            }
-                        }
+                    for (int n = 0; n < NT; ++n) {
+                        uint4 yv[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) yv[u] = yk[(size_t)n * y_tile_vecs + (c + u) * 4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            mma_bf16_16816(acc[n][u % CH], lo[u].x, hi[u].x, lo[u].y, hi[u].y, yv[u].x, yv[u].y);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            mma_bf16_16816(acc[n][u % CH], lo[u].z, hi[u].z, lo[u].w, hi[u].w, yv[u].z, yv[u].w);
                     }
                 }
+                for (; c < nch; ++c) {                                 // remainder, and the chunk that straddles d
+                    uint4 lo = *reinterpret_cast<const uint4*>(a_lo + c * 64);
+                    uint4 hi = *reinterpret_cast<const uint4*>(a_hi + c * 64);
+                    if (k_ragged && k0 + c * 32 + t * 8 >= p.d) {      // beyond d: whatever the ring holds
+                        lo = make_uint4(0, 0, 0, 0);
+                        hi = make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        const uint4 yv = yk[(size_t)n * y_tile_vecs + c * 4];
+                        mma_bf16_16816(acc[n][0], lo.x, hi.x, lo.y, hi.y, yv.x, yv.y);
+                        mma_bf16_16816(acc[n][0], lo.z, hi.z, lo.w, hi.w, yv.z, yv.w);
+                    }
+                }
+                // The slot has been read; hand it back to the copy engine for this warp's next stage.
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(empty_bar(slot));  // the stage may be refilled
+                if (issued < my_stages) {
+                    ptx::fence_proxy_async();
+                    issue_stage(issued);
+                    ++issued;
+                }
             }
             if (!ok) break;
             // The 16 x MPAD logits of this row group are complete.
@@ -276,8 +316,19 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
                 }
             }
         }
+        if (!ok && lane == 0) {
+            // Let this warp's copies that are still in flight land before the CTA gives its shared memory back.
+            for (int q = max(0, issued - p.slots_per_warp); q < issued; ++q) {
+                const int slot = warp * p.slots_per_warp + q % p.slots_per_warp;
+                const uint32_t par = (uint32_t)(q / p.slots_per_warp) & 1u;
+                for (uint32_t n = 0; n < (1u << 14) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
+            }
+        }
+    }
 
+    {
         // Merge over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then own tokens 2t, 2t+1.
+        const int g = lane >> 2, t = lane & 3;
 #pragma unroll
         for (int n = 0; n < NT; ++n)
 #pragma unroll
@@ -292,10 +343,10 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     }
     __syncthreads();
 
-    // Merge over the CTA's consumer warps; publish the CTA partial.
+    // Merge over the CTA's warps; publish the CTA partial.
     if (threadIdx.x < MPAD) {
         State a = wpart[threadIdx.x];
-        for (int w = 1; w < kConsumerWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
+        for (int w = 1; w < kWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
         p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = a;
         __threadfence();
     }
@@ -307,12 +358,21 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     __syncthreads();
     if (!s_is_last) return;
 
-    // Last CTA: merge the partials of all CTAs, one warp per token, and decide.
+    // Last CTA: merge the partials of all CTAs and decide.  The partials are first pulled into shared memory
+    // with independent, coalesced loads (the ring is free by now); then one warp per token merges them
+    // (lane-strided over the CTAs, then a butterfly).
     __threadfence();
-    for (int tok = warp; tok < p.M; tok += kThreads / 32) {
+    const int n_part = (int)gridDim.x * MPAD;
+    const bool via_smem = (size_t)n_part * sizeof(State) <= (size_t)p.n_stages * stage_bytes;
+    State* part_s = reinterpret_cast<State*>(ring);
+    if (via_smem) {
+        for (int i = threadIdx.x; i < n_part; i += kThreads) part_s[i] = state_load_cg(p.partials + i);
+        __syncthreads();
+    }
+    for (int tok = warp; tok < p.M; tok += kWarps) {
         State a = state_empty();
         for (int b = lane; b < (int)gridDim.x; b += 32) {
-            const State o = state_load_cg(p.partials + (size_t)b * MPAD + tok);
+            const State o = via_smem ? part_s[b * MPAD + tok] : state_load_cg(p.partials + (size_t)b * MPAD + tok);
             state_merge(a, o);
         }
 #pragma unroll
@@ -332,40 +392,76 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
 // Host side: shared-memory plan and launch
 // ---------------------------------------------------------------------------------------------
 struct SmemPlan {
-    int seg_cols, n_segs, stage_row_bytes, n_stages, n_consumers, slots_per_warp;
+    int seg_cols, n_segs, stage_row_bytes, n_stages, n_workers, slots_per_warp, contiguous;
     size_t bytes;
 };
 
+// Splits n ring slots of `stage` bytes into private rings: the split with the most slots wins, with at
+// least min(6, n) workers (the MMAs of several stages then overlap) and at most four slots per worker.
+bool split_slots(long long n, int min_workers, SmemPlan& s) {
+    int best_total = 0;
+    for (int c = kWarps; c >= 1; --c) {
+        int b = (int)(n / c);
+        if (b < 1) continue;
+        if (b > 4) b = 4;
+        if (c < 6 && c < n) continue;
+        if (c < min_workers && n >= min_workers) continue;
+        if (c * b > best_total) {
+            best_total = c * b;
+            s.n_workers = c;
+            s.slots_per_warp = b;
+        }
+    }
+    s.n_stages = best_total;
+    return best_total > 0;
+}
+
 // Ring geometry for hidden size d with 8*nt rows of y resident; n_stages = 0 if it does not fit.
-// Stages hold up to 1024 columns (2 KB per row); narrower stages are chosen when y leaves little room,
-// so that at least four stages are in flight.
 SmemPlan plan_smem(int d, int nt) {
-    SmemPlan best;
-    best.n_stages = 0;
-    best.bytes = 0;
+    SmemPlan none = {};
     const int d64 = (d + 63) / 64 * 64;
     const size_t fixed = (size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
-                         (size_t)kConsumerWarps * 8 * nt * sizeof(State) + 2 * kMaxStages * sizeof(uint64_t);
+                         (size_t)kWarps * 8 * nt * sizeof(State) + (size_t)2 * d * sizeof(float) +
+                         kMaxStages * sizeof(uint64_t);
     const long long room = (long long)kSmemBudget - (long long)fixed;
+    if (room <= 0) return none;
+    if (d <= kSegMax) {
+        // Rows of up to 2 KB: a stage is 16 whole rows, contiguous in W, fetched by a single copy into an
+        // unpadded block (adjacent rows then share banks: a two-way conflict on the A loads, which is cheap
+        // next to issuing sixteen copies of about a hundred cycles each).
+        SmemPlan s = {};
+        s.contiguous = 1;
+        s.seg_cols = d;
+        s.n_segs = 1;
+        s.stage_row_bytes = 2 * d;
+        const long long stage = (long long)kStageRows * s.stage_row_bytes;
+        long long n = room / stage;
+        if (n > kMaxStages) n = kMaxStages;
+        if (n >= 2 && split_slots(n, 1, s)) {
+            s.bytes = fixed + (size_t)s.n_stages * (size_t)stage;
+            return s;
+        }
+    }
+    // Wider rows: column segments of up to 1024 / 512 / 256, rows padded by 64 bytes (conflict-free), one copy
+    // per row; enough workers to issue the copies faster than HBM delivers them.
+    SmemPlan best = none;
+    long long best_bytes = 0;
     for (int seg = kSegMax; seg >= 256; seg >>= 1) {
-        SmemPlan s;
+        SmemPlan s = {};
+        s.contiguous = 0;
         s.seg_cols = d64 < seg ? d64 : seg;
         s.n_segs = (d + s.seg_cols - 1) / s.seg_cols;
         s.stage_row_bytes = 2 * s.seg_cols + 64;
         const long long stage = (long long)kStageRows * s.stage_row_bytes;
-        long long n = room > 0 ? room / stage : 0;
+        long long n = room / stage;
         if (n > kMaxStages) n = kMaxStages;
-        // Split the slots into private rings: n_consumers warps x slots_per_warp, as many slots as fit.
-        s.n_consumers = 0;
-        s.slots_per_warp = 0;
-        for (int c = kConsumerWarps; c >= 1; --c) {
-            if (c < 4 && c < n) continue;                       // keep at least four warps busy when slots allow
-            const int b = (int)(n / c);
-            if (b >= 1 && c * b > s.n_consumers * s.slots_per_warp) { s.n_consumers = c; s.slots_per_warp = b; }
+        int min_workers = (1700 + s.seg_cols - 1) / s.seg_cols;
+        if (min_workers > kWarps) min_workers = kWarps;
+        if (n >= 2 && split_slots(n, min_workers, s) && (long long)s.n_stages * stage > best_bytes) {
+            best_bytes = (long long)s.n_stages * stage;
+            s.bytes = fixed + (size_t)best_bytes;
+            best = s;
         }
-        s.n_stages = s.n_consumers * s.slots_per_warp;
-        s.bytes = fixed + (size_t)s.n_stages * (size_t)stage;
-        if (s.n_stages >= 4 || (seg == 256 && s.n_stages >= 2)) return s;
         if (d64 <= seg / 2) break;          // a narrower cap would not change the stage
     }
     return best;
@@ -379,8 +475,9 @@ ee_status launch_one(StreamParams& p, int grid, int device, cudaStream_t stream)
     p.n_segs = plan.n_segs;
     p.stage_row_bytes = plan.stage_row_bytes;
     p.n_stages = plan.n_stages;
-    p.n_consumers = plan.n_consumers;
+    p.n_workers = plan.n_workers;
     p.slots_per_warp = plan.slots_per_warp;
+    p.contiguous = plan.contiguous;
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
         if (cudaFuncSetAttribute(exit_head_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -388,8 +485,17 @@ ee_status launch_one(StreamParams& p, int grid, int device, cudaStream_t stream)
             return EE_ERR_CUDA;
         configured[device] = true;
     }
-    exit_head_stream_kernel<NT><<<grid, kThreads, plan.bytes, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = plan.bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, exit_head_stream_kernel<NT>, p) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 }  // namespace
