@@ -37,7 +37,9 @@ typedef enum {
 typedef enum {
     EE_PATH_AUTO = 0,      /* by M: streaming kernel for decode-sized M, tensor-core kernel above   */
     EE_PATH_STREAM = 1,    /* fused LayerNorm + split-V streaming kernel (any M, in slabs of rows)  */
-    EE_PATH_TCGEN05 = 2    /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics     */
+    EE_PATH_TCGEN05 = 2,   /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics     */
+    EE_PATH_SKINNY = 3     /* one-launch tcgen05 kernel with W as the MMA's M operand: M <= 64, d % 64 == 0,
+                              M_pad * d <= 64 Ki elements; other sizes return EE_ERR_SHAPE                */
 } ee_path;
 
 /* Static, human-readable name of a status code. */

@@ -10,7 +10,7 @@ import torch
 
 from . import _lib
 
-EE_PATH_AUTO, EE_PATH_STREAM, EE_PATH_TCGEN05 = 0, 1, 2
+EE_PATH_AUTO, EE_PATH_STREAM, EE_PATH_TCGEN05, EE_PATH_SKINNY = 0, 1, 2, 3
 
 
 class EExitError(RuntimeError):

@@ -48,6 +48,7 @@ size_t workspace_bytes(int M, int d, int V) {
     size_t need = gemm_workspace_bytes(M, d, V);
     const size_t s = stream_workspace_bytes(M, d, V);
     if (s > need) need = s;
+    if (skinny_workspace_bytes() > need) need = skinny_workspace_bytes();
     return kCtrlBytes + need;
 }
 
@@ -84,6 +85,7 @@ int ee_exit_head_launches(int M, int d, int V, int path) {
         const int slab = stream_slab_rows(d);
         return slab > 0 ? (M + slab - 1) / slab : 0;
     }
+    if (path == EE_PATH_SKINNY) return skinny_supports(M, d) ? 1 : 0;
     return path == EE_PATH_TCGEN05 ? 3 : 0;      // LayerNorm, GEMM with fused statistics, merge
 }
 
@@ -100,7 +102,7 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
                             float* entropy, float* maxprob, unsigned char* exit_mask, void* workspace,
                             size_t workspace_bytes_, void* stream, int path) {
     if (!sizes_ok(M, d, V)) return EE_ERR_SHAPE;
-    if (path != EE_PATH_AUTO && path != EE_PATH_STREAM && path != EE_PATH_TCGEN05) return EE_ERR_SHAPE;
+    if (path < EE_PATH_AUTO || path > EE_PATH_SKINNY) return EE_ERR_SHAPE;
     if (M == 0) return EE_OK;
     if (!h || !gamma || !beta || !W || !argmax || !entropy || !maxprob || !exit_mask || !workspace) return EE_ERR_NULL;
     if (ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
@@ -119,6 +121,7 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
 
     if (path == EE_PATH_AUTO) path = auto_path(M, d);
     if (path == EE_PATH_STREAM) return stream_launch(a);
+    if (path == EE_PATH_SKINNY) return skinny_launch(a);
     return gemm_launch(a);
 }
 

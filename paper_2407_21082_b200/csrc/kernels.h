@@ -38,6 +38,12 @@ int stream_slab_rows(int d);               // rows one launch can take for this 
 size_t stream_workspace_bytes(int M, int d, int V);
 ee_status stream_launch(const HeadArgs& a);
 
+// ---- skinny tensor-core kernel (one launch, weights as the MMA's M operand, 1 <= M <= 64, d % 64 == 0) ----
+constexpr int kSkinnyMaxRows = 64;
+bool skinny_supports(int M, int d);
+size_t skinny_workspace_bytes();
+ee_status skinny_launch(const HeadArgs& a);
+
 // ---- tensor-core kernel (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge) ----
 int gemm_tile_n(int M);                    // vocabulary tile width used for M rows
 size_t gemm_workspace_bytes(int M, int d, int V);

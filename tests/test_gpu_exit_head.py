@@ -35,10 +35,15 @@ SMALL = [
 ]
 
 
-@pytest.mark.parametrize("path_name", ["stream", "tcgen05"])
-@pytest.mark.parametrize("name,M,d,V", SMALL)
+PATHS = {"stream": 1, "tcgen05": 2, "skinny": 3}
+
+
+@pytest.mark.parametrize("path_name", ["stream", "tcgen05", "skinny"])
+@pytest.mark.parametrize("name,M,d,V", SMALL + [("sk_n32", 17, 192, 3001), ("sk_n64", 64, 512, 2500), ("sk_n64b", 33, 1024, 1500)])
 def test_small_shapes_match_oracle(ee, path_name, name, M, d, V):
-    path = ee.EE_PATH_STREAM if path_name == "stream" else ee.EE_PATH_TCGEN05
+    path = PATHS[path_name]
+    if ee.ee_exit_head_launches(M, d, V, path) == 0:
+        pytest.skip(f"{path_name} kernel does not take M={M}, d={d}")
     for planted in (False, True):
         cfg = gen.make_config("c0", seed=11, planted=planted, M=M, d=d, V=V)
         tau = 1.0 if planted else float(np.log(V) - 0.05) if V > 1 else 1.0
@@ -57,7 +62,7 @@ def test_exact_small_integer_case(ee):
                 W=gen.bf16_bits_from_f32(Wv.astype(np.float32)))
     h = gen.bf16_bits_from_f32(x.astype(np.float32))
     ref = oracle.exit_head(h, head["gamma"], head["beta"], 1e-5, head["W"], 1.0)
-    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05, ee.EE_PATH_SKINNY):
         hd = head_to_dev(head)
         out = ee.ee_exit_head(dev_bf16(h), hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, path=path)
         got = {k: v.cpu().numpy() for k, v in out.items()}
@@ -72,7 +77,7 @@ def test_uniform_logits_give_ln_V_and_lowest_index(ee):
     cfg = gen.make_config("c0", seed=1, M=M, d=d, V=8)
     Wz = torch.zeros((V, d), dtype=torch.bfloat16, device="cuda")
     hd = head_to_dev(cfg["heads"][0])
-    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+    for path in (ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05, ee.EE_PATH_SKINNY):
         out = ee.ee_exit_head(dev_bf16(cfg["h"]), hd["gamma"], hd["beta"], 1e-5, Wz, 11.0, path=path)
         assert torch.all(out["argmax"] == 0)
         assert np.allclose(out["entropy"].cpu().numpy(), 10.825839875788878, atol=2e-4)
@@ -99,7 +104,7 @@ def test_c1_three_heads_full_size(ee, planted):
         for M in gen.CONFIGS["c1"]["Ms"]:
             sub = dict(cfg, h=cfg["h"][:M])
             ref = {k: v[:M] for k, v in ref64.items()}
-            for path in (ee.EE_PATH_AUTO, ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05):
+            for path in (ee.EE_PATH_AUTO, ee.EE_PATH_STREAM, ee.EE_PATH_TCGEN05, ee.EE_PATH_SKINNY):
                 assert_head_matches(_run(ee, sub, hid, cfg["tau"], path), ref, label=f"c1 head{hid} M={M} path={path}")
     if planted:
         assert 0 < exits < 3 * 64          # the planted inputs exercise both outcomes
@@ -138,8 +143,11 @@ def test_both_kernels_agree_and_runs_are_bit_identical(ee):
     b = _run(ee, cfg, 0, 1.0, ee.EE_PATH_STREAM)
     c = _run(ee, cfg, 0, 1.0, ee.EE_PATH_TCGEN05)
     e = _run(ee, cfg, 0, 1.0, ee.EE_PATH_TCGEN05)
+    f = _run(ee, cfg, 0, 1.0, ee.EE_PATH_SKINNY)
+    g = _run(ee, cfg, 0, 1.0, ee.EE_PATH_SKINNY)
     for k in a:
-        assert torch.equal(a[k], b[k]) and torch.equal(c[k], e[k]), k
+        assert torch.equal(a[k], b[k]) and torch.equal(c[k], e[k]) and torch.equal(f[k], g[k]), k
+    assert torch.allclose(a["entropy"], f["entropy"], atol=1e-3) and torch.equal(a["argmax"], f["argmax"])
     assert torch.allclose(a["entropy"], c["entropy"], atol=1e-3) and torch.equal(a["argmax"], c["argmax"])
 
 
@@ -184,4 +192,9 @@ def test_device_side_argument_errors(ee):
     assert e.value.code in (3, 4)
     with pytest.raises(ee.EExitError) as e:
         ee.ee_exit_head(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, workspace=ws, path=7)
+    assert e.value.code == 2
+    odd = gen.make_config("c0", seed=2, M=4, d=72, V=100)              # d % 64 != 0: not for the skinny kernel
+    ohd = head_to_dev(odd["heads"][0])
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_exit_head(dev_bf16(odd["h"]), ohd["gamma"], ohd["beta"], 1e-5, ohd["W"], 1.0, path=ee.EE_PATH_SKINNY)
     assert e.value.code == 2
