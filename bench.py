@@ -107,10 +107,11 @@ def _algorithmic(M, d, V):
 class Workload:
     """Device tensors of one workload and a `step()` that runs the whole hot path once."""
 
-    def __init__(self, name: str, M: int | None, seed: int, n_copies: int):
+    def __init__(self, name: str, M: int | None, seed: int, n_copies: int, path: int = 0):
         import torch
         import paper_2407_21082_b200 as ee
         self.torch, self.ee = torch, ee
+        self.path = path
         cfg = gen.make_config(name, seed=seed, planted=False, M=M)
         self.name, self.cfg = name, cfg
         self.M, self.d, self.V = cfg["M"], cfg["d"], cfg["V"]
@@ -140,7 +141,7 @@ class Workload:
         self.acc = {n: torch.empty(max(self.S, 1), dtype=torch.int32, device="cuda") for n in ("draft_len", "accept_len", "next_tok")}
         self.calls = 0
         self.n_copies = n_copies
-        self.head_launches = ee.ee_exit_head_launches(self.M, self.d, self.V)
+        self.head_launches = ee.ee_exit_head_launches(self.M, self.d, self.V, path)
         self.launches_per_step = len(self.heads) * self.head_launches + 1 + (1 if self.S > 0 else 0)
         self.bytes_per_call, self.flops_per_call = _algorithmic(self.M, self.d, self.V)
         self.w_bytes_total = sum(w.numel() * 2 for hd in self.heads for w in hd["W"])
@@ -150,7 +151,7 @@ class Workload:
         """Marshals every call of a step once (the binding's PreparedCall), so the loop is a few C calls."""
         ee = self.ee
         self.head_calls = [[ee.prepare_exit_head(self.h[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], self.tau,
-                                                 out=self.outs[i], workspace=self.ws)
+                                                 out=self.outs[i], workspace=self.ws, path=self.path)
                             for i, hd in enumerate(self.heads)] for c in range(self.n_copies)]
         self.compact_call = ee.prepare_compact(self.outs[0]["exit_mask"], self.h[0], out=self.comp)
         self.accept_call = None
@@ -327,6 +328,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--rows", type=int, default=None, help="override M of the workload")
+    ap.add_argument("--path", default="auto", choices=["auto", "stream", "tcgen05", "skinny"], help="force a kernel")
+    ap.add_argument("--sweep", action="store_true", help="time every kernel that accepts the size, for c1 at several M")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-config table and the CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -364,7 +367,9 @@ def main():
     peaks, peak_src = load_peaks()
 
     n_copies = {"c0": 8, "c1": 2}.get(args.workload, 2)
-    wl = Workload(args.workload, M, seed=rank, n_copies=n_copies)
+    path = dict(auto=0, stream=1, tcgen05=2, skinny=3)[args.path]
+    wl = Workload(args.workload, M, seed=rank, n_copies=n_copies, path=path)
+    config["kernel"] = args.path
     sampler = ClockSampler(local_rank) if rank == 0 else None
     res = measure(wl, args.steps, args.warmup, dist, sampler)
     n_heads = len(wl.heads)
@@ -399,6 +404,18 @@ def main():
             del w
             torch.cuda.empty_cache()
         line["configs"] = extra
+        if args.sweep:
+            sweep = {}
+            for rows in (1, 8, 16, 32, 64):
+                for pname, pid in (("stream", 1), ("skinny", 3), ("tcgen05", 2)):
+                    w = Workload("c1", rows, seed=0, n_copies=2, path=pid)
+                    if w.head_launches == 0:
+                        continue
+                    r = measure(w, 300, 5)
+                    sweep[f"c1_M{rows}_{pname}"] = round(r["head_call_us"], 2)
+                    del w
+                    torch.cuda.empty_cache()
+            line["sweep_head_call_us"] = sweep
         cfg = gen.make_config(args.workload, seed=0, planted=False, M=M)
         line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0)
     if rank == 0:
