@@ -6,9 +6,11 @@
 // CTA normalises them itself, writing the swizzled layout directly).  The MMAs are issued by one thread and
 // cost the SM nothing else, so a ring slot is free again as soon as the tensor core has read it.  The
 // accumulator [128 vocabulary rows x N tokens] lives in TMEM (two buffers).  Epilogue warps read it back with
-// the vocabulary row on the lane, reduce each token's column across the warp (redux for the maximum, ballot
-// for its position, shuffles for the two sums) and fold the result into per-token online states kept by owner
-// lanes.  Per-CTA partial states, atomic ticket, last CTA merges and decides, as in the streaming kernel.
+// the vocabulary row on the lane; every thread keeps one online state per token (at most 32 tokens per thread:
+// for N = 64 a second set of epilogue warps takes tokens 32..63), so a tile costs one state update per logit and
+// no cross-lane traffic.  At the end the per-lane states are transposed through shared memory (the ring is
+// free by then) and merged per token.  Per-CTA partial states, atomic ticket, last CTA merges and decides, as
+// in the streaming kernel.
 #include "common.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -18,8 +20,9 @@ namespace ee {
 
 namespace {
 
-constexpr int kSkThreads = 192;            // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-constexpr int kSkWarps = kSkThreads / 32;
+// warp 0 TMA, warp 1 MMA, then four epilogue warps per group of up to 32 tokens
+__host__ __device__ constexpr int sk_groups(int n) { return n <= 32 ? 1 : n / 32; }
+__host__ __device__ constexpr int sk_threads(int n) { return 64 + 128 * sk_groups(n); }
 constexpr int kTileRows = 128;             // MMA M
 constexpr int kBK = 64;
 constexpr int kStageBytes = kTileRows * kBK * 2;      // 16 KB
@@ -55,13 +58,6 @@ __device__ __forceinline__ void sk_cp_async_wait_all() {
     asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
-// Order-preserving map float -> int, so that the warp maximum can use one redux instruction.
-__device__ __forceinline__ int ordered_int(float f) {
-    const int i = __float_as_int(f);
-    return i >= 0 ? i : i ^ 0x7fffffff;
-}
-__device__ __forceinline__ float ordered_float(int i) { return __int_as_float(i >= 0 ? i : i ^ 0x7fffffff); }
-
 // Address of 16-byte vector c (columns 8c .. 8c+7) of activation row r inside the swizzled y tiles:
 // tile kb = c / 8 holds [N rows][64 columns], rows of 128 bytes, 16-byte chunks XOR-ed with (row & 7).
 template <int N>
@@ -71,9 +67,12 @@ __device__ __forceinline__ uint4* y_vec(unsigned char* y_tiles, int r, int c) {
 }
 
 template <int N>
-__global__ void __launch_bounds__(kSkThreads, 1)
+__global__ void __launch_bounds__(sk_threads(N), 1)
 exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyParams p) {
-    constexpr int NSLOT = (N + 31) / 32;                         // tokens owned per lane
+    constexpr int TOK = N < 32 ? N : 32;                          // tokens per epilogue thread
+    constexpr int GROUPS = sk_groups(N);
+    constexpr int kSkThreads = sk_threads(N);
+    constexpr int kSkWarps = kSkThreads / 32;
     constexpr int TMEM_COLS = (2 * N < 32) ? 32 : 2 * N;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -107,7 +106,7 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4);
+            ptx::mbar_init(tempty_bar(b), 4 * GROUPS);
         }
         ptx::mbar_init(drain_bar, 1);
         *abort_flag = 0;
@@ -177,10 +176,6 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
         ptx::fence_proxy_async();                                 // y was written by threads, is read by the MMA
         __syncthreads();
     }
-
-    State own[NSLOT];
-#pragma unroll
-    for (int s = 0; s < NSLOT; ++s) own[s] = state_empty();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (continues the ring)
@@ -252,9 +247,13 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2 ..)
         const int quarter = warp & 3;                             // TMEM lanes 32*quarter .. +31
+        const int group = (warp - 2) >> 2;                        // tokens group*32 .. +TOK-1
         const int row_in_tile = quarter * 32 + lane;
+        State own[TOK];
+#pragma unroll
+        for (int k = 0; k < TOK; ++k) own[k] = state_empty();
         for (int tile = 0; tile < n_tiles; ++tile) {
             const int buf = tile & 1;
             const uint32_t acc_phase = (uint32_t)(tile >> 1) & 1u;
@@ -270,48 +269,32 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
             ptx::tc_fence_after_sync();
             const int row = r_begin + tile * p.box_rows + row_in_tile;       // this lane's vocabulary row
             const bool valid = row_in_tile < p.box_rows && row < r_end;
-            const int warp_row0 = r_begin + tile * p.box_rows + quarter * 32;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * N);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * N + group * 32);
 #pragma unroll
-            for (int c = 0; c < N / 16; ++c) {
+            for (int c = 0; c < TOK / 16; ++c) {
                 float v[16];
                 ptx::tmem_ld_32x16(taddr + c * 16, v);
                 ptx::tmem_ld_wait();
+                if (valid) {
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    const int j = c * 16 + jj;                    // token (compile-time after unrolling)
-                    const float z = valid ? v[jj] : -CUDART_INF_F;
-                    const float mw = ordered_float(__reduce_max_sync(0xffffffffu, ordered_int(z)));
-                    const unsigned eq = __ballot_sync(0xffffffffu, valid && z == mw);
-                    const float m_run = __shfl_sync(0xffffffffu, own[j >> 5].m, j & 31);
-                    const float m_new = fmaxf(m_run, mw);
-                    const float dz = z - m_new;
-                    const float e = valid ? ex2(dz * kLog2e) : 0.f;
-                    const float s_w = warp_sum(e);
-                    const float t_w = warp_sum(valid ? e * dz : 0.f);
-                    if (lane == (j & 31)) {
-                        State& o = own[j >> 5];
-                        if (mw > m_run) {                         // the maximum moves into this tile
-                            const float dl = m_run - m_new;
-                            const bool was_empty = (o.s == 0.f);
-                            const float al = was_empty ? 0.f : ex2(dl * kLog2e);
-                            o.t = was_empty ? 0.f : al * fmaf(dl, o.s, o.t);
-                            o.s = al * o.s;
-                            o.m = m_new;
-                            o.idx = warp_row0 + __ffs(eq) - 1;
-                        }
-                        o.s += s_w;
-                        o.t += t_w;
-                    }
+                    for (int jj = 0; jj < 16; ++jj) state_push(own[c * 16 + jj], v[jj], row);
                 }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
         }
+        // Transpose through shared memory (ring and y are no longer read: the last tile's MMAs have completed):
+        // lane t then merges token t's 32 per-lane states in row order.
+        State* stash = reinterpret_cast<State*>(smem) + (size_t)(warp - 2) * 32 * TOK;
 #pragma unroll
-        for (int s = 0; s < NSLOT; ++s)
-            if (lane + 32 * s < N) qpart[quarter * N + lane + 32 * s] = own[s];
+        for (int k = 0; k < TOK; ++k) stash[lane * TOK + (k ^ (lane & (TOK - 1)))] = own[k];   // XOR spreads the banks
+        __syncwarp();
+        if (lane < TOK) {
+            State a = stash[lane];                                // row lane 0 holds token k at column k
+            for (int l = 1; l < 32; ++l) state_merge(a, stash[l * TOK + (lane ^ (l & (TOK - 1)))]);
+            qpart[quarter * N + group * 32 + lane] = a;
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -392,7 +375,7 @@ ee_status launch_skinny(const CUtensorMap& tm_w, const SkinnyParams& p, int grid
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kSkThreads);
+    cfg.blockDim = dim3(sk_threads(N));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
