@@ -174,4 +174,109 @@ __device__ __forceinline__ float vec8_sqdev(uint4 v, float mu, float acc) {
     return acc;
 }
 
+// ---------------------------------------------------------------------------------------------
+// LayerNorm of rows that already sit in shared memory as raw bf16 (16-byte vectors reached through
+// vec(row, c)), in place.  A warp keeps R whole rows in registers (up to VPL vectors per lane), so each row is
+// read once and the R dependency chains (two warp reductions each) overlap.  Requires nvec <= 32 * VPL.
+// ---------------------------------------------------------------------------------------------
+template <int R, int VPL, class VecFn>
+__device__ __forceinline__ void layer_norm_rows_in_regs(VecFn vec, const int (&rows)[R], int n_rows, int nvec, float inv_d,
+                                                        float ln_eps, const float* gamma_s, const float* beta_s,
+                                                        int lane) {
+    uint4 x[R][VPL];
+    float mu[R], rstd[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            x[i][k] = (i < n_rows && c < nvec) ? *vec(rows[i], c) : make_uint4(0, 0, 0, 0);
+            sum += vec8_sum(x[i][k]);
+        }
+        mu[i] = sum;
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) mu[i] = warp_sum(mu[i]) * inv_d;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float sq = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (lane + 32 * k < nvec) sq = vec8_sqdev(x[i][k], mu[i], sq);
+        rstd[i] = sq;
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) rstd[i] = 1.f / sqrtf(warp_sum(rstd[i]) * inv_d + ln_eps);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int c = lane + 32 * k;
+        if (c < nvec) {
+            const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
+            const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
+            const float4 g0 = g4[0], g1 = g4[1], b0 = b4[0], b1 = b4[1];
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+                if (i < n_rows) *vec(rows[i], c) = layer_norm_vec8(x[i][k], mu[i], rstd[i], g0, g1, b0, b1);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Completion ticket and final merge shared by the one-launch kernels.
+// ---------------------------------------------------------------------------------------------
+// Thread 0 of a CTA, after a CTA-wide barrier that follows the CTA's partial-state stores: one acquire-release
+// atomic publishes those stores and tells whether every other CTA has published before.
+__device__ __forceinline__ bool ticket_arrive_is_last(Control* ctrl, unsigned int n_cta) {
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&ctrl->ticket) : "memory");
+    return old == n_cta - 1;
+}
+
+// Every thread of the last CTA: merge partials [n_cta][np] per token (lane-strided over the CTAs, then a
+// butterfly; four tokens per warp at a time so that their chains overlap) and write the outputs.  `scratch`
+// is shared memory the partials are first copied to with independent loads, if it is large enough.
+template <int THREADS>
+__device__ void merge_partials_and_decide(const State* partials, int n_cta, int np, int M, State* scratch,
+                                          size_t scratch_bytes, const float* tau_per_row, float tau, int* argmax,
+                                          float* entropy, float* maxprob, unsigned char* exit_mask) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_part = n_cta * np;
+    const bool via_smem = (size_t)n_part * sizeof(State) <= scratch_bytes;
+    if (via_smem) {
+        for (int i = threadIdx.x; i < n_part; i += THREADS) scratch[i] = state_load_cg(partials + i);
+        __syncthreads();
+    }
+    for (int tok0 = warp * 4; tok0 < M; tok0 += (THREADS / 32) * 4) {
+        State a[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) a[q] = state_empty();
+        for (int b = lane; b < n_cta; b += 32) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (tok0 + q < M) {
+                    const size_t i = (size_t)b * np + tok0 + q;
+                    const State o = via_smem ? scratch[i] : state_load_cg(partials + i);
+                    state_merge(a[q], o);
+                }
+        }
+#pragma unroll
+        for (int msk = 1; msk <= 16; msk <<= 1) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const State o = state_shfl_xor(a[q], msk);
+                state_merge(a[q], o);
+            }
+        }
+        if (lane < 4 && tok0 + lane < M) {
+            State mine = a[0];
+#pragma unroll
+            for (int q = 1; q < 4; ++q)
+                if (lane == q) mine = a[q];
+            const int tok = tok0 + lane;
+            state_finish(mine, tau_per_row ? tau_per_row[tok] : tau, argmax, entropy, maxprob, exit_mask, tok);
+        }
+    }
+}
+
 }  // namespace ee

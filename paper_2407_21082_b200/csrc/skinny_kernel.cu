@@ -155,22 +155,31 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
         sk_cp_async_wait_all();
         __syncthreads();
         const float inv_d = 1.f / (float)p.d;
-        for (int r = warp; r < N; r += kSkWarps) {
-            if (r >= p.M) {
-                for (int c = lane; c < nvec; c += 32) *y_vec<N>(y_tiles, r, c) = make_uint4(0, 0, 0, 0);
-                continue;
+        auto vec = [&](int r, int c) { return y_vec<N>(y_tiles, r, c); };
+        for (int r = p.M + warp; r < N; r += kSkWarps)            // padding rows
+            for (int c = lane; c < nvec; c += 32) *vec(r, c) = make_uint4(0, 0, 0, 0);
+        if (nvec <= 256) {
+            // Rows held in registers: one pass over shared memory, two rows at a time.
+            for (int r = warp; r < p.M; r += 2 * kSkWarps) {
+                const int rows[2] = {r, r + kSkWarps};
+                const int live = 1 + (rows[1] < p.M);
+                if (nvec <= 128) layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+                else layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
             }
-            float sum = 0.f;
-            for (int c = lane; c < nvec; c += 32) sum += vec8_sum(*y_vec<N>(y_tiles, r, c));
-            const float mu = warp_sum(sum) * inv_d;
-            float sq = 0.f;
-            for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(*y_vec<N>(y_tiles, r, c), mu, sq);
-            const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
-            for (int c = lane; c < nvec; c += 32) {
-                const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
-                const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-                uint4* v = y_vec<N>(y_tiles, r, c);
-                *v = layer_norm_vec8(*v, mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+        } else {
+            for (int r = warp; r < p.M; r += kSkWarps) {
+                float sum = 0.f;
+                for (int c = lane; c < nvec; c += 32) sum += vec8_sum(*vec(r, c));
+                const float mu = warp_sum(sum) * inv_d;
+                float sq = 0.f;
+                for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(*vec(r, c), mu, sq);
+                const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
+                for (int c = lane; c < nvec; c += 32) {
+                    const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
+                    const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
+                    uint4* v = vec(r, c);
+                    *v = layer_norm_vec8(*v, mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+                }
             }
         }
         ptx::fence_proxy_async();                                 // y was written by threads, is read by the MMA
@@ -291,9 +300,17 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
         for (int k = 0; k < TOK; ++k) stash[lane * TOK + (k ^ (lane & (TOK - 1)))] = own[k];   // XOR spreads the banks
         __syncwarp();
         if (lane < TOK) {
-            State a = stash[lane];                                // row lane 0 holds token k at column k
-            for (int l = 1; l < 32; ++l) state_merge(a, stash[l * TOK + (lane ^ (l & (TOK - 1)))]);
-            qpart[quarter * N + group * 32 + lane] = a;
+            State a[4];                                           // four interleaved chains over the 32 rows
+#pragma unroll
+            for (int q = 0; q < 4; ++q) a[q] = stash[q * TOK + (lane ^ (q & (TOK - 1)))];
+            for (int l = 4; l < 32; l += 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) state_merge(a[q], stash[(l + q) * TOK + (lane ^ ((l + q) & (TOK - 1)))]);
+            }
+            state_merge(a[0], a[1]);
+            state_merge(a[2], a[3]);
+            state_merge(a[0], a[2]);
+            qpart[quarter * N + group * 32 + lane] = a[0];
         }
     }
 
@@ -310,41 +327,16 @@ exit_head_skinny_kernel(const __grid_constant__ CUtensorMap tm_w, const SkinnyPa
         State a = qpart[threadIdx.x];
         for (int q = 1; q < 4; ++q) state_merge(a, qpart[q * N + threadIdx.x]);
         p.partials[(size_t)blockIdx.x * N + threadIdx.x] = a;
-        __threadfence();
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int old = atomicAdd(&p.ctrl->ticket, 1u);
-        s_is_last = (old == gridDim.x - 1);
-    }
+    if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(p.ctrl, gridDim.x);
     __syncthreads();
     if (!s_is_last) return;
 
-    // Last CTA: pull all partials into shared memory (ring and y are free by now), merge per token, decide.
-    __threadfence();
-    const int n_part = (int)gridDim.x * N;
-    State* part_s = reinterpret_cast<State*>(smem);
-    const bool via_smem = (size_t)n_part * sizeof(State) <= (size_t)S * kStageBytes + (size_t)p.k_blocks * N * 128;
-    if (via_smem) {
-        for (int i = threadIdx.x; i < n_part; i += kSkThreads) part_s[i] = state_load_cg(p.partials + i);
-        __syncthreads();
-    }
-    for (int tok = warp; tok < p.M; tok += kSkWarps) {
-        State a = state_empty();
-        for (int b = lane; b < (int)gridDim.x; b += 32) {
-            const State o = via_smem ? part_s[b * N + tok] : state_load_cg(p.partials + (size_t)b * N + tok);
-            state_merge(a, o);
-        }
-#pragma unroll
-        for (int msk = 1; msk <= 16; msk <<= 1) {
-            const State o = state_shfl_xor(a, msk);
-            state_merge(a, o);
-        }
-        if (lane == 0) {
-            const float tau = p.tau_per_row ? p.tau_per_row[tok] : p.tau;
-            state_finish(a, tau, p.argmax, p.entropy, p.maxprob, p.exit_mask, tok);
-        }
-    }
+    // Last CTA: merge the partials of all CTAs and decide (ring and y are free by now and serve as scratch).
+    merge_partials_and_decide<kSkThreads>(p.partials, (int)gridDim.x, N, p.M, reinterpret_cast<State*>(smem),
+                                          (size_t)S * kStageBytes + (size_t)p.k_blocks * N * 128, p.tau_per_row, p.tau,
+                                          p.argmax, p.entropy, p.maxprob, p.exit_mask);
     if (threadIdx.x == 0) p.ctrl->ticket = 0;                     // ready for the next call
 }
 
@@ -423,7 +415,7 @@ ee_status skinny_launch(const HeadArgs& a) {
     // so that the last tile of a CTA reaches at most a few rows into its neighbour's range.
     const int rows_max = (a.V + grid - 1) / grid;
     const int tiles = (rows_max + kTileRows - 1) / kTileRows;
-    int box = ((rows_max + tiles - 1) / tiles + 7) / 8 * 8;
+    int box = (rows_max + tiles - 1) / tiles;
     if (box > kTileRows) box = kTileRows;
     p.box_rows = box;
     p.n_stages = skinny_stages(n, a.d);

@@ -112,6 +112,24 @@ __device__ void layer_norm_in_smem(const StreamParams& p, __nv_bfloat16* y_s, co
     const int nvec = p.d >> 3;                                   // 16-byte vectors per row
     const int svec = p.y_stride >> 3;
     const float inv_d = 1.f / (float)p.d;
+    auto vec = [&](int r, int c) { return reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c; };
+    if (nvec <= 256) {
+        // Rows held in registers: one pass over shared memory, two rows at a time.
+        for (int i = 0; i < NT; i += 2) {
+            const int rows[2] = {warp + i * kWarps, warp + (i + 1) * kWarps};
+            const int live = (rows[0] < p.M) + (i + 1 < NT && rows[1] < p.M);
+            if (live == 0) break;
+            if (nvec <= 128) layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+            else layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+        }
+#pragma unroll
+        for (int i = 0; i < NT; ++i) {
+            const int r = warp + i * kWarps;
+            uint4* yrow = vec(r, 0);
+            for (int c = (r < p.M ? nvec : 0) + lane; c < svec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < NT; ++i) {
         const int r = warp + i * kWarps;
@@ -348,43 +366,16 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         State a = wpart[threadIdx.x];
         for (int w = 1; w < kWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
         p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = a;
-        __threadfence();
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int old = atomicAdd(&p.ctrl->ticket, 1u);
-        s_is_last = (old == gridDim.x - 1);
-    }
+    if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(p.ctrl, gridDim.x);
     __syncthreads();
     if (!s_is_last) return;
 
-    // Last CTA: merge the partials of all CTAs and decide.  The partials are first pulled into shared memory
-    // with independent, coalesced loads (the ring is free by now); then one warp per token merges them
-    // (lane-strided over the CTAs, then a butterfly).
-    __threadfence();
-    const int n_part = (int)gridDim.x * MPAD;
-    const bool via_smem = (size_t)n_part * sizeof(State) <= (size_t)p.n_stages * stage_bytes;
-    State* part_s = reinterpret_cast<State*>(ring);
-    if (via_smem) {
-        for (int i = threadIdx.x; i < n_part; i += kThreads) part_s[i] = state_load_cg(p.partials + i);
-        __syncthreads();
-    }
-    for (int tok = warp; tok < p.M; tok += kWarps) {
-        State a = state_empty();
-        for (int b = lane; b < (int)gridDim.x; b += 32) {
-            const State o = via_smem ? part_s[b * MPAD + tok] : state_load_cg(p.partials + (size_t)b * MPAD + tok);
-            state_merge(a, o);
-        }
-#pragma unroll
-        for (int msk = 1; msk <= 16; msk <<= 1) {
-            const State o = state_shfl_xor(a, msk);
-            state_merge(a, o);
-        }
-        if (lane == 0) {
-            const float tau = p.tau_per_row ? p.tau_per_row[tok] : p.tau;
-            state_finish(a, tau, p.argmax, p.entropy, p.maxprob, p.exit_mask, tok);
-        }
-    }
+    // Last CTA: merge the partials of all CTAs and decide (the ring is free by now and serves as scratch).
+    merge_partials_and_decide<kThreads>(p.partials, (int)gridDim.x, MPAD, p.M, reinterpret_cast<State*>(ring),
+                                        (size_t)p.n_stages * stage_bytes, p.tau_per_row, p.tau, p.argmax, p.entropy,
+                                        p.maxprob, p.exit_mask);
     if (threadIdx.x == 0) p.ctrl->ticket = 0;                     // ready for the next call
 }
 
