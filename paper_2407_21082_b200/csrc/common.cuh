@@ -103,7 +103,9 @@ struct Control {
     unsigned int ticket;      // completion counter of the streaming kernel; returns to 0 after every call
     unsigned int error;       // 0, or a code recorded by a bounded wait that gave up
     unsigned int error_info;  // where it gave up (role << 24 | stage << 16 | low bits of the tile index)
-    unsigned int pad[61];
+    unsigned int pad0;
+    unsigned int head_ticket[8];   // completion counters of the heads of a multi-head launch; return to 0 as well
+    unsigned int pad[52];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -227,27 +229,19 @@ __device__ __forceinline__ void layer_norm_rows_in_regs(VecFn vec, const int (&r
 // ---------------------------------------------------------------------------------------------
 // Thread 0 of a CTA, after a CTA-wide barrier that follows the CTA's partial-state stores: one acquire-release
 // atomic publishes those stores and tells whether every other CTA has published before.
-__device__ __forceinline__ bool ticket_arrive_is_last(Control* ctrl, unsigned int n_cta) {
+__device__ __forceinline__ bool ticket_arrive_is_last(unsigned int* counter, unsigned int n_cta) {
     unsigned int old;
-    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&ctrl->ticket) : "memory");
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
     return old == n_cta - 1;
 }
 
-// Every thread of the last CTA: merge partials [n_cta][np] per token (lane-strided over the CTAs, then a
-// butterfly; four tokens per warp at a time so that their chains overlap) and write the outputs.  `scratch`
-// is shared memory the partials are first copied to with independent loads, if it is large enough.
-template <int THREADS>
-__device__ void merge_partials_and_decide(const State* partials, int n_cta, int np, int M, State* scratch,
-                                          size_t scratch_bytes, const float* tau_per_row, float tau, int* argmax,
-                                          float* entropy, float* maxprob, unsigned char* exit_mask) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_part = n_cta * np;
-    const bool via_smem = (size_t)n_part * sizeof(State) <= scratch_bytes;
-    if (via_smem) {
-        for (int i = threadIdx.x; i < n_part; i += THREADS) scratch[i] = state_load_cg(partials + i);
-        __syncthreads();
-    }
-    for (int tok0 = warp * 4; tok0 < M; tok0 += (THREADS / 32) * 4) {
+// The threads of the last CTA that take part (n_warps whole warps, this one being number `warp`): merge
+// partials [n_cta][np] per token (lane-strided over the CTAs, then a butterfly; four tokens per warp at a time
+// so that their chains overlap) and write the outputs.
+__device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem, int n_cta, int np, int M, int warp,
+                                             int n_warps, int lane, const float* tau_per_row, float tau, int* argmax,
+                                             float* entropy, float* maxprob, unsigned char* exit_mask) {
+    for (int tok0 = warp * 4; tok0 < M; tok0 += n_warps * 4) {
         State a[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) a[q] = state_empty();
@@ -256,7 +250,7 @@ __device__ void merge_partials_and_decide(const State* partials, int n_cta, int 
             for (int q = 0; q < 4; ++q)
                 if (tok0 + q < M) {
                     const size_t i = (size_t)b * np + tok0 + q;
-                    const State o = via_smem ? scratch[i] : state_load_cg(partials + i);
+                    const State o = src_is_smem ? src[i] : state_load_cg(src + i);
                     state_merge(a[q], o);
                 }
         }
@@ -277,6 +271,22 @@ __device__ void merge_partials_and_decide(const State* partials, int n_cta, int 
             state_finish(mine, tau_per_row ? tau_per_row[tok] : tau, argmax, entropy, maxprob, exit_mask, tok);
         }
     }
+}
+
+// Whole-CTA variant: `scratch` is shared memory the partials are first copied to with independent loads, if it
+// is large enough.
+template <int THREADS>
+__device__ void merge_partials_and_decide(const State* partials, int n_cta, int np, int M, State* scratch,
+                                          size_t scratch_bytes, const float* tau_per_row, float tau, int* argmax,
+                                          float* entropy, float* maxprob, unsigned char* exit_mask) {
+    const int n_part = n_cta * np;
+    const bool via_smem = (size_t)n_part * sizeof(State) <= scratch_bytes;
+    if (via_smem) {
+        for (int i = threadIdx.x; i < n_part; i += THREADS) scratch[i] = state_load_cg(partials + i);
+        __syncthreads();
+    }
+    merge_tokens(via_smem ? scratch : partials, via_smem, n_cta, np, M, threadIdx.x >> 5, THREADS / 32, threadIdx.x & 31,
+                 tau_per_row, tau, argmax, entropy, maxprob, exit_mask);
 }
 
 }  // namespace ee

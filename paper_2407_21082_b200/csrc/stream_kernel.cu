@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = a;
     }
     __syncthreads();
-    if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(p.ctrl, gridDim.x);
+    if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(&p.ctrl->ticket, gridDim.x);
     __syncthreads();
     if (!s_is_last) return;
 
