@@ -88,6 +88,32 @@ ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const 
                        int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Several heads on batches of the same shape in one call -- what the calibration pass of section 3.4.1 does
+ * (every head is evaluated on every token of the calibration set) and what a verify step with several
+ * heads does.  Equivalent to n_heads calls of ee_exit_head with the same M, d, V, ln_eps and workspace; when
+ * the sizes allow (M <= 64, d % 64 == 0) up to four heads share one kernel launch, which keeps the weight
+ * stream going across the per-head LayerNorm and merge steps.  `heads` is a HOST array read during the call;
+ * the pointers inside follow the rules of ee_exit_head (each head has its own h, LayerNorm parameters, W,
+ * thresholds and outputs; h may be the same for all).  Workspace: ee_exit_head_multi_workspace_bytes().
+ */
+typedef struct {
+    const void* h;             /* bf16 [M, d], row stride ld_h */
+    long long ld_h;
+    const float* gamma;        /* fp32 [d] */
+    const float* beta;         /* fp32 [d] */
+    const void* W;             /* bf16 [V, d] */
+    const float* tau_per_row;  /* fp32 [M] or NULL */
+    float tau;
+    int* argmax;               /* int32 [M] */
+    float* entropy;            /* fp32 [M] */
+    float* maxprob;            /* fp32 [M] */
+    unsigned char* exit_mask;  /* uint8 [M] */
+} ee_head;
+size_t    ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V);
+ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
 /* Same operation with the kernel chosen by the caller (`path` is an ee_path); used to cross-check the
  * kernels against each other and to time them separately. */
 ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,

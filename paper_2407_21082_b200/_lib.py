@@ -9,6 +9,14 @@ from . import build as _build
 _LIB = None
 
 _p = C.c_void_p
+
+
+class EEHead(C.Structure):
+    """Mirror of `ee_head` in include/eexit.h."""
+    _fields_ = [("h", _p), ("ld_h", C.c_longlong), ("gamma", _p), ("beta", _p), ("W", _p), ("tau_per_row", _p),
+                ("tau", C.c_float), ("argmax", _p), ("entropy", _p), ("maxprob", _p), ("exit_mask", _p)]
+
+
 PROTOTYPES = {
     "ee_status_string": (C.c_char_p, [C.c_int]),
     "ee_exit_head_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
@@ -16,6 +24,8 @@ PROTOTYPES = {
     "ee_workspace_init": (C.c_int, [_p, C.c_size_t, _p]),
     "ee_exit_head": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_exit_head_multi_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
+    "ee_exit_head_multi": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, _p, C.c_size_t, _p]),
     "ee_exit_head_path": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                     _p, _p, _p, _p, _p, C.c_size_t, _p, C.c_int]),
     "ee_exit_head_host": (C.c_int, [_p, _p, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,

@@ -124,6 +124,59 @@ class PreparedCall:
         return self.out
 
 
+def ee_exit_head_multi_workspace_bytes(n_heads: int, M: int, d: int, V: int) -> int:
+    return int(_lib.load().ee_exit_head_multi_workspace_bytes(int(n_heads), int(M), int(d), int(V)))
+
+
+def _multi_args(heads, ln_eps, workspace):
+    """heads: list of dicts with h, gamma, beta, W, tau and optionally out (see new_outputs)."""
+    n = len(heads)
+    arr = (_lib.EEHead * n)()
+    keep, outs = [], []
+    M, d = _bf16(heads[0]["h"]).shape
+    V = heads[0]["W"].shape[0]
+    for i, hd in enumerate(heads):
+        h, W = _bf16(_dev(hd["h"], "h")), _bf16(_dev(hd["W"], "W"))
+        if h.shape != (M, d) or W.shape != (V, d) or not W.is_contiguous() or h.stride(1) != 1:
+            raise ValueError("all heads must share M, d, V; W contiguous [V, d]; h row-major [M, d]")
+        out = hd.get("out") or new_outputs(M, h.device)
+        tau = hd["tau"]
+        tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+        e = arr[i]
+        e.h, e.ld_h, e.gamma, e.beta, e.W = _ptr(h), (h.stride(0) if M > 1 else max(h.stride(0), d)), _ptr(hd["gamma"]), _ptr(hd["beta"]), _ptr(W)
+        e.tau_per_row, e.tau = _ptr(tau_t), tau_f
+        e.argmax, e.entropy, e.maxprob, e.exit_mask = (_ptr(out[k]) for k in ("argmax", "entropy", "maxprob", "exit_mask"))
+        keep.append((h, W, hd["gamma"], hd["beta"], tau_t, out))
+        outs.append(out)
+    if workspace is None:
+        nbytes = ee_exit_head_multi_workspace_bytes(n, M, d, V)
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=heads[0]["h"].device)
+        ee_workspace_init(workspace)
+    args = (arr, n, float(ln_eps), M, d, V, _ptr(workspace), workspace.numel(), _stream())
+    return args, outs, (arr, keep, workspace)
+
+
+def ee_exit_head_multi(heads, ln_eps, *, workspace=None) -> list:
+    """ee_exit_head for several heads on batches of the same shape in one call; returns one output dict per head."""
+    args, outs, _ = _multi_args(heads, ln_eps, workspace)
+    _check(_lib.load().ee_exit_head_multi(*args), "ee_exit_head_multi")
+    return outs
+
+
+class PreparedMulti:
+    """ee_exit_head_multi with its argument block built once (see PreparedCall)."""
+    __slots__ = ("_args", "_keep", "out")
+
+    def __init__(self, heads, ln_eps, workspace=None):
+        self._args, self.out, self._keep = _multi_args(heads, ln_eps, workspace)
+
+    def __call__(self):
+        code = _lib.load().ee_exit_head_multi(*self._args)
+        if code:
+            raise EExitError(code, "ee_exit_head_multi")
+        return self.out
+
+
 def prepare_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> PreparedCall:
     """ee_exit_head with the arguments marshalled once; see PreparedCall."""
     args, out, keep = _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path)

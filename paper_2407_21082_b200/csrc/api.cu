@@ -48,7 +48,7 @@ size_t workspace_bytes(int M, int d, int V) {
     size_t need = gemm_workspace_bytes(M, d, V);
     const size_t s = stream_workspace_bytes(M, d, V);
     if (s > need) need = s;
-    if (skinny_workspace_bytes() > need) need = skinny_workspace_bytes();
+    if (skinny_workspace_bytes(1) > need) need = skinny_workspace_bytes(1);
     return kCtrlBytes + need;
 }
 
@@ -121,8 +121,58 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
 
     if (path == EE_PATH_AUTO) path = auto_path(M, d);
     if (path == EE_PATH_STREAM) return stream_launch(a);
-    if (path == EE_PATH_SKINNY) return skinny_launch(a);
+    if (path == EE_PATH_SKINNY) return skinny_launch(&a, 1);
     return gemm_launch(a);
+}
+
+size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
+    if (!sizes_ok(M, d, V) || n_heads < 1) return 0;
+    size_t need = workspace_bytes(M, d, V);
+    const int per_launch = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
+    if (kCtrlBytes + skinny_workspace_bytes(per_launch) > need) need = kCtrlBytes + skinny_workspace_bytes(per_launch);
+    return need;
+}
+
+ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, void* workspace,
+                             size_t workspace_bytes_, void* stream) {
+    if (!sizes_ok(M, d, V) || n_heads < 0) return EE_ERR_SHAPE;
+    if (n_heads == 0 || M == 0) return EE_OK;
+    if (!heads || !workspace) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < ee_exit_head_multi_workspace_bytes(n_heads, M, d, V)) return EE_ERR_WORKSPACE;
+    for (int k = 0; k < n_heads; ++k) {
+        const ee_head& e = heads[k];
+        if (!e.h || !e.gamma || !e.beta || !e.W || !e.argmax || !e.entropy || !e.maxprob || !e.exit_mask) return EE_ERR_NULL;
+        if (e.ld_h < d || (e.ld_h % 8) != 0) return EE_ERR_SHAPE;
+        if (!aligned(e.h, 16) || !aligned(e.W, 16) || !aligned(e.gamma, 16) || !aligned(e.beta, 16)) return EE_ERR_ALIGN;
+    }
+    HeadArgs base;
+    const ee_status dev = current_device(&base.device, &base.num_sms);
+    if (dev != EE_OK) return dev;
+    const bool batched = skinny_supports(M, d) && auto_path(M, d) == EE_PATH_SKINNY;
+    for (int k0 = 0; k0 < n_heads; k0 += kSkinnyMaxHeads) {
+        HeadArgs a[kSkinnyMaxHeads];
+        const int n = n_heads - k0 < kSkinnyMaxHeads ? n_heads - k0 : kSkinnyMaxHeads;
+        for (int k = 0; k < n; ++k) {
+            const ee_head& e = heads[k0 + k];
+            a[k] = base;
+            a[k].h = e.h; a[k].ld_h = e.ld_h; a[k].gamma = e.gamma; a[k].beta = e.beta; a[k].ln_eps = ln_eps; a[k].W = e.W;
+            a[k].M = M; a[k].d = d; a[k].V = V; a[k].tau_per_row = e.tau_per_row; a[k].tau = e.tau;
+            a[k].argmax = e.argmax; a[k].entropy = e.entropy; a[k].maxprob = e.maxprob; a[k].exit_mask = e.exit_mask;
+            a[k].workspace = workspace; a[k].workspace_bytes = workspace_bytes_;
+            a[k].stream = static_cast<cudaStream_t>(stream);
+        }
+        if (batched) {
+            const ee_status st = skinny_launch(a, n);
+            if (st != EE_OK) return st;
+        } else {
+            for (int k = 0; k < n; ++k) {
+                const ee_status st = auto_path(M, d) == EE_PATH_STREAM ? stream_launch(a[k]) : gemm_launch(a[k]);
+                if (st != EE_OK) return st;
+            }
+        }
+    }
+    return EE_OK;
 }
 
 ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,

@@ -38,11 +38,15 @@ int stream_slab_rows(int d);               // rows one launch can take for this 
 size_t stream_workspace_bytes(int M, int d, int V);
 ee_status stream_launch(const HeadArgs& a);
 
-// ---- skinny tensor-core kernel (one launch, weights as the MMA's M operand, 1 <= M <= 64, d % 64 == 0) ----
+// ---- skinny tensor-core kernel (one launch for up to four heads, weights as the MMA's M operand,
+//      1 <= M <= 64, d % 64 == 0) ----
 constexpr int kSkinnyMaxRows = 64;
+constexpr int kSkinnyMaxHeads = 4;
 bool skinny_supports(int M, int d);
-size_t skinny_workspace_bytes();
-ee_status skinny_launch(const HeadArgs& a);
+size_t skinny_workspace_bytes(int n_heads);
+// heads[0 .. n_heads) share M, d, V, ln_eps, workspace, stream and device; each has its own h, LayerNorm
+// parameters, W, thresholds and outputs.
+ee_status skinny_launch(const HeadArgs* heads, int n_heads);
 
 // ---- tensor-core kernel (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge) ----
 int gemm_tile_n(int M);                    // vocabulary tile width used for M rows

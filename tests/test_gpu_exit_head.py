@@ -198,3 +198,43 @@ def test_device_side_argument_errors(ee):
     with pytest.raises(ee.EExitError) as e:
         ee.ee_exit_head(dev_bf16(odd["h"]), ohd["gamma"], ohd["beta"], 1e-5, ohd["W"], 1.0, path=ee.EE_PATH_SKINNY)
     assert e.value.code == 2
+
+
+@pytest.mark.parametrize("name,M,d,V,n_heads", [
+    ("c1_shape_small_v", 8, 1024, 3000, 3),       # two activation buffers
+    ("n32_two_launches", 20, 256, 2111, 5),       # five heads: a launch of four and a launch of one
+    ("n64_single_buffer", 64, 1024, 1200, 3),     # activations too large for a second buffer
+    ("wide_single_buffer", 12, 2560, 900, 2),
+    ("not_batched", 40, 72, 500, 3),              # d % 64 != 0: falls back to one launch per head
+])
+def test_multi_head_call_matches_oracle(ee, name, M, d, V, n_heads):
+    cfg = gen.make_config("c1", seed=17, planted=True, M=M, d=d, V=V, heads=n_heads)
+    h = dev_bf16(cfg["h"])
+    taus = [0.5 + 0.5 * k for k in range(n_heads)]
+    heads = []
+    for k in range(n_heads):
+        hd = head_to_dev(cfg["heads"][k])
+        heads.append(dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=taus[k]))
+    outs = ee.ee_exit_head_multi(heads, 1e-5)
+    torch.cuda.synchronize()
+    again = ee.ee_exit_head_multi(heads, 1e-5)
+    torch.cuda.synchronize()
+    for k in range(n_heads):
+        ref = oracle_head(cfg["h"], cfg["heads"][k], taus[k])
+        assert_head_matches(outs[k], ref, label=f"{name} head {k}")
+        for key in outs[k]:
+            assert torch.equal(outs[k][key], again[k][key]), (name, k, key)
+
+
+def test_multi_head_full_size_c1(ee):
+    cfg = gen.make_config("c1", seed=0, planted=True)
+    for M in (1, 16, 64):
+        h = dev_bf16(cfg["h"][:M])
+        heads = []
+        for k in range(3):
+            hd = head_to_dev(cfg["heads"][k])
+            heads.append(dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=cfg["tau"]))
+        outs = ee.ee_exit_head_multi(heads, 1e-5)
+        for k in range(3):
+            ref = oracle_head(cfg["h"][:M], cfg["heads"][k], cfg["tau"])
+            assert_head_matches(outs[k], ref, label=f"c1 multi M={M} head {k}")
