@@ -149,7 +149,7 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     HeadArgs base;
     const ee_status dev = current_device(&base.device, &base.num_sms);
     if (dev != EE_OK) return dev;
-    const bool batched = skinny_supports(M, d) && auto_path(M, d) == EE_PATH_SKINNY;
+    const bool batched = skinny_supports(M, d);
     for (int k0 = 0; k0 < n_heads; k0 += kSkinnyMaxHeads) {
         HeadArgs a[kSkinnyMaxHeads];
         const int n = n_heads - k0 < kSkinnyMaxHeads ? n_heads - k0 : kSkinnyMaxHeads;
