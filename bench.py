@@ -107,11 +107,12 @@ def _algorithmic(M, d, V):
 class Workload:
     """Device tensors of one workload and a `step()` that runs the whole hot path once."""
 
-    def __init__(self, name: str, M: int | None, seed: int, n_copies: int, path: int = 0):
+    def __init__(self, name: str, M: int | None, seed: int, n_copies: int, path: int = 0, multi: bool = True):
         import torch
         import paper_2407_21082_b200 as ee
         self.torch, self.ee = torch, ee
         self.path = path
+        self.multi = multi and path == 0
         cfg = gen.make_config(name, seed=seed, planted=False, M=M)
         self.name, self.cfg = name, cfg
         self.M, self.d, self.V = cfg["M"], cfg["d"], cfg["V"]
@@ -133,7 +134,11 @@ class Workload:
             self.k = 8
             self.S = self.M // self.k
         self.tau = torch.from_numpy(cfg["tau_per_row"]).cuda() if "tau_per_row" in cfg else float(cfg["tau"])
-        self.ws = ee.new_workspace(self.M, self.d, self.V)
+        self.multi = self.multi and len(self.heads) > 1 and len({hh.data_ptr() for hh in self.h}) >= 1
+        ws_bytes = max(ee.ee_exit_head_workspace_bytes(self.M, self.d, self.V),
+                       ee.ee_exit_head_multi_workspace_bytes(len(self.heads), self.M, self.d, self.V))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        ee.ee_workspace_init(self.ws)
         self.outs = [ee.new_outputs(self.M) for _ in self.heads]
         self.comp = dict(kept_idx=torch.empty(self.M, dtype=torch.int32, device="cuda"),
                          kept_count=torch.zeros(1, dtype=torch.int32, device="cuda"),
@@ -142,7 +147,9 @@ class Workload:
         self.calls = 0
         self.n_copies = n_copies
         self.head_launches = ee.ee_exit_head_launches(self.M, self.d, self.V, path)
-        self.launches_per_step = len(self.heads) * self.head_launches + 1 + (1 if self.S > 0 else 0)
+        heads_launches = (ee.ee_exit_head_multi_launches(len(self.heads), self.M, self.d, self.V) if self.multi
+                          else len(self.heads) * self.head_launches)
+        self.launches_per_step = heads_launches + 1 + (1 if self.S > 0 else 0)
         self.bytes_per_call, self.flops_per_call = _algorithmic(self.M, self.d, self.V)
         self.w_bytes_total = sum(w.numel() * 2 for hd in self.heads for w in hd["W"])
         self.prepare()
@@ -150,9 +157,14 @@ class Workload:
     def prepare(self):
         """Marshals every call of a step once (the binding's PreparedCall), so the loop is a few C calls."""
         ee = self.ee
-        self.head_calls = [[ee.prepare_exit_head(self.h[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], self.tau,
-                                                 out=self.outs[i], workspace=self.ws, path=self.path)
-                            for i, hd in enumerate(self.heads)] for c in range(self.n_copies)]
+        if self.multi:       # all heads of the step in one call
+            self.head_calls = [[ee.PreparedMulti([dict(h=self.h[i], gamma=hd["gamma"], beta=hd["beta"], W=hd["W"][c],
+                                                       tau=self.tau, out=self.outs[i]) for i, hd in enumerate(self.heads)],
+                                                 1e-5, self.ws)] for c in range(self.n_copies)]
+        else:
+            self.head_calls = [[ee.prepare_exit_head(self.h[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], self.tau,
+                                                     out=self.outs[i], workspace=self.ws, path=self.path)
+                                for i, hd in enumerate(self.heads)] for c in range(self.n_copies)]
         self.compact_call = ee.prepare_compact(self.outs[0]["exit_mask"], self.h[0], out=self.comp)
         self.accept_call = None
         if self.S > 0:
@@ -382,8 +394,10 @@ def main():
                 data="synthetic", config=config, clocks=res["clocks"], gpu_launches=wl.launches_per_step * args.steps,
                 head_call_us=res["head_call_us"], tail_us=res["tail_us"])
     line["roofline"] = roofline(wl, res["head_call_us"], peaks, peak_src)
-    line["roofline"]["kernel"] = ("one ee_exit_head call (%d launch(es)); duration = CUDA events around the %d head calls of "
-                                  "each step, averaged" % (wl.head_launches, n_heads))
+    line["roofline"]["kernel"] = (("ee_exit_head_multi: %d heads in one launch; " % n_heads if wl.multi else
+                                   "one ee_exit_head call (%d launch(es)); " % wl.head_launches) +
+                                  "duration = CUDA events around the head evaluations of each step, averaged per head")
+    config["heads_call"] = "ee_exit_head_multi" if wl.multi else "ee_exit_head per head"
     if rank == 0:
         line["e2e"] = measure_e2e(wl, max(10, args.steps // 4), 3)
         if world > 1:
@@ -407,8 +421,12 @@ def main():
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):
+                w = Workload("c1", rows, seed=0, n_copies=2)
+                sweep[f"c1_M{rows}_multi"] = round(measure(w, 300, 5)["head_call_us"], 2)
+                del w
+                torch.cuda.empty_cache()
                 for pname, pid in (("stream", 1), ("skinny", 3), ("tcgen05", 2)):
-                    w = Workload("c1", rows, seed=0, n_copies=2, path=pid)
+                    w = Workload("c1", rows, seed=0, n_copies=2, path=pid, multi=False)
                     if w.head_launches == 0:
                         continue
                     r = measure(w, 300, 5)

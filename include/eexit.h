@@ -111,6 +111,7 @@ typedef struct {
     unsigned char* exit_mask;  /* uint8 [M] */
 } ee_head;
 size_t    ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V);
+int       ee_exit_head_multi_launches(int n_heads, int M, int d, int V);   /* kernels one call launches; host-only */
 ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
                              void* workspace, size_t workspace_bytes, void* stream);
 

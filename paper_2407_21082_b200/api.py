@@ -128,6 +128,10 @@ def ee_exit_head_multi_workspace_bytes(n_heads: int, M: int, d: int, V: int) -> 
     return int(_lib.load().ee_exit_head_multi_workspace_bytes(int(n_heads), int(M), int(d), int(V)))
 
 
+def ee_exit_head_multi_launches(n_heads: int, M: int, d: int, V: int) -> int:
+    return int(_lib.load().ee_exit_head_multi_launches(int(n_heads), int(M), int(d), int(V)))
+
+
 def _multi_args(heads, ln_eps, workspace):
     """heads: list of dicts with h, gamma, beta, W, tau and optionally out (see new_outputs)."""
     n = len(heads)

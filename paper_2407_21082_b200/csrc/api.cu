@@ -133,6 +133,12 @@ size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
     return need;
 }
 
+int ee_exit_head_multi_launches(int n_heads, int M, int d, int V) {
+    if (!sizes_ok(M, d, V) || n_heads < 1 || M == 0) return 0;
+    if (skinny_supports(M, d)) return (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
+    return n_heads * ee_exit_head_launches(M, d, V, EE_PATH_AUTO);
+}
+
 ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, void* workspace,
                              size_t workspace_bytes_, void* stream) {
     if (!sizes_ok(M, d, V) || n_heads < 0) return EE_ERR_SHAPE;
