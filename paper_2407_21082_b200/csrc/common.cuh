@@ -86,6 +86,49 @@ __device__ __forceinline__ State state_load_cg(const State* p) {
     return o;
 }
 
+// Merge of C states held by one thread, and of one state per lane across the lanes that differ in the bits
+// LO, 2*LO, .., HI of the lane index.  Unlike a chain of state_merge calls these take the maximum first and
+// then add the rescaled sums, so the work per state is independent of the others (and pipelines) and the
+// cross-lane part is plain shuffles of scalars.  The result is bitwise identical in every participating lane.
+template <int C>
+__device__ __forceinline__ State state_combine(const State (&v)[C]) {
+    float m = -CUDART_INF_F;
+#pragma unroll
+    for (int c = 0; c < C; ++c) m = fmaxf(m, v[c].m);
+    float s = 0.f, t = 0.f;
+    int idx = 0x7fffffff;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const bool live = !(v[c].s == 0.f);                        // NaN counts as live and propagates
+        const float dl = v[c].m - m;
+        const float al = live ? ex2(dl * kLog2e) : 0.f;
+        s += live ? al * v[c].s : 0.f;
+        t += live ? al * fmaf(dl, v[c].s, v[c].t) : 0.f;
+        idx = (live && v[c].m == m) ? min(idx, v[c].idx) : idx;
+    }
+    return State{(s == 0.f) ? -CUDART_INF_F : m, s, t, idx};
+}
+
+template <int LO, int HI>
+__device__ __forceinline__ State state_reduce_lanes(const State& a) {
+    float m = a.m;
+#pragma unroll
+    for (int msk = LO; msk <= HI; msk <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, msk));
+    const bool live = !(a.s == 0.f);
+    const float dl = a.m - m;
+    const float al = live ? ex2(dl * kLog2e) : 0.f;
+    float s = live ? al * a.s : 0.f;
+    float t = live ? al * fmaf(dl, a.s, a.t) : 0.f;
+    int idx = (live && a.m == m) ? a.idx : 0x7fffffff;
+#pragma unroll
+    for (int msk = LO; msk <= HI; msk <<= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, msk);
+        t += __shfl_xor_sync(0xffffffffu, t, msk);
+        idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, msk));
+    }
+    return State{(s == 0.f) ? -CUDART_INF_F : m, s, t, idx};
+}
+
 // Final statistics of a full-vocabulary state, and the exit decision.
 __device__ __forceinline__ void state_finish(const State& a, float tau, int* argmax, float* entropy,
                                              float* maxprob, unsigned char* exit_mask, int row) {
@@ -236,37 +279,34 @@ __device__ __forceinline__ bool ticket_arrive_is_last(unsigned int* counter, uns
 }
 
 // The threads of the last CTA that take part (n_warps whole warps, this one being number `warp`): merge
-// partials [n_cta][np] per token (lane-strided over the CTAs, then a butterfly; four tokens per warp at a time
-// so that their chains overlap) and write the outputs.
+// partials [n_cta][np] per token and write the outputs.  A warp takes four tokens at a time; every lane first
+// loads all the states it is responsible for (CTAs lane, lane + 32, ..; at most 256 CTAs), so the loads are
+// one round trip, then combines them and the lanes reduce.
 __device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem, int n_cta, int np, int M, int warp,
                                              int n_warps, int lane, const float* tau_per_row, float tau, int* argmax,
                                              float* entropy, float* maxprob, unsigned char* exit_mask) {
     for (int tok0 = warp * 4; tok0 < M; tok0 += n_warps * 4) {
-        State a[4];
+        State v[4][8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) a[q] = state_empty();
-        for (int b = lane; b < n_cta; b += 32) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (tok0 + q < M) {
-                    const size_t i = (size_t)b * np + tok0 + q;
-                    const State o = src_is_smem ? src[i] : state_load_cg(src + i);
-                    state_merge(a[q], o);
-                }
-        }
-#pragma unroll
-        for (int msk = 1; msk <= 16; msk <<= 1) {
+        for (int i = 0; i < 8; ++i) {
+            const int b = lane + 32 * i;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const State o = state_shfl_xor(a[q], msk);
-                state_merge(a[q], o);
+                v[q][i] = state_empty();
+                if (b < n_cta && tok0 + q < M) {
+                    const size_t at = (size_t)b * np + tok0 + q;
+                    v[q][i] = src_is_smem ? src[at] : state_load_cg(src + at);
+                }
             }
         }
+        State r[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) r[q] = state_reduce_lanes<1, 16>(state_combine<8>(v[q]));
         if (lane < 4 && tok0 + lane < M) {
-            State mine = a[0];
+            State mine = r[0];
 #pragma unroll
             for (int q = 1; q < 4; ++q)
-                if (lane == q) mine = a[q];
+                if (lane == q) mine = r[q];
             const int tok = tok0 + lane;
             state_finish(mine, tau_per_row ? tau_per_row[tok] : tau, argmax, entropy, maxprob, exit_mask, tok);
         }

@@ -293,16 +293,18 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
-    State a = state_empty();
-    for (int n = lane; n < n_tiles; n += 32) {
-        const State o = state_load_cg(partials + (size_t)row * n_tiles + n);
-        state_merge(a, o);
-    }
+    // Lane-strided over the tiles, eight independent loads at a time; then the lanes reduce.
+    State v[9];
+    v[8] = state_empty();                                         // running result of this lane
+    for (int n0 = lane; n0 < n_tiles; n0 += 256) {
 #pragma unroll
-    for (int msk = 1; msk <= 16; msk <<= 1) {
-        const State o = state_shfl_xor(a, msk);
-        state_merge(a, o);
+        for (int i = 0; i < 8; ++i) {
+            const int n = n0 + 32 * i;
+            v[i] = n < n_tiles ? state_load_cg(partials + (size_t)row * n_tiles + n) : state_empty();
+        }
+        v[8] = state_combine<9>(v);
     }
+    const State a = state_reduce_lanes<1, 16>(v[8]);
     if (lane == 0) state_finish(a, tau_per_row ? tau_per_row[row] : tau, argmax, entropy, maxprob, exit_mask, row);
 }
 

@@ -144,32 +144,32 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
     constexpr int kSkWarps = kSkThreads / 32;
     constexpr int kEpiWarps = 4 * GROUPS;
     constexpr int kEpiThreads = 32 * kEpiWarps;
-    constexpr int TMEM_COLS = (2 * N < 32) ? 32 : 2 * N;
+    constexpr int ACC = 4;                                        // accumulator buffers in TMEM
+    constexpr int TMEM_COLS = ACC * N;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
     const int S = p.n_stages;
     const int y_bytes = p.k_blocks * N * 128;
-    // layout: W stages | y buffers | gamma, beta | per-quarter states | transposition buffers | barriers
+    // layout: W stages | y buffers | gamma, beta | per-quarter states | barriers
     unsigned char* y_all = smem + (size_t)S * p.stage_stride;
     float* gamma_s = reinterpret_cast<float*>(y_all + (size_t)p.y_bufs * y_bytes);
     float* beta_s = gamma_s + p.d;
     State* qpart = reinterpret_cast<State*>(beta_s + p.d);       // [4][N]
-    State* xbuf = qpart + 4 * N;                                  // [epilogue warp][2 tokens][32 lanes]
-    unsigned char* bar_mem = reinterpret_cast<unsigned char*>(xbuf + kEpiWarps * 64);
+    unsigned char* bar_mem = reinterpret_cast<unsigned char*>(qpart + 4 * N);
     const uint32_t w_base = ptx::smem_addr(smem);
     const uint32_t y_base = ptx::smem_addr(y_all);
     const uint32_t bar_base = ptx::smem_addr(bar_mem);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kSkMaxStages + s); };
     auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * kSkMaxStages + b); };
-    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * kSkMaxStages + 2 + b); };
-    const uint32_t drain_bar = bar_base + 8u * (2 * kSkMaxStages + 4);
-    auto yready_bar = [&](int b) { return bar_base + 8u * (2 * kSkMaxStages + 5 + b); };
-    const uint32_t epi_bar = bar_base + 8u * (2 * kSkMaxStages + 7);          // barrier among the epilogue threads
-    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_mem + 8 * (2 * kSkMaxStages + 8));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * kSkMaxStages + 8) + 4);
-    volatile int* last_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * kSkMaxStages + 9));
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * kSkMaxStages + 4 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * kSkMaxStages + 8);
+    auto yready_bar = [&](int b) { return bar_base + 8u * (2 * kSkMaxStages + 9 + b); };
+    const uint32_t epi_bar = bar_base + 8u * (2 * kSkMaxStages + 11);         // barrier among the epilogue threads
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_mem + 8 * (2 * kSkMaxStages + 12));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * kSkMaxStages + 12) + 4);
+    volatile int* last_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * kSkMaxStages + 13));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -179,11 +179,11 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
             ptx::mbar_init(full_bar(s), 1);
             ptx::mbar_init(empty_bar(s), 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < ACC; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
             ptx::mbar_init(tempty_bar(b), kEpiWarps);
-            ptx::mbar_init(yready_bar(b), kEpiWarps);
         }
+        for (int b = 0; b < 2; ++b) ptx::mbar_init(yready_bar(b), kEpiWarps);
         ptx::mbar_init(drain_bar, 1);
         ptx::mbar_init(epi_bar, kEpiThreads);
         *abort_flag = 0;
@@ -267,8 +267,8 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
                     }
                 }
                 for (int tile = 0; ok && tile < n_tiles; ++tile, ++t) {
-                    const int buf = t & 1;
-                    const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
+                    const int buf = t % ACC;
+                    const uint32_t acc_phase = (uint32_t)(t / ACC) & 1u;
                     if (!ptx::mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag)) {
                         if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
                             p.ctrl->error_info = (2u << 24) | (0x80u << 16) | ((unsigned)t & 0xffffu);
@@ -335,8 +335,8 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
 #pragma unroll
             for (int q = 0; q < TOK; ++q) own[q] = state_empty();
             for (int tile = 0; tile < n_tiles; ++tile, ++t) {
-                const int buf = t & 1;
-                const uint32_t acc_phase = (uint32_t)(t >> 1) & 1u;
+                const int buf = t % ACC;
+                const uint32_t acc_phase = (uint32_t)(t / ACC) & 1u;
                 const bool landed = ptx::mbar_wait(tfull_bar(buf), acc_phase, abort_flag);
                 if (!__all_sync(0xffffffffu, landed)) {
                     if (lane == 0) {
@@ -366,26 +366,11 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
                 if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
             }
             if (!ok) break;
-            // Cross-lane merge of this warp's states, two tokens at a time through a small transposition buffer:
-            // lane (q, s) merges rows 2s, 2s+1 of token q, then four shuffle steps over s.
-            {
-                State* xb = xbuf + ew * 64;
-                const int q = lane >> 4, s = lane & 15;
+            // Cross-lane reduction of this warp's states: per token a warp maximum, then sums of rescaled terms.
 #pragma unroll
-                for (int c = 0; c < TOK; c += 2) {
-                    xb[lane] = own[c];
-                    xb[32 + lane] = own[c + 1];
-                    __syncwarp();
-                    State a = xb[q * 32 + s * 2];
-                    state_merge(a, xb[q * 32 + s * 2 + 1]);
-#pragma unroll
-                    for (int msk = 1; msk <= 8; msk <<= 1) {
-                        const State o = state_shfl_xor(a, msk);
-                        state_merge(a, o);
-                    }
-                    if (s == 0) qpart[quarter * N + group * 32 + c + q] = a;
-                    __syncwarp();
-                }
+            for (int c = 0; c < TOK; ++c) {
+                const State a = state_reduce_lanes<1, 16>(own[c]);
+                if (lane == 0) qpart[quarter * N + group * 32 + c] = a;
             }
             // Head k's MMAs are complete.  With a single buffer the next head's activations are prepared now (the
             // per-thread states have just been handed over, which frees the registers LayerNorm needs).
@@ -399,9 +384,8 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
             // Merge the four quarters; publish the CTA partial of head k.
             State* part_k = p.partials + (size_t)k * gridDim.x * N;
             if (et < N) {
-                State a = qpart[et];
-                for (int qq = 1; qq < 4; ++qq) state_merge(a, qpart[qq * N + et]);
-                part_k[(size_t)blockIdx.x * N + et] = a;
+                const State four[4] = {qpart[et], qpart[N + et], qpart[2 * N + et], qpart[3 * N + et]};
+                part_k[(size_t)blockIdx.x * N + et] = state_combine<4>(four);
             }
             if (!(ok = epi_sync())) break;
             if (et == 0) *last_flag = ticket_arrive_is_last(&p.ctrl->head_ticket[k], gridDim.x) ? 1 : 0;
@@ -430,7 +414,7 @@ int pad_rows(int M) { return M <= 16 ? 16 : (M <= 32 ? 32 : 64); }
 // Shared-memory bytes besides the W ring, with `y_bufs` activation buffers.
 size_t skinny_fixed_bytes(int n, int d, int y_bufs) {
     return (size_t)y_bufs * n * d * 2 + (size_t)2 * d * sizeof(float) + (size_t)4 * n * sizeof(State) +
-           (size_t)4 * sk_groups(n) * 64 * sizeof(State) + (size_t)(2 * kSkMaxStages + 10) * 8 + 1024;
+           (size_t)(2 * kSkMaxStages + 16) * 8 + 1024;
 }
 
 int stage_stride_bytes(int box_rows) { return (box_rows * 128 + 1023) / 1024 * 1024; }

@@ -351,11 +351,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         for (int n = 0; n < NT; ++n)
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-#pragma unroll
-                for (int msk = 4; msk <= 16; msk <<= 1) {
-                    const State o = state_shfl_xor(st[n][e], msk);
-                    state_merge(st[n][e], o);
-                }
+                st[n][e] = state_reduce_lanes<4, 16>(st[n][e]);
                 if (g == 0) wpart[warp * MPAD + n * 8 + t * 2 + e] = st[n][e];
             }
     }
@@ -363,9 +359,10 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
 
     // Merge over the CTA's warps; publish the CTA partial.
     if (threadIdx.x < MPAD) {
-        State a = wpart[threadIdx.x];
-        for (int w = 1; w < kWarps; ++w) state_merge(a, wpart[w * MPAD + threadIdx.x]);
-        p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = a;
+        State all[kWarps];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) all[w] = wpart[w * MPAD + threadIdx.x];
+        p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = state_combine<kWarps>(all);
     }
     __syncthreads();
     if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(&p.ctrl->ticket, gridDim.x);
