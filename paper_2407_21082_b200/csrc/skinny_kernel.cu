@@ -491,7 +491,8 @@ ee_status skinny_launch(const HeadArgs* heads, int n_heads) {
         s.entropy = h.entropy;
         s.maxprob = h.maxprob;
         s.exit_mask = h.exit_mask;
-        if (!make_tile_map(&maps.w[k], h.W, a.V, a.d, box)) return EE_ERR_CUDA;
+        // W is streamed once, front to back: 256-byte promotion fetches the next k-block's half of the line pair too.
+        if (!make_tile_map(&maps.w[k], h.W, a.V, a.d, box, CU_TENSOR_MAP_L2_PROMOTION_L2_256B)) return EE_ERR_CUDA;
     }
     for (int k = n_heads; k < kSkinnyMaxHeads; ++k) {
         p.head[k] = p.head[0];

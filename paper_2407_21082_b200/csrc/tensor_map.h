@@ -25,7 +25,8 @@ inline EncodeTiledFn encode_tiled_fn() {
 }
 
 // bf16 matrix [rows, cols] row-major (row stride = cols), box = [box_rows x 64 columns], 128-byte swizzle.
-inline bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+inline bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols, int box_rows,
+                          CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_128B) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -33,7 +34,7 @@ inline bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols
     const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
