@@ -421,10 +421,13 @@ def main():
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):
-                w = Workload("c1", rows, seed=0, n_copies=2)
-                sweep[f"c1_M{rows}_multi"] = round(measure(w, 300, 5)["head_call_us"], 2)
-                del w
-                torch.cuda.empty_cache()
+                for mk in ("stream", "skinny"):
+                    os.environ["EE_MULTI_KERNEL"] = mk
+                    w = Workload("c1", rows, seed=0, n_copies=2)
+                    sweep[f"c1_M{rows}_multi_{mk}"] = round(measure(w, 300, 5)["head_call_us"], 2)
+                    del w
+                    torch.cuda.empty_cache()
+                os.environ.pop("EE_MULTI_KERNEL", None)
                 for pname, pid in (("stream", 1), ("skinny", 3), ("tcgen05", 2)):
                     w = Workload("c1", rows, seed=0, n_copies=2, path=pid, multi=False)
                     if w.head_launches == 0:

@@ -35,7 +35,7 @@ typedef enum {
 
 /* Kernel selection for ee_exit_head_path(). */
 typedef enum {
-    EE_PATH_AUTO = 0,      /* by M: streaming kernel for decode-sized M, tensor-core kernel above   */
+    EE_PATH_AUTO = 0,      /* by M: streaming kernel up to 16 rows, tensor-core GEMM kernel above   */
     EE_PATH_STREAM = 1,    /* fused LayerNorm + split-V streaming kernel (any M, in slabs of rows)  */
     EE_PATH_TCGEN05 = 2,   /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics     */
     EE_PATH_SKINNY = 3     /* one-launch tcgen05 kernel with W as the MMA's M operand: M <= 64, d % 64 == 0,
@@ -92,8 +92,8 @@ ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const 
  * Several heads on batches of the same shape in one call -- what the calibration pass of section 3.4.1 does
  * (every head is evaluated on every token of the calibration set) and what a verify step with several
  * heads does.  Equivalent to n_heads calls of ee_exit_head with the same M, d, V, ln_eps and workspace; when
- * the sizes allow (M <= 64, d % 64 == 0) up to four heads share one kernel launch, which keeps the weight
- * stream going across the per-head LayerNorm and merge steps.  `heads` is a HOST array read during the call;
+ * the batch is decode-sized (M <= 16 rows) up to four heads share one kernel launch, which keeps the weight
+ * stream going across the per-head LayerNorm and merge steps; larger batches run head by head.  `heads` is a HOST array read during the call;
  * the pointers inside follow the rules of ee_exit_head (each head has its own h, LayerNorm parameters, W,
  * thresholds and outputs; h may be the same for all).  Workspace: ee_exit_head_multi_workspace_bytes().
  */

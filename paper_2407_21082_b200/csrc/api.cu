@@ -1,5 +1,7 @@
 // The C ABI: argument validation, device checks, kernel selection.  No compute happens here.
 #include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -40,13 +42,13 @@ bool sizes_ok(int M, int d, int V) { return M >= 0 && V >= 1 && d >= 8 && d <= 8
 
 // Kernel used for M rows when the caller does not choose.
 int auto_path(int M, int d) {
-    const int slab = stream_slab_rows(d);
-    return (slab > 0 && M <= slab) ? EE_PATH_STREAM : EE_PATH_TCGEN05;
+    const int slab = stream_slab_rows(d, 1);
+    return (slab > 0 && M <= slab && M <= 16) ? EE_PATH_STREAM : EE_PATH_TCGEN05;
 }
 
 size_t workspace_bytes(int M, int d, int V) {
     size_t need = gemm_workspace_bytes(M, d, V);
-    const size_t s = stream_workspace_bytes(M, d, V);
+    const size_t s = stream_workspace_bytes(1);
     if (s > need) need = s;
     if (skinny_workspace_bytes(1) > need) need = skinny_workspace_bytes(1);
     return kCtrlBytes + need;
@@ -82,7 +84,7 @@ int ee_exit_head_launches(int M, int d, int V, int path) {
     if (!sizes_ok(M, d, V) || M == 0) return 0;
     if (path == EE_PATH_AUTO) path = auto_path(M, d);
     if (path == EE_PATH_STREAM) {
-        const int slab = stream_slab_rows(d);
+        const int slab = stream_slab_rows(d, 1);
         return slab > 0 ? (M + slab - 1) / slab : 0;
     }
     if (path == EE_PATH_SKINNY) return skinny_supports(M, d) ? 1 : 0;
@@ -120,7 +122,7 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
     a.stream = static_cast<cudaStream_t>(stream);
 
     if (path == EE_PATH_AUTO) path = auto_path(M, d);
-    if (path == EE_PATH_STREAM) return stream_launch(a);
+    if (path == EE_PATH_STREAM) return stream_launch(&a, 1);
     if (path == EE_PATH_SKINNY) return skinny_launch(&a, 1);
     return gemm_launch(a);
 }
@@ -130,12 +132,15 @@ size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
     size_t need = workspace_bytes(M, d, V);
     const int per_launch = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
     if (kCtrlBytes + skinny_workspace_bytes(per_launch) > need) need = kCtrlBytes + skinny_workspace_bytes(per_launch);
+    if (kCtrlBytes + stream_workspace_bytes(per_launch) > need) need = kCtrlBytes + stream_workspace_bytes(per_launch);
     return need;
 }
 
 int ee_exit_head_multi_launches(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1 || M == 0) return 0;
-    if (skinny_supports(M, d)) return (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
+    const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
+    if ((M <= 8 && stream_slab_rows(d, chunk) >= M) || (M <= 16 && skinny_supports(M, d)))
+        return (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
     return n_heads * ee_exit_head_launches(M, d, V, EE_PATH_AUTO);
 }
 
@@ -155,7 +160,19 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     HeadArgs base;
     const ee_status dev = current_device(&base.device, &base.num_sms);
     if (dev != EE_OK) return dev;
-    const bool batched = skinny_supports(M, d);
+    // Which kernel batches the heads: the streaming kernel up to 8 rows (its mma.sync math keeps up with HBM
+    // there), the skinny tcgen05 kernel up to 16; larger batches run head by head.  EE_MULTI_KERNEL=stream |
+    // skinny | none overrides the choice (for A/B timing).
+    enum { kNone, kStream, kSkinny } mode = kNone;
+    const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
+    const bool stream_ok = stream_slab_rows(d, chunk) >= M;
+    if (M <= 8 && stream_ok) mode = kStream;
+    else if (M <= 16 && skinny_supports(M, d)) mode = kSkinny;
+    if (const char* force = getenv("EE_MULTI_KERNEL")) {
+        if (!strcmp(force, "stream") && stream_ok) mode = kStream;
+        else if (!strcmp(force, "skinny") && skinny_supports(M, d)) mode = kSkinny;
+        else if (!strcmp(force, "none")) mode = kNone;
+    }
     for (int k0 = 0; k0 < n_heads; k0 += kSkinnyMaxHeads) {
         HeadArgs a[kSkinnyMaxHeads];
         const int n = n_heads - k0 < kSkinnyMaxHeads ? n_heads - k0 : kSkinnyMaxHeads;
@@ -168,12 +185,12 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
             a[k].workspace = workspace; a[k].workspace_bytes = workspace_bytes_;
             a[k].stream = static_cast<cudaStream_t>(stream);
         }
-        if (batched) {
-            const ee_status st = skinny_launch(a, n);
+        if (mode != kNone) {
+            const ee_status st = mode == kStream ? stream_launch(a, n) : skinny_launch(a, n);
             if (st != EE_OK) return st;
         } else {
             for (int k = 0; k < n; ++k) {
-                const ee_status st = auto_path(M, d) == EE_PATH_STREAM ? stream_launch(a[k]) : gemm_launch(a[k]);
+                const ee_status st = auto_path(M, d) == EE_PATH_STREAM ? stream_launch(&a[k], 1) : gemm_launch(a[k]);
                 if (st != EE_OK) return st;
             }
         }

@@ -31,12 +31,13 @@ struct HeadArgs {
     int num_sms;      // its multiprocessor count
 };
 
-// ---- streaming kernel (fused LayerNorm + split-V mma.sync GEMV + last-CTA merge) ----
+// ---- streaming kernel (fused LayerNorm + split-V mma.sync GEMV + last-CTA merge; up to four heads per launch) ----
 constexpr int kStreamMaxCtas = 256;        // upper bound on the grid, used for workspace sizing
 constexpr int kStreamMaxRows = 32;         // rows per launch (slab)
-int stream_slab_rows(int d);               // rows one launch can take for this d (0 if d does not fit)
-size_t stream_workspace_bytes(int M, int d, int V);
-ee_status stream_launch(const HeadArgs& a);
+constexpr int kStreamMaxHeads = 4;
+int stream_slab_rows(int d, int n_heads);  // rows one launch can take for this d (0 if d does not fit)
+size_t stream_workspace_bytes(int n_heads);
+ee_status stream_launch(const HeadArgs* heads, int n_heads);
 
 // ---- skinny tensor-core kernel (one launch for up to four heads, weights as the MMA's M operand,
 //      1 <= M <= 64, d % 64 == 0) ----

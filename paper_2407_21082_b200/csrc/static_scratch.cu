@@ -46,7 +46,7 @@ extern "C" ee_status ee_exit_head_static(const void* h, long long ld_h, const fl
     if (M < 0 || V < 1 || d < 8 || d > 8192 || (d % 8) != 0) return EE_ERR_SHAPE;
     if (M > EE_STATIC_MAX_ROWS) return EE_ERR_SHAPE;              // beyond the built-in scratch
     if (M == 0) return EE_OK;
-    if (stream_slab_rows(d) < M) return EE_ERR_SHAPE;              // rows of this width do not fit one launch
+    if (stream_slab_rows(d, 1) < M) return EE_ERR_SHAPE;              // rows of this width do not fit one launch
     if (!h || !gamma || !beta || !W || !argmax || !entropy || !maxprob || !exit_mask) return EE_ERR_NULL;
     if (ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
     auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
@@ -69,5 +69,5 @@ extern "C" ee_status ee_exit_head_static(const void* h, long long ld_h, const fl
     a.argmax = argmax; a.entropy = entropy; a.maxprob = maxprob; a.exit_mask = exit_mask;
     a.workspace = scratch;
     a.workspace_bytes = kStaticScratchBytes;
-    return stream_launch(a);
+    return stream_launch(&a, 1);
 }

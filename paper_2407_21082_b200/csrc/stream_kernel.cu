@@ -27,21 +27,26 @@ constexpr int kSegMax = 1024;                         // columns of W per stage 
 constexpr int kMaxStages = 32;
 constexpr size_t kSmemBudget = 226 * 1024;
 
-struct StreamParams {
+struct StreamHead {
     const __nv_bfloat16* h;
     long long ld_h;
     const float* gamma;
     const float* beta;
-    float ln_eps;
     const __nv_bfloat16* W;
-    int M, d, V;                           // M: rows of this slab
     const float* tau_per_row;
     float tau;
     int* argmax;
     float* entropy;
     float* maxprob;
     unsigned char* exit_mask;
-    State* partials;                       // [gridDim.x][8 * NT]
+};
+
+struct StreamParams {
+    StreamHead head[kStreamMaxHeads];
+    int n_heads;
+    float ln_eps;
+    int M, d, V;                           // M: rows of this slab
+    State* partials;                       // [n_heads][gridDim.x][8 * NT]
     Control* ctrl;
     int y_stride;                          // bf16 elements between rows of y in shared memory
     int seg_cols;                          // columns of W per stage
@@ -90,16 +95,17 @@ __device__ __forceinline__ void cp_async_wait_all() {
 
 // Starts the asynchronous copies of everything LayerNorm reads -- the slab's rows of h (into their rows of
 // y), gamma and beta -- 16 bytes per thread and step.
-__device__ void stage_layer_norm_inputs(const StreamParams& p, __nv_bfloat16* y_s, float* gamma_s, float* beta_s) {
+__device__ void stage_layer_norm_inputs(const StreamParams& p, const StreamHead& hd, __nv_bfloat16* y_s, float* gamma_s,
+                                        float* beta_s) {
     const int nvec = p.d >> 3;
     for (int i = threadIdx.x; i < p.M * nvec; i += kThreads) {
         const int r = i / nvec, c = i - r * nvec;
         cp_async_16(reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c,
-                    reinterpret_cast<const uint4*>(p.h + (size_t)r * p.ld_h) + c);
+                    reinterpret_cast<const uint4*>(hd.h + (size_t)r * hd.ld_h) + c);
     }
     for (int i = threadIdx.x; i < (p.d >> 2); i += kThreads) {
-        cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(p.gamma) + i);
-        cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(p.beta) + i);
+        cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(hd.gamma) + i);
+        cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(hd.beta) + i);
     }
 }
 
@@ -161,16 +167,16 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     constexpr int MPAD = 8 * NT;
     constexpr int CH = (NT >= 4) ? 1 : 4 / NT;                    // independent accumulator chains per n-tile
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // layout: ring stages | y | per-warp partial states | gamma, beta (fp32) | barriers
+    // layout: ring stages | y of every head | per-warp partial states of every head | gamma, beta (fp32) | barriers
     const int stage_bytes = kStageRows * p.stage_row_bytes;
+    const size_t y_head_elems = (size_t)MPAD * p.y_stride;
     unsigned char* ring = smem_raw;
-    __nv_bfloat16* y_s = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_stages * stage_bytes);
-    State* wpart = reinterpret_cast<State*>(reinterpret_cast<unsigned char*>(y_s) +
-                                            (size_t)MPAD * p.y_stride * sizeof(__nv_bfloat16));
-    float* gamma_s = reinterpret_cast<float*>(wpart + kWarps * MPAD);
+    __nv_bfloat16* y_all = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_stages * stage_bytes);
+    State* wpart = reinterpret_cast<State*>(y_all + p.n_heads * y_head_elems);      // [head][warp][MPAD]
+    float* gamma_s = reinterpret_cast<float*>(wpart + p.n_heads * kWarps * MPAD);
     float* beta_s = gamma_s + p.d;
     uint64_t* bars = reinterpret_cast<uint64_t*>(beta_s + p.d);
-    __shared__ int s_is_last;
+    __shared__ int s_is_last[kStreamMaxHeads];
     __shared__ int s_abort;
     const uint32_t bar_base = ptx::smem_addr(bars);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -191,22 +197,19 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     const int ngroups = (r_end - r_begin + kStageRows - 1) / kStageRows;
     const uint32_t ring_addr = ptx::smem_addr(ring);
 
-    State st[NT][2];
-#pragma unroll
-    for (int n = 0; n < NT; ++n) {
-        st[n][0] = state_empty();
-        st[n][1] = state_empty();
-    }
-
     // Row group grp belongs to worker warp grp % n_workers.  The warp's stages, in order, are the column
     // segments of its groups; stage j of the warp uses its private slot j % slots_per_warp, phase
     // (j / slots_per_warp) & 1.  One warp arms, waits for, reads and re-arms a slot, so parity waits are exact.
+    // With several heads the sequence simply continues with the next head's weights (same rows, same groups).
     const bool worker = warp < p.n_workers;
     const int my_groups = worker ? (ngroups - warp + p.n_workers - 1) / p.n_workers : 0;
-    const int my_stages = my_groups * p.n_segs;
+    const int stages_per_head = my_groups * p.n_segs;
+    const int my_stages = stages_per_head * p.n_heads;
     auto issue_stage = [&](int j) {
-        const int grp = warp + (j / p.n_segs) * p.n_workers;
-        const int seg = j % p.n_segs;
+        const int hk = j / stages_per_head, jj = j - hk * stages_per_head;
+        const __nv_bfloat16* W = p.head[hk].W;
+        const int grp = warp + (jj / p.n_segs) * p.n_workers;
+        const int seg = jj % p.n_segs;
         const int slot = warp * p.slots_per_warp + j % p.slots_per_warp;
         const int row0 = r_begin + grp * kStageRows;
         const int nrows = min(kStageRows, r_end - row0);
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         if (p.contiguous) {
             if (lane == 0) {
                 ptx::mbar_arrive_expect_tx(full_bar(slot), seg_bytes * nrows);
-                bulk_copy_g2s(ring_addr + slot * stage_bytes, p.W + (size_t)row0 * p.d, seg_bytes * nrows, full_bar(slot));
+                bulk_copy_g2s(ring_addr + slot * stage_bytes, W + (size_t)row0 * p.d, seg_bytes * nrows, full_bar(slot));
             }
             return;
         }
@@ -223,25 +226,35 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         __syncwarp();
         if (lane < nrows)
             bulk_copy_g2s(ring_addr + slot * stage_bytes + lane * p.stage_row_bytes,
-                          p.W + (size_t)(row0 + lane) * p.d + k0, seg_bytes, full_bar(slot));
+                          W + (size_t)(row0 + lane) * p.d + k0, seg_bytes, full_bar(slot));
     };
     int issued = 0;
     for (; issued < my_stages && issued < p.slots_per_warp; ++issued) issue_stage(issued);   // W is in flight ...
 
     grid_dependency_wait();                                       // h and the workspace may come from earlier kernels
-    stage_layer_norm_inputs(p, y_s, gamma_s, beta_s);
-    cp_async_wait_all();
-    __syncthreads();
-    layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, warp, lane);  // ... while LayerNorm runs
-    __syncthreads();
+    for (int hk = 0; hk < p.n_heads; ++hk) {                      // ... while LayerNorm of every head runs
+        __nv_bfloat16* y_s = y_all + hk * y_head_elems;
+        stage_layer_norm_inputs(p, p.head[hk], y_s, gamma_s, beta_s);
+        cp_async_wait_all();
+        __syncthreads();
+        layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, warp, lane);
+        __syncthreads();
+    }
 
-    if (worker) {
-        const int g = lane >> 2, t = lane & 3;
-        const uint4* y_lane = reinterpret_cast<const uint4*>(y_s + (size_t)g * p.y_stride + t * 8);
+    const int g = lane >> 2, t = lane & 3;
+    bool ok = true;
+    int j = 0;                                                    // this warp's stage counter over all heads
+    for (int hk = 0; hk < p.n_heads; ++hk) {
+      State st[NT][2];
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+          st[n][0] = state_empty();
+          st[n][1] = state_empty();
+      }
+      if (worker && ok) {
+        const uint4* y_lane = reinterpret_cast<const uint4*>(y_all + hk * y_head_elems + (size_t)g * p.y_stride + t * 8);
         const int y_tile_vecs = p.y_stride;                       // 8 rows * y_stride elements / 8 per vector
         const bool k_ragged = (p.d & 31) != 0;
-        bool ok = true;
-        int j = 0;                                                // this warp's stage counter
         for (int grp = warp; ok && grp < ngroups; grp += p.n_workers) {
             float acc[NT][CH][4];
 #pragma unroll
@@ -334,46 +347,50 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
                 }
             }
         }
-        if (!ok && lane == 0) {
-            // Let this warp's copies that are still in flight land before the CTA gives its shared memory back.
-            for (int q = max(0, issued - p.slots_per_warp); q < issued; ++q) {
-                const int slot = warp * p.slots_per_warp + q % p.slots_per_warp;
-                const uint32_t par = (uint32_t)(q / p.slots_per_warp) & 1u;
-                for (uint32_t n = 0; n < (1u << 14) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
-            }
+      }
+      // Head hk of this warp is done: reduce over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then
+      // hold tokens 2t, 2t+1.  No CTA-wide barrier here: the warp goes straight on to the next head's stages.
+#pragma unroll
+      for (int n = 0; n < NT; ++n)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+              const State r = state_reduce_lanes<4, 16>(st[n][e]);
+              if (g == 0) wpart[(hk * kWarps + warp) * MPAD + n * 8 + t * 2 + e] = r;
+          }
+    }
+    if (worker && !ok && lane == 0) {
+        // Let this warp's copies that are still in flight land before the CTA gives its shared memory back.
+        for (int q = max(0, issued - p.slots_per_warp); q < issued; ++q) {
+            const int slot = warp * p.slots_per_warp + q % p.slots_per_warp;
+            const uint32_t par = (uint32_t)(q / p.slots_per_warp) & 1u;
+            for (uint32_t n = 0; n < (1u << 14) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
         }
     }
-
-    {
-        // Merge over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then own tokens 2t, 2t+1.
-        const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-        for (int n = 0; n < NT; ++n)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                st[n][e] = state_reduce_lanes<4, 16>(st[n][e]);
-                if (g == 0) wpart[warp * MPAD + n * 8 + t * 2 + e] = st[n][e];
-            }
-    }
     __syncthreads();
 
-    // Merge over the CTA's warps; publish the CTA partial.
-    if (threadIdx.x < MPAD) {
+    // Merge over the CTA's warps; publish the CTA partial of every head.
+    for (int i = threadIdx.x; i < p.n_heads * MPAD; i += kThreads) {
+        const int hk = i / MPAD, tok = i - hk * MPAD;
         State all[kWarps];
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) all[w] = wpart[w * MPAD + threadIdx.x];
-        p.partials[(size_t)blockIdx.x * MPAD + threadIdx.x] = state_combine<kWarps>(all);
+        for (int w = 0; w < kWarps; ++w) all[w] = wpart[(hk * kWarps + w) * MPAD + tok];
+        p.partials[((size_t)hk * gridDim.x + blockIdx.x) * MPAD + tok] = state_combine<kWarps>(all);
     }
     __syncthreads();
-    if (threadIdx.x == 0) s_is_last = ticket_arrive_is_last(&p.ctrl->ticket, gridDim.x);
+    if (threadIdx.x < p.n_heads) s_is_last[threadIdx.x] = ticket_arrive_is_last(&p.ctrl->head_ticket[threadIdx.x], gridDim.x);
     __syncthreads();
-    if (!s_is_last) return;
 
-    // Last CTA: merge the partials of all CTAs and decide (the ring is free by now and serves as scratch).
-    merge_partials_and_decide<kThreads>(p.partials, (int)gridDim.x, MPAD, p.M, reinterpret_cast<State*>(ring),
-                                        (size_t)p.n_stages * stage_bytes, p.tau_per_row, p.tau, p.argmax, p.entropy,
-                                        p.maxprob, p.exit_mask);
-    if (threadIdx.x == 0) p.ctrl->ticket = 0;                     // ready for the next call
+    // The last CTA to arrive for a head merges that head's partials of all CTAs and decides (the ring is free
+    // by now and serves as scratch).
+    for (int hk = 0; hk < p.n_heads; ++hk) {
+        if (!s_is_last[hk]) continue;
+        const StreamHead& hd = p.head[hk];
+        merge_partials_and_decide<kThreads>(p.partials + (size_t)hk * gridDim.x * MPAD, (int)gridDim.x, MPAD, p.M,
+                                            reinterpret_cast<State*>(ring), (size_t)p.n_stages * stage_bytes, hd.tau_per_row,
+                                            hd.tau, hd.argmax, hd.entropy, hd.maxprob, hd.exit_mask);
+        if (threadIdx.x == 0) p.ctrl->head_ticket[hk] = 0;        // ready for the next call
+        __syncthreads();                                          // the scratch is reused by the next head
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -405,12 +422,12 @@ bool split_slots(long long n, int min_workers, SmemPlan& s) {
 }
 
 // Ring geometry for hidden size d with 8*nt rows of y resident; n_stages = 0 if it does not fit.
-SmemPlan plan_smem(int d, int nt) {
+SmemPlan plan_smem(int d, int nt, int n_heads) {
     SmemPlan none = {};
     const int d64 = (d + 63) / 64 * 64;
-    const size_t fixed = (size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
-                         (size_t)kWarps * 8 * nt * sizeof(State) + (size_t)2 * d * sizeof(float) +
-                         kMaxStages * sizeof(uint64_t);
+    const size_t fixed = (size_t)n_heads * ((size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
+                                            (size_t)kWarps * 8 * nt * sizeof(State)) +
+                         (size_t)2 * d * sizeof(float) + kMaxStages * sizeof(uint64_t);
     const long long room = (long long)kSmemBudget - (long long)fixed;
     if (room <= 0) return none;
     if (d <= kSegMax) {
@@ -457,7 +474,7 @@ SmemPlan plan_smem(int d, int nt) {
 
 template <int NT>
 ee_status launch_one(StreamParams& p, int grid, int device, cudaStream_t stream) {
-    const SmemPlan plan = plan_smem(p.d, NT);
+    const SmemPlan plan = plan_smem(p.d, NT, p.n_heads);
     if (plan.n_stages == 0) return EE_ERR_SHAPE;
     p.seg_cols = plan.seg_cols;
     p.n_segs = plan.n_segs;
@@ -488,40 +505,48 @@ ee_status launch_one(StreamParams& p, int grid, int device, cudaStream_t stream)
 
 }  // namespace
 
-int stream_slab_rows(int d) {
+int stream_slab_rows(int d, int n_heads) {
     for (int nt = kStreamMaxRows / 8; nt >= 1; nt >>= 1)
-        if (plan_smem(d, nt).n_stages > 0) return 8 * nt;
+        if (plan_smem(d, nt, n_heads).n_stages > 0) return 8 * nt;
     return 0;
 }
 
-size_t stream_workspace_bytes(int M, int d, int V) {
-    (void)M; (void)d; (void)V;
-    return (size_t)kStreamMaxCtas * kStreamMaxRows * sizeof(State);
+size_t stream_workspace_bytes(int n_heads) {
+    return (size_t)n_heads * kStreamMaxCtas * kStreamMaxRows * sizeof(State);
 }
 
-ee_status stream_launch(const HeadArgs& a) {
-    const int slab = stream_slab_rows(a.d);
-    if (slab == 0) return EE_ERR_SHAPE;
+// heads[0 .. n_heads) share M, d, V, ln_eps, workspace and stream.  Several heads go into one launch when all
+// M rows fit one slab with every head's activations resident; a single head may be cut into slabs of rows.
+ee_status stream_launch(const HeadArgs* heads, int n_heads) {
+    const HeadArgs& a = heads[0];
+    if (n_heads < 1 || n_heads > kStreamMaxHeads) return EE_ERR_SHAPE;
+    const int slab = stream_slab_rows(a.d, n_heads);
+    if (slab == 0 || (n_heads > 1 && a.M > slab)) return EE_ERR_SHAPE;
     const int grid = a.num_sms < kStreamMaxCtas ? a.num_sms : kStreamMaxCtas;
     unsigned char* ws = static_cast<unsigned char*>(a.workspace);
     for (int m0 = 0; m0 < a.M; m0 += slab) {
         const int rows = (a.M - m0 < slab) ? a.M - m0 : slab;
         StreamParams p;
-        p.h = static_cast<const __nv_bfloat16*>(a.h) + (size_t)m0 * a.ld_h;
-        p.ld_h = a.ld_h;
-        p.gamma = a.gamma;
-        p.beta = a.beta;
+        for (int k = 0; k < kStreamMaxHeads; ++k) {
+            const HeadArgs& h = heads[k < n_heads ? k : 0];
+            StreamHead& s = p.head[k];
+            s.h = static_cast<const __nv_bfloat16*>(h.h) + (size_t)m0 * h.ld_h;
+            s.ld_h = h.ld_h;
+            s.gamma = h.gamma;
+            s.beta = h.beta;
+            s.W = static_cast<const __nv_bfloat16*>(h.W);
+            s.tau_per_row = h.tau_per_row ? h.tau_per_row + m0 : nullptr;
+            s.tau = h.tau;
+            s.argmax = h.argmax + m0;
+            s.entropy = h.entropy + m0;
+            s.maxprob = h.maxprob + m0;
+            s.exit_mask = h.exit_mask + m0;
+        }
+        p.n_heads = n_heads;
         p.ln_eps = a.ln_eps;
-        p.W = static_cast<const __nv_bfloat16*>(a.W);
         p.M = rows;
         p.d = a.d;
         p.V = a.V;
-        p.tau_per_row = a.tau_per_row ? a.tau_per_row + m0 : nullptr;
-        p.tau = a.tau;
-        p.argmax = a.argmax + m0;
-        p.entropy = a.entropy + m0;
-        p.maxprob = a.maxprob + m0;
-        p.exit_mask = a.exit_mask + m0;
         p.partials = reinterpret_cast<State*>(ws + kCtrlBytes);
         p.ctrl = reinterpret_cast<Control*>(ws);
         p.y_stride = y_stride_elems(a.d);
