@@ -12,6 +12,10 @@
 // as bf16.  Each thread folds the logits it owns into an online (max, sum exp, sum exp*(z-max), argmax)
 // state; states merge by warp shuffles, through shared memory across warps, and the last CTA to finish
 // (atomic ticket, no spinning) merges the per-CTA partials and writes argmax / entropy / max-prob / exit mask.
+//
+// Up to four heads can share a launch: a worker simply continues with the next head's weights, warps that own no
+// ring slots normalise the later heads' activations meanwhile, and the last worker of a CTA to finish a head
+// publishes that head's partial and takes its ticket at once, so only the last head's merge is not hidden.
 #include "common.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -96,68 +100,60 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // Starts the asynchronous copies of everything LayerNorm reads -- the slab's rows of h (into their rows of
 // y), gamma and beta -- 16 bytes per thread and step.
 __device__ void stage_layer_norm_inputs(const StreamParams& p, const StreamHead& hd, __nv_bfloat16* y_s, float* gamma_s,
-                                        float* beta_s) {
+                                        float* beta_s, int tid, int nthreads) {
     const int nvec = p.d >> 3;
-    for (int i = threadIdx.x; i < p.M * nvec; i += kThreads) {
+    for (int i = tid; i < p.M * nvec; i += nthreads) {
         const int r = i / nvec, c = i - r * nvec;
         cp_async_16(reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c,
                     reinterpret_cast<const uint4*>(hd.h + (size_t)r * hd.ld_h) + c);
     }
-    for (int i = threadIdx.x; i < (p.d >> 2); i += kThreads) {
+    for (int i = tid; i < (p.d >> 2); i += nthreads) {
         cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(hd.gamma) + i);
         cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(hd.beta) + i);
     }
 }
 
-// LayerNorm in shared memory: the rows of y hold raw h on entry and the normalised bf16 rows on exit.
-// Warp w owns rows w, w + 8, ...  Rows >= M and the k padding are zero-filled so that they contribute nothing
-// and stay finite.
+// LayerNorm in shared memory: the rows of y hold raw h on entry and the normalised bf16 rows on exit.  The
+// 8 * NT rows are shared out over the `nw` warps of a group (this warp being number `w`).  Rows >= M and the k
+// padding are zero-filled so that they contribute nothing and stay finite.
 template <int NT>
 __device__ void layer_norm_in_smem(const StreamParams& p, __nv_bfloat16* y_s, const float* gamma_s,
-                                   const float* beta_s, int warp, int lane) {
+                                   const float* beta_s, int w, int nw, int lane) {
+    constexpr int MPAD = 8 * NT;
     const int nvec = p.d >> 3;                                   // 16-byte vectors per row
     const int svec = p.y_stride >> 3;
     const float inv_d = 1.f / (float)p.d;
     auto vec = [&](int r, int c) { return reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c; };
-    if (nvec <= 256) {
-        // Rows held in registers: one pass over shared memory, two rows at a time.
-        for (int i = 0; i < NT; i += 2) {
-            const int rows[2] = {warp + i * kWarps, warp + (i + 1) * kWarps};
-            const int live = (rows[0] < p.M) + (i + 1 < NT && rows[1] < p.M);
-            if (live == 0) break;
-            if (nvec <= 128) layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
-            else layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
-        }
-#pragma unroll
-        for (int i = 0; i < NT; ++i) {
-            const int r = warp + i * kWarps;
-            uint4* yrow = vec(r, 0);
-            for (int c = (r < p.M ? nvec : 0) + lane; c < svec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
-        }
-        return;
-    }
-#pragma unroll
-    for (int i = 0; i < NT; ++i) {
-        const int r = warp + i * kWarps;
-        uint4* yrow = reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride);
-        if (r >= p.M) {
-            for (int c = lane; c < svec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
-            continue;
-        }
-        float sum = 0.f;
-        for (int c = lane; c < nvec; c += 32) sum += vec8_sum(yrow[c]);
-        const float mu = warp_sum(sum) * inv_d;
-        float sq = 0.f;
-        for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(yrow[c], mu, sq);
-        const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
-        for (int c = lane; c < svec; c += 32) {
-            if (c < nvec) {
-                const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
-                const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-                yrow[c] = layer_norm_vec8(yrow[c], mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+    for (int r0 = w; r0 < MPAD; r0 += 2 * nw) {
+        const int rows[2] = {r0, r0 + nw};
+        const int live = (rows[0] < p.M) + (rows[1] < MPAD && rows[1] < p.M);
+        if (live > 0) {
+            if (nvec <= 128) {
+                layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+            } else if (nvec <= 256) {
+                layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
             } else {
-                yrow[c] = make_uint4(0, 0, 0, 0);
+                for (int i = 0; i < live; ++i) {
+                    uint4* yrow = vec(rows[i], 0);
+                    float sum = 0.f;
+                    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(yrow[c]);
+                    const float mu = warp_sum(sum) * inv_d;
+                    float sq = 0.f;
+                    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(yrow[c], mu, sq);
+                    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
+                    for (int c = lane; c < nvec; c += 32) {
+                        const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
+                        const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
+                        yrow[c] = layer_norm_vec8(yrow[c], mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+                    }
+                }
             }
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int r = rows[i];
+            if (r < MPAD)
+                for (int c = (r < p.M ? nvec : 0) + lane; c < svec; c += 32) *vec(r, c) = make_uint4(0, 0, 0, 0);
         }
     }
 }
@@ -176,16 +172,21 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     float* gamma_s = reinterpret_cast<float*>(wpart + p.n_heads * kWarps * MPAD);
     float* beta_s = gamma_s + p.d;
     uint64_t* bars = reinterpret_cast<uint64_t*>(beta_s + p.d);
-    __shared__ int s_is_last[kStreamMaxHeads];
+    __shared__ int s_head_done[kStreamMaxHeads];                  // workers of this CTA that have finished a head
     __shared__ int s_abort;
     const uint32_t bar_base = ptx::smem_addr(bars);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto yready_bar = [&](int k) { return bar_base + 8u * (kMaxStages + k); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.n_stages; ++s) ptx::mbar_init(full_bar(s), 1);
+        for (int k = 0; k < kStreamMaxHeads; ++k) {
+            ptx::mbar_init(yready_bar(k), kWarps - p.n_workers > 0 ? kWarps - p.n_workers : 1);
+            s_head_done[k] = 0;
+        }
         s_abort = 0;
         ptx::fence_mbar_init();
     }
@@ -232,13 +233,31 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     for (; issued < my_stages && issued < p.slots_per_warp; ++issued) issue_stage(issued);   // W is in flight ...
 
     grid_dependency_wait();                                       // h and the workspace may come from earlier kernels
-    for (int hk = 0; hk < p.n_heads; ++hk) {                      // ... while LayerNorm of every head runs
+    // ... while LayerNorm runs.  Every warp works on the first head; the later heads are left to the warps that
+    // own no ring slots (if there are any), which signal yready[k] when head k's activations are in place.
+    const int n_helpers = kWarps - p.n_workers;
+    const int heads_by_all = n_helpers > 0 ? 1 : p.n_heads;
+    for (int hk = 0; hk < heads_by_all; ++hk) {
         __nv_bfloat16* y_s = y_all + hk * y_head_elems;
-        stage_layer_norm_inputs(p, p.head[hk], y_s, gamma_s, beta_s);
+        stage_layer_norm_inputs(p, p.head[hk], y_s, gamma_s, beta_s, threadIdx.x, kThreads);
         cp_async_wait_all();
         __syncthreads();
-        layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, warp, lane);
+        layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, warp, kWarps, lane);
         __syncthreads();
+    }
+    if (warp >= p.n_workers) {
+        const int hw = warp - p.n_workers;
+        for (int hk = 1; hk < p.n_heads; ++hk) {
+            __nv_bfloat16* y_s = y_all + hk * y_head_elems;
+            stage_layer_norm_inputs(p, p.head[hk], y_s, gamma_s, beta_s, hw * 32 + lane, n_helpers * 32);
+            cp_async_wait_all();
+            asm volatile("bar.sync 2, %0;" ::"r"(n_helpers * 32) : "memory");
+            layer_norm_in_smem<NT>(p, y_s, gamma_s, beta_s, hw, n_helpers, lane);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(yready_bar(hk));
+            asm volatile("bar.sync 2, %0;" ::"r"(n_helpers * 32) : "memory");      // gamma_s / beta_s are reused
+        }
+        return;
     }
 
     const int g = lane >> 2, t = lane & 3;
@@ -250,6 +269,17 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
       for (int n = 0; n < NT; ++n) {
           st[n][0] = state_empty();
           st[n][1] = state_empty();
+      }
+      if (ok && hk > 0 && n_helpers > 0) {
+          const bool ready = ptx::mbar_wait(yready_bar(hk), 0, &s_abort);
+          if (!__all_sync(0xffffffffu, ready)) {
+              if (lane == 0) {
+                  if (atomicCAS(&p.ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
+                      p.ctrl->error_info = (4u << 24) | (unsigned)hk;
+                  s_abort = 1;
+              }
+              ok = false;
+          }
       }
       if (worker && ok) {
         const uint4* y_lane = reinterpret_cast<const uint4*>(y_all + hk * y_head_elems + (size_t)g * p.y_stride + t * 8);
@@ -349,7 +379,8 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         }
       }
       // Head hk of this warp is done: reduce over the eight row lanes of the warp (lane bits 2..4); lanes 0..3 then
-      // hold tokens 2t, 2t+1.  No CTA-wide barrier here: the warp goes straight on to the next head's stages.
+      // hold tokens 2t, 2t+1.  No CTA-wide barrier: the last worker of the CTA to get here finishes the head (CTA
+      // partial, ticket, and in the last CTA the final merge) while the others are already on the next head.
 #pragma unroll
       for (int n = 0; n < NT; ++n)
 #pragma unroll
@@ -357,39 +388,40 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
               const State r = state_reduce_lanes<4, 16>(st[n][e]);
               if (g == 0) wpart[(hk * kWarps + warp) * MPAD + n * 8 + t * 2 + e] = r;
           }
+      __threadfence_block();
+      __syncwarp();
+      int arrived = 0;
+      if (lane == 0) arrived = atomicAdd(&s_head_done[hk], 1);
+      arrived = __shfl_sync(0xffffffffu, arrived, 0);
+      if (arrived == p.n_workers - 1) {
+          __threadfence_block();
+          State* part = p.partials + ((size_t)hk * gridDim.x + blockIdx.x) * MPAD;
+          for (int tok = lane; tok < MPAD; tok += 32) {
+              State all[kWarps];
+#pragma unroll
+              for (int w = 0; w < kWarps; ++w)
+                  all[w] = w < p.n_workers ? wpart[(hk * kWarps + w) * MPAD + tok] : state_empty();
+              part[tok] = state_combine<kWarps>(all);
+          }
+          __syncwarp();
+          int last = 0;
+          if (lane == 0) last = ticket_arrive_is_last(&p.ctrl->head_ticket[hk], gridDim.x) ? 1 : 0;
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last) {
+              const StreamHead& hd = p.head[hk];
+              merge_tokens(p.partials + (size_t)hk * gridDim.x * MPAD, false, (int)gridDim.x, MPAD, p.M, 0, 1, lane,
+                           hd.tau_per_row, hd.tau, hd.argmax, hd.entropy, hd.maxprob, hd.exit_mask);
+              if (lane == 0) p.ctrl->head_ticket[hk] = 0;          // ready for the next call
+          }
+      }
     }
-    if (worker && !ok && lane == 0) {
+    if (!ok && lane == 0) {
         // Let this warp's copies that are still in flight land before the CTA gives its shared memory back.
         for (int q = max(0, issued - p.slots_per_warp); q < issued; ++q) {
             const int slot = warp * p.slots_per_warp + q % p.slots_per_warp;
             const uint32_t par = (uint32_t)(q / p.slots_per_warp) & 1u;
             for (uint32_t n = 0; n < (1u << 14) && !ptx::mbar_try_wait(full_bar(slot), par); ++n) __nanosleep(100);
         }
-    }
-    __syncthreads();
-
-    // Merge over the CTA's warps; publish the CTA partial of every head.
-    for (int i = threadIdx.x; i < p.n_heads * MPAD; i += kThreads) {
-        const int hk = i / MPAD, tok = i - hk * MPAD;
-        State all[kWarps];
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) all[w] = wpart[(hk * kWarps + w) * MPAD + tok];
-        p.partials[((size_t)hk * gridDim.x + blockIdx.x) * MPAD + tok] = state_combine<kWarps>(all);
-    }
-    __syncthreads();
-    if (threadIdx.x < p.n_heads) s_is_last[threadIdx.x] = ticket_arrive_is_last(&p.ctrl->head_ticket[threadIdx.x], gridDim.x);
-    __syncthreads();
-
-    // The last CTA to arrive for a head merges that head's partials of all CTAs and decides (the ring is free
-    // by now and serves as scratch).
-    for (int hk = 0; hk < p.n_heads; ++hk) {
-        if (!s_is_last[hk]) continue;
-        const StreamHead& hd = p.head[hk];
-        merge_partials_and_decide<kThreads>(p.partials + (size_t)hk * gridDim.x * MPAD, (int)gridDim.x, MPAD, p.M,
-                                            reinterpret_cast<State*>(ring), (size_t)p.n_stages * stage_bytes, hd.tau_per_row,
-                                            hd.tau, hd.argmax, hd.entropy, hd.maxprob, hd.exit_mask);
-        if (threadIdx.x == 0) p.ctrl->head_ticket[hk] = 0;        // ready for the next call
-        __syncthreads();                                          // the scratch is reused by the next head
     }
 }
 
@@ -427,7 +459,7 @@ SmemPlan plan_smem(int d, int nt, int n_heads) {
     const int d64 = (d + 63) / 64 * 64;
     const size_t fixed = (size_t)n_heads * ((size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
                                             (size_t)kWarps * 8 * nt * sizeof(State)) +
-                         (size_t)2 * d * sizeof(float) + kMaxStages * sizeof(uint64_t);
+                         (size_t)2 * d * sizeof(float) + (kMaxStages + kStreamMaxHeads) * sizeof(uint64_t);
     const long long room = (long long)kSmemBudget - (long long)fixed;
     if (room <= 0) return none;
     if (d <= kSegMax) {
