@@ -14,8 +14,9 @@
 // (atomic ticket, no spinning) merges the per-CTA partials and writes argmax / entropy / max-prob / exit mask.
 //
 // Up to four heads can share a launch: a worker simply continues with the next head's weights, warps that own no
-// ring slots normalise the later heads' activations meanwhile, and the last worker of a CTA to finish a head
-// publishes that head's partial and takes its ticket at once, so only the last head's merge is not hidden.
+// ring slots normalise the later heads' activations meanwhile, and one of them completes each head (CTA partial,
+// ticket, final merge in the last CTA) as soon as the workers are through with it, so that only the last head's
+// merge is not hidden behind the stream.
 #include "common.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
@@ -177,6 +178,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     const uint32_t bar_base = ptx::smem_addr(bars);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto yready_bar = [&](int k) { return bar_base + 8u * (kMaxStages + k); };
+    auto hdone_bar = [&](int k) { return bar_base + 8u * (kMaxStages + kStreamMaxHeads + k); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -185,6 +187,7 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         for (int s = 0; s < p.n_stages; ++s) ptx::mbar_init(full_bar(s), 1);
         for (int k = 0; k < kStreamMaxHeads; ++k) {
             ptx::mbar_init(yready_bar(k), kWarps - p.n_workers > 0 ? kWarps - p.n_workers : 1);
+            ptx::mbar_init(hdone_bar(k), p.n_workers);
             s_head_done[k] = 0;
         }
         s_abort = 0;
@@ -233,6 +236,29 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
     for (; issued < my_stages && issued < p.slots_per_warp; ++issued) issue_stage(issued);   // W is in flight ...
 
     grid_dependency_wait();                                       // h and the workspace may come from earlier kernels
+    // Completion of head hk in this CTA, by one warp, once every worker has stored its per-warp states: CTA
+    // partial, ticket, and in the last CTA to arrive the final merge and the decision.
+    auto finalize_head = [&](int hk) {
+        State* part = p.partials + ((size_t)hk * gridDim.x + blockIdx.x) * MPAD;
+        for (int tok = lane; tok < MPAD; tok += 32) {
+            State all[kWarps];
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w)
+                all[w] = w < p.n_workers ? wpart[(hk * kWarps + w) * MPAD + tok] : state_empty();
+            part[tok] = state_combine<kWarps>(all);
+        }
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = ticket_arrive_is_last(&p.ctrl->head_ticket[hk], gridDim.x) ? 1 : 0;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            const StreamHead& hd = p.head[hk];
+            merge_tokens(p.partials + (size_t)hk * gridDim.x * MPAD, false, (int)gridDim.x, MPAD, p.M, 0, 1, lane,
+                         hd.tau_per_row, hd.tau, hd.argmax, hd.entropy, hd.maxprob, hd.exit_mask);
+            if (lane == 0) p.ctrl->head_ticket[hk] = 0;            // ready for the next call
+        }
+    };
+
     // ... while LayerNorm runs.  Every warp works on the first head; the later heads are left to the warps that
     // own no ring slots (if there are any), which signal yready[k] when head k's activations are in place.
     const int n_helpers = kWarps - p.n_workers;
@@ -256,6 +282,15 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(yready_bar(hk));
             asm volatile("bar.sync 2, %0;" ::"r"(n_helpers * 32) : "memory");      // gamma_s / beta_s are reused
+        }
+        // The first of these warps then completes each head as soon as the workers are through with it, so that
+        // no worker ever leaves its ring waiting.
+        if (hw == 0) {
+            for (int hk = 0; hk < p.n_heads; ++hk) {
+                const bool done = ptx::mbar_wait(hdone_bar(hk), 0, &s_abort);
+                if (!__all_sync(0xffffffffu, done)) break;        // a worker gave up; it has recorded the error
+                finalize_head(hk);
+            }
         }
         return;
     }
@@ -388,30 +423,18 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
               const State r = state_reduce_lanes<4, 16>(st[n][e]);
               if (g == 0) wpart[(hk * kWarps + warp) * MPAD + n * 8 + t * 2 + e] = r;
           }
-      __threadfence_block();
       __syncwarp();
-      int arrived = 0;
-      if (lane == 0) arrived = atomicAdd(&s_head_done[hk], 1);
-      arrived = __shfl_sync(0xffffffffu, arrived, 0);
-      if (arrived == p.n_workers - 1) {
+      if (n_helpers > 0) {
+          if (lane == 0) ptx::mbar_arrive(hdone_bar(hk));         // release: the states above are visible to the waiter
+      } else {
+          // No idle warp: the last worker of the CTA to get here completes the head itself.
           __threadfence_block();
-          State* part = p.partials + ((size_t)hk * gridDim.x + blockIdx.x) * MPAD;
-          for (int tok = lane; tok < MPAD; tok += 32) {
-              State all[kWarps];
-#pragma unroll
-              for (int w = 0; w < kWarps; ++w)
-                  all[w] = w < p.n_workers ? wpart[(hk * kWarps + w) * MPAD + tok] : state_empty();
-              part[tok] = state_combine<kWarps>(all);
-          }
-          __syncwarp();
-          int last = 0;
-          if (lane == 0) last = ticket_arrive_is_last(&p.ctrl->head_ticket[hk], gridDim.x) ? 1 : 0;
-          last = __shfl_sync(0xffffffffu, last, 0);
-          if (last) {
-              const StreamHead& hd = p.head[hk];
-              merge_tokens(p.partials + (size_t)hk * gridDim.x * MPAD, false, (int)gridDim.x, MPAD, p.M, 0, 1, lane,
-                           hd.tau_per_row, hd.tau, hd.argmax, hd.entropy, hd.maxprob, hd.exit_mask);
-              if (lane == 0) p.ctrl->head_ticket[hk] = 0;          // ready for the next call
+          int arrived = 0;
+          if (lane == 0) arrived = atomicAdd(&s_head_done[hk], 1);
+          arrived = __shfl_sync(0xffffffffu, arrived, 0);
+          if (arrived == p.n_workers - 1) {
+              __threadfence_block();
+              finalize_head(hk);
           }
       }
     }
@@ -459,7 +482,7 @@ SmemPlan plan_smem(int d, int nt, int n_heads) {
     const int d64 = (d + 63) / 64 * 64;
     const size_t fixed = (size_t)n_heads * ((size_t)8 * nt * y_stride_elems(d) * sizeof(__nv_bfloat16) +
                                             (size_t)kWarps * 8 * nt * sizeof(State)) +
-                         (size_t)2 * d * sizeof(float) + (kMaxStages + kStreamMaxHeads) * sizeof(uint64_t);
+                         (size_t)2 * d * sizeof(float) + (kMaxStages + 2 * kStreamMaxHeads) * sizeof(uint64_t);
     const long long room = (long long)kSmemBudget - (long long)fixed;
     if (room <= 0) return none;
     if (d <= kSegMax) {
