@@ -279,19 +279,21 @@ __device__ __forceinline__ bool ticket_arrive_is_last(unsigned int* counter, uns
 }
 
 // The threads of the last CTA that take part (n_warps whole warps, this one being number `warp`): merge
-// partials [n_cta][np] per token and write the outputs.  A warp takes four tokens at a time; every lane first
-// loads all the states it is responsible for (CTAs lane, lane + 32, ..; at most 256 CTAs), so the loads are
-// one round trip, then combines them and the lanes reduce.
-__device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem, int n_cta, int np, int M, int warp,
-                                             int n_warps, int lane, const float* tau_per_row, float tau, int* argmax,
-                                             float* entropy, float* maxprob, unsigned char* exit_mask) {
-    for (int tok0 = warp * 4; tok0 < M; tok0 += n_warps * 4) {
-        State v[4][8];
+// partials [n_cta][np] per token and write the outputs.  A warp takes TB tokens at a time; every lane first
+// loads all the states it is responsible for (CTAs lane, lane + 32, .., NL of them), so the loads of a batch
+// are one round trip, then combines them and the lanes reduce.
+template <int TB, int NL>
+__device__ __forceinline__ void merge_token_batches(const State* src, bool src_is_smem, int n_cta, int np, int M,
+                                                    int warp, int n_warps, int lane, const float* tau_per_row, float tau,
+                                                    int* argmax, float* entropy, float* maxprob,
+                                                    unsigned char* exit_mask) {
+    for (int tok0 = warp * TB; tok0 < M; tok0 += n_warps * TB) {
+        State v[TB][NL];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < NL; ++i) {
             const int b = lane + 32 * i;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < TB; ++q) {
                 v[q][i] = state_empty();
                 if (b < n_cta && tok0 + q < M) {
                     const size_t at = (size_t)b * np + tok0 + q;
@@ -299,18 +301,29 @@ __device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem,
                 }
             }
         }
-        State r[4];
+        State mine = state_empty();
 #pragma unroll
-        for (int q = 0; q < 4; ++q) r[q] = state_reduce_lanes<1, 16>(state_combine<8>(v[q]));
-        if (lane < 4 && tok0 + lane < M) {
-            State mine = r[0];
-#pragma unroll
-            for (int q = 1; q < 4; ++q)
-                if (lane == q) mine = r[q];
+        for (int q = 0; q < TB; ++q) {
+            const State r = state_reduce_lanes<1, 16>(state_combine<NL>(v[q]));
+            if (lane == q) mine = r;
+        }
+        if (lane < TB && tok0 + lane < M) {
             const int tok = tok0 + lane;
             state_finish(mine, tau_per_row ? tau_per_row[tok] : tau, argmax, entropy, maxprob, exit_mask, tok);
         }
     }
+}
+
+// Up to 256 CTAs; grids of at most 160 CTAs (a B200 has 148 SMs) take eight tokens per batch.
+__device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem, int n_cta, int np, int M, int warp,
+                                             int n_warps, int lane, const float* tau_per_row, float tau, int* argmax,
+                                             float* entropy, float* maxprob, unsigned char* exit_mask) {
+    if (n_cta <= 160)
+        merge_token_batches<8, 5>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
+                                  maxprob, exit_mask);
+    else
+        merge_token_batches<4, 8>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
+                                  maxprob, exit_mask);
 }
 
 // Whole-CTA variant: `scratch` is shared memory the partials are first copied to with independent loads, if it
