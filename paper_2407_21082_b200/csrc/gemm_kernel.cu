@@ -1,6 +1,7 @@
 // Verify/prefill-sized exit head: LayerNorm kernel -> persistent TMA + tcgen05 GEMM whose epilogue reduces
 // every 128 x BN block of logits to per-row softmax states straight out of tensor memory -> merge kernel.
-// The M x V logits are never written anywhere.
+// The M x V logits are never written anywhere.  The three kernels are chained by programmatic dependent
+// launch, and the GEMM requests its first weight tiles before it waits for the LayerNorm kernel.
 //
 // GEMM kernel, one CTA per SM, 192 threads:
 //   warp 0 (one lane)  TMA producer: y tile [128 x 64] and W tile [BN x 64] per k-block into a smem ring
@@ -24,13 +25,18 @@ constexpr int kGemmThreads = 192;
 constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile order
 constexpr int kATileBytes = BM * BK * 2;    // 16 KB
 
-template <int BN>
+constexpr int kBarBytes = 256;
+constexpr int kMaxGemmStages = 12;
+constexpr size_t kGemmSmemBudget = 226 * 1024;
+
+// BN_T = 256: the tile width is a compile-time constant (large M).  BN_T = 0: the width comes from the
+// parameters (any multiple of 16 up to 256), chosen so that the tiles fill whole waves of CTAs.
+template <int BN_T>
 struct Cfg {
-    static constexpr int kStages = (BN >= 256) ? 4 : 6;
-    static constexpr int kBTileBytes = BN * BK * 2;
+    static constexpr int kStages = 4;
+    static constexpr int kBTileBytes = 256 * BK * 2;
     static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-    static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;       // power of two for BN in {16..256}
-    static constexpr int kBarBytes = 256;
+    static constexpr int kTmemCols = 512;                             // two accumulator buffers of 256 columns
     static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;   // + slack to align to 1024
 };
 
@@ -39,7 +45,15 @@ struct GemmParams {
     int m_tiles, n_tiles, k_blocks;
     State* partials;       // [M][n_tiles]
     Control* ctrl;
+    int bn;                // tile width (vocabulary rows per tile), a multiple of 16, <= 256
+    int n_stages;          // smem ring depth
 };
+
+// Programmatic dependent launch: the next kernel of the stream may start once every CTA of this one has passed
+// launch_dependents(); a kernel calls grid_dependency_wait() before it touches anything an earlier kernel
+// of the stream writes (it returns when those kernels have completed and their stores are visible).
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
     const int per_group = kGroupM * n_tiles;
@@ -93,18 +107,22 @@ __device__ __forceinline__ void fold_chunk(State& st, const float (&v)[32], int 
     st.t = fmaf(t2, kLn2, st.t);
 }
 
-template <int BN>
+template <int BN_T>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
                       const GemmParams p) {
-    using C = Cfg<BN>;
-    constexpr int S = C::kStages;
+    using C = Cfg<BN_T>;
+    const int BN = BN_T ? BN_T : p.bn;
+    const int S = BN_T ? C::kStages : p.n_stages;
+    const int b_tile_bytes = BN * BK * 2;
+    const int stage_bytes = kATileBytes + b_tile_bytes;
+    constexpr int kAccStride = 256;                               // TMEM columns between the two accumulators
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
     const uint32_t a_base = ptx::smem_addr(smem);
     const uint32_t b_base = a_base + S * kATileBytes;
-    unsigned char* bar_mem = smem + S * C::kStageBytes;
+    unsigned char* bar_mem = smem + S * stage_bytes;
     const uint32_t bar_base = ptx::smem_addr(bar_mem);
     // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -116,6 +134,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 5) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -149,18 +168,38 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
             int stage = 0;
             uint32_t phase = 0, armed = 0, armed_parity = 0;
             bool ok = true;
+            // The weights do not depend on earlier kernels of the stream: the W tiles of the first stages are
+            // requested before the dependency wait, the y tiles (written by the LayerNorm kernel) after it.
+            int n_pre = 0;
+            if ((int)blockIdx.x < total_tiles) {
+                int m_tile, n_tile;
+                tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                n_pre = min(S, p.k_blocks);
+                for (int kb = 0; kb < n_pre; ++kb) {
+                    ptx::mbar_arrive_expect_tx(full_bar(kb), stage_bytes);
+                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &tm_w, kb * BK, n_tile * BN, full_bar(kb));
+                    armed |= 1u << kb;
+                }
+            }
+            grid_dependency_wait();
+            int issued = 0;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 int m_tile, n_tile;
                 tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
+                    if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
+                        ptx::tma_load_2d(a_base + stage * kATileBytes, &tm_y, kb * BK, m_tile * BM, full_bar(stage));
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
                         record_failure(p.ctrl, abort_flag, 1, stage, tile);
                         ok = false;
                         break;
                     }
-                    ptx::mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
+                    ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
                     ptx::tma_load_2d(a_base + stage * kATileBytes, &tm_y, kb * BK, m_tile * BM, full_bar(stage));
-                    ptx::tma_load_2d(b_base + stage * C::kBTileBytes, &tm_w, kb * BK, n_tile * BN, full_bar(stage));
+                    ptx::tma_load_2d(b_base + stage * b_tile_bytes, &tm_w, kb * BK, n_tile * BN, full_bar(stage));
                     armed |= 1u << stage;
                     armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -178,7 +217,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+            const uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -191,7 +230,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
                         record_failure(p.ctrl, abort_flag, 2, stage, tile);
@@ -200,7 +239,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
                     }
                     ptx::tc_fence_after_sync();
                     const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
-                    const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * C::kBTileBytes);
+                    const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units per step
                         ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
@@ -220,6 +259,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
         const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31 belong to this warp
         const int row_in_tile = quarter * 32 + lane;
         int local = 0;
+        grid_dependency_wait();                           // the partial states may still be read by an earlier merge
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
             int m_tile, n_tile;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
@@ -233,7 +273,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
             ptx::tc_fence_after_sync();
             const int n0 = n_tile * BN;
             const int ncols = min(BN, p.V - n0);
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccStride);
             State st = state_empty();
             for (int c = 0; c * 32 < ncols; ++c) {
                 float v[32];
@@ -261,12 +301,15 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------
-// LayerNorm: h [M, d] (row stride ld_h) -> y [M, d] bf16, one warp per row.
+// LayerNorm: h [M, d] (row stride ld_h) -> y [M, d] bf16, one warp per row.  With VPL > 0 the row stays in
+// registers (VPL 16-byte vectors per lane, d <= 256 * VPL) and is read once; VPL = 0 re-reads it per pass.
 // ---------------------------------------------------------------------------------------------
+template <int VPL>
 __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat16* __restrict__ h, long long ld_h,
                                                               const float* __restrict__ gamma,
                                                               const float* __restrict__ beta, float ln_eps,
                                                               __nv_bfloat16* __restrict__ y, int M, int d) {
+    launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -274,13 +317,37 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat1
     const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)row * ld_h);
     uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
     const float inv_d = 1.f / (float)d;
-    float sum = 0.f;
-    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
-    const float mu = warp_sum(sum) * inv_d;
-    float sq = 0.f;
-    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
-    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
-    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+    grid_dependency_wait();                              // h may be an earlier kernel's output; y may still be read
+    if constexpr (VPL > 0) {
+        uint4 x[VPL];
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            x[k] = c < nvec ? ld_stream_v4(hrow + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) sum += vec8_sum(x[k]);
+        const float mu = warp_sum(sum) * inv_d;
+        float sq = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (lane + 32 * k < nvec) sq = vec8_sqdev(x[k], mu, sq);
+        const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            if (c < nvec) yrow[c] = layer_norm_vec8(x[k], mu, rstd, gamma, beta, c);
+        }
+    } else {
+        float sum = 0.f;
+        for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
+        const float mu = warp_sum(sum) * inv_d;
+        float sq = 0.f;
+        for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
+        const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
+        for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -290,9 +357,11 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
                                                          const float* __restrict__ tau_per_row, float tau,
                                                          int* argmax, float* entropy, float* maxprob,
                                                          unsigned char* exit_mask) {
+    launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
+    grid_dependency_wait();                              // the partial states come from the GEMM kernel
     // Lane-strided over the tiles, eight independent loads at a time; then the lanes reduce.
     State v[9];
     v[8] = state_empty();                                         // running result of this lane
@@ -311,28 +380,76 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-template <int BN>
+// Every kernel of the path is launched with programmatic stream serialization: its prologue (and, in the
+// GEMM, the first weight tiles) overlaps the tail of the kernel before it.
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+constexpr int kMinTileN = 64;
+
+// Ring depth for a runtime tile width.
+int stages_for(int bn) {
+    const size_t stage = kATileBytes + (size_t)bn * BK * 2;
+    const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
+    return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
+}
+
+template <int BN_T>
 ee_status launch_gemm(const CUtensorMap& tm_y, const CUtensorMap& tm_w, const GemmParams& p, int grid, int device,
                       cudaStream_t stream) {
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
-        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<BN>::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kGemmSmemBudget) != cudaSuccess)
             return EE_ERR_CUDA;
         configured[device] = true;
     }
-    exit_head_gemm_kernel<BN><<<grid, kGemmThreads, Cfg<BN>::kSmemBytes, stream>>>(tm_y, tm_w, p);
-    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
+                             : (size_t)p.n_stages * (kATileBytes + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
+    return launch_pdl(exit_head_gemm_kernel<BN_T>, grid, kGemmThreads, smem, stream, tm_y, tm_w, p) == cudaSuccess
+               ? EE_OK
+               : EE_ERR_CUDA;
 }
 
+// Upper bound on the partial states of M rows whatever tile width the launch picks.
 size_t partials_bytes(int M, int V) {
-    const int bn = gemm_tile_n(M);
+    const int bn = M > 1024 ? 256 : kMinTileN;
     return align_up((size_t)M * ((V + bn - 1) / bn) * sizeof(State), 256);
 }
 
 }  // namespace
 
-int gemm_tile_n(int M) { return M > 1024 ? 256 : 128; }
+// Large M: 256, the widest accumulator (two fit in tensor memory), which maximises the reuse of each y tile.
+// Up to 1024 rows the weights are read about once and the launch is bound by HBM and by how evenly the
+// tiles fill the SMs: the width in 64..256 (multiple of 16) that minimises waves x (width + fixed cost).
+int gemm_tile_n(int M, int V, int num_sms) {
+    if (M > 1024) return 256;
+    const long long m_tiles = (M + BM - 1) / BM;
+    int best = 128;
+    long long best_cost = -1;
+    for (int bn = kMinTileN; bn <= 256; bn += 16) {
+        const long long tiles = m_tiles * ((V + bn - 1) / bn);
+        const long long waves = (tiles + num_sms - 1) / num_sms;
+        const long long cost = waves * (bn + 16);
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && bn > best)) {
+            best = bn;
+            best_cost = cost;
+        }
+    }
+    return best;
+}
 
 size_t gemm_workspace_bytes(int M, int d, int V) {
     return partials_bytes(M, V) + align_up((size_t)M * d * sizeof(__nv_bfloat16), 256);
@@ -342,11 +459,18 @@ ee_status gemm_launch(const HeadArgs& a) {
     unsigned char* ws = static_cast<unsigned char*>(a.workspace);
     State* partials = reinterpret_cast<State*>(ws + kCtrlBytes);
     __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + partials_bytes(a.M, a.V));
-    const int bn = gemm_tile_n(a.M);
+    const int bn = gemm_tile_n(a.M, a.V, a.num_sms);
 
-    layer_norm_rows_kernel<<<(a.M + 7) / 8, 256, 0, a.stream>>>(static_cast<const __nv_bfloat16*>(a.h), a.ld_h, a.gamma,
-                                                                a.beta, a.ln_eps, y, a.M, a.d);
-    if (cudaGetLastError() != cudaSuccess) return EE_ERR_CUDA;
+    const __nv_bfloat16* h = static_cast<const __nv_bfloat16*>(a.h);
+    const int ln_grid = (a.M + 7) / 8;
+    cudaError_t err;
+    if (a.d <= 1024)
+        err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
+    else if (a.d <= 2048)
+        err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
+    else
+        err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
+    if (err != cudaSuccess) return EE_ERR_CUDA;
 
     CUtensorMap tm_y, tm_w;
     if (!make_tile_map(&tm_y, y, a.M, a.d, BM) || !make_tile_map(&tm_w, a.W, a.V, a.d, bn)) return EE_ERR_CUDA;
@@ -360,15 +484,17 @@ ee_status gemm_launch(const HeadArgs& a) {
     p.k_blocks = (a.d + BK - 1) / BK;
     p.partials = partials;
     p.ctrl = reinterpret_cast<Control*>(ws);
+    p.bn = bn;
+    p.n_stages = stages_for(bn);
     const long long total = (long long)p.m_tiles * p.n_tiles;
     const int grid = (int)(total < a.num_sms ? total : a.num_sms);
-    const ee_status st = (bn == 256) ? launch_gemm<256>(tm_y, tm_w, p, grid, a.device, a.stream)
-                                     : launch_gemm<128>(tm_y, tm_w, p, grid, a.device, a.stream);
+    const ee_status st = (a.M > 1024) ? launch_gemm<256>(tm_y, tm_w, p, grid, a.device, a.stream)
+                                      : launch_gemm<0>(tm_y, tm_w, p, grid, a.device, a.stream);
     if (st != EE_OK) return st;
 
-    merge_rows_kernel<<<(a.M + 7) / 8, 256, 0, a.stream>>>(partials, p.n_tiles, a.M, a.tau_per_row, a.tau, a.argmax,
-                                                           a.entropy, a.maxprob, a.exit_mask);
-    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    err = launch_pdl(merge_rows_kernel, (a.M + 7) / 8, 256, 0, a.stream, (const State*)partials, p.n_tiles, a.M,
+                     a.tau_per_row, a.tau, a.argmax, a.entropy, a.maxprob, a.exit_mask);
+    return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 }  // namespace ee

@@ -50,7 +50,7 @@ size_t skinny_workspace_bytes(int n_heads);
 ee_status skinny_launch(const HeadArgs* heads, int n_heads);
 
 // ---- tensor-core kernel (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge) ----
-int gemm_tile_n(int M);                    // vocabulary tile width used for M rows
+int gemm_tile_n(int M, int V, int num_sms);   // vocabulary tile width used for M rows on num_sms SMs
 size_t gemm_workspace_bytes(int M, int d, int V);
 ee_status gemm_launch(const HeadArgs& a);
 
