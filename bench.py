@@ -220,14 +220,12 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
         torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     wl.check()
-    total_ms = t0.elapsed_time(t1)
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    from paper_2407_21082_b200 import replicas
+    agg = replicas.aggregate_timing(t0.elapsed_time(t1), float(steps * len(wl.heads) * wl.M), dist, device="cuda")
+    total_ms = agg["elapsed_ms"]                     # the slowest rank
     heads_ms = sum(a.elapsed_time(b) for a, b in ev)
     n_heads = len(wl.heads)
-    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, head_call_us=1e3 * heads_ms / (steps * n_heads),
+    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"], head_call_us=1e3 * heads_ms / (steps * n_heads),
                 tail_us=1e3 * (total_ms - heads_ms) / steps, clocks=clocks)
 
 
@@ -380,12 +378,13 @@ def main():
 
     n_copies = {"c0": 8, "c1": 2}.get(args.workload, 2)
     path = dict(auto=0, stream=1, tcgen05=2, skinny=3)[args.path]
-    wl = Workload(args.workload, M, seed=rank, n_copies=n_copies, path=path)
+    from paper_2407_21082_b200 import replicas
+    wl = Workload(args.workload, M, seed=replicas.rank_seed(0, rank), n_copies=n_copies, path=path)
     config["kernel"] = args.path
     sampler = ClockSampler(local_rank) if rank == 0 else None
     res = measure(wl, args.steps, args.warmup, dist, sampler)
     n_heads = len(wl.heads)
-    value = world * n_heads * wl.M / (res["ms_per_step"] * 1e-3)
+    value = res["units_per_s"]                       # head evaluations of all ranks / time of the slowest rank
     config["l2"] = (f"inputs larger than L2: the step cycles through {wl.w_bytes_total / 1e6:.0f} MB of head weights "
                     f"({n_heads} heads x {n_copies} copies) against a 126 MB L2")
     config["parallelism"] = f"replicas x{world} (independent batches, no collective)"
