@@ -268,6 +268,32 @@ __device__ __forceinline__ void layer_norm_rows_in_regs(VecFn vec, const int (&r
 }
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  The next kernel of the stream may start once every CTA of this one has
+// passed launch_dependents(); a kernel calls grid_dependency_wait() before it touches anything an earlier
+// kernel of the stream writes or still reads (it returns when those kernels have completed and their stores
+// are visible).  Every kernel of the library is launched through launch_pdl, so completions stay in stream
+// order: a kernel cannot complete before it has passed its own wait.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Completion ticket and final merge shared by the one-launch kernels.
 // ---------------------------------------------------------------------------------------------
 // Thread 0 of a CTA, after a CTA-wide barrier that follows the CTA's partial-state stores: one acquire-release

@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned
     __shared__ int s_base, s_n;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row0 = blockIdx.x * kRowsPerCta;
+    launch_dependents();
+    grid_dependency_wait();                              // the mask and h come from earlier kernels of the stream
 
     int cnt = 0;
     for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (exit_mask[i] == 0);
@@ -65,7 +67,9 @@ __global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ dra
                                                      int* __restrict__ next_tok) {
     const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
+    launch_dependents();
     if (s >= S) return;
+    grid_dependency_wait();                              // tokens and mask come from earlier kernels of the stream
     int n = k;             // first slot that is not confident (draft length)
     int first_mis = k;     // first slot whose drafted token differs from the verifier's
     for (int base = 0; base < k; base += 32) {
@@ -92,17 +96,19 @@ ee_status compact_launch(const unsigned char* exit_mask, const void* h, long lon
                          int* kept_count, void* h_out, cudaStream_t stream) {
     if (M == 0) return cudaMemsetAsync(kept_count, 0, sizeof(int), stream) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
     const int grid = (M + kRowsPerCta - 1) / kRowsPerCta;
-    compact_kernel<<<grid, kCompactThreads, 0, stream>>>(exit_mask, static_cast<const __nv_bfloat16*>(h), ld_h, M, d,
-                                                         kept_idx, kept_count, static_cast<__nv_bfloat16*>(h_out));
-    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    return launch_pdl(compact_kernel, grid, kCompactThreads, 0, stream, exit_mask, static_cast<const __nv_bfloat16*>(h),
+                      ld_h, M, d, kept_idx, kept_count, static_cast<__nv_bfloat16*>(h_out)) == cudaSuccess
+               ? EE_OK
+               : EE_ERR_CUDA;
 }
 
 ee_status accept_launch(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k,
                         int kv, int* draft_len, int* accept_len, int* next_tok, cudaStream_t stream) {
     if (S == 0) return EE_OK;
-    accept_kernel<<<(S + 3) / 4, 128, 0, stream>>>(draft_tok, draft_exit_mask, verify_tok, S, k, kv, draft_len,
-                                                   accept_len, next_tok);
-    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    return launch_pdl(accept_kernel, (S + 3) / 4, 128, 0, stream, draft_tok, draft_exit_mask, verify_tok, S, k, kv,
+                      draft_len, accept_len, next_tok) == cudaSuccess
+               ? EE_OK
+               : EE_ERR_CUDA;
 }
 
 }  // namespace ee

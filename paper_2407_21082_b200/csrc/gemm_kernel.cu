@@ -49,12 +49,6 @@ struct GemmParams {
     int n_stages;          // smem ring depth
 };
 
-// Programmatic dependent launch: the next kernel of the stream may start once every CTA of this one has passed
-// launch_dependents(); a kernel calls grid_dependency_wait() before it touches anything an earlier kernel
-// of the stream writes (it returns when those kernels have completed and their stores are visible).
-__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
     const int per_group = kGroupM * n_tiles;
     const int grp = tile / per_group;
@@ -380,23 +374,6 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-// Every kernel of the path is launched with programmatic stream serialization: its prologue (and, in the
-// GEMM, the first weight tiles) overlaps the tail of the kernel before it.
-template <class... KArgs, class... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
-}
-
 constexpr int kMinTileN = 64;
 
 // Ring depth for a runtime tile width.

@@ -85,12 +85,6 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
                  : "memory");
 }
 
-// Programmatic dependent launch: the next kernel in the stream may start its preamble once every CTA of this
-// one has passed launch_dependents(); a kernel must call grid_dependency_wait() before it touches anything an
-// earlier kernel in the stream produces (here: h, the workspace and the outputs -- not the weights).
-__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 __device__ __forceinline__ void cp_async_16(void* dst_smem, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_addr(dst_smem)), "l"(src) : "memory");
 }
