@@ -420,7 +420,7 @@ def main():
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):
-                for mk in ("stream", "skinny"):
+                for mk in ("stream", "skinny", "gemm"):
                     os.environ["EE_MULTI_KERNEL"] = mk
                     w = Workload("c1", rows, seed=0, n_copies=2)
                     sweep[f"c1_M{rows}_multi_{mk}"] = round(measure(w, 300, 5)["head_call_us"], 2)

@@ -47,7 +47,7 @@ int auto_path(int M, int d) {
 }
 
 size_t workspace_bytes(int M, int d, int V) {
-    size_t need = gemm_workspace_bytes(M, d, V);
+    size_t need = gemm_workspace_bytes(M, d, V, 1);
     const size_t s = stream_workspace_bytes(1);
     if (s > need) need = s;
     if (skinny_workspace_bytes(1) > need) need = skinny_workspace_bytes(1);
@@ -124,7 +124,7 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
     if (path == EE_PATH_AUTO) path = auto_path(M, d);
     if (path == EE_PATH_STREAM) return stream_launch(&a, 1);
     if (path == EE_PATH_SKINNY) return skinny_launch(&a, 1);
-    return gemm_launch(a);
+    return gemm_launch(&a, 1);
 }
 
 size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
@@ -133,15 +133,16 @@ size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
     const int per_launch = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
     if (kCtrlBytes + skinny_workspace_bytes(per_launch) > need) need = kCtrlBytes + skinny_workspace_bytes(per_launch);
     if (kCtrlBytes + stream_workspace_bytes(per_launch) > need) need = kCtrlBytes + stream_workspace_bytes(per_launch);
+    if (kCtrlBytes + gemm_workspace_bytes(M, d, V, per_launch) > need) need = kCtrlBytes + gemm_workspace_bytes(M, d, V, per_launch);
     return need;
 }
 
 int ee_exit_head_multi_launches(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1 || M == 0) return 0;
     const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
-    if ((M <= 8 && stream_slab_rows(d, chunk) >= M) || (M <= 16 && skinny_supports(M, d)))
-        return (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
-    return n_heads * ee_exit_head_launches(M, d, V, EE_PATH_AUTO);
+    const int calls = (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
+    if (M <= 8 && stream_slab_rows(d, chunk) >= M) return calls;
+    return 3 * calls;                                  // LayerNorm, GEMM with fused statistics, merge
 }
 
 ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, void* workspace,
@@ -161,16 +162,16 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     const ee_status dev = current_device(&base.device, &base.num_sms);
     if (dev != EE_OK) return dev;
     // Which kernel batches the heads: the streaming kernel up to 8 rows (its mma.sync math keeps up with HBM
-    // there), the skinny tcgen05 kernel up to 16; larger batches run head by head.  EE_MULTI_KERNEL=stream |
-    // skinny | none overrides the choice (for A/B timing).
-    enum { kNone, kStream, kSkinny } mode = kNone;
+    // there), the tensor-core path (one LayerNorm, one GEMM, one merge launch for the batch of heads) above.
+    // EE_MULTI_KERNEL=stream | skinny | gemm | none overrides the choice (for A/B timing).
+    enum { kNone, kStream, kSkinny, kGemm } mode = kGemm;
     const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
     const bool stream_ok = stream_slab_rows(d, chunk) >= M;
     if (M <= 8 && stream_ok) mode = kStream;
-    else if (M <= 16 && skinny_supports(M, d)) mode = kSkinny;
     if (const char* force = getenv("EE_MULTI_KERNEL")) {
         if (!strcmp(force, "stream") && stream_ok) mode = kStream;
         else if (!strcmp(force, "skinny") && skinny_supports(M, d)) mode = kSkinny;
+        else if (!strcmp(force, "gemm")) mode = kGemm;
         else if (!strcmp(force, "none")) mode = kNone;
     }
     for (int k0 = 0; k0 < n_heads; k0 += kSkinnyMaxHeads) {
@@ -186,11 +187,11 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
             a[k].stream = static_cast<cudaStream_t>(stream);
         }
         if (mode != kNone) {
-            const ee_status st = mode == kStream ? stream_launch(a, n) : skinny_launch(a, n);
+            const ee_status st = mode == kStream ? stream_launch(a, n) : mode == kSkinny ? skinny_launch(a, n) : gemm_launch(a, n);
             if (st != EE_OK) return st;
         } else {
             for (int k = 0; k < n; ++k) {
-                const ee_status st = auto_path(M, d) == EE_PATH_STREAM ? stream_launch(&a[k], 1) : gemm_launch(a[k]);
+                const ee_status st = auto_path(M, d) == EE_PATH_STREAM ? stream_launch(&a[k], 1) : gemm_launch(&a[k], 1);
                 if (st != EE_OK) return st;
             }
         }

@@ -26,6 +26,7 @@ constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile
 constexpr int kATileBytes = BM * BK * 2;    // 16 KB
 
 constexpr int kBarBytes = 256;
+constexpr int kGemmMaxHeads = kGemmLaunchMaxHeads;
 constexpr int kMaxGemmStages = 12;
 constexpr size_t kGemmSmemBudget = 226 * 1024;
 
@@ -40,10 +41,17 @@ struct Cfg {
     static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;   // + slack to align to 1024
 };
 
+// One launch evaluates up to kGemmMaxHeads heads that share M, d and V: the tile list runs head by head.
+struct GemmMaps {
+    CUtensorMap y;                     // LayerNorm outputs of all heads stacked: [n_heads * M, d]
+    CUtensorMap w[kGemmMaxHeads];      // each head's weights [V, d]
+};
+
 struct GemmParams {
     int M, V, d;
     int m_tiles, n_tiles, k_blocks;
-    State* partials;       // [M][n_tiles]
+    int n_heads;
+    State* partials;       // [head][M][n_tiles]
     Control* ctrl;
     int bn;                // tile width (vocabulary rows per tile), a multiple of 16, <= 256
     int n_stages;          // smem ring depth
@@ -103,8 +111,7 @@ __device__ __forceinline__ void fold_chunk(State& st, const float (&v)[32], int 
 
 template <int BN_T>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
-                      const GemmParams p) {
+exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p) {
     using C = Cfg<BN_T>;
     const int BN = BN_T ? BN_T : p.bn;
     const int S = BN_T ? C::kStages : p.n_stages;
@@ -142,8 +149,8 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
         ptx::mbar_init(drain_bar, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
-        ptx::prefetch_tensormap(&tm_y);
-        ptx::prefetch_tensormap(&tm_w);
+        ptx::prefetch_tensormap(&maps.y);
+        for (int k = 0; k < p.n_heads; ++k) ptx::prefetch_tensormap(&maps.w[k]);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), C::kTmemCols);
@@ -154,7 +161,13 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
 
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int tiles_per_head = p.m_tiles * p.n_tiles;
+    const int total_tiles = p.n_heads * tiles_per_head;
+    // tile -> (head, m_tile, n_tile); within a head the order keeps concurrent CTAs on the same W tiles
+    auto locate = [&](int tile, int& head, int& m_tile, int& n_tile) {
+        head = tile / tiles_per_head;
+        tile_coords(tile - head * tiles_per_head, p.m_tiles, p.n_tiles, m_tile, n_tile);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -166,23 +179,24 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
             // requested before the dependency wait, the y tiles (written by the LayerNorm kernel) after it.
             int n_pre = 0;
             if ((int)blockIdx.x < total_tiles) {
-                int m_tile, n_tile;
-                tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                int head, m_tile, n_tile;
+                locate(blockIdx.x, head, m_tile, n_tile);
                 n_pre = min(S, p.k_blocks);
                 for (int kb = 0; kb < n_pre; ++kb) {
                     ptx::mbar_arrive_expect_tx(full_bar(kb), stage_bytes);
-                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &tm_w, kb * BK, n_tile * BN, full_bar(kb));
+                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN, full_bar(kb));
                     armed |= 1u << kb;
                 }
             }
             grid_dependency_wait();
             int issued = 0;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                int m_tile, n_tile;
-                tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                int head, m_tile, n_tile;
+                locate(tile, head, m_tile, n_tile);
+                const int y_row = head * p.M + m_tile * BM;   // rows past the head's M are never looked at
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
-                        ptx::tma_load_2d(a_base + stage * kATileBytes, &tm_y, kb * BK, m_tile * BM, full_bar(stage));
+                        ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                         continue;
                     }
@@ -192,8 +206,8 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
                         break;
                     }
                     ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
-                    ptx::tma_load_2d(a_base + stage * kATileBytes, &tm_y, kb * BK, m_tile * BM, full_bar(stage));
-                    ptx::tma_load_2d(b_base + stage * b_tile_bytes, &tm_w, kb * BK, n_tile * BN, full_bar(stage));
+                    ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                    ptx::tma_load_2d(b_base + stage * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN, full_bar(stage));
                     armed |= 1u << stage;
                     armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -255,8 +269,8 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
         int local = 0;
         grid_dependency_wait();                           // the partial states may still be read by an earlier merge
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
-            int m_tile, n_tile;
-            tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+            int head, m_tile, n_tile;
+            locate(tile, head, m_tile, n_tile);
             const int buf = local & 1;
             const uint32_t acc_phase = (local >> 1) & 1u;
             const bool landed = ptx::mbar_wait(tfull_bar(buf), acc_phase, abort_flag);
@@ -281,7 +295,7 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
             const int row = m_tile * BM + row_in_tile;
-            if (row < p.M) p.partials[(size_t)row * p.n_tiles + n_tile] = st;
+            if (row < p.M) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
         }
     }
 
@@ -295,24 +309,45 @@ exit_head_gemm_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------
-// LayerNorm: h [M, d] (row stride ld_h) -> y [M, d] bf16, one warp per row.  With VPL > 0 the row stays in
-// registers (VPL 16-byte vectors per lane, d <= 256 * VPL) and is read once; VPL = 0 re-reads it per pass.
+// LayerNorm of every head's input: h_k [M, d] (row stride ld_h) -> y [k][M, d] bf16, one warp per row,
+// blockIdx.y = head.  With VPL > 0 the row stays in registers (VPL 16-byte vectors per lane, d <= 256 * VPL)
+// and is read once; VPL = 0 re-reads it per pass.
 // ---------------------------------------------------------------------------------------------
+struct LnHeads {
+    const __nv_bfloat16* h[kGemmMaxHeads];
+    long long ld_h[kGemmMaxHeads];
+    const float* gamma[kGemmMaxHeads];
+    const float* beta[kGemmMaxHeads];
+};
+
 template <int VPL>
-__global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat16* __restrict__ h, long long ld_h,
-                                                              const float* __restrict__ gamma,
-                                                              const float* __restrict__ beta, float ln_eps,
-                                                              __nv_bfloat16* __restrict__ y, int M, int d) {
+__global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps,
+                                                              __nv_bfloat16* __restrict__ y_all, int M, int d) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
+    const int head = blockIdx.y;
     if (row >= M) return;
     const int nvec = d >> 3;
-    const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)row * ld_h);
-    uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
+    const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
+    const float* gamma = hs.gamma[head];
+    const float* beta = hs.beta[head];
+    uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * M + row) * d);
     const float inv_d = 1.f / (float)d;
-    grid_dependency_wait();                              // h may be an earlier kernel's output; y may still be read
     if constexpr (VPL > 0) {
+        // The LayerNorm parameters are weights, not results of an earlier kernel: fetched before the wait.
+        float4 g[VPL][2], b[VPL][2];
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            if (c < nvec) {
+                g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+                g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+                b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+                b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+            }
+        }
+        grid_dependency_wait();                          // h may be an earlier kernel's output; y may still be read
         uint4 x[VPL];
         float sum = 0.f;
 #pragma unroll
@@ -331,9 +366,10 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat1
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
-            if (c < nvec) yrow[c] = layer_norm_vec8(x[k], mu, rstd, gamma, beta, c);
+            if (c < nvec) yrow[c] = layer_norm_vec8(x[k], mu, rstd, g[k][0], g[k][1], b[k][0], b[k][1]);
         }
     } else {
+        grid_dependency_wait();
         float sum = 0.f;
         for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
         const float mu = warp_sum(sum) * inv_d;
@@ -346,15 +382,25 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __nv_bfloat1
 
 // ---------------------------------------------------------------------------------------------
 // Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
+// blockIdx.y = head.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials, int n_tiles, int M,
-                                                         const float* __restrict__ tau_per_row, float tau,
-                                                         int* argmax, float* entropy, float* maxprob,
-                                                         unsigned char* exit_mask) {
+struct MergeHeads {
+    const float* tau_per_row[kGemmMaxHeads];
+    float tau[kGemmMaxHeads];
+    int* argmax[kGemmMaxHeads];
+    float* entropy[kGemmMaxHeads];
+    float* maxprob[kGemmMaxHeads];
+    unsigned char* exit_mask[kGemmMaxHeads];
+};
+
+__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials_all, int n_tiles, int M,
+                                                         const __grid_constant__ MergeHeads hs) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
+    const int head = blockIdx.y;
     if (row >= M) return;
+    const State* partials = partials_all + ((size_t)head * M + row) * n_tiles;
     grid_dependency_wait();                              // the partial states come from the GEMM kernel
     // Lane-strided over the tiles, eight independent loads at a time; then the lanes reduce.
     State v[9];
@@ -363,12 +409,14 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int n = n0 + 32 * i;
-            v[i] = n < n_tiles ? state_load_cg(partials + (size_t)row * n_tiles + n) : state_empty();
+            v[i] = n < n_tiles ? state_load_cg(partials + n) : state_empty();
         }
         v[8] = state_combine<9>(v);
     }
     const State a = state_reduce_lanes<1, 16>(v[8]);
-    if (lane == 0) state_finish(a, tau_per_row ? tau_per_row[row] : tau, argmax, entropy, maxprob, exit_mask, row);
+    if (lane == 0)
+        state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
+                     hs.maxprob[head], hs.exit_mask[head], row);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -384,8 +432,7 @@ int stages_for(int bn) {
 }
 
 template <int BN_T>
-ee_status launch_gemm(const CUtensorMap& tm_y, const CUtensorMap& tm_w, const GemmParams& p, int grid, int device,
-                      cudaStream_t stream) {
+ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int device, cudaStream_t stream) {
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
         if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -395,12 +442,12 @@ ee_status launch_gemm(const CUtensorMap& tm_y, const CUtensorMap& tm_w, const Ge
     }
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
                              : (size_t)p.n_stages * (kATileBytes + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
-    return launch_pdl(exit_head_gemm_kernel<BN_T>, grid, kGemmThreads, smem, stream, tm_y, tm_w, p) == cudaSuccess
+    return launch_pdl(exit_head_gemm_kernel<BN_T>, grid, kGemmThreads, smem, stream, maps, p) == cudaSuccess
                ? EE_OK
                : EE_ERR_CUDA;
 }
 
-// Upper bound on the partial states of M rows whatever tile width the launch picks.
+// Upper bound on the partial states of M rows of one head whatever tile width the launch picks.
 size_t partials_bytes(int M, int V) {
     const int bn = M > 1024 ? 256 : kMinTileN;
     return align_up((size_t)M * ((V + bn - 1) / bn) * sizeof(State), 256);
@@ -411,13 +458,13 @@ size_t partials_bytes(int M, int V) {
 // Large M: 256, the widest accumulator (two fit in tensor memory), which maximises the reuse of each y tile.
 // Up to 1024 rows the weights are read about once and the launch is bound by HBM and by how evenly the
 // tiles fill the SMs: the width in 64..256 (multiple of 16) that minimises waves x (width + fixed cost).
-int gemm_tile_n(int M, int V, int num_sms) {
+int gemm_tile_n(int M, int V, int n_heads, int num_sms) {
     if (M > 1024) return 256;
     const long long m_tiles = (M + BM - 1) / BM;
     int best = 128;
     long long best_cost = -1;
     for (int bn = kMinTileN; bn <= 256; bn += 16) {
-        const long long tiles = m_tiles * ((V + bn - 1) / bn);
+        const long long tiles = n_heads * m_tiles * ((V + bn - 1) / bn);
         const long long waves = (tiles + num_sms - 1) / num_sms;
         const long long cost = waves * (bn + 16);
         if (best_cost < 0 || cost < best_cost || (cost == best_cost && bn > best)) {
@@ -428,29 +475,47 @@ int gemm_tile_n(int M, int V, int num_sms) {
     return best;
 }
 
-size_t gemm_workspace_bytes(int M, int d, int V) {
-    return partials_bytes(M, V) + align_up((size_t)M * d * sizeof(__nv_bfloat16), 256);
+size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
+    return (size_t)n_heads * (partials_bytes(M, V) + align_up((size_t)M * d * sizeof(__nv_bfloat16), 256));
 }
 
-ee_status gemm_launch(const HeadArgs& a) {
+ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
+    if (n_heads < 1 || n_heads > kGemmMaxHeads) return EE_ERR_SHAPE;
+    const HeadArgs& a = heads[0];
     unsigned char* ws = static_cast<unsigned char*>(a.workspace);
     State* partials = reinterpret_cast<State*>(ws + kCtrlBytes);
-    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + partials_bytes(a.M, a.V));
-    const int bn = gemm_tile_n(a.M, a.V, a.num_sms);
+    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + (size_t)n_heads * partials_bytes(a.M, a.V));
+    const int bn = gemm_tile_n(a.M, a.V, n_heads, a.num_sms);
 
-    const __nv_bfloat16* h = static_cast<const __nv_bfloat16*>(a.h);
-    const int ln_grid = (a.M + 7) / 8;
+    LnHeads ln = {};
+    MergeHeads mg = {};
+    for (int k = 0; k < n_heads; ++k) {
+        ln.h[k] = static_cast<const __nv_bfloat16*>(heads[k].h);
+        ln.ld_h[k] = heads[k].ld_h;
+        ln.gamma[k] = heads[k].gamma;
+        ln.beta[k] = heads[k].beta;
+        mg.tau_per_row[k] = heads[k].tau_per_row;
+        mg.tau[k] = heads[k].tau;
+        mg.argmax[k] = heads[k].argmax;
+        mg.entropy[k] = heads[k].entropy;
+        mg.maxprob[k] = heads[k].maxprob;
+        mg.exit_mask[k] = heads[k].exit_mask;
+    }
+    const dim3 row_grid((a.M + 7) / 8, n_heads);
     cudaError_t err;
-    if (a.d <= 1024)
-        err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
-    else if (a.d <= 2048)
-        err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
-    else
-        err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, h, a.ld_h, a.gamma, a.beta, a.ln_eps, y, a.M, a.d);
+    if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else err = launch_pdl(layer_norm_rows_kernel<0>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     if (err != cudaSuccess) return EE_ERR_CUDA;
 
-    CUtensorMap tm_y, tm_w;
-    if (!make_tile_map(&tm_y, y, a.M, a.d, BM) || !make_tile_map(&tm_w, a.W, a.V, a.d, bn)) return EE_ERR_CUDA;
+    // 256-byte L2 promotion for the weights while they are read about once: a tile load touches 128 bytes of
+    // each row, and fetching the neighbouring 128 bytes (the next k-block's) with it lets the row-strided
+    // pattern stream from HBM at the rate of a contiguous copy (measured: 6.9 against 5.5 TB/s).
+    const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+    GemmMaps maps;
+    if (!make_tile_map(&maps.y, y, n_heads * a.M, a.d, BM)) return EE_ERR_CUDA;
+    for (int k = 0; k < kGemmMaxHeads; ++k)
+        if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, bn, promo)) return EE_ERR_CUDA;
 
     GemmParams p;
     p.M = a.M;
@@ -459,18 +524,18 @@ ee_status gemm_launch(const HeadArgs& a) {
     p.m_tiles = (a.M + BM - 1) / BM;
     p.n_tiles = (a.V + bn - 1) / bn;
     p.k_blocks = (a.d + BK - 1) / BK;
+    p.n_heads = n_heads;
     p.partials = partials;
     p.ctrl = reinterpret_cast<Control*>(ws);
     p.bn = bn;
     p.n_stages = stages_for(bn);
-    const long long total = (long long)p.m_tiles * p.n_tiles;
+    const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
     const int grid = (int)(total < a.num_sms ? total : a.num_sms);
-    const ee_status st = (a.M > 1024) ? launch_gemm<256>(tm_y, tm_w, p, grid, a.device, a.stream)
-                                      : launch_gemm<0>(tm_y, tm_w, p, grid, a.device, a.stream);
+    const ee_status st = (a.M > 1024) ? launch_gemm<256>(maps, p, grid, a.device, a.stream)
+                                      : launch_gemm<0>(maps, p, grid, a.device, a.stream);
     if (st != EE_OK) return st;
 
-    err = launch_pdl(merge_rows_kernel, (a.M + 7) / 8, 256, 0, a.stream, (const State*)partials, p.n_tiles, a.M,
-                     a.tau_per_row, a.tau, a.argmax, a.entropy, a.maxprob, a.exit_mask);
+    err = launch_pdl(merge_rows_kernel, row_grid, 256, 0, a.stream, (const State*)partials, p.n_tiles, a.M, mg);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 

@@ -49,10 +49,12 @@ size_t skinny_workspace_bytes(int n_heads);
 // parameters, W, thresholds and outputs.
 ee_status skinny_launch(const HeadArgs* heads, int n_heads);
 
-// ---- tensor-core kernel (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge) ----
-int gemm_tile_n(int M, int V, int num_sms);   // vocabulary tile width used for M rows on num_sms SMs
-size_t gemm_workspace_bytes(int M, int d, int V);
-ee_status gemm_launch(const HeadArgs& a);
+// ---- tensor-core path (LayerNorm kernel, TMA + tcgen05 GEMM with fused statistics, merge): three launches
+//      for up to four heads that share M, d, V, ln_eps, workspace, stream and device ----
+constexpr int kGemmLaunchMaxHeads = 4;
+int gemm_tile_n(int M, int V, int n_heads, int num_sms);   // vocabulary tile width used for M rows on num_sms SMs
+size_t gemm_workspace_bytes(int M, int d, int V, int n_heads);
+ee_status gemm_launch(const HeadArgs* heads, int n_heads);
 
 // ---- compaction and DSSD accept ----
 ee_status compact_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,

@@ -205,9 +205,15 @@ def test_device_side_argument_errors(ee):
     ("n32_two_launches", 20, 256, 2111, 5),       # five heads: a launch of four and a launch of one
     ("n64_single_buffer", 64, 1024, 1200, 3),     # activations too large for a second buffer
     ("wide_single_buffer", 12, 2560, 900, 2),
-    ("not_batched", 40, 72, 500, 3),              # d % 64 != 0: falls back to one launch per head
+    ("odd_width", 40, 72, 500, 3),                # d % 64 != 0: the tensor-core path's ragged last k-block
+    ("two_m_tiles", 150, 128, 1000, 3),           # stacked LayerNorm outputs: a 128-row tile reaches into the next head
+    ("one_row", 1, 512, 777, 4),
 ])
-def test_multi_head_call_matches_oracle(ee, name, M, d, V, n_heads):
+@pytest.mark.parametrize("kernel", ["auto", "stream", "skinny", "gemm", "none"])
+def test_multi_head_call_matches_oracle(ee, monkeypatch, name, M, d, V, n_heads, kernel):
+    # The library reads EE_MULTI_KERNEL per call; a kernel that does not take the shape leaves the default choice.
+    if kernel != "auto":
+        monkeypatch.setenv("EE_MULTI_KERNEL", kernel)
     cfg = gen.make_config("c1", seed=17, planted=True, M=M, d=d, V=V, heads=n_heads)
     h = dev_bf16(cfg["h"])
     taus = [0.5 + 0.5 * k for k in range(n_heads)]
