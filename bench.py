@@ -229,6 +229,45 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
                 tail_us=1e3 * (total_ms - heads_ms) / steps, clocks=clocks)
 
 
+# DRAM bytes (read + write) one launch of the dominant kernel moved in the ncu captures summarised under
+# profiles/, by (workload, rows).  A figure holds only for the kernel sources it was taken on: it is reported
+# while the SHA-256 of those sources still matches and as null afterwards.
+CSRC = os.path.join(ROOT, "paper_2407_21082_b200", "csrc")
+TRAFFIC = {
+    ("c1", 64): dict(bytes=309.605376e6 + 4.559360e6, heads_per_launch=3, kernel="exit_head_gemm_kernel<0>",
+                     sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
+                     sha256="21185e39d99e5d8990c5fe13ac3f06b2c3062d443b7a68ea9c7c9d829e064cca", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
+    ("c1", 8): dict(bytes=309.227008e6 + 4.190464e6, heads_per_launch=3, kernel="exit_head_stream_kernel<1>",
+                    sources=("stream_kernel.cu", "common.cuh", "sm100_ptx.cuh"),
+                    sha256="9c82612b27bc4a17d5700ef60f3929fd4964868a364d404a5e7a9a69e99a81f3", profile="profiles/exit_head_stream_kernel_c1_M8.md"),
+    ("c4", 16384): dict(bytes=2146.557e6 + 53.811456e6, heads_per_launch=1, kernel="exit_head_gemm_kernel<256>",
+                        sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
+                        sha256="21185e39d99e5d8990c5fe13ac3f06b2c3062d443b7a68ea9c7c9d829e064cca", profile="profiles/exit_head_gemm_kernel_c4.md"),
+}
+
+
+def sources_sha256(names) -> str:
+    import hashlib
+    hsh = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(CSRC, n), "rb") as f:
+            hsh.update(f.read())
+    return hsh.hexdigest()
+
+
+def measured_traffic(wl: "Workload"):
+    """(bytes per launch, note) from the committed ncu capture of this workload's dominant kernel, or (None, why)."""
+    t = TRAFFIC.get((wl.name, wl.M))
+    if t is None or not wl.path == 0:
+        return None, "no ncu capture of this workload"
+    heads_per_launch = len(wl.heads) if wl.multi else 1
+    if heads_per_launch != t["heads_per_launch"]:
+        return None, "no ncu capture of this launch shape"
+    if sources_sha256(t["sources"]) != t["sha256"]:
+        return None, "kernel sources changed since the ncu capture in " + t["profile"]
+    return t["bytes"], f"dram read+write of one {t['kernel']} launch ({t['heads_per_launch']} head(s)), {t['profile']}"
+
+
 def roofline(wl: Workload, head_call_us: float, peaks: dict, src: str) -> dict:
     gbs = wl.bytes_per_call / (head_call_us * 1e-6) / 1e9
     tfs = wl.flops_per_call / (head_call_us * 1e-6) / 1e12
@@ -393,6 +432,12 @@ def main():
                 data="synthetic", config=config, clocks=res["clocks"], gpu_launches=wl.launches_per_step * args.steps,
                 head_call_us=res["head_call_us"], tail_us=res["tail_us"])
     line["roofline"] = roofline(wl, res["head_call_us"], peaks, peak_src)
+    traffic, traffic_note = measured_traffic(wl)
+    heads_per_launch = n_heads if wl.multi else 1
+    line["roofline"].update(traffic=traffic, traffic_note=traffic_note,
+                            launch=dict(heads=heads_per_launch, algorithmic_bytes=heads_per_launch * wl.bytes_per_call,
+                                        flops=heads_per_launch * wl.flops_per_call,
+                                        us=heads_per_launch * res["head_call_us"]))
     line["roofline"]["kernel"] = (("ee_exit_head_multi: %d heads in one launch; " % n_heads if wl.multi else
                                    "one ee_exit_head call (%d launch(es)); " % wl.head_launches) +
                                   "duration = CUDA events around the head evaluations of each step, averaged per head")
