@@ -195,38 +195,58 @@ class Workload:
 
 
 def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSampler | None = None) -> dict:
-    """Times `steps` steps with CUDA events on the launching stream; also the head calls alone inside them."""
+    """Times `steps` whole steps, then the head evaluations of `steps` steps alone, with CUDA events on the
+    launching stream.
+
+    The kernels of a step are chained by programmatic dependent launch, and an event recorded between two
+    launches breaks that chain (measured: about 5 us per event), so neither region has events inside it: the
+    first gives the step time (the metric), the second the duration of the dominant launch for the roofline.
+    A third, shorter region with an event pair around the head evaluation of every step is reported beside
+    them (`head_call_us_inner_events`) to show what the events cost.
+    """
     torch = wl.torch
     for _ in range(warmup):
         wl.step()
     wl.check()
     if dist is not None:
         dist.barrier()
-        torch.cuda.synchronize()
+    torch.cuda.synchronize()
     if sampler:
         sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0, t1, t2, t3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
     t0.record()
-    for a, b in ev:
-        a.record()
-        wl.run_heads()
-        b.record()
-        wl.run_tail()
+    for _ in range(steps):
+        wl.step()
     t1.record()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
+    t2.record()
+    for _ in range(steps):
+        wl.run_heads()
+    t3.record()
+    torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
+    n_inner = min(steps, 500)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inner)]
+    for a, b in ev:
+        a.record()
+        wl.run_heads()
+        b.record()
+        wl.run_tail()
+    torch.cuda.synchronize()
     wl.check()
     from paper_2407_21082_b200 import replicas
-    agg = replicas.aggregate_timing(t0.elapsed_time(t1), float(steps * len(wl.heads) * wl.M), dist, device="cuda")
-    total_ms = agg["elapsed_ms"]                     # the slowest rank
-    heads_ms = sum(a.elapsed_time(b) for a, b in ev)
     n_heads = len(wl.heads)
-    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"], head_call_us=1e3 * heads_ms / (steps * n_heads),
-                tail_us=1e3 * (total_ms - heads_ms) / steps, clocks=clocks)
+    agg = replicas.aggregate_timing(t0.elapsed_time(t1), float(steps * n_heads * wl.M), dist, device="cuda")
+    total_ms = agg["elapsed_ms"]                     # the slowest rank
+    heads_ms = t2.elapsed_time(t3)
+    inner_ms = sum(a.elapsed_time(b) for a, b in ev)
+    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"],
+                head_call_us=1e3 * heads_ms / (steps * n_heads),
+                head_call_us_inner_events=1e3 * inner_ms / (n_inner * n_heads),
+                tail_us=1e3 * (t0.elapsed_time(t1) - heads_ms) / steps, clocks=clocks)
 
 
 # DRAM bytes (read + write) one launch of the dominant kernel moved in the ncu captures summarised under
@@ -430,7 +450,8 @@ def main():
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                 data="synthetic", config=config, clocks=res["clocks"], gpu_launches=wl.launches_per_step * args.steps,
-                head_call_us=res["head_call_us"], tail_us=res["tail_us"])
+                head_call_us=res["head_call_us"], head_call_us_inner_events=res["head_call_us_inner_events"],
+                tail_us=res["tail_us"])
     line["roofline"] = roofline(wl, res["head_call_us"], peaks, peak_src)
     traffic, traffic_note = measured_traffic(wl)
     heads_per_launch = n_heads if wl.multi else 1
@@ -440,7 +461,9 @@ def main():
                                         us=heads_per_launch * res["head_call_us"]))
     line["roofline"]["kernel"] = (("ee_exit_head_multi: %d heads in one launch; " % n_heads if wl.multi else
                                    "one ee_exit_head call (%d launch(es)); " % wl.head_launches) +
-                                  "duration = CUDA events around the head evaluations of each step, averaged per head")
+                                  "duration = CUDA events around `steps` consecutive head evaluations (no event between launches: "
+                                  "one would break their programmatic dependent launch chain), averaged per head; "
+                                  "tail_us = step time minus that")
     config["heads_call"] = "ee_exit_head_multi" if wl.multi else "ee_exit_head per head"
     if rank == 0:
         line["e2e"] = measure_e2e(wl, max(10, args.steps // 4), 3)

@@ -40,11 +40,10 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 bool sizes_ok(int M, int d, int V) { return M >= 0 && V >= 1 && d >= 8 && d <= 8192 && (d % 8) == 0; }
 
-// Kernel used for M rows when the caller does not choose.
-int auto_path(int M, int d) {
-    const int slab = stream_slab_rows(d, 1);
-    return (slab > 0 && M <= slab && M <= 16) ? EE_PATH_STREAM : EE_PATH_TCGEN05;
-}
+// Kernel used when the caller does not choose: the tensor-core path for every size.  (Measured per head call,
+// d = 512..2560, V = 50304: it is ahead of the streaming kernel from M = 1 on, 16.3 against 17.4 us at
+// d = 512 M = 1 and 41.8 against 56.7 us at d = 2048 M = 16; the other two kernels stay selectable.)
+int auto_path(int, int) { return EE_PATH_TCGEN05; }
 
 size_t workspace_bytes(int M, int d, int V) {
     size_t need = gemm_workspace_bytes(M, d, V, 1);
@@ -139,9 +138,7 @@ size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
 
 int ee_exit_head_multi_launches(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1 || M == 0) return 0;
-    const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
     const int calls = (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
-    if (M <= 8 && stream_slab_rows(d, chunk) >= M) return calls;
     return 3 * calls;                                  // LayerNorm, GEMM with fused statistics, merge
 }
 
@@ -161,13 +158,12 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     HeadArgs base;
     const ee_status dev = current_device(&base.device, &base.num_sms);
     if (dev != EE_OK) return dev;
-    // Which kernel batches the heads: the streaming kernel up to 8 rows (its mma.sync math keeps up with HBM
-    // there), the tensor-core path (one LayerNorm, one GEMM, one merge launch for the batch of heads) above.
-    // EE_MULTI_KERNEL=stream | skinny | gemm | none overrides the choice (for A/B timing).
+    // The tensor-core path batches the heads (one LayerNorm, one GEMM, one merge launch for up to four).
+    // EE_MULTI_KERNEL=stream | skinny | gemm | none overrides the choice (for A/B timing; a kernel that does
+    // not take the shape leaves the default).
     enum { kNone, kStream, kSkinny, kGemm } mode = kGemm;
     const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
     const bool stream_ok = stream_slab_rows(d, chunk) >= M;
-    if (M <= 8 && stream_ok) mode = kStream;
     if (const char* force = getenv("EE_MULTI_KERNEL")) {
         if (!strcmp(force, "stream") && stream_ok) mode = kStream;
         else if (!strcmp(force, "skinny") && skinny_supports(M, d)) mode = kSkinny;

@@ -43,7 +43,7 @@ struct Cfg {
 
 // One launch evaluates up to kGemmMaxHeads heads that share M, d and V: the tile list runs head by head.
 struct GemmMaps {
-    CUtensorMap y;                     // LayerNorm outputs of all heads stacked: [n_heads * M, d]
+    CUtensorMap y;                     // LayerNorm outputs of all heads, each padded to whole tiles: [n_heads * m_tiles * 128, d]
     CUtensorMap w[kGemmMaxHeads];      // each head's weights [V, d]
 };
 
@@ -193,7 +193,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                 int head, m_tile, n_tile;
                 locate(tile, head, m_tile, n_tile);
-                const int y_row = head * p.M + m_tile * BM;   // rows past the head's M are never looked at
+                const int y_row = (head * p.m_tiles + m_tile) * BM;   // each head's rows are padded to whole tiles
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
                         ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
@@ -327,12 +327,19 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int head = blockIdx.y;
-    if (row >= M) return;
+    const int m_pad = (M + BM - 1) / BM * BM;            // a head's rows are padded to whole 128-row tiles
+    if (row >= m_pad) return;
     const int nvec = d >> 3;
+    uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * m_pad + row) * d);
+    if (row >= M) {
+        // Padding row: zeros, so that the rows of a tile that carry no token cost the tensor pipe no switching.
+        grid_dependency_wait();
+        for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
     const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
     const float* gamma = hs.gamma[head];
     const float* beta = hs.beta[head];
-    uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * M + row) * d);
     const float inv_d = 1.f / (float)d;
     if constexpr (VPL > 0) {
         // The LayerNorm parameters are weights, not results of an earlier kernel: fetched before the wait.
@@ -453,6 +460,12 @@ size_t partials_bytes(int M, int V) {
     return align_up((size_t)M * ((V + bn - 1) / bn) * sizeof(State), 256);
 }
 
+// The stacked LayerNorm outputs, every head's rows padded to whole 128-row tiles (padding rows are written as
+// zeros): each tile the GEMM loads lies inside the buffer, a plain copy for the TMA unit, which it serves
+// faster than a tile it has to fill with zeros itself, and no tile holds another head's rows.
+size_t y_rows(int M, int n_heads) { return (size_t)n_heads * (size_t)((M + BM - 1) / BM) * BM; }
+size_t y_bytes(int M, int d, int n_heads) { return align_up(y_rows(M, n_heads) * d * sizeof(__nv_bfloat16), 256); }
+
 }  // namespace
 
 // Large M: 256, the widest accumulator (two fit in tensor memory), which maximises the reuse of each y tile.
@@ -476,7 +489,7 @@ int gemm_tile_n(int M, int V, int n_heads, int num_sms) {
 }
 
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
-    return (size_t)n_heads * (partials_bytes(M, V) + align_up((size_t)M * d * sizeof(__nv_bfloat16), 256));
+    return (size_t)n_heads * partials_bytes(M, V) + y_bytes(M, d, n_heads);
 }
 
 ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
@@ -502,10 +515,11 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         mg.exit_mask[k] = heads[k].exit_mask;
     }
     const dim3 row_grid((a.M + 7) / 8, n_heads);
+    const dim3 ln_grid((a.M + BM - 1) / BM * (BM / 8), n_heads);
     cudaError_t err;
-    if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else err = launch_pdl(layer_norm_rows_kernel<0>, row_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     if (err != cudaSuccess) return EE_ERR_CUDA;
 
     // 256-byte L2 promotion for the weights while they are read about once: a tile load touches 128 bytes of
@@ -513,7 +527,7 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     // pattern stream from HBM at the rate of a contiguous copy (measured: 6.9 against 5.5 TB/s).
     const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     GemmMaps maps;
-    if (!make_tile_map(&maps.y, y, n_heads * a.M, a.d, BM)) return EE_ERR_CUDA;
+    if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, BM)) return EE_ERR_CUDA;
     for (int k = 0; k < kGemmMaxHeads; ++k)
         if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, bn, promo)) return EE_ERR_CUDA;
 
