@@ -149,7 +149,7 @@ class Workload:
         self.head_launches = ee.ee_exit_head_launches(self.M, self.d, self.V, path)
         heads_launches = (ee.ee_exit_head_multi_launches(len(self.heads), self.M, self.d, self.V) if self.multi
                           else len(self.heads) * self.head_launches)
-        self.launches_per_step = heads_launches + 1 + (1 if self.S > 0 else 0)
+        self.launches_per_step = heads_launches + 1          # + one launch for compaction and accept together
         self.bytes_per_call, self.flops_per_call = _algorithmic(self.M, self.d, self.V)
         self.w_bytes_total = sum(w.numel() * 2 for hd in self.heads for w in hd["W"])
         self.prepare()
@@ -165,13 +165,18 @@ class Workload:
             self.head_calls = [[ee.prepare_exit_head(self.h[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], self.tau,
                                                      out=self.outs[i], workspace=self.ws, path=self.path)
                                 for i, hd in enumerate(self.heads)] for c in range(self.n_copies)]
-        self.compact_call = ee.prepare_compact(self.outs[0]["exit_mask"], self.h[0], out=self.comp)
-        self.accept_call = None
-        if self.S > 0:
-            n = self.S * self.k
-            self.accept_call = ee.prepare_accept(self.outs[0]["argmax"][:n].view(self.S, self.k),
-                                                 self.outs[0]["exit_mask"][:n].view(self.S, self.k),
-                                                 self.outs[-1]["argmax"][:n].view(self.S, self.k), out=self.acc)
+        self.tail_call = self.prepare_tail(self.h[0])
+
+    def prepare_tail(self, h):
+        """Compaction of head 0's survivors (with the gather from `h`) and the DSSD count, in one launch."""
+        ee = self.ee
+        if self.S == 0:
+            return ee.prepare_compact(self.outs[0]["exit_mask"], h, out=self.comp)
+        n = self.S * self.k
+        return ee.prepare_compact_accept(self.outs[0]["exit_mask"], h, self.outs[0]["argmax"][:n].view(self.S, self.k),
+                                         self.outs[0]["exit_mask"][:n].view(self.S, self.k),
+                                         self.outs[-1]["argmax"][:n].view(self.S, self.k),
+                                         out=dict(compact=self.comp, accept=self.acc))
 
     def run_heads(self):
         for call in self.head_calls[self.calls % self.n_copies]:
@@ -179,9 +184,7 @@ class Workload:
         self.calls += 1
 
     def run_tail(self):
-        self.compact_call()
-        if self.accept_call is not None:
-            self.accept_call()
+        self.tail_call()
 
     def step(self):
         self.run_heads()
@@ -315,15 +318,13 @@ def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
     host_calls = [[ee.prepare_exit_head_host(h_host[i], h_dev[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], wl.tau,
                                              out_host[i], wl.outs[i], wl.ws)
                    for i, hd in enumerate(wl.heads)] for c in range(wl.n_copies)]
-    compact_call = ee.prepare_compact(wl.outs[0]["exit_mask"], h_dev[0], out=wl.comp)
+    tail_call = wl.prepare_tail(h_dev[0])
 
     def step():
         for call in host_calls[wl.calls % wl.n_copies]:
             call()
         wl.calls += 1
-        compact_call()
-        if wl.accept_call is not None:
-            wl.accept_call()
+        tail_call()
         small_host["kept_count"].copy_(wl.comp["kept_count"], non_blocking=True)
         for k in wl.acc:
             small_host[k].copy_(wl.acc[k], non_blocking=True)
@@ -409,7 +410,7 @@ def main():
     M = args.rows if args.rows is not None else spec["M"]
     config = dict(workload=f"{args.workload}: Pythia-shaped exit heads d={spec['d']} V={spec['V']} M={M} heads={spec['heads']}",
                   rows_per_gpu=M, heads=spec["heads"], d=spec["d"], V=spec["V"], seed=0,
-                  step="all heads on the batch, ee_compact of head 0's survivors, dssd_accept(head 0 vs last head, k=8)")
+                  step="ee_exit_head_multi on the batch, then ee_compact_accept: compaction of head 0's survivors + dssd_accept(head 0 vs last head, k=8)")
 
     if args.impl == "reference":
         if rank != 0:

@@ -192,6 +192,18 @@ ee_status dssd_accept(const int* draft_tok, const unsigned char* draft_exit_mask
                       int S, int k, int kv, int* draft_len, int* accept_len, int* next_tok, void* stream);
 
 /*
+ * ee_compact and dssd_accept in one kernel launch, for a decoding step that needs both (section 3.4.2 and
+ * section 4.3.1): both read the heads' outputs and write disjoint results, so one launch does the work of two
+ * and a step saves a launch boundary.  Arguments, layouts and results are exactly those of the two calls;
+ * the mask given to the compaction (exit_mask, M rows) and the one given to the draft-length count
+ * (draft_exit_mask, S x k) may be the same buffer or different ones.
+ */
+ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
+                            int* kept_idx, int* kept_count, void* h_out, const int* draft_tok,
+                            const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k, int kv,
+                            int* draft_len, int* accept_len, int* next_tok, void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the error word of the workspace's control block.
  * Every device-side wait in the tensor-core kernel is bounded; one that gives up records itself there
  * and the kernel drains and returns.  EE_OK if nothing was recorded, EE_ERR_TIMEOUT otherwise (outputs

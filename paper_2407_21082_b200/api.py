@@ -270,6 +270,24 @@ def prepare_accept(draft_tok, draft_exit_mask, verify_tok, *, out=None) -> Prepa
     return PreparedCall(_lib.load().dssd_accept, args, "dssd_accept", keep, out)
 
 
+def _compact_accept_args(exit_mask, h, draft_tok, draft_exit_mask, verify_tok, gather, out):
+    c_args, c_out, c_keep = _compact_args(exit_mask, h, gather, None if out is None else out["compact"])
+    a_args, a_out, a_keep = _accept_args(draft_tok, draft_exit_mask, verify_tok, None if out is None else out["accept"])
+    return c_args[:-1] + a_args, dict(compact=c_out, accept=a_out), (c_keep, a_keep)
+
+
+def ee_compact_accept(exit_mask, h, draft_tok, draft_exit_mask, verify_tok, *, gather=True, out=None) -> dict:
+    """`ee_compact` and `dssd_accept` in one launch; returns dict(compact=..., accept=...) of their results."""
+    args, out, _ = _compact_accept_args(exit_mask, h, draft_tok, draft_exit_mask, verify_tok, gather, out)
+    _check(_lib.load().ee_compact_accept(*args), "ee_compact_accept")
+    return out
+
+
+def prepare_compact_accept(exit_mask, h, draft_tok, draft_exit_mask, verify_tok, *, gather=True, out=None) -> PreparedCall:
+    args, out, keep = _compact_accept_args(exit_mask, h, draft_tok, draft_exit_mask, verify_tok, gather, out)
+    return PreparedCall(_lib.load().ee_compact_accept, args, "ee_compact_accept", keep, out)
+
+
 def _accept_args(draft_tok, draft_exit_mask, verify_tok, out):
     S, k = draft_tok.shape
     kv = verify_tok.shape[1]

@@ -252,6 +252,27 @@ ee_status dssd_accept(const int* draft_tok, const unsigned char* draft_exit_mask
                          static_cast<cudaStream_t>(stream));
 }
 
+ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d, int* kept_idx,
+                            int* kept_count, void* h_out, const int* draft_tok, const unsigned char* draft_exit_mask,
+                            const int* verify_tok, int S, int k, int kv, int* draft_len, int* accept_len,
+                            int* next_tok, void* stream) {
+    if (M < 0 || S < 0 || k < 1 || kv < k) return EE_ERR_SHAPE;
+    if (!kept_count) return EE_ERR_NULL;
+    if (M > 0 && (!exit_mask || !kept_idx)) return EE_ERR_NULL;
+    if (h_out) {
+        if (M > 0 && !h) return EE_ERR_NULL;
+        if (d < 8 || (d % 8) != 0 || ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
+        if (!aligned(h, 16) || !aligned(h_out, 16)) return EE_ERR_ALIGN;
+    }
+    if (S > 0 && (!draft_tok || !verify_tok || !draft_len || !accept_len || !next_tok)) return EE_ERR_NULL;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return compact_accept_launch(exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out, draft_tok, draft_exit_mask,
+                                 verify_tok, S, k, kv, draft_len, accept_len, next_tok,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_query_async_error(void* workspace, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -12,18 +12,15 @@ constexpr int kRowsPerCta = 32;           // one ballot's worth of rows per CTA
 
 // CTA b owns rows [32b, 32b + 32).  Its output offset is the number of surviving rows before 32b, which it
 // counts itself from the mask (M bytes at most, L2-resident), so no CTA waits for another.
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned char* __restrict__ exit_mask,
-                                                                  const __nv_bfloat16* __restrict__ h, long long ld_h,
-                                                                  int M, int d, int* __restrict__ kept_idx,
-                                                                  int* __restrict__ kept_count,
-                                                                  __nv_bfloat16* __restrict__ h_out) {
+__device__ __forceinline__ void compact_body(int cta, const unsigned char* __restrict__ exit_mask,
+                                             const __nv_bfloat16* __restrict__ h, long long ld_h, int M, int d,
+                                             int* __restrict__ kept_idx, int* __restrict__ kept_count,
+                                             __nv_bfloat16* __restrict__ h_out) {
     __shared__ int s_warp_cnt[kCompactThreads / 32];
     __shared__ int s_src[kRowsPerCta];
     __shared__ int s_base, s_n;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row0 = blockIdx.x * kRowsPerCta;
-    launch_dependents();
-    grid_dependency_wait();                              // the mask and h come from earlier kernels of the stream
+    const int row0 = cta * kRowsPerCta;
 
     int cnt = 0;
     for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (exit_mask[i] == 0);
@@ -59,17 +56,22 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned
     }
 }
 
-// One warp per sequence; lane j looks at draft slot j (slots beyond 32 in further rounds).
-__global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ draft_tok,
-                                                     const unsigned char* __restrict__ draft_exit_mask,
-                                                     const int* __restrict__ verify_tok, int S, int k, int kv,
-                                                     int* __restrict__ draft_len, int* __restrict__ accept_len,
-                                                     int* __restrict__ next_tok) {
-    const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned char* __restrict__ exit_mask,
+                                                                  const __nv_bfloat16* __restrict__ h, long long ld_h,
+                                                                  int M, int d, int* __restrict__ kept_idx,
+                                                                  int* __restrict__ kept_count,
+                                                                  __nv_bfloat16* __restrict__ h_out) {
     launch_dependents();
-    if (s >= S) return;
-    grid_dependency_wait();                              // tokens and mask come from earlier kernels of the stream
+    grid_dependency_wait();                              // the mask and h come from earlier kernels of the stream
+    compact_body(blockIdx.x, exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out);
+}
+
+// One warp per sequence s; lane j looks at draft slot j (slots beyond 32 in further rounds).
+__device__ __forceinline__ void accept_body(int s, int lane, const int* __restrict__ draft_tok,
+                                            const unsigned char* __restrict__ draft_exit_mask,
+                                            const int* __restrict__ verify_tok, int k, int kv,
+                                            int* __restrict__ draft_len, int* __restrict__ accept_len,
+                                            int* __restrict__ next_tok) {
     int n = k;             // first slot that is not confident (draft length)
     int first_mis = k;     // first slot whose drafted token differs from the verifier's
     for (int base = 0; base < k; base += 32) {
@@ -87,6 +89,51 @@ __global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ dra
         draft_len[s] = n;
         accept_len[s] = a;
         next_tok[s] = (a < kv) ? verify_tok[(size_t)s * kv + a] : -1;
+    }
+}
+
+__global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ draft_tok,
+                                                     const unsigned char* __restrict__ draft_exit_mask,
+                                                     const int* __restrict__ verify_tok, int S, int k, int kv,
+                                                     int* __restrict__ draft_len, int* __restrict__ accept_len,
+                                                     int* __restrict__ next_tok) {
+    const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
+    launch_dependents();
+    if (s >= S) return;
+    grid_dependency_wait();                              // tokens and mask come from earlier kernels of the stream
+    accept_body(s, threadIdx.x & 31, draft_tok, draft_exit_mask, verify_tok, k, kv, draft_len, accept_len, next_tok);
+}
+
+// Both in one launch: the first n_compact CTAs compact, the others take eight sequences each.  The two parts
+// read the same head outputs and write disjoint results, so they need no order between them.
+struct TailArgs {
+    const unsigned char* exit_mask;
+    const __nv_bfloat16* h;
+    long long ld_h;
+    int M, d;
+    int* kept_idx;
+    int* kept_count;
+    __nv_bfloat16* h_out;
+    const int* draft_tok;
+    const unsigned char* draft_exit_mask;
+    const int* verify_tok;
+    int S, k, kv;
+    int* draft_len;
+    int* accept_len;
+    int* next_tok;
+    int n_compact;
+};
+
+__global__ void __launch_bounds__(kCompactThreads) compact_accept_kernel(const __grid_constant__ TailArgs a) {
+    launch_dependents();
+    grid_dependency_wait();
+    if ((int)blockIdx.x < a.n_compact) {
+        compact_body(blockIdx.x, a.exit_mask, a.h, a.ld_h, a.M, a.d, a.kept_idx, a.kept_count, a.h_out);
+    } else {
+        const int s = ((int)blockIdx.x - a.n_compact) * (kCompactThreads / 32) + (threadIdx.x >> 5);
+        if (s < a.S)
+            accept_body(s, threadIdx.x & 31, a.draft_tok, a.draft_exit_mask, a.verify_tok, a.k, a.kv, a.draft_len,
+                        a.accept_len, a.next_tok);
     }
 }
 
@@ -109,6 +156,26 @@ ee_status accept_launch(const int* draft_tok, const unsigned char* draft_exit_ma
                       draft_len, accept_len, next_tok) == cudaSuccess
                ? EE_OK
                : EE_ERR_CUDA;
+}
+
+ee_status compact_accept_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
+                                int* kept_idx, int* kept_count, void* h_out, const int* draft_tok,
+                                const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k, int kv,
+                                int* draft_len, int* accept_len, int* next_tok, cudaStream_t stream) {
+    if (M == 0 || S == 0) {      // one part is empty: the plain launches handle it
+        const ee_status st = compact_launch(exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out, stream);
+        if (st != EE_OK) return st;
+        return accept_launch(draft_tok, draft_exit_mask, verify_tok, S, k, kv, draft_len, accept_len, next_tok, stream);
+    }
+    TailArgs a;
+    a.exit_mask = exit_mask; a.h = static_cast<const __nv_bfloat16*>(h); a.ld_h = ld_h; a.M = M; a.d = d;
+    a.kept_idx = kept_idx; a.kept_count = kept_count; a.h_out = static_cast<__nv_bfloat16*>(h_out);
+    a.draft_tok = draft_tok; a.draft_exit_mask = draft_exit_mask; a.verify_tok = verify_tok;
+    a.S = S; a.k = k; a.kv = kv; a.draft_len = draft_len; a.accept_len = accept_len; a.next_tok = next_tok;
+    a.n_compact = (M + kRowsPerCta - 1) / kRowsPerCta;
+    const int per_cta = kCompactThreads / 32;
+    const int grid = a.n_compact + (S + per_cta - 1) / per_cta;
+    return launch_pdl(compact_accept_kernel, grid, kCompactThreads, 0, stream, a) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 
 }  // namespace ee

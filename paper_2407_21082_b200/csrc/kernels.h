@@ -63,4 +63,9 @@ ee_status accept_launch(const int* draft_tok, const unsigned char* draft_exit_ma
                         int S, int k, int kv, int* draft_len, int* accept_len, int* next_tok,
                         cudaStream_t stream);
 
+ee_status compact_accept_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
+                                int* kept_idx, int* kept_count, void* h_out, const int* draft_tok,
+                                const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k, int kv,
+                                int* draft_len, int* accept_len, int* next_tok, cudaStream_t stream);
+
 }  // namespace ee

@@ -140,3 +140,28 @@ def test_c3_pipeline_draft_verify_accept(ee, planted):
         assert a_ref["draft_len"].max() > 0          # some sequences draft at least one token
     else:
         assert a_ref["draft_len"].max() == 0         # the literal inputs are never confident
+
+
+@pytest.mark.parametrize("M,d,S,k,kv", [(64, 1024, 8, 8, 8), (1, 8, 1, 1, 1), (33, 72, 70, 5, 9), (1000, 40, 3, 40, 40),
+                                        (40, 16, 0, 4, 4), (0, 16, 9, 4, 6)])
+def test_compact_accept_one_launch_matches_oracle(ee, M, d, S, k, kv):
+    """The fused call gives bit for bit what the oracle gives for the two operations, twice in a row."""
+    rng = np.random.default_rng(1000 * M + S)
+    h = rng.integers(0, 65536, size=(M, d)).astype(np.uint16)
+    mask = (rng.random(M) < 0.4).astype(np.uint8) * rng.integers(1, 256, size=M).astype(np.uint8)
+    case = gen.random_token_case(seed=M + S, S=max(S, 1), k=k, kv=kv)
+    draft, conf, verify = (case[n][:S] for n in ("draft_tok", "draft_exit_mask", "verify_tok"))
+    ref_c = oracle.compact(mask, h)
+    ref_a = oracle.dssd_accept(draft, conf, verify) if S else None
+    h_dev = dev_bf16(h) if M else torch.empty((0, d), dtype=torch.bfloat16, device="cuda")
+    for _ in range(2):
+        out = ee.ee_compact_accept(dev(mask), h_dev, dev(draft.reshape(S, k)), dev(conf.reshape(S, k)),
+                                   dev(verify.reshape(S, kv)))
+        n = int(out["compact"]["kept_count"].item())
+        assert n == ref_c["kept_count"]
+        assert np.array_equal(out["compact"]["kept_idx"].cpu().numpy()[:n], ref_c["kept_idx"])
+        got = out["compact"]["h_out"].view(torch.int16).cpu().numpy().view(np.uint16)[:n]
+        assert np.array_equal(got, ref_c["h_out"])
+        if S:
+            for name in ("draft_len", "accept_len", "next_tok"):
+                assert np.array_equal(out["accept"][name].cpu().numpy(), ref_a[name]), name
