@@ -55,6 +55,7 @@ struct GemmParams {
     Control* ctrl;
     int bn;                // tile width (vocabulary rows per tile), a multiple of 16, <= 256
     int n_stages;          // smem ring depth
+    int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
 };
 
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
@@ -116,13 +117,17 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     const int BN = BN_T ? BN_T : p.bn;
     const int S = BN_T ? C::kStages : p.n_stages;
     const int b_tile_bytes = BN * BK * 2;
-    const int stage_bytes = kATileBytes + b_tile_bytes;
+    // With at most 64 rows per head the MMA is issued with M = 64: half the tensor work (and power) of a
+    // 128-row MMA whose lower half would be padding, and an 8 KB instead of a 16 KB y tile per stage.
+    const int mma_m = BN_T ? BM : p.mma_m;
+    const int a_tile_bytes = mma_m * BK * 2;
+    const int stage_bytes = a_tile_bytes + b_tile_bytes;
     constexpr int kAccStride = 256;                               // TMEM columns between the two accumulators
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
     const uint32_t a_base = ptx::smem_addr(smem);
-    const uint32_t b_base = a_base + S * kATileBytes;
+    const uint32_t b_base = a_base + S * a_tile_bytes;
     unsigned char* bar_mem = smem + S * stage_bytes;
     const uint32_t bar_base = ptx::smem_addr(bar_mem);
     // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
@@ -196,7 +201,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 const int y_row = (head * p.m_tiles + m_tile) * BM;   // each head's rows are padded to whole tiles
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
-                        ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                        ptx::tma_load_2d(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, full_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                         continue;
                     }
@@ -206,7 +211,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                         break;
                     }
                     ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
-                    ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                    ptx::tma_load_2d(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, full_bar(stage));
                     ptx::tma_load_2d(b_base + stage * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN, full_bar(stage));
                     armed |= 1u << stage;
                     armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
@@ -225,7 +230,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+            const uint32_t idesc = ptx::idesc_bf16_f32(mma_m, BN);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -246,7 +251,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
+                    const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * a_tile_bytes);
                     const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units per step
@@ -265,7 +270,9 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int row_in_tile = quarter * 32 + lane;
+        // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in the first 16 lanes of
+        // quarter q, the other 16 lanes hold nothing.
+        const int row_in_tile = mma_m == 64 ? (lane < 16 ? quarter * 16 + lane : BM) : quarter * 32 + lane;
         int local = 0;
         grid_dependency_wait();                           // the partial states may still be read by an earlier merge
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
@@ -283,19 +290,24 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             const int ncols = min(BN, p.V - n0);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccStride);
             State st = state_empty();
-            for (int c = 0; c * 32 < ncols; ++c) {
-                float v[32];
-                ptx::tmem_ld_32x32(taddr + c * 32, v);
-                ptx::tmem_ld_wait();
-                const int nvalid = ncols - c * 32;
-                if (nvalid >= 32) fold_chunk<true>(st, v, n0 + c * 32, 32);
-                else fold_chunk<false>(st, v, n0 + c * 32, nvalid);
+            const int row = m_tile * BM + row_in_tile;
+            const bool live = row < p.M;                  // padding rows are neither read nor folded
+            if (__any_sync(0xffffffffu, live)) {
+                for (int c = 0; c * 32 < ncols; ++c) {
+                    float v[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, v);
+                    ptx::tmem_ld_wait();
+                    const int nvalid = ncols - c * 32;
+                    if (live) {
+                        if (nvalid >= 32) fold_chunk<true>(st, v, n0 + c * 32, 32);
+                        else fold_chunk<false>(st, v, n0 + c * 32, nvalid);
+                    }
+                }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
-            const int row = m_tile * BM + row_in_tile;
-            if (row < p.M) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+            if (live) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
         }
     }
 
@@ -432,8 +444,8 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 constexpr int kMinTileN = 64;
 
 // Ring depth for a runtime tile width.
-int stages_for(int bn) {
-    const size_t stage = kATileBytes + (size_t)bn * BK * 2;
+int stages_for(int bn, int mma_m) {
+    const size_t stage = (size_t)mma_m * BK * 2 + (size_t)bn * BK * 2;
     const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
@@ -448,7 +460,7 @@ ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int d
         configured[device] = true;
     }
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
-                             : (size_t)p.n_stages * (kATileBytes + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
+                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
     return launch_pdl(exit_head_gemm_kernel<BN_T>, grid, kGemmThreads, smem, stream, maps, p) == cudaSuccess
                ? EE_OK
                : EE_ERR_CUDA;
@@ -527,7 +539,8 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     // pattern stream from HBM at the rate of a contiguous copy (measured: 6.9 against 5.5 TB/s).
     const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     GemmMaps maps;
-    if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, BM)) return EE_ERR_CUDA;
+    const int mma_m = a.M <= 64 ? 64 : BM;
+    if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)) return EE_ERR_CUDA;
     for (int k = 0; k < kGemmMaxHeads; ++k)
         if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, bn, promo)) return EE_ERR_CUDA;
 
@@ -542,7 +555,8 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.partials = partials;
     p.ctrl = reinterpret_cast<Control*>(ws);
     p.bn = bn;
-    p.n_stages = stages_for(bn);
+    p.mma_m = mma_m;
+    p.n_stages = stages_for(bn, mma_m);
     const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
     const int grid = (int)(total < a.num_sms ? total : a.num_sms);
     const ee_status st = (a.M > 1024) ? launch_gemm<256>(maps, p, grid, a.device, a.stream)
