@@ -3,10 +3,11 @@
 // The M x V logits are never written anywhere.  The three kernels are chained by programmatic dependent
 // launch, and the GEMM requests its first weight tiles before it waits for the LayerNorm kernel.
 //
-// GEMM kernel, one CTA per SM, 192 threads:
+// GEMM kernel, one CTA per SM, 320 threads:
 //   warp 0 (one lane)  TMA producer: y tile [128 x 64] and W tile [BN x 64] per k-block into a smem ring
 //   warp 1 (one lane)  tcgen05.mma issuer; accumulators [128 x BN] fp32 double-buffered in TMEM
-//   warps 2..5         epilogue: tcgen05.ld 32 columns at a time, thread = row, online softmax state,
+//   warps 2..9         epilogue (two warps per quarter of the TMEM lanes, even / odd 32-column chunks):
+//                      tcgen05.ld 32 columns at a time, thread = row, online softmax state,
 //                      one 16-byte partial state per (row, vocabulary tile)
 // All mbarrier waits are bounded; a wait that gives up records an error word, raises the CTA's abort
 // flag, and every role drains to the common exit where TMEM is released.
@@ -21,11 +22,11 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;           // producer warp, MMA warp, eight epilogue warps
 constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile order
 constexpr int kATileBytes = BM * BK * 2;    // 16 KB
 
-constexpr int kBarBytes = 256;
+constexpr int kBarBytes = 512 + 2048;          // barriers and flags (512 B), then 128 states exchanged between epilogue warps
 constexpr int kGemmMaxHeads = kGemmLaunchMaxHeads;
 constexpr int kMaxGemmStages = 12;
 constexpr size_t kGemmSmemBudget = 226 * 1024;
@@ -138,9 +139,16 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     const uint32_t drain_bar = bar_base + 8u * (2 * S + 4);
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_mem + 8 * (2 * S + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 5) + 4);
+    // per quarter of the TMEM lanes: "state of the odd chunks is in the exchange slot" / "slot has been read"
+    auto xfull_bar = [&](int q) { return bar_base + 8u * (2 * S + 6 + q); };
+    auto xfree_bar = [&](int q) { return bar_base + 8u * (2 * S + 10 + q); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    launch_dependents();
+    // The runtime-width variant (launches of tens of microseconds) lets its dependents start at once; their few
+    // CTAs wait beside this one.  The 256-wide variant runs for milliseconds and its merge has thousands of
+    // CTAs: resident and waiting they cost it about a tenth of its speed, so it triggers them only when a CTA
+    // starts its last tile (see the producer).
+    if (BN_T == 0) launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -149,7 +157,11 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4);
+            ptx::mbar_init(tempty_bar(b), BN_T ? 4 : 8);
+        }
+        for (int q = 0; q < 4; ++q) {
+            ptx::mbar_init(xfull_bar(q), 1);
+            ptx::mbar_init(xfree_bar(q), 1);
         }
         ptx::mbar_init(drain_bar, 1);
         *abort_flag = 0;
@@ -199,6 +211,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 int head, m_tile, n_tile;
                 locate(tile, head, m_tile, n_tile);
                 const int y_row = (head * p.m_tiles + m_tile) * BM;   // each head's rows are padded to whole tiles
+                if (BN_T != 0 && tile + (int)gridDim.x >= total_tiles) launch_dependents();
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
                         ptx::tma_load_2d(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, full_bar(stage));
@@ -268,14 +281,21 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        // Two warps share each quarter of the TMEM lanes: one folds the even 32-column chunks of a tile, the
+        // other the odd ones, and the first adds the second's state to its own before it stores the partial.
         const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31 belong to this warp
+        // (The compile-time 256-wide variant is tensor-bound and its epilogue hides behind the next tile's MMAs:
+        // there one warp per quarter folds all chunks and the other four warps stay out of the way.)
+        constexpr bool kSplit = BN_T == 0;
+        const int half = (warp - 2) >> 2;
+        State* xchg = reinterpret_cast<State*>(bar_mem + 512) + quarter * 32 + lane;
         // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in the first 16 lanes of
         // quarter q, the other 16 lanes hold nothing.
         const int row_in_tile = mma_m == 64 ? (lane < 16 ? quarter * 16 + lane : BM) : quarter * 32 + lane;
         int local = 0;
         grid_dependency_wait();                           // the partial states may still be read by an earlier merge
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+        for (int tile = blockIdx.x; (kSplit || half == 0) && tile < total_tiles; tile += gridDim.x, ++local) {
             int head, m_tile, n_tile;
             locate(tile, head, m_tile, n_tile);
             const int buf = local & 1;
@@ -293,7 +313,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             const int row = m_tile * BM + row_in_tile;
             const bool live = row < p.M;                  // padding rows are neither read nor folded
             if (__any_sync(0xffffffffu, live)) {
-                for (int c = 0; c * 32 < ncols; ++c) {
+                for (int c = kSplit ? half : 0; c * 32 < ncols; c += kSplit ? 2 : 1) {
                     float v[32];
                     ptx::tmem_ld_32x32(taddr + c * 32, v);
                     ptx::tmem_ld_wait();
@@ -307,7 +327,33 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
-            if (live) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+            const uint32_t x_phase = (uint32_t)local & 1u;
+            if (!kSplit) {
+                if (live) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+            } else if (half == 1) {
+                // the slot is free once the partner has read the state of the tile before
+                const bool free_ = local == 0 || ptx::mbar_wait(xfree_bar(quarter), x_phase ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, free_)) {
+                    if (lane == 0) record_failure(p.ctrl, abort_flag, 5, quarter, tile);
+                    break;
+                }
+                *xchg = st;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(xfull_bar(quarter));
+            } else {
+                const bool there = ptx::mbar_wait(xfull_bar(quarter), x_phase, abort_flag);
+                if (!__all_sync(0xffffffffu, there)) {
+                    if (lane == 0) record_failure(p.ctrl, abort_flag, 6, quarter, tile);
+                    break;
+                }
+                const State other = *xchg;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(xfree_bar(quarter));
+                if (live) {
+                    state_merge(st, other);
+                    p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                }
+            }
         }
     }
 
@@ -366,7 +412,14 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
                 b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
             }
         }
-        grid_dependency_wait();                          // h may be an earlier kernel's output; y may still be read
+        // h may be an earlier kernel's output, so it is read after the wait; asking L2 for its lines before
+        // the wait is harmless (L2 is the point of coherence) and hides a DRAM round trip when h is not cached.
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            if (c < nvec && (c & 7) == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(hrow + c));
+        }
+        grid_dependency_wait();                          // y may still be read by the GEMM of the call before
         uint4 x[VPL];
         float sum = 0.f;
 #pragma unroll
