@@ -87,7 +87,7 @@ int ee_exit_head_launches(int M, int d, int V, int path) {
         return slab > 0 ? (M + slab - 1) / slab : 0;
     }
     if (path == EE_PATH_SKINNY) return skinny_supports(M, d) ? 1 : 0;
-    return path == EE_PATH_TCGEN05 ? 3 : 0;      // LayerNorm, GEMM with fused statistics, merge
+    return path == EE_PATH_TCGEN05 ? gemm_launches(M, 1) : 0;
 }
 
 ee_status ee_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {
@@ -138,8 +138,10 @@ size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
 
 int ee_exit_head_multi_launches(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1 || M == 0) return 0;
-    const int calls = (n_heads + kSkinnyMaxHeads - 1) / kSkinnyMaxHeads;
-    return 3 * calls;                                  // LayerNorm, GEMM with fused statistics, merge
+    int launches = 0;
+    for (int k0 = 0; k0 < n_heads; k0 += kGemmLaunchMaxHeads)
+        launches += gemm_launches(M, n_heads - k0 < kGemmLaunchMaxHeads ? n_heads - k0 : kGemmLaunchMaxHeads);
+    return launches;
 }
 
 ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, void* workspace,

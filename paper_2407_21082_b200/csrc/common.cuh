@@ -143,12 +143,13 @@ __device__ __forceinline__ void state_finish(const State& a, float tau, int* arg
 // Workspace layout.  [0, 256): control block.  Then the partial states, then (tensor-core path) y.
 // ---------------------------------------------------------------------------------------------
 struct Control {
-    unsigned int ticket;      // completion counter of the streaming kernel; returns to 0 after every call
+    unsigned int ticket;      // CTAs that have stored their partial states; returns to 0 after every call
     unsigned int error;       // 0, or a code recorded by a bounded wait that gave up
     unsigned int error_info;  // where it gave up (role << 24 | stage << 16 | low bits of the tile index)
     unsigned int pad0;
     unsigned int head_ticket[8];   // completion counters of the heads of a multi-head launch; return to 0 as well
-    unsigned int pad[52];
+    unsigned int merge_seen;  // tensor-core kernel, in-kernel merge: rows merged so far; returns to 0 as well
+    unsigned int pad[51];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 

@@ -48,6 +48,35 @@ struct GemmMaps {
     CUtensorMap w[kGemmMaxHeads];      // each head's weights [V, d]
 };
 
+struct MergeHeads {
+    const float* tau_per_row[kGemmMaxHeads];
+    float tau[kGemmMaxHeads];
+    int* argmax[kGemmMaxHeads];
+    float* entropy[kGemmMaxHeads];
+    float* maxprob[kGemmMaxHeads];
+    unsigned char* exit_mask[kGemmMaxHeads];
+};
+
+// One warp: merge of the n_tiles partial states of one row (lane-strided, eight independent loads at a
+// time, then the lanes reduce) and the final decision for that row.
+__device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ partials, int n_tiles, int head, int row,
+                                                     const MergeHeads& hs, int lane) {
+    State v[9];
+    v[8] = state_empty();                                         // running result of this lane
+    for (int n0 = lane; n0 < n_tiles; n0 += 256) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int n = n0 + 32 * i;
+            v[i] = n < n_tiles ? state_load_cg(partials + n) : state_empty();
+        }
+        v[8] = state_combine<9>(v);
+    }
+    const State a = state_reduce_lanes<1, 16>(v[8]);
+    if (lane == 0)
+        state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
+                     hs.maxprob[head], hs.exit_mask[head], row);
+}
+
 struct GemmParams {
     int M, V, d;
     int m_tiles, n_tiles, k_blocks;
@@ -57,6 +86,8 @@ struct GemmParams {
     int bn;                // tile width (vocabulary rows per tile), a multiple of 16, <= 256
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
+    int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
+    MergeHeads mg;
 };
 
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
@@ -355,6 +386,46 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 }
             }
         }
+        if (kSplit && p.fused_merge) {
+            // With few rows the merge runs here instead of in a kernel of its own (one launch boundary less per
+            // call).  Every CTA publishes its partial states with a ticket; epilogue warp w of CTA c owns rows
+            // 8c + w, 8c + w + 8 * grid, ..: a warp that owns a row waits, bounded, until all CTAs have
+            // published, then merges and decides.  CTAs without rows leave at once.  The warp that finishes
+            // the last row returns both counters to zero.
+            __threadfence();
+            asm volatile("bar.sync 1, 256;" ::: "memory");            // the eight epilogue warps, whatever path they took
+            if (warp == 2 && lane == 0)
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&p.ctrl->ticket) : "memory");
+            const int total_rows = p.n_heads * p.M;
+            const int first = (int)blockIdx.x * 8 + (warp - 2);
+            if (first < total_rows) {
+                bool there = false;
+                for (uint32_t i = 0; i < ptx::kWaitPolls; ++i) {
+                    unsigned int v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(&p.ctrl->ticket) : "memory");
+                    if (v >= gridDim.x) { there = true; break; }
+                    if (*abort_flag) break;
+                    __nanosleep(i < 4096 ? 40 : 400);
+                }
+                there = __all_sync(0xffffffffu, there);
+                if (!there) {
+                    if (lane == 0) record_failure(p.ctrl, abort_flag, 7, 0, blockIdx.x);
+                } else {
+                    int mine = 0;
+                    for (int r = first; r < total_rows; r += (int)gridDim.x * 8, ++mine) {
+                        const int head = r / p.M, row = r - head * p.M;
+                        merge_row_and_decide(p.partials + (size_t)r * p.n_tiles, p.n_tiles, head, row, p.mg, lane);
+                    }
+                    if (lane == 0) {
+                        const unsigned int old = atomicAdd(&p.ctrl->merge_seen, (unsigned int)mine);
+                        if (old + (unsigned int)mine == (unsigned int)total_rows) {
+                            p.ctrl->ticket = 0;
+                            p.ctrl->merge_seen = 0;
+                        }
+                    }
+                }
+            }
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -456,15 +527,6 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
 // Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
 // blockIdx.y = head.
 // ---------------------------------------------------------------------------------------------
-struct MergeHeads {
-    const float* tau_per_row[kGemmMaxHeads];
-    float tau[kGemmMaxHeads];
-    int* argmax[kGemmMaxHeads];
-    float* entropy[kGemmMaxHeads];
-    float* maxprob[kGemmMaxHeads];
-    unsigned char* exit_mask[kGemmMaxHeads];
-};
-
 __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials_all, int n_tiles, int M,
                                                          const __grid_constant__ MergeHeads hs) {
     launch_dependents();
@@ -474,27 +536,14 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
     if (row >= M) return;
     const State* partials = partials_all + ((size_t)head * M + row) * n_tiles;
     grid_dependency_wait();                              // the partial states come from the GEMM kernel
-    // Lane-strided over the tiles, eight independent loads at a time; then the lanes reduce.
-    State v[9];
-    v[8] = state_empty();                                         // running result of this lane
-    for (int n0 = lane; n0 < n_tiles; n0 += 256) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int n = n0 + 32 * i;
-            v[i] = n < n_tiles ? state_load_cg(partials + n) : state_empty();
-        }
-        v[8] = state_combine<9>(v);
-    }
-    const State a = state_reduce_lanes<1, 16>(v[8]);
-    if (lane == 0)
-        state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
-                     hs.maxprob[head], hs.exit_mask[head], row);
+    merge_row_and_decide(partials, n_tiles, head, row, hs, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
 constexpr int kMinTileN = 64;
+constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
 
 // Ring depth for a runtime tile width.
 int stages_for(int bn, int mma_m) {
@@ -553,6 +602,9 @@ int gemm_tile_n(int M, int V, int n_heads, int num_sms) {
     return best;
 }
 
+// LayerNorm and GEMM; plus the merge kernel when the rows are too many for the GEMM kernel to merge itself.
+int gemm_launches(int M, int n_heads) { return n_heads * M <= kFusedMergeMaxRows ? 2 : 3; }
+
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
     return (size_t)n_heads * partials_bytes(M, V) + y_bytes(M, d, n_heads);
 }
@@ -609,12 +661,15 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.ctrl = reinterpret_cast<Control*>(ws);
     p.bn = bn;
     p.mma_m = mma_m;
+    p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
+    p.mg = mg;
     p.n_stages = stages_for(bn, mma_m);
     const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
     const int grid = (int)(total < a.num_sms ? total : a.num_sms);
     const ee_status st = (a.M > 1024) ? launch_gemm<256>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<0>(maps, p, grid, a.device, a.stream);
     if (st != EE_OK) return st;
+    if (p.fused_merge) return EE_OK;
 
     err = launch_pdl(merge_rows_kernel, row_grid, 256, 0, a.stream, (const State*)partials, p.n_tiles, a.M, mg);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;

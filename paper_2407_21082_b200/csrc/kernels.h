@@ -55,6 +55,7 @@ constexpr int kGemmLaunchMaxHeads = 4;
 int gemm_tile_n(int M, int V, int n_heads, int num_sms);   // vocabulary tile width used for M rows on num_sms SMs
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads);
 ee_status gemm_launch(const HeadArgs* heads, int n_heads);
+int gemm_launches(int M, int n_heads);     // kernels one gemm_launch call starts
 
 // ---- compaction and DSSD accept ----
 ee_status compact_launch(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d,
