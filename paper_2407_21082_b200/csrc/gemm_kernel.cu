@@ -57,21 +57,22 @@ struct MergeHeads {
     unsigned char* exit_mask[kGemmMaxHeads];
 };
 
-// One warp: merge of the n_tiles partial states of one row (lane-strided, eight independent loads at a
-// time, then the lanes reduce) and the final decision for that row.
+// One warp: merge of the n_tiles partial states of one row (lane-strided, twelve independent loads at a
+// time -- one round trip for up to 384 tiles -- then the lanes reduce) and the final decision for that row.
 __device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ partials, int n_tiles, int head, int row,
                                                      const MergeHeads& hs, int lane) {
-    State v[9];
-    v[8] = state_empty();                                         // running result of this lane
-    for (int n0 = lane; n0 < n_tiles; n0 += 256) {
+    constexpr int kBatch = 12;
+    State v[kBatch + 1];
+    v[kBatch] = state_empty();                                    // running result of this lane
+    for (int n0 = lane; n0 < n_tiles; n0 += 32 * kBatch) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < kBatch; ++i) {
             const int n = n0 + 32 * i;
             v[i] = n < n_tiles ? state_load_cg(partials + n) : state_empty();
         }
-        v[8] = state_combine<9>(v);
+        v[kBatch] = state_combine<kBatch + 1>(v);
     }
-    const State a = state_reduce_lanes<1, 16>(v[8]);
+    const State a = state_reduce_lanes<1, 16>(v[kBatch]);
     if (lane == 0)
         state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
                      hs.maxprob[head], hs.exit_mask[head], row);
@@ -392,7 +393,8 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             // 8c + w, 8c + w + 8 * grid, ..: a warp that owns a row waits, bounded, until all CTAs have
             // published, then merges and decides.  CTAs without rows leave at once.  The warp that finishes
             // the last row returns both counters to zero.
-            __threadfence();
+            // The barrier orders the epilogue threads' stores before thread 64's release, which is cumulative:
+            // a warp that acquires the full ticket count sees every CTA's partial states.
             asm volatile("bar.sync 1, 256;" ::: "memory");            // the eight epilogue warps, whatever path they took
             if (warp == 2 && lane == 0)
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&p.ctrl->ticket) : "memory");
