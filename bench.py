@@ -308,26 +308,36 @@ def roofline(wl: Workload, head_call_us: float, peaks: dict, src: str) -> dict:
 
 
 def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
-    """Same step driven through ee_exit_head_host: h comes from pinned host memory and the results go back to it."""
+    """The same step through the host-buffer API: every step copies the heads' input rows from pinned host
+    memory (one copy), evaluates the heads (ee_exit_head_multi_host), copies the packed results back (one
+    copy), runs compaction + accept on the device results, copies their counts back and synchronises,
+    because the caller reads its results every step.  Wall-clock around the loop."""
     torch, ee = wl.torch, wl.ee
-    h_host = [h.cpu().pin_memory() for h in wl.h]
-    h_dev = [torch.empty_like(h) for h in wl.h]
-    out_host = [{k: v.cpu().pin_memory() for k, v in o.items()} for o in wl.outs]
-    small_host = {k: v.cpu().pin_memory() for k, v in {**wl.acc, "kept_count": wl.comp["kept_count"]}.items()}
-
-    host_calls = [[ee.prepare_exit_head_host(h_host[i], h_dev[i], hd["gamma"], hd["beta"], 1e-5, hd["W"][c], wl.tau,
-                                             out_host[i], wl.outs[i], wl.ws)
-                   for i, hd in enumerate(wl.heads)] for c in range(wl.n_copies)]
-    tail_call = wl.prepare_tail(h_dev[0])
+    n_heads, S, k = len(wl.heads), wl.S, wl.k
+    h_host = torch.stack([h.cpu() for h in wl.h]).pin_memory()                  # [n_heads, M, d]
+    calls = [ee.PreparedMultiHost([dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"][c], tau=wl.tau) for hd in wl.heads],
+                                  1e-5, h_host, wl.ws) for c in range(wl.n_copies)]
+    small_dev = torch.zeros(1 + 3 * max(S, 1), dtype=torch.int32, device="cuda")  # kept_count | draft_len | accept_len | next_tok
+    small_host = torch.zeros_like(small_dev, device="cpu").pin_memory()
+    comp = dict(kept_idx=wl.comp["kept_idx"], kept_count=small_dev[0:1], h_out=wl.comp["h_out"])
+    acc = {n: small_dev[1 + i * max(S, 1):1 + (i + 1) * max(S, 1)] for i, n in enumerate(("draft_len", "accept_len", "next_tok"))}
+    tails = []
+    for call in calls:
+        o = call.out_dev
+        if S == 0:
+            tails.append(ee.prepare_compact(o[0]["exit_mask"], call.h_dev[0], out=comp))
+        else:
+            n = S * k
+            tails.append(ee.prepare_compact_accept(o[0]["exit_mask"], call.h_dev[0], o[0]["argmax"][:n].view(S, k),
+                                                   o[0]["exit_mask"][:n].view(S, k), o[-1]["argmax"][:n].view(S, k),
+                                                   out=dict(compact=comp, accept=acc)))
 
     def step():
-        for call in host_calls[wl.calls % wl.n_copies]:
-            call()
+        c = wl.calls % wl.n_copies
         wl.calls += 1
-        tail_call()
-        small_host["kept_count"].copy_(wl.comp["kept_count"], non_blocking=True)
-        for k in wl.acc:
-            small_host[k].copy_(wl.acc[k], non_blocking=True)
+        calls[c]()
+        tails[c]()
+        small_host.copy_(small_dev, non_blocking=True)
         torch.cuda.synchronize()          # the caller reads its results every step
 
     for _ in range(warmup):
@@ -341,11 +351,11 @@ def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
     t1.record()
     torch.cuda.synchronize()
     wall = time.perf_counter() - wall0
-    n_heads = len(wl.heads)
-    h2d = n_heads * wl.M * wl.d * 2
-    d2h = n_heads * wl.M * 13 + 4 + 3 * 4 * max(wl.S, 1)
-    return dict(value=n_heads * wl.M * steps / wall, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-                ms_per_step=1e3 * wall / steps, device_ms_per_step=t0.elapsed_time(t1) / steps)
+    wl.check()
+    return dict(value=n_heads * wl.M * steps / wall, unit=UNIT, h2d_bytes_per_step=calls[0].h2d_bytes,
+                d2h_bytes_per_step=calls[0].d2h_bytes + small_host.numel() * 4,
+                ms_per_step=1e3 * wall / steps, device_ms_per_step=t0.elapsed_time(t1) / steps,
+                api="ee_exit_head_multi_host + ee_compact_accept, three copies and one synchronise per step")
 
 
 def oracle_threads() -> int:

@@ -91,9 +91,9 @@ ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const 
 /*
  * Several heads on batches of the same shape in one call -- what the calibration pass of section 3.4.1 does
  * (every head is evaluated on every token of the calibration set) and what a verify step with several
- * heads does.  Equivalent to n_heads calls of ee_exit_head with the same M, d, V, ln_eps and workspace; when
- * the batch is decode-sized (M <= 16 rows) up to four heads share one kernel launch, which keeps the weight
- * stream going across the per-head LayerNorm and merge steps; larger batches run head by head.  `heads` is a HOST array read during the call;
+ * heads does.  Equivalent to n_heads calls of ee_exit_head with the same M, d, V, ln_eps and workspace; up to
+ * four heads share one sequence of kernel launches, which keeps the weight stream going from one head to
+ * the next and pays the LayerNorm and merge steps once.  `heads` is a HOST array read during the call;
  * the pointers inside follow the rules of ee_exit_head (each head has its own h, LayerNorm parameters, W,
  * thresholds and outputs; h may be the same for all).  Workspace: ee_exit_head_multi_workspace_bytes().
  */
@@ -162,6 +162,24 @@ ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma,
 ee_status ee_exit_head_static(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
                               const void* W, int M, int d, int V, const float* tau_per_row, float tau,
                               int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask, void* stream);
+
+/*
+ * ee_exit_head_multi for a caller whose activations and results live in HOST memory: one copy in, the heads,
+ * one copy out (same passage as ee_exit_head_multi; pinned host memory makes the copies asynchronous).
+ *   h_host        bf16 [n_heads][M][d], dense: head k's input rows
+ *   h_dev         device staging of the same size
+ *   results_host  packed results, ee_exit_head_results_bytes(n_heads, M) bytes; head k's block starts at
+ *                 byte k * ee_exit_head_results_bytes(1, M) and holds argmax int32 [M], entropy fp32 [M],
+ *                 maxprob fp32 [M], exit_mask uint8 [M] back to back (the block is padded to 16 bytes)
+ *   results_dev   device staging of the same size and layout; the device copies of the results stay valid
+ *                 there for later calls on the stream (ee_compact, dssd_accept)
+ * Of each ee_head only gamma, beta, W, tau_per_row and tau are read; its h, ld_h and output pointers are
+ * ignored.  Returns without synchronising: results_host is valid after the caller synchronises `stream`.
+ */
+size_t    ee_exit_head_results_bytes(int n_heads, int M);      /* host-only, pure; 0 if a size is invalid */
+ee_status ee_exit_head_multi_host(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
+                                  const void* h_host, void* h_dev, void* results_host, void* results_dev,
+                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Continuation of the rows that did not exit (section 3.4.2: an input keeps going through the model's

@@ -31,6 +31,9 @@ PROTOTYPES = {
                                     _p, _p, _p, _p, _p, C.c_size_t, _p, C.c_int]),
     "ee_exit_head_host": (C.c_int, [_p, _p, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                     _p, _p, _p, _p, _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_exit_head_results_bytes": (C.c_size_t, [C.c_int, C.c_int]),
+    "ee_exit_head_multi_host": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int,
+                                          _p, _p, _p, _p, _p, C.c_size_t, _p]),
     "ee_exit_head_static": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                       _p, _p, _p, _p, _p]),
     "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),

@@ -181,6 +181,60 @@ class PreparedMulti:
         return self.out
 
 
+def ee_exit_head_results_bytes(n_heads: int, M: int) -> int:
+    return int(_lib.load().ee_exit_head_results_bytes(n_heads, M))
+
+
+def results_views(block: torch.Tensor, n_heads: int, M: int) -> list:
+    """Views (no copies) of a packed result block (uint8, host or device) as one output dict per head."""
+    stride = ee_exit_head_results_bytes(1, M)
+    outs = []
+    for k in range(n_heads):
+        b = block[k * stride:(k + 1) * stride]
+        outs.append(dict(argmax=b[0:4 * M].view(torch.int32), entropy=b[4 * M:8 * M].view(torch.float32),
+                         maxprob=b[8 * M:12 * M].view(torch.float32), exit_mask=b[12 * M:13 * M]))
+    return outs
+
+
+class PreparedMultiHost:
+    """ee_exit_head_multi_host with its argument block built once.
+
+    heads: list of dicts with gamma, beta, W, tau (device tensors / floats).  h_host: pinned bf16
+    [n_heads, M, d].  The staging buffers and the pinned result block are created here, once; `out_host`
+    and `out_dev` are per-head views into the packed result blocks.
+    """
+    __slots__ = ("_args", "_keep", "out_host", "out_dev", "h_dev", "h2d_bytes", "d2h_bytes")
+
+    def __init__(self, heads, ln_eps, h_host, workspace):
+        n, (_, M, d) = len(heads), h_host.shape
+        V = heads[0]["W"].shape[0]
+        dev = workspace.device
+        arr = (_lib.EEHead * n)()
+        keep = []
+        for i, hd in enumerate(heads):
+            W = _bf16(_dev(hd["W"], "W"))
+            tau = hd["tau"]
+            tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+            e = arr[i]
+            e.gamma, e.beta, e.W, e.tau_per_row, e.tau = _ptr(hd["gamma"]), _ptr(hd["beta"]), _ptr(W), _ptr(tau_t), tau_f
+            keep.append((W, hd["gamma"], hd["beta"], tau_t))
+        nbytes = ee_exit_head_results_bytes(n, M)
+        self.h_dev = torch.empty((n, M, d), dtype=torch.bfloat16, device=dev)
+        res_dev = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+        res_host = torch.zeros(nbytes, dtype=torch.uint8).pin_memory()
+        self.out_dev, self.out_host = results_views(res_dev, n, M), results_views(res_host, n, M)
+        self.h2d_bytes, self.d2h_bytes = h_host.numel() * 2, nbytes
+        self._args = (arr, n, float(ln_eps), M, d, V, _ptr(h_host), _ptr(self.h_dev), _ptr(res_host), _ptr(res_dev),
+                      _ptr(workspace), workspace.numel(), _stream())
+        self._keep = (arr, keep, h_host, res_dev, res_host, workspace)
+
+    def __call__(self):
+        code = _lib.load().ee_exit_head_multi_host(*self._args)
+        if code:
+            raise EExitError(code, "ee_exit_head_multi_host")
+        return self.out_host
+
+
 def prepare_exit_head(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None, path=EE_PATH_AUTO) -> PreparedCall:
     """ee_exit_head with the arguments marshalled once; see PreparedCall."""
     args, out, keep = _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path)

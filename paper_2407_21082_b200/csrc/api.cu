@@ -226,6 +226,39 @@ ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma,
     return EE_OK;
 }
 
+size_t ee_exit_head_results_bytes(int n_heads, int M) {
+    if (n_heads < 1 || M < 0) return 0;
+    return (size_t)n_heads * (((size_t)13 * M + 15) / 16 * 16);
+}
+
+ee_status ee_exit_head_multi_host(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
+                                  const void* h_host, void* h_dev, void* results_host, void* results_dev,
+                                  void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!sizes_ok(M, d, V) || n_heads < 0 || n_heads > 64) return EE_ERR_SHAPE;
+    if (n_heads == 0 || M == 0) return EE_OK;
+    if (!heads || !h_host || !h_dev || !results_host || !results_dev) return EE_ERR_NULL;
+    if (!aligned(h_dev, 16) || !aligned(results_dev, 16)) return EE_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t h_bytes = (size_t)M * d * 2, block = ee_exit_head_results_bytes(1, M);
+    ee_head dev_heads[64];
+    for (int k = 0; k < n_heads; ++k) {
+        unsigned char* r = static_cast<unsigned char*>(results_dev) + k * block;
+        dev_heads[k] = heads[k];
+        dev_heads[k].h = static_cast<unsigned char*>(h_dev) + k * h_bytes;
+        dev_heads[k].ld_h = d;
+        dev_heads[k].argmax = reinterpret_cast<int*>(r);
+        dev_heads[k].entropy = reinterpret_cast<float*>(r + (size_t)4 * M);
+        dev_heads[k].maxprob = reinterpret_cast<float*>(r + (size_t)8 * M);
+        dev_heads[k].exit_mask = r + (size_t)12 * M;
+    }
+    if (cudaMemcpyAsync(h_dev, h_host, n_heads * h_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return EE_ERR_CUDA;
+    const ee_status st = ee_exit_head_multi(dev_heads, n_heads, ln_eps, M, d, V, workspace, workspace_bytes_, stream);
+    if (st != EE_OK) return st;
+    if (cudaMemcpyAsync(results_host, results_dev, n_heads * block, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return EE_ERR_CUDA;
+    return EE_OK;
+}
+
 ee_status ee_compact(const unsigned char* exit_mask, const void* h, long long ld_h, int M, int d, int* kept_idx,
                      int* kept_count, void* h_out, void* stream) {
     if (M < 0) return EE_ERR_SHAPE;

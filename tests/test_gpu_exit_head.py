@@ -244,3 +244,27 @@ def test_multi_head_full_size_c1(ee):
         for k in range(3):
             ref = oracle_head(cfg["h"][:M], cfg["heads"][k], cfg["tau"])
             assert_head_matches(outs[k], ref, label=f"c1 multi M={M} head {k}")
+
+
+def test_multi_head_host_call_matches_oracle(ee):
+    """Packed host-buffer variant: one copy in, the heads, one copy out; device copies of the results stay usable."""
+    M, d, V, n_heads = 20, 256, 1500, 3
+    cfg = gen.make_config("c1", seed=23, planted=True, M=M, d=d, V=V, heads=n_heads)
+    hds = [head_to_dev(cfg["heads"][k]) for k in range(n_heads)]
+    taus = [0.7, 1.0, 2.0]
+    h_one = dev_bf16(cfg["h"]).cpu()
+    h_host = torch.stack([h_one] * n_heads).pin_memory()
+    ws = torch.empty(ee.ee_exit_head_multi_workspace_bytes(n_heads, M, d, V), dtype=torch.uint8, device="cuda")
+    ee.ee_workspace_init(ws)
+    call = ee.PreparedMultiHost([dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=t) for hd, t in zip(hds, taus)],
+                                1e-5, h_host, ws)
+    assert call.d2h_bytes == ee.ee_exit_head_results_bytes(n_heads, M) == n_heads * ((13 * M + 15) // 16 * 16)
+    for _ in range(2):
+        out = call()
+        torch.cuda.synchronize()
+        for k in range(n_heads):
+            ref = oracle_head(cfg["h"], cfg["heads"][k], taus[k])
+            assert_head_matches(out[k], ref, label=f"host multi head {k}")
+            for key in out[k]:
+                assert torch.equal(out[k][key], call.out_dev[k][key].cpu()), (k, key)
+    assert ee.ee_query_async_error(ws) == 0
