@@ -35,9 +35,10 @@ typedef enum {
 
 /* Kernel selection for ee_exit_head_path(). */
 typedef enum {
-    EE_PATH_AUTO = 0,      /* by M: streaming kernel up to 16 rows, tensor-core GEMM kernel above   */
+    EE_PATH_AUTO = 0,      /* the library's choice: the tensor-core path for every size             */
     EE_PATH_STREAM = 1,    /* fused LayerNorm + split-V streaming kernel (any M, in slabs of rows)  */
-    EE_PATH_TCGEN05 = 2,   /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics     */
+    EE_PATH_TCGEN05 = 2,   /* LayerNorm kernel + TMA/tcgen05 GEMM with fused softmax statistics
+                              (+ a merge kernel above 512 rows)                                      */
     EE_PATH_SKINNY = 3     /* one-launch tcgen05 kernel with W as the MMA's M operand: M <= 64, d % 64 == 0,
                               M_pad * d <= 64 Ki elements; other sizes return EE_ERR_SHAPE                */
 } ee_path;
