@@ -14,3 +14,4 @@ from .exit_head import (  # noqa: F401
     dssd_accept,
     decisive_rows,
 )
+from .calibrate import calibrate_threshold, calibrate_threshold_bruteforce, correctness  # noqa: F401,E402
