@@ -358,6 +358,42 @@ def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
                 api="ee_exit_head_multi_host + ee_compact_accept, three copies and one synchronise per step")
 
 
+def measure_calibration(peaks: dict, src: str, n: int = 1 << 22, calls: int = 30) -> dict:
+    """ee_calibrate (threshold of one head from n calibration tokens) timed with CUDA events, and the oracle on
+    the same set.  The sort has no fixed algorithmic byte count; `bytes_by_design` is what this implementation's
+    passes must move (pack 12 + 8 B, five passes of 8 + 8 + 8 B, two reads of 8 B per token)."""
+    import torch
+    import oracle
+    import paper_2407_21082_b200 as ee
+    cs = gen.make_calibration_set(0, n)
+    dev = {k: torch.from_numpy(v).cuda() for k, v in cs.items()}
+    call = ee.prepare_calibrate(dev["entropy"], dev["argmax_head"], dev["argmax_final"], 0.9)
+    for _ in range(3):
+        call()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(calls):
+        call()
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / calls
+    c0 = time.perf_counter()
+    ref = oracle.calibrate_threshold(cs["entropy"], oracle.correctness(cs["argmax_head"], cs["argmax_final"]), 0.9)
+    cpu_s = time.perf_counter() - c0
+    got = call.out if hasattr(call, "out") else None
+    counts = got["counts"].cpu().tolist()
+    assert counts == [ref["n_exit"], ref["n_correct"], ref["j_hat"]], (counts, ref)
+    by_design = (12 + 8 + 5 * 24 + 16) * n
+    gbs = by_design / (us * 1e-6) / 1e9
+    return dict(n_tokens=n, epsilon=0.9, us_per_call=round(us, 1), tokens_per_s=n / (us * 1e-6), launches=19,
+                roofline=dict(bound="hbm", bytes_by_design=by_design, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                              frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None),
+                result=dict(tau=float(got["tau"].item()), n_exit=counts[0], n_correct=counts[1]),
+                cpu_baseline=dict(value=n / cpu_s, unit="calibration tokens/s", seconds=round(cpu_s, 3), kind="oracle",
+                                  cores=oracle_threads(), sample="the same n tokens (numpy fp64, stable argsort + cumsum)"))
+
+
 def oracle_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -496,6 +532,7 @@ def main():
             del w
             torch.cuda.empty_cache()
         line["configs"] = extra
+        line["calibration"] = measure_calibration(peaks, peak_src)
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):

@@ -13,4 +13,5 @@ from .synth import (  # noqa: F401
     make_config,
     make_dssd_hidden,
     random_token_case,
+    make_calibration_set,
 )

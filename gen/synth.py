@@ -153,3 +153,21 @@ def random_token_case(seed: int, S: int, k: int, kv: int, alphabet: int = 3, p_c
     verify[:, :k] = np.where(keep, draft, verify[:, :k])
     return dict(draft_tok=draft, verify_tok=verify,
                 draft_exit_mask=(rng.random((S, k)) < p_confident).astype(np.uint8))
+
+
+def make_calibration_set(seed: int, n: int, V: int = 50304, ties: bool = False) -> dict:
+    """A stand-in for the scores a calibration epoch stores per head: an entropy per token (nats, spread over
+    0 .. ln V like the planted workloads' entropies: a surer half and a diffuse half), the head's token and the
+    full model's token, which agree more often where the entropy is low.  `ties` rounds the entropies to two
+    decimals so that many tokens share a value."""
+    rng = _rng(seed, "calibration", n, V)
+    sure = rng.random(n) < 0.45
+    H = np.where(sure, rng.gamma(1.2, 0.25, size=n), np.log(V) - rng.gamma(2.0, 1.2, size=n))
+    H = np.clip(H, 0.0, np.log(V)).astype(np.float32)
+    if ties:
+        H = np.round(H, 2).astype(np.float32)
+    final = rng.integers(0, V, size=n).astype(np.int32)
+    agree = rng.random(n) < np.exp(-H.astype(np.float64) / 2.5)
+    head = np.where(agree, final, (final + 1 + rng.integers(0, V - 1, size=n)) % V).astype(np.int32)
+    return dict(entropy=H, argmax_head=head, argmax_final=final)
+

@@ -223,6 +223,28 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
                             int* draft_len, int* accept_len, int* next_tok, void* stream);
 
 /*
+ * Calibration of one head's threshold from a calibration set (section 3.4.1, "Calibration of Confidence
+ * Thresholds": Eq. 3 and the two equations that define the index j-hat and tau_k = c_{k, j-hat}), with the
+ * entropy as the confidence metric.  Over n calibration tokens:
+ *   t_j = [argmax_head[j] == argmax_final[j]]                                   (Eq. 3)
+ *   the candidate sets are { j : entropy[j] <= v } for the distinct entropies v (tokens of equal entropy
+ *   enter together, so the result does not depend on how equal values are ordered);
+ *   the largest candidate set whose proportion of t_j = 1 is >= epsilon is chosen (the comparison
+ *   correct >= epsilon * count is made in fp64) -- the paper's smallest index j-hat in ascending confidence.
+ * Outputs (device): tau fp32 [1] = the largest entropy inside the chosen set (the paper's tau; a token AT the
+ * threshold is inside the set, so a caller of ee_exit_head, whose rule is H < tau, passes the next float
+ * above it), or -inf if no set qualifies (the head then never exits); counts int32 [3] = size of the chosen
+ * set, number of correct predictions in it, j-hat (1-based, 0 if none).
+ * entropy fp32 [n] must not contain NaN; argmax_head, argmax_final int32 [n]; 0 <= epsilon <= 1; n = 0 gives
+ * tau = -inf.  Workspace: ee_calibrate_workspace_bytes(n) bytes, 256-byte aligned (two copies of one
+ * 64-bit word per token and the sort's histograms); needs no initialisation.
+ */
+size_t    ee_calibrate_workspace_bytes(int n);       /* host-only, pure; 0 if n < 0 */
+ee_status ee_calibrate(const float* entropy, const int* argmax_head, const int* argmax_final, int n,
+                       double epsilon, float* tau, int* counts, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the error word of the workspace's control block.
  * Every device-side wait in the tensor-core kernel is bounded; one that gives up records itself there
  * and the kernel drains and returns.  EE_OK if nothing was recorded, EE_ERR_TIMEOUT otherwise (outputs

@@ -342,6 +342,34 @@ def prepare_compact_accept(exit_mask, h, draft_tok, draft_exit_mask, verify_tok,
     return PreparedCall(_lib.load().ee_compact_accept, args, "ee_compact_accept", keep, out)
 
 
+def _calibrate_args(entropy, argmax_head, argmax_final, epsilon, out, workspace):
+    n = entropy.numel()
+    dev = entropy.device
+    if not (entropy.dtype == torch.float32 and argmax_head.dtype == torch.int32 and argmax_final.dtype == torch.int32):
+        raise TypeError("entropy must be float32, the argmax arrays int32")
+    if not (entropy.is_contiguous() and argmax_head.is_contiguous() and argmax_final.is_contiguous()):
+        raise ValueError("calibration arrays must be contiguous")
+    if out is None:
+        out = dict(tau=torch.empty(1, dtype=torch.float32, device=dev), counts=torch.empty(3, dtype=torch.int32, device=dev))
+    if workspace is None:
+        workspace = torch.empty(int(_lib.load().ee_calibrate_workspace_bytes(n)), dtype=torch.uint8, device=dev)
+    args = (_ptr(entropy), _ptr(argmax_head), _ptr(argmax_final), n, float(epsilon), _ptr(out["tau"]), _ptr(out["counts"]),
+            _ptr(workspace), workspace.numel(), _stream())
+    return args, out, (entropy, argmax_head, argmax_final, workspace, out)
+
+
+def ee_calibrate(entropy, argmax_head, argmax_final, epsilon, *, out=None, workspace=None) -> dict:
+    """Threshold of one head from a calibration set (see include/eexit.h): dict(tau [1], counts [3]) on the device."""
+    args, out, _ = _calibrate_args(entropy, argmax_head, argmax_final, epsilon, out, workspace)
+    _check(_lib.load().ee_calibrate(*args), "ee_calibrate")
+    return out
+
+
+def prepare_calibrate(entropy, argmax_head, argmax_final, epsilon, *, out=None, workspace=None) -> PreparedCall:
+    args, out, keep = _calibrate_args(entropy, argmax_head, argmax_final, epsilon, out, workspace)
+    return PreparedCall(_lib.load().ee_calibrate, args, "ee_calibrate", keep, out)
+
+
 def _accept_args(draft_tok, draft_exit_mask, verify_tok, out):
     S, k = draft_tok.shape
     kv = verify_tok.shape[1]

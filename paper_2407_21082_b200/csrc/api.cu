@@ -308,6 +308,22 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
                                  static_cast<cudaStream_t>(stream));
 }
 
+size_t ee_calibrate_workspace_bytes(int n) { return n < 0 ? 0 : calibrate_workspace_bytes(n); }
+
+ee_status ee_calibrate(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
+                       float* tau, int* counts, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (n < 0 || !(epsilon >= 0.0 && epsilon <= 1.0)) return EE_ERR_SHAPE;
+    if (!tau || !counts || !workspace) return EE_ERR_NULL;
+    if (n > 0 && (!entropy || !argmax_head || !argmax_final)) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < calibrate_workspace_bytes(n)) return EE_ERR_WORKSPACE;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return calibrate_launch(entropy, argmax_head, argmax_final, n, epsilon, tau, counts, workspace,
+                            static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_query_async_error(void* workspace, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -1,0 +1,278 @@
+// Calibration of a head's threshold (paper section 3.4.1): joint sort of (confidence, correctness) over the
+// calibration tokens, running count of correct predictions, and the most permissive threshold whose set of
+// tokens is correct with proportion >= epsilon.
+//
+// The metric is the entropy H (smaller = surer).  Each token becomes one 64-bit word
+//     word = (monotone 32-bit key of H) << 1 | t        t = [argmax_head == argmax_final]   (Eq. 3)
+// and the words are sorted ascending by a least-significant-digit radix sort: five stable passes of 8 bits
+// over the 33 significant bits (per-tile digit histogram -> exclusive scan over (digit, tile) -> stable
+// scatter).  A last pass over the sorted words counts the correct predictions before each position and
+// tests  correct >= epsilon * count  (fp64) at every position that closes a group of equal entropies; the
+// largest such position wins (64-bit atomic max of (count << 32 | correct)).
+// Integer work throughout, except that one comparison.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ee {
+
+namespace {
+
+constexpr int kSortThreads = 256;
+constexpr int kItems = 16;                              // words per thread
+constexpr int kTile = kSortThreads * kItems;            // 4096 words per CTA
+constexpr int kWarpChunk = 32 * kItems;                 // 512 consecutive words per warp
+constexpr int kDigits = 256;
+constexpr int kPasses = 5;                              // 33 significant bits
+
+typedef unsigned long long u64;
+
+// Order-preserving map of a float onto unsigned integers (negative floats reversed below the positive ones;
+// the two zeros compare equal, so both take the key of +0).
+__device__ __forceinline__ unsigned int float_key(float f) {
+    const unsigned int b = f == 0.f ? 0u : __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(unsigned int k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+__global__ void __launch_bounds__(kSortThreads) calib_pack_kernel(const float* __restrict__ entropy,
+                                                                  const int* __restrict__ argmax_head,
+                                                                  const int* __restrict__ argmax_final, int n,
+                                                                  u64* __restrict__ words, u64* __restrict__ best) {
+    const int i = blockIdx.x * kSortThreads + threadIdx.x;
+    if (i == 0) *best = 0ull;
+    if (i >= n) return;
+    const unsigned int t = argmax_head[i] == argmax_final[i] ? 1u : 0u;
+    words[i] = ((u64)float_key(entropy[i]) << 1) | t;
+}
+
+// hist[digit * n_tiles + tile] = number of words of the tile whose digit of this pass is `digit`.
+__global__ void __launch_bounds__(kSortThreads) calib_hist_kernel(const u64* __restrict__ words, int n, int shift,
+                                                                  unsigned int* __restrict__ hist, int n_tiles) {
+    __shared__ unsigned int cnt[kDigits];
+    cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const int base = blockIdx.x * kTile;
+#pragma unroll
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * kSortThreads + threadIdx.x;
+        if (i < n) atomicAdd(&cnt[(unsigned int)(words[i] >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    hist[(size_t)threadIdx.x * n_tiles + blockIdx.x] = cnt[threadIdx.x];
+}
+
+// In-place exclusive scan of `len` counters by one CTA of 1024 threads (each thread a contiguous piece).
+__global__ void __launch_bounds__(1024) calib_scan_kernel(unsigned int* __restrict__ a, int len) {
+    __shared__ unsigned int warp_sum[32];
+    const int per = (len + 1023) / 1024;
+    const int lo = min(len, (int)threadIdx.x * per), hi = min(len, lo + per);
+    unsigned int s = 0;
+    for (int i = lo; i < hi; ++i) s += a[i];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned int incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned int w = warp_sum[lane], wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += v;
+        }
+        warp_sum[lane] = wi - w;                         // exclusive over warps
+    }
+    __syncthreads();
+    unsigned int run = warp_sum[warp] + incl - s;        // exclusive prefix of this thread's piece
+    for (int i = lo; i < hi; ++i) {
+        const unsigned int v = a[i];
+        a[i] = run;
+        run += v;
+    }
+}
+
+// Stable scatter of one tile.  Warp w owns words [512 w, 512 w + 512) of the tile and walks them 32 at a time,
+// so the order of equal digits inside the tile is (warp, round, lane) = their order in memory.
+__global__ void __launch_bounds__(kSortThreads) calib_scatter_kernel(const u64* __restrict__ src, u64* __restrict__ dst,
+                                                                     int n, int shift,
+                                                                     const unsigned int* __restrict__ offsets,
+                                                                     int n_tiles) {
+    __shared__ unsigned int cnt[kSortThreads / 32][kDigits];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < (kSortThreads / 32) * kDigits; i += kSortThreads) (&cnt[0][0])[i] = 0;
+    __syncthreads();
+    const int base = blockIdx.x * kTile + warp * kWarpChunk;
+    u64 v[kItems];
+    unsigned int rank[kItems];
+#pragma unroll
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * 32 + lane;
+        const bool valid = i < n;
+        v[r] = valid ? src[i] : 0ull;
+        const unsigned int d = valid ? ((unsigned int)(v[r] >> shift) & 255u) : 0xffffffffu;
+        const unsigned int peers = __match_any_sync(0xffffffffu, d);
+        const unsigned int before = valid ? cnt[warp][d] : 0u;                // all peers read, then the leader adds
+        __syncwarp();
+        if (valid && lane == __ffs(peers) - 1) cnt[warp][d] = before + __popc(peers);
+        __syncwarp();
+        rank[r] = before + __popc(peers & ((1u << lane) - 1u));
+    }
+    __syncthreads();
+    {   // thread = digit: where each warp's words of that digit start in the output
+        const unsigned int d = threadIdx.x;
+        unsigned int run = offsets[(size_t)d * n_tiles + blockIdx.x];
+#pragma unroll
+        for (int w = 0; w < kSortThreads / 32; ++w) {
+            const unsigned int c = cnt[w][d];
+            cnt[w][d] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * 32 + lane;
+        if (i < n) dst[cnt[warp][(unsigned int)(v[r] >> shift) & 255u] + rank[r]] = v[r];
+    }
+}
+
+// Correct predictions per tile of the sorted words.
+__global__ void __launch_bounds__(kSortThreads) calib_tile_sum_kernel(const u64* __restrict__ sorted, int n,
+                                                                      unsigned int* __restrict__ tile_sum) {
+    __shared__ unsigned int warp_part[kSortThreads / 32];
+    const int base = blockIdx.x * kTile;
+    unsigned int s = 0;
+#pragma unroll
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * kSortThreads + threadIdx.x;
+        if (i < n) s += (unsigned int)sorted[i] & 1u;
+    }
+    s = __reduce_add_sync(0xffffffffu, s);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int t = 0;
+        for (int w = 0; w < kSortThreads / 32; ++w) t += warp_part[w];
+        tile_sum[blockIdx.x] = t;
+    }
+}
+
+// Position i (0-based, surest first) closes a group when the next word has another key.  There the set of the
+// i + 1 surest tokens is tested; the largest qualifying set wins.
+__global__ void __launch_bounds__(kSortThreads) calib_select_kernel(const u64* __restrict__ sorted, int n,
+                                                                    const unsigned int* __restrict__ tile_sum,
+                                                                    double epsilon, u64* __restrict__ best) {
+    __shared__ unsigned int part[kSortThreads / 32];
+    __shared__ unsigned int s_before;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // correct predictions in the tiles before this one
+    unsigned int before = 0;
+    for (int b = threadIdx.x; b < (int)blockIdx.x; b += kSortThreads) before += tile_sum[b];
+    before = __reduce_add_sync(0xffffffffu, before);
+    if (lane == 0) part[warp] = before;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int t = 0;
+        for (int w = 0; w < kSortThreads / 32; ++w) t += part[w];
+        s_before = t;
+    }
+    __syncthreads();
+    before = s_before;
+    __syncthreads();
+    // thread = 16 consecutive positions
+    const int i0 = blockIdx.x * kTile + threadIdx.x * kItems;
+    u64 w[kItems + 1];
+#pragma unroll
+    for (int j = 0; j <= kItems; ++j) w[j] = (i0 + j < n) ? sorted[i0 + j] : ~0ull;
+    unsigned int mine = 0;
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) mine += (i0 + j < n) ? ((unsigned int)w[j] & 1u) : 0u;
+    unsigned int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+    }
+    if (lane == 31) part[warp] = incl;
+    __syncthreads();
+    unsigned int run = before + incl - mine;
+    for (int k = 0; k < warp; ++k) run += part[k];
+    u64 local_best = 0;
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+        const int i = i0 + j;
+        if (i < n) {
+            run += (unsigned int)w[j] & 1u;                        // correct among the i + 1 surest
+            const bool closes = (i + 1 == n) || ((w[j + 1] >> 1) != (w[j] >> 1));
+            if (closes && (double)run >= epsilon * (double)(i + 1)) local_best = ((u64)(i + 1) << 32) | run;
+        }
+    }
+    if (local_best) atomicMax(best, local_best);
+}
+
+__global__ void calib_output_kernel(const u64* __restrict__ sorted, int n, const u64* __restrict__ best,
+                                    float* __restrict__ tau, int* __restrict__ counts) {
+    const u64 b = *best;
+    const int n_exit = (int)(b >> 32);
+    counts[0] = n_exit;
+    counts[1] = (int)(b & 0xffffffffull);
+    counts[2] = n_exit ? n - n_exit + 1 : 0;
+    *tau = n_exit ? key_float((unsigned int)(sorted[n_exit - 1] >> 1)) : -CUDART_INF_F;
+}
+
+__global__ void calib_empty_kernel(float* __restrict__ tau, int* __restrict__ counts) {
+    counts[0] = counts[1] = counts[2] = 0;
+    *tau = -CUDART_INF_F;
+}
+
+size_t words_bytes(int n) { return align_up((size_t)n * sizeof(u64), 256); }
+int tiles_of(int n) { return (n + kTile - 1) / kTile; }
+
+}  // namespace
+
+size_t calibrate_workspace_bytes(int n) {
+    const int n_tiles = tiles_of(n);
+    return 256 + 2 * words_bytes(n) + align_up((size_t)kDigits * n_tiles * sizeof(unsigned int), 256) +
+           align_up((size_t)n_tiles * sizeof(unsigned int), 256);
+}
+
+int calibrate_launches(int n) { return n > 0 ? 1 + 3 * kPasses + 3 : 1; }
+
+ee_status calibrate_launch(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
+                           float* tau, int* counts, void* workspace, cudaStream_t stream) {
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    u64* best = reinterpret_cast<u64*>(ws);
+    u64* a = reinterpret_cast<u64*>(ws + 256);
+    u64* b = reinterpret_cast<u64*>(ws + 256 + words_bytes(n));
+    const int n_tiles = tiles_of(n);
+    unsigned int* hist = reinterpret_cast<unsigned int*>(ws + 256 + 2 * words_bytes(n));
+    unsigned int* tile_sum = hist + align_up((size_t)kDigits * n_tiles * sizeof(unsigned int), 256) / sizeof(unsigned int);
+    if (n == 0) {
+        calib_empty_kernel<<<1, 1, 0, stream>>>(tau, counts);
+        return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    }
+    calib_pack_kernel<<<(n + kSortThreads - 1) / kSortThreads, kSortThreads, 0, stream>>>(entropy, argmax_head,
+                                                                                           argmax_final, n, a, best);
+    u64 *src = a, *dst = b;
+    for (int pass = 0; pass < kPasses; ++pass) {
+        const int shift = 8 * pass;
+        calib_hist_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, n, shift, hist, n_tiles);
+        calib_scan_kernel<<<1, 1024, 0, stream>>>(hist, kDigits * n_tiles);
+        calib_scatter_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, dst, n, shift, hist, n_tiles);
+        u64* t = src;
+        src = dst;
+        dst = t;
+    }
+    calib_tile_sum_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, n, tile_sum);
+    calib_select_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, n, tile_sum, epsilon, best);
+    calib_output_kernel<<<1, 1, 0, stream>>>(src, n, best, tau, counts);
+    return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+}  // namespace ee

@@ -69,4 +69,10 @@ ee_status compact_accept_launch(const unsigned char* exit_mask, const void* h, l
                                 const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k, int kv,
                                 int* draft_len, int* accept_len, int* next_tok, cudaStream_t stream);
 
+// ---- calibration of a head's threshold (radix sort of the calibration tokens by entropy, scan, selection) ----
+size_t calibrate_workspace_bytes(int n);
+int calibrate_launches(int n);
+ee_status calibrate_launch(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
+                           float* tau, int* counts, void* workspace, cudaStream_t stream);
+
 }  // namespace ee
