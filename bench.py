@@ -361,7 +361,7 @@ def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
 def measure_calibration(peaks: dict, src: str, n: int = 1 << 22, calls: int = 30) -> dict:
     """ee_calibrate (threshold of one head from n calibration tokens) timed with CUDA events, and the oracle on
     the same set.  The sort has no fixed algorithmic byte count; `bytes_by_design` is what this implementation's
-    passes must move (pack 12 + 8 B, five passes of 8 + 8 + 8 B, two reads of 8 B per token)."""
+    passes must move (pack 12 + 8 B, four passes of 8 + 8 + 8 B, two reads of 8 B per token)."""
     import torch
     import oracle
     import paper_2407_21082_b200 as ee
@@ -384,9 +384,9 @@ def measure_calibration(peaks: dict, src: str, n: int = 1 << 22, calls: int = 30
     got = call.out if hasattr(call, "out") else None
     counts = got["counts"].cpu().tolist()
     assert counts == [ref["n_exit"], ref["n_correct"], ref["j_hat"]], (counts, ref)
-    by_design = (12 + 8 + 5 * 24 + 16) * n
+    by_design = (12 + 8 + 4 * 24 + 16) * n
     gbs = by_design / (us * 1e-6) / 1e9
-    return dict(n_tokens=n, epsilon=0.9, us_per_call=round(us, 1), tokens_per_s=n / (us * 1e-6), launches=19,
+    return dict(n_tokens=n, epsilon=0.9, us_per_call=round(us, 1), tokens_per_s=n / (us * 1e-6), launches=16,
                 roofline=dict(bound="hbm", bytes_by_design=by_design, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
                               frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None),
                 result=dict(tau=float(got["tau"].item()), n_exit=counts[0], n_correct=counts[1]),

@@ -4,9 +4,9 @@
 //
 // The metric is the entropy H (smaller = surer).  Each token becomes one 64-bit word
 //     word = (monotone 32-bit key of H) << 1 | t        t = [argmax_head == argmax_final]   (Eq. 3)
-// and the words are sorted ascending by a least-significant-digit radix sort: five stable passes of 8 bits
-// over the 33 significant bits (per-tile digit histogram -> exclusive scan over (digit, tile) -> stable
-// scatter).  A last pass over the sorted words counts the correct predictions before each position and
+// and the words are sorted ascending by key with a least-significant-digit radix sort: four stable passes of
+// 8 bits over the key's 32 bits (per-tile digit histogram -> per-digit exclusive scan over the tiles -> stable
+// scatter); t rides along in bit 0 and is not sorted on, because tokens of equal entropy are judged as one group.  A last pass over the sorted words counts the correct predictions before each position and
 // tests  correct >= epsilon * count  (fp64) at every position that closes a group of equal entropies; the
 // largest such position wins (64-bit atomic max of (count << 32 | correct)).
 // Integer work throughout, except that one comparison.
@@ -22,7 +22,7 @@ constexpr int kItems = 16;                              // words per thread
 constexpr int kTile = kSortThreads * kItems;            // 4096 words per CTA
 constexpr int kWarpChunk = 32 * kItems;                 // 512 consecutive words per warp
 constexpr int kDigits = 256;
-constexpr int kPasses = 5;                              // 33 significant bits
+constexpr int kPasses = 4;                              // the 32 key bits; bit 0 (t) is carried, not sorted on
 
 typedef unsigned long long u64;
 
@@ -63,51 +63,66 @@ __global__ void __launch_bounds__(kSortThreads) calib_hist_kernel(const u64* __r
     hist[(size_t)threadIdx.x * n_tiles + blockIdx.x] = cnt[threadIdx.x];
 }
 
-// In-place exclusive scan of `len` counters by one CTA of 1024 threads (each thread a contiguous piece).
-__global__ void __launch_bounds__(1024) calib_scan_kernel(unsigned int* __restrict__ a, int len) {
+// One CTA per digit: in-place exclusive scan of the digit's row hist[digit][0 .. n_tiles) (where each tile's
+// words of that digit start among all words of that digit) and the row total.
+__global__ void __launch_bounds__(1024) calib_scan_kernel(unsigned int* __restrict__ hist, int n_tiles,
+                                                          unsigned int* __restrict__ digit_total) {
     __shared__ unsigned int warp_sum[32];
-    const int per = (len + 1023) / 1024;
-    const int lo = min(len, (int)threadIdx.x * per), hi = min(len, lo + per);
-    unsigned int s = 0;
-    for (int i = lo; i < hi; ++i) s += a[i];
+    __shared__ unsigned int s_carry;
+    unsigned int* row = hist + (size_t)blockIdx.x * n_tiles;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned int incl = s;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sum[warp] = incl;
+    if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
-    if (warp == 0) {
-        unsigned int w = warp_sum[lane], wi = w;
+    for (int t0 = 0; t0 < n_tiles; t0 += 1024) {
+        const int t = t0 + threadIdx.x;
+        const unsigned int v = t < n_tiles ? row[t] : 0u;
+        unsigned int incl = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const unsigned int v = __shfl_up_sync(0xffffffffu, wi, o);
-            if (lane >= o) wi += v;
+            const unsigned int x = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += x;
         }
-        warp_sum[lane] = wi - w;                         // exclusive over warps
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned int w = warp_sum[lane];
+            unsigned int wi = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int x = __shfl_up_sync(0xffffffffu, wi, o);
+                if (lane >= o) wi += x;
+            }
+            warp_sum[lane] = wi - w;                     // exclusive over warps
+        }
+        __syncthreads();
+        const unsigned int carry = s_carry;
+        if (t < n_tiles) row[t] = carry + warp_sum[warp] + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) s_carry = carry + warp_sum[31] + incl;
+        __syncthreads();
     }
-    __syncthreads();
-    unsigned int run = warp_sum[warp] + incl - s;        // exclusive prefix of this thread's piece
-    for (int i = lo; i < hi; ++i) {
-        const unsigned int v = a[i];
-        a[i] = run;
-        run += v;
-    }
+    if (threadIdx.x == 0) digit_total[blockIdx.x] = s_carry;
 }
 
 // Stable scatter of one tile.  Warp w owns words [512 w, 512 w + 512) of the tile and walks them 32 at a time,
-// so the order of equal digits inside the tile is (warp, round, lane) = their order in memory.
-__global__ void __launch_bounds__(kSortThreads) calib_scatter_kernel(const u64* __restrict__ src, u64* __restrict__ dst,
+// so the order of equal digits inside the tile is (warp, round, lane) = their order in memory.  The tile is
+// first put in output order in shared memory, so that consecutive threads then write consecutive words of a
+// digit's run to global memory.
+__global__ void __launch_bounds__(kSortThreads, 3) calib_scatter_kernel(const u64* __restrict__ src, u64* __restrict__ dst,
                                                                      int n, int shift,
-                                                                     const unsigned int* __restrict__ offsets,
+                                                                     const unsigned int* __restrict__ tile_start,
+                                                                     const unsigned int* __restrict__ digit_total,
                                                                      int n_tiles) {
     __shared__ unsigned int cnt[kSortThreads / 32][kDigits];
+    __shared__ unsigned int local_start[kDigits];      // where the digit's words start inside the sorted tile
+    __shared__ unsigned int global_start[kDigits];     // where this tile's words of the digit start in the output
+    __shared__ unsigned int warp_part[kSortThreads / 32];
+    __shared__ u64 staged[kTile];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < (kSortThreads / 32) * kDigits; i += kSortThreads) (&cnt[0][0])[i] = 0;
     __syncthreads();
-    const int base = blockIdx.x * kTile + warp * kWarpChunk;
+    const int tile_base = blockIdx.x * kTile;
+    const int base = tile_base + warp * kWarpChunk;
     u64 v[kItems];
     unsigned int rank[kItems];
 #pragma unroll
@@ -124,9 +139,33 @@ __global__ void __launch_bounds__(kSortThreads) calib_scatter_kernel(const u64* 
         rank[r] = before + __popc(peers & ((1u << lane) - 1u));
     }
     __syncthreads();
-    {   // thread = digit: where each warp's words of that digit start in the output
+    {   // thread = digit d: the tile's count of d, the exclusive scan of the counts over the digits (inside the
+        // tile) and of the digit totals (over all words), and each warp's start inside the digit's run
         const unsigned int d = threadIdx.x;
-        unsigned int run = offsets[(size_t)d * n_tiles + blockIdx.x];
+        unsigned int mine = 0;
+#pragma unroll
+        for (int w = 0; w < kSortThreads / 32; ++w) mine += cnt[w][d];
+        const unsigned int total = digit_total[d];
+        unsigned int incl = mine, gincl = total;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int x = __shfl_up_sync(0xffffffffu, incl, o);
+            const unsigned int g = __shfl_up_sync(0xffffffffu, gincl, o);
+            if (lane >= o) { incl += x; gincl += g; }
+        }
+        if (lane == 31) warp_part[warp] = incl;
+        __syncthreads();
+        unsigned int lbase = 0;
+        for (int w = 0; w < warp; ++w) lbase += warp_part[w];
+        __syncthreads();
+        if (lane == 31) warp_part[warp] = gincl;
+        __syncthreads();
+        unsigned int gbase = 0;
+        for (int w = 0; w < warp; ++w) gbase += warp_part[w];
+        const unsigned int lstart = lbase + incl - mine;
+        local_start[d] = lstart;
+        global_start[d] = gbase + gincl - total + tile_start[(size_t)d * n_tiles + blockIdx.x];
+        unsigned int run = lstart;
 #pragma unroll
         for (int w = 0; w < kSortThreads / 32; ++w) {
             const unsigned int c = cnt[w][d];
@@ -138,7 +177,14 @@ __global__ void __launch_bounds__(kSortThreads) calib_scatter_kernel(const u64* 
 #pragma unroll
     for (int r = 0; r < kItems; ++r) {
         const int i = base + r * 32 + lane;
-        if (i < n) dst[cnt[warp][(unsigned int)(v[r] >> shift) & 255u] + rank[r]] = v[r];
+        if (i < n) staged[cnt[warp][(unsigned int)(v[r] >> shift) & 255u] + rank[r]] = v[r];
+    }
+    __syncthreads();
+    const int in_tile = min(kTile, n - tile_base);
+    for (int k = threadIdx.x; k < in_tile; k += kSortThreads) {
+        const u64 w = staged[k];
+        const unsigned int d = (unsigned int)(w >> shift) & 255u;
+        dst[global_start[d] + ((unsigned int)k - local_start[d])] = w;
     }
 }
 
@@ -164,56 +210,70 @@ __global__ void __launch_bounds__(kSortThreads) calib_tile_sum_kernel(const u64*
 }
 
 // Position i (0-based, surest first) closes a group when the next word has another key.  There the set of the
-// i + 1 surest tokens is tested; the largest qualifying set wins.
+// i + 1 surest tokens is tested; the largest qualifying set wins.  Warp w walks positions [512 w, 512 w + 512)
+// of the tile 32 at a time (held in registers), after the warps have exchanged their counts.
 __global__ void __launch_bounds__(kSortThreads) calib_select_kernel(const u64* __restrict__ sorted, int n,
                                                                     const unsigned int* __restrict__ tile_sum,
                                                                     double epsilon, u64* __restrict__ best) {
     __shared__ unsigned int part[kSortThreads / 32];
-    __shared__ unsigned int s_before;
+    __shared__ unsigned int warp_total[kSortThreads / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // correct predictions in the tiles before this one
-    unsigned int before = 0;
+    unsigned int before = 0;                                   // correct predictions in the tiles before this one
     for (int b = threadIdx.x; b < (int)blockIdx.x; b += kSortThreads) before += tile_sum[b];
     before = __reduce_add_sync(0xffffffffu, before);
-    if (lane == 0) part[warp] = before;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned int t = 0;
-        for (int w = 0; w < kSortThreads / 32; ++w) t += part[w];
-        s_before = t;
-    }
-    __syncthreads();
-    before = s_before;
-    __syncthreads();
-    // thread = 16 consecutive positions
-    const int i0 = blockIdx.x * kTile + threadIdx.x * kItems;
-    u64 w[kItems + 1];
-#pragma unroll
-    for (int j = 0; j <= kItems; ++j) w[j] = (i0 + j < n) ? sorted[i0 + j] : ~0ull;
+    const int base = blockIdx.x * kTile + warp * kWarpChunk;
+    u64 w[kItems];
     unsigned int mine = 0;
 #pragma unroll
-    for (int j = 0; j < kItems; ++j) mine += (i0 + j < n) ? ((unsigned int)w[j] & 1u) : 0u;
-    unsigned int incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned int x = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += x;
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * 32 + lane;
+        w[r] = i < n ? sorted[i] : ~0ull;
+        mine += i < n ? ((unsigned int)w[r] & 1u) : 0u;
     }
-    if (lane == 31) part[warp] = incl;
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if (lane == 0) { part[warp] = before; warp_total[warp] = mine; }
     __syncthreads();
-    unsigned int run = before + incl - mine;
-    for (int k = 0; k < warp; ++k) run += part[k];
+    unsigned int run = 0;
+    for (int k = 0; k < kSortThreads / 32; ++k) run += part[k] + (k < warp ? warp_total[k] : 0u);
+    // the word after this warp's chunk (the first of the next warp's, or of the next tile)
+    const int after = base + kWarpChunk;
+    const u64 chunk_next = after < n ? sorted[after] : ~0ull;
     u64 local_best = 0;
 #pragma unroll
-    for (int j = 0; j < kItems; ++j) {
-        const int i = i0 + j;
-        if (i < n) {
-            run += (unsigned int)w[j] & 1u;                        // correct among the i + 1 surest
-            const bool closes = (i + 1 == n) || ((w[j + 1] >> 1) != (w[j] >> 1));
-            if (closes && (double)run >= epsilon * (double)(i + 1)) local_best = ((u64)(i + 1) << 32) | run;
+    for (int r = 0; r < kItems; ++r) {
+        const int i = base + r * 32 + lane;
+        const unsigned int t = i < n ? ((unsigned int)w[r] & 1u) : 0u;
+        unsigned int incl = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int x = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += x;
         }
+        u64 next = __shfl_down_sync(0xffffffffu, w[r], 1);
+        const u64 first_of_next = (r + 1 < kItems) ? w[(r + 1) % kItems] : chunk_next;   // lane 0's follows lane 31's word
+        const u64 next_round = __shfl_sync(0xffffffffu, first_of_next, 0);
+        if (lane == 31) next = next_round;
+        if (i < n) {
+            const unsigned int correct = run + incl;               // correct among the i + 1 surest
+            const bool closes = (i + 1 == n) || ((next >> 1) != (w[r] >> 1));
+            if (closes && (double)correct >= epsilon * (double)(i + 1)) local_best = ((u64)(i + 1) << 32) | correct;
+        }
+        run += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (local_best) atomicMax(best, local_best);
+    // one atomic per CTA: the candidates of a CTA are reduced first (positions grow with lane, round and warp)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const u64 x = __shfl_xor_sync(0xffffffffu, local_best, o);
+        local_best = x > local_best ? x : local_best;
+    }
+    __shared__ u64 warp_best[kSortThreads / 32];
+    if (lane == 0) warp_best[warp] = local_best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u64 m = 0;
+        for (int k = 0; k < kSortThreads / 32; ++k) m = warp_best[k] > m ? warp_best[k] : m;
+        if (m) atomicMax(best, m);
+    }
 }
 
 __global__ void calib_output_kernel(const u64* __restrict__ sorted, int n, const u64* __restrict__ best,
@@ -231,6 +291,8 @@ __global__ void calib_empty_kernel(float* __restrict__ tau, int* __restrict__ co
     *tau = -CUDART_INF_F;
 }
 
+constexpr size_t kCalibHeader = 2048;      // the result word and the 256 digit totals
+
 size_t words_bytes(int n) { return align_up((size_t)n * sizeof(u64), 256); }
 int tiles_of(int n) { return (n + kTile - 1) / kTile; }
 
@@ -238,7 +300,7 @@ int tiles_of(int n) { return (n + kTile - 1) / kTile; }
 
 size_t calibrate_workspace_bytes(int n) {
     const int n_tiles = tiles_of(n);
-    return 256 + 2 * words_bytes(n) + align_up((size_t)kDigits * n_tiles * sizeof(unsigned int), 256) +
+    return kCalibHeader + 2 * words_bytes(n) + align_up((size_t)kDigits * n_tiles * sizeof(unsigned int), 256) +
            align_up((size_t)n_tiles * sizeof(unsigned int), 256);
 }
 
@@ -248,11 +310,12 @@ ee_status calibrate_launch(const float* entropy, const int* argmax_head, const i
                            float* tau, int* counts, void* workspace, cudaStream_t stream) {
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     u64* best = reinterpret_cast<u64*>(ws);
-    u64* a = reinterpret_cast<u64*>(ws + 256);
-    u64* b = reinterpret_cast<u64*>(ws + 256 + words_bytes(n));
+    u64* a = reinterpret_cast<u64*>(ws + kCalibHeader);
+    u64* b = reinterpret_cast<u64*>(ws + kCalibHeader + words_bytes(n));
     const int n_tiles = tiles_of(n);
-    unsigned int* hist = reinterpret_cast<unsigned int*>(ws + 256 + 2 * words_bytes(n));
+    unsigned int* hist = reinterpret_cast<unsigned int*>(ws + kCalibHeader + 2 * words_bytes(n));
     unsigned int* tile_sum = hist + align_up((size_t)kDigits * n_tiles * sizeof(unsigned int), 256) / sizeof(unsigned int);
+    unsigned int* digit_total = reinterpret_cast<unsigned int*>(ws + 8);        // 256 counters inside the first 2 KB
     if (n == 0) {
         calib_empty_kernel<<<1, 1, 0, stream>>>(tau, counts);
         return cudaGetLastError() == cudaSuccess ? EE_OK : EE_ERR_CUDA;
@@ -261,10 +324,10 @@ ee_status calibrate_launch(const float* entropy, const int* argmax_head, const i
                                                                                            argmax_final, n, a, best);
     u64 *src = a, *dst = b;
     for (int pass = 0; pass < kPasses; ++pass) {
-        const int shift = 8 * pass;
+        const int shift = 1 + 8 * pass;
         calib_hist_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, n, shift, hist, n_tiles);
-        calib_scan_kernel<<<1, 1024, 0, stream>>>(hist, kDigits * n_tiles);
-        calib_scatter_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, dst, n, shift, hist, n_tiles);
+        calib_scan_kernel<<<kDigits, 1024, 0, stream>>>(hist, n_tiles, digit_total);
+        calib_scatter_kernel<<<n_tiles, kSortThreads, 0, stream>>>(src, dst, n, shift, hist, digit_total, n_tiles);
         u64* t = src;
         src = dst;
         dst = t;
