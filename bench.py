@@ -403,14 +403,17 @@ def oracle_threads() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_step(cfg: dict, rows: int, heads: int):
+def oracle_step(cfg: dict, rows: int, heads: int, keep: list | None = None):
     """The oracle's version of a step on the first `rows` rows and `heads` heads.  Returns rows*heads."""
     import oracle
     hb = cfg["h_draft" if "h_draft" in cfg else "h"][:rows]
     tau = cfg["tau_per_row"][:rows] if "tau_per_row" in cfg else cfg["tau"]
     outs = []
-    for hd in cfg["heads"][:heads]:
-        outs.append(oracle.exit_head(hb, hd["gamma"], hd["beta"], hd["ln_eps"], hd["W"], tau))
+    for k, hd in enumerate(cfg["heads"][:heads]):
+        hk = cfg["h_verify"][:rows] if ("h_verify" in cfg and k > 0) else hb      # the verify head reads its own rows
+        outs.append(oracle.exit_head(hk, hd["gamma"], hd["beta"], hd["ln_eps"], hd["W"], tau))
+    if keep is not None:
+        keep.extend(outs)
     oracle.compact(outs[0]["exit_mask"], hb)
     S = rows // 8
     if S:
@@ -419,15 +422,35 @@ def oracle_step(cfg: dict, rows: int, heads: int):
     return rows * heads
 
 
-def cpu_baseline(cfg: dict, steps: int = 1, warmup: int = 0) -> dict:
+def parity_report(gpu_outs: list, ref_outs: list) -> dict:
+    """The timed workload's device results against the oracle's on the rows the oracle evaluated."""
+    import oracle
+    rep = dict(rows=int(ref_outs[0]["entropy"].size), heads=len(ref_outs), max_abs_dH=0.0, max_abs_dP=0.0,
+               argmax_mismatch=0, mask_mismatch=0, excluded_argmax=0, excluded_mask=0, exit_fraction=0.0)
+    for got, ref in zip(gpu_outs, ref_outs):
+        n = ref["entropy"].size
+        keep = oracle.decisive_rows(ref, 1e-3, 1e-3)
+        g = {k: v[:n] for k, v in got.items()}
+        rep["max_abs_dH"] = max(rep["max_abs_dH"], float(np.abs(g["entropy"].astype(np.float64) - ref["entropy"]).max()))
+        rep["max_abs_dP"] = max(rep["max_abs_dP"], float(np.abs(g["maxprob"].astype(np.float64) - ref["maxprob"]).max()))
+        rep["argmax_mismatch"] += int(((g["argmax"] != ref["argmax"]) & keep["argmax"]).sum())
+        rep["mask_mismatch"] += int(((g["exit_mask"] != ref["exit_mask"]) & keep["exit_mask"]).sum())
+        rep["excluded_argmax"] += int((~keep["argmax"]).sum())
+        rep["excluded_mask"] += int((~keep["exit_mask"]).sum())
+        rep["exit_fraction"] += float(ref["exit_mask"].mean()) / len(ref_outs)
+    rep["tolerance"] = "entropy, maxprob within 2e-3; argmax / mask exact outside top-2 gap < 1e-3 and |H - tau| < 1e-3"
+    return rep
+
+
+def cpu_baseline(cfg: dict, steps: int = 1, warmup: int = 0, keep: list | None = None) -> dict:
     """Times the oracle, as it stands, on the host cores on a bounded sample of the headline workload."""
     rows, heads = min(cfg["M"], 64), len(cfg["heads"])
     for _ in range(warmup):
         oracle_step(cfg, rows, heads)
     t0 = time.perf_counter()
     done = 0
-    for _ in range(steps):
-        done += oracle_step(cfg, rows, heads)
+    for i in range(steps):
+        done += oracle_step(cfg, rows, heads, keep if i == 0 else None)
     dt = time.perf_counter() - t0
     return dict(value=done / dt, unit=UNIT, cores=oracle_threads(), kind="oracle", seconds=round(dt, 2),
                 sample=f"{steps} step(s) of all {rows} rows x {heads} heads of the workload (fp64 numpy, weights decoded per call)")
@@ -512,6 +535,7 @@ def main():
                                   "one would break their programmatic dependent launch chain), averaged per head; "
                                   "tail_us = step time minus that")
     config["heads_call"] = "ee_exit_head_multi" if wl.multi else "ee_exit_head per head"
+    gpu_outs = [{k: v.cpu().numpy() for k, v in o.items()} for o in wl.outs] if rank == 0 else None
     if rank == 0:
         line["e2e"] = measure_e2e(wl, max(10, args.steps // 4), 3)
         if world > 1:
@@ -553,7 +577,9 @@ def main():
                     torch.cuda.empty_cache()
             line["sweep_head_call_us"] = sweep
         cfg = gen.make_config(args.workload, seed=0, planted=False, M=M)
-        line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0)
+        ref_outs = []
+        line["cpu_baseline"] = cpu_baseline(cfg, steps=1, warmup=0, keep=ref_outs)
+        line["parity"] = parity_report(gpu_outs, ref_outs)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -32,6 +32,12 @@ SMALL = [
     ("v1", 3, 64, 1), ("tiny", 1, 8, 5), ("ragged", 5, 72, 257), ("k_tail", 8, 520, 1000),
     ("two_ntiles", 16, 128, 300), ("slab_edge", 32, 256, 2049), ("slab_over", 33, 264, 1031),
     ("mtile_edge", 128, 64, 700), ("mtile_over", 129, 320, 515), ("wide_d", 4, 4096, 600),
+    # vocabulary sizes around one tile, the smallest d, and row counts at the tensor-core path's switches:
+    # 64 / 65 rows (64- vs 128-row MMAs), 512 / 513 (merge inside the GEMM kernel vs merge kernel),
+    # 1024 / 1025 (runtime-width vs 256-wide variant)
+    ("v2", 2, 8, 2), ("v127", 3, 64, 127), ("v128", 127, 64, 128), ("v129", 1, 64, 129),
+    ("m64", 64, 128, 400), ("m65", 65, 128, 400), ("m512", 512, 64, 300), ("m513", 513, 64, 300),
+    ("m1024", 1024, 64, 300), ("m1025", 1025, 64, 520),
 ]
 
 
