@@ -132,10 +132,10 @@ __global__ void __launch_bounds__(kSortThreads, 3) calib_scatter_kernel(const u6
         v[r] = valid ? src[i] : 0ull;
         const unsigned int d = valid ? ((unsigned int)(v[r] >> shift) & 255u) : 0xffffffffu;
         const unsigned int peers = __match_any_sync(0xffffffffu, d);
-        const unsigned int before = valid ? cnt[warp][d] : 0u;                // all peers read, then the leader adds
-        __syncwarp();
-        if (valid && lane == __ffs(peers) - 1) cnt[warp][d] = before + __popc(peers);
-        __syncwarp();
+        const int leader = __ffs(peers) - 1;
+        unsigned int before = 0;                                             // the leader reserves the group's ranks
+        if (valid && lane == leader) before = atomicAdd(&cnt[warp][d], (unsigned int)__popc(peers));
+        before = __shfl_sync(0xffffffffu, before, leader);
         rank[r] = before + __popc(peers & ((1u << lane) - 1u));
     }
     __syncthreads();
