@@ -15,3 +15,4 @@ from .exit_head import (  # noqa: F401
     decisive_rows,
 )
 from .calibrate import calibrate_threshold, calibrate_threshold_bruteforce, correctness  # noqa: F401,E402
+from .cascade import cascade  # noqa: F401,E402
