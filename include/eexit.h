@@ -223,6 +223,25 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
                             int* draft_len, int* accept_len, int* next_tok, void* stream);
 
 /*
+ * The inference-time cascade of section 3.4.2 ("Inference Process") for a batch: the heads are tried in the
+ * order given; head k is evaluated (as by ee_exit_head, scalar threshold heads[k].tau, rule H < tau) on the
+ * rows that no earlier head answered, reading row i of the batch from ITS OWN hidden states heads[k].h
+ * (bf16 [M, d], row stride heads[k].ld_h: the batch at head k's layer); a row stops at the first head that
+ * answers it.  A last head with tau = +infinity plays the full model.
+ * Outputs (device): exit_head int32 [M] = index of the answering head, n_heads if none; token int32 [M] = that
+ * head's argmax, -1 if none; entropy fp32 [M] = that head's entropy, NaN if none; rows_in int32 [n_heads] =
+ * the number of rows each head was evaluated on (head usage = rows_in[k] - rows_in[k+1]).
+ * Of each ee_head the output pointers are ignored and tau_per_row must be NULL.  The row counts stay on the
+ * device: no synchronisation between heads; head k's weights are streamed once whatever the count, its
+ * LayerNorm and statistics run on the surviving rows only.  Workspace: ee_cascade_workspace_bytes(M, d, V),
+ * 256-byte aligned, initialised once with ee_workspace_init.  M = 0 writes rows_in = 0.
+ */
+size_t    ee_cascade_workspace_bytes(int M, int d, int V);      /* host-only, pure; 0 if a size is invalid */
+ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, int* exit_head,
+                     int* token, float* entropy, int* rows_in, void* workspace, size_t workspace_bytes,
+                     void* stream);
+
+/*
  * Calibration of one head's threshold from a calibration set (section 3.4.1, "Calibration of Confidence
  * Thresholds": Eq. 3 and the two equations that define the index j-hat and tau_k = c_{k, j-hat}), with the
  * entropy as the confidence metric.  Over n calibration tokens:

@@ -40,6 +40,9 @@ PROTOTYPES = {
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_compact_accept": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p,
                                     _p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
+    "ee_cascade_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
+    "ee_cascade": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p,
+                             _p, C.c_size_t, _p]),
     "ee_calibrate_workspace_bytes": (C.c_size_t, [C.c_int]),
     "ee_calibrate": (C.c_int, [_p, _p, _p, C.c_int, C.c_double, _p, _p, _p, C.c_size_t, _p]),
     "ee_query_async_error": (C.c_int, [_p, _p]),

@@ -342,6 +342,53 @@ def prepare_compact_accept(exit_mask, h, draft_tok, draft_exit_mask, verify_tok,
     return PreparedCall(_lib.load().ee_compact_accept, args, "ee_compact_accept", keep, out)
 
 
+def _cascade_args(heads, ln_eps, out, workspace):
+    n = len(heads)
+    arr = (_lib.EEHead * n)()
+    keep = []
+    M, d = _bf16(heads[0]["h"]).shape
+    V = heads[0]["W"].shape[0]
+    dev = heads[0]["h"].device
+    for i, hd in enumerate(heads):
+        h, W = _bf16(_dev(hd["h"], "h")), _bf16(_dev(hd["W"], "W"))
+        if h.shape != (M, d) or W.shape != (V, d) or not W.is_contiguous() or h.stride(1) != 1:
+            raise ValueError("all heads must share M, d, V; W contiguous [V, d]; h row-major [M, d]")
+        e = arr[i]
+        e.h, e.ld_h, e.gamma, e.beta, e.W = _ptr(h), (h.stride(0) if M > 1 else max(h.stride(0), d)), _ptr(hd["gamma"]), _ptr(hd["beta"]), _ptr(W)
+        e.tau_per_row, e.tau = None, float(hd["tau"])
+        keep.append((h, W, hd["gamma"], hd["beta"]))
+    if out is None:
+        out = dict(exit_head=torch.empty(M, dtype=torch.int32, device=dev), token=torch.empty(M, dtype=torch.int32, device=dev),
+                   entropy=torch.empty(M, dtype=torch.float32, device=dev), rows_in=torch.empty(n, dtype=torch.int32, device=dev))
+    if workspace is None:
+        workspace = torch.empty(int(_lib.load().ee_cascade_workspace_bytes(M, d, V)), dtype=torch.uint8, device=dev)
+        ee_workspace_init(workspace)
+    args = (arr, n, float(ln_eps), M, d, V, _ptr(out["exit_head"]), _ptr(out["token"]), _ptr(out["entropy"]), _ptr(out["rows_in"]),
+            _ptr(workspace), workspace.numel(), _stream())
+    return args, out, (arr, keep, workspace, out)
+
+
+def ee_cascade(heads, ln_eps, *, out=None, workspace=None) -> dict:
+    """Cascade of heads on a batch (see include/eexit.h): heads is a list of dicts with h, gamma, beta, W, tau."""
+    args, out, _ = _cascade_args(heads, ln_eps, out, workspace)
+    _check(_lib.load().ee_cascade(*args), "ee_cascade")
+    return out
+
+
+class PreparedCascade:
+    """ee_cascade with its argument block built once (see PreparedCall)."""
+    __slots__ = ("_args", "_keep", "out")
+
+    def __init__(self, heads, ln_eps, out=None, workspace=None):
+        self._args, self.out, self._keep = _cascade_args(heads, ln_eps, out, workspace)
+
+    def __call__(self):
+        code = _lib.load().ee_cascade(*self._args)
+        if code:
+            raise EExitError(code, "ee_cascade")
+        return self.out
+
+
 def _calibrate_args(entropy, argmax_head, argmax_final, epsilon, out, workspace):
     n = entropy.numel()
     dev = entropy.device

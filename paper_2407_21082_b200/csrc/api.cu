@@ -111,7 +111,7 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
         return EE_ERR_ALIGN;
     if (workspace_bytes_ < workspace_bytes(M, d, V)) return EE_ERR_WORKSPACE;
 
-    HeadArgs a;
+    HeadArgs a{};
     const ee_status dev = current_device(&a.device, &a.num_sms);
     if (dev != EE_OK) return dev;
     a.h = h; a.ld_h = ld_h; a.gamma = gamma; a.beta = beta; a.ln_eps = ln_eps; a.W = W;
@@ -157,7 +157,7 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
         if (e.ld_h < d || (e.ld_h % 8) != 0) return EE_ERR_SHAPE;
         if (!aligned(e.h, 16) || !aligned(e.W, 16) || !aligned(e.gamma, 16) || !aligned(e.beta, 16)) return EE_ERR_ALIGN;
     }
-    HeadArgs base;
+    HeadArgs base{};
     const ee_status dev = current_device(&base.device, &base.num_sms);
     if (dev != EE_OK) return dev;
     // The tensor-core path batches the heads (one LayerNorm, one GEMM, one merge launch for up to four).
@@ -306,6 +306,61 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
     return compact_accept_launch(exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out, draft_tok, draft_exit_mask,
                                  verify_tok, S, k, kv, draft_len, accept_len, next_tok,
                                  static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+size_t cascade_head_ws(int M, int d, int V) { return align_up(kCtrlBytes + gemm_workspace_bytes(M, d, V, 1), 256); }
+size_t cascade_rows_bytes(int M) { return align_up((size_t)M * 4, 256); }
+}  // namespace
+
+size_t ee_cascade_workspace_bytes(int M, int d, int V) {
+    if (!sizes_ok(M, d, V)) return 0;
+    return cascade_head_ws(M, d, V) + 6 * cascade_rows_bytes(M) + 256;
+}
+
+ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, int* exit_head, int* token,
+                     float* entropy, int* rows_in, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!sizes_ok(M, d, V) || n_heads < 1 || n_heads > 64) return EE_ERR_SHAPE;
+    if (!heads || !rows_in || !workspace) return EE_ERR_NULL;
+    if (M > 0 && (!exit_head || !token || !entropy)) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < ee_cascade_workspace_bytes(M, d, V)) return EE_ERR_WORKSPACE;
+    for (int k = 0; k < n_heads; ++k) {
+        const ee_head& e = heads[k];
+        if (M > 0 && (!e.h || !e.gamma || !e.beta || !e.W)) return EE_ERR_NULL;
+        if (e.tau_per_row) return EE_ERR_SHAPE;          // thresholds belong to heads here, not to rows
+        if (e.ld_h < d || (e.ld_h % 8) != 0) return EE_ERR_SHAPE;
+        if (!aligned(e.h, 16) || !aligned(e.W, 16) || !aligned(e.gamma, 16) || !aligned(e.beta, 16)) return EE_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (M == 0) return cudaMemsetAsync(rows_in, 0, (size_t)n_heads * sizeof(int), s) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+    HeadArgs a{};
+    const ee_status dev = current_device(&a.device, &a.num_sms);
+    if (dev != EE_OK) return dev;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    unsigned char* p = ws + cascade_head_ws(M, d, V);
+    const size_t rb = cascade_rows_bytes(M);
+    int* t_argmax = reinterpret_cast<int*>(p);
+    float* t_entropy = reinterpret_cast<float*>(p + rb);
+    float* t_maxprob = reinterpret_cast<float*>(p + 2 * rb);
+    unsigned char* t_mask = p + 3 * rb;
+    int* idx[2] = {reinterpret_cast<int*>(p + 4 * rb), reinterpret_cast<int*>(p + 5 * rb)};
+    int* count = reinterpret_cast<int*>(p + 6 * rb);         // count[0], count[1]: survivors, ping-pong
+    for (int k = 0; k < n_heads; ++k) {
+        const ee_head& e = heads[k];
+        a.h = e.h; a.ld_h = e.ld_h; a.gamma = e.gamma; a.beta = e.beta; a.ln_eps = ln_eps; a.W = e.W;
+        a.M = M; a.d = d; a.V = V; a.tau_per_row = nullptr; a.tau = e.tau;
+        a.argmax = t_argmax; a.entropy = t_entropy; a.maxprob = t_maxprob; a.exit_mask = t_mask;
+        a.workspace = workspace; a.workspace_bytes = cascade_head_ws(M, d, V); a.stream = s;
+        a.row_idx = k ? idx[(k - 1) & 1] : nullptr;
+        a.m_dev = k ? count + ((k - 1) & 1) : nullptr;
+        ee_status st = gemm_launch(&a, 1);
+        if (st != EE_OK) return st;
+        st = cascade_step_launch(t_mask, t_argmax, t_entropy, a.row_idx, a.m_dev, M, k, k == n_heads - 1, n_heads, exit_head,
+                                 token, entropy, idx[k & 1], count + (k & 1), rows_in, s);
+        if (st != EE_OK) return st;
+    }
+    return EE_OK;
 }
 
 size_t ee_calibrate_workspace_bytes(int n) { return n < 0 ? 0 : calibrate_workspace_bytes(n); }

@@ -525,6 +525,40 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
     }
 }
 
+// LayerNorm of a gathered subset of one head's rows: output row j = LayerNorm(h[row_idx[j]]) for j < *m_dev,
+// zeros from there to the end of the padded tile rows.  The list and the count come from an earlier kernel of
+// the stream (the cascade of heads), so everything is read after the dependency wait.  Warp per row.
+__global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloat16* __restrict__ h, long long ld_h,
+                                                                const float* __restrict__ gamma,
+                                                                const float* __restrict__ beta, float ln_eps,
+                                                                const int* __restrict__ row_idx,
+                                                                const int* __restrict__ m_dev,
+                                                                __nv_bfloat16* __restrict__ y, int M, int d) {
+    launch_dependents();
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int m_pad = (M + BM - 1) / BM * BM;
+    if (row >= m_pad) return;
+    const int nvec = d >> 3;
+    uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
+    grid_dependency_wait();
+    const int m_live = m_dev ? min(max(*m_dev, 0), M) : M;
+    if (row >= m_live) {
+        for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const int src = row_idx ? row_idx[row] : row;
+    const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)src * ld_h);
+    const float inv_d = 1.f / (float)d;
+    float sum = 0.f;
+    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
+    const float mu = warp_sum(sum) * inv_d;
+    float sq = 0.f;
+    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
+    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
+    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
 // blockIdx.y = head.
@@ -636,7 +670,11 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     const dim3 row_grid((a.M + 7) / 8, n_heads);
     const dim3 ln_grid((a.M + BM - 1) / BM * (BM / 8), n_heads);
     cudaError_t err;
-    if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    if (a.row_idx || a.m_dev) {
+        if (n_heads != 1) return EE_ERR_SHAPE;
+        err = launch_pdl(layer_norm_gather_kernel, dim3(ln_grid.x), 256, 0, a.stream, ln.h[0], a.ld_h, a.gamma, a.beta,
+                         a.ln_eps, a.row_idx, a.m_dev, y, a.M, a.d);
+    } else if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     else err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     if (err != cudaSuccess) return EE_ERR_CUDA;

@@ -29,6 +29,12 @@ struct HeadArgs {
     cudaStream_t stream;
     int device;       // current device ordinal
     int num_sms;      // its multiprocessor count
+    // Optional (tensor-core path, one head per launch): evaluate the rows h[row_idx[j]], j < *m_dev, instead of
+    // rows 0 .. M-1; output row j belongs to input row row_idx[j], output rows at and beyond *m_dev are
+    // meaningless.  Either may be NULL (identity / M).  Both are device pointers read after the stream's
+    // earlier kernels have finished.
+    const int* row_idx;
+    const int* m_dev;
 };
 
 // ---- streaming kernel (fused LayerNorm + split-V mma.sync GEMV + last-CTA merge; up to four heads per launch) ----
@@ -74,5 +80,11 @@ size_t calibrate_workspace_bytes(int n);
 int calibrate_launches(int n);
 ee_status calibrate_launch(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
                            float* tau, int* counts, void* workspace, cudaStream_t stream);
+
+// ---- one step of the cascade of heads: rows answered by head k are recorded, the others move on ----
+ee_status cascade_step_launch(const unsigned char* exit_mask, const int* argmax, const float* entropy,
+                              const int* idx_in, const int* m_in, int M, int k, int is_last, int n_heads,
+                              int* exit_head, int* token, float* entropy_out, int* idx_out, int* m_out, int* rows_in,
+                              cudaStream_t stream);
 
 }  // namespace ee

@@ -52,7 +52,7 @@ extern "C" ee_status ee_exit_head_static(const void* h, long long ld_h, const fl
     auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
     if (misaligned(h) || misaligned(W) || misaligned(gamma) || misaligned(beta)) return EE_ERR_ALIGN;
 
-    HeadArgs a;
+    HeadArgs a{};
     if (cudaGetDevice(&a.device) != cudaSuccess || a.device < 0 || a.device >= kMaxDevices) return EE_ERR_CUDA;
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, a.device) != cudaSuccess ||
