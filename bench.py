@@ -394,6 +394,51 @@ def measure_calibration(peaks: dict, src: str, n: int = 1 << 22, calls: int = 30
                                   cores=oracle_threads(), sample="the same n tokens (numpy fp64, stable argsort + cumsum)"))
 
 
+def measure_cascade(peaks: dict, src: str, M: int = 64, calls: int = 300) -> dict:
+    """ee_cascade on the c1 shape (three heads in depth order, the last one with tau = +inf playing the full
+    model) with planted inputs so that rows do exit; two copies of every W in rotation (cold L2)."""
+    import torch
+    import oracle
+    import paper_2407_21082_b200 as ee
+    cfg = gen.make_config("c1", seed=0, planted=True, M=M)
+    taus = [1.0, 1.0, float("inf")]
+
+    def bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    h = bf16(cfg["h"])
+    ws = torch.empty(ee.ee_cascade_workspace_bytes(M, cfg["d"], cfg["V"]), dtype=torch.uint8, device="cuda")
+    ee.ee_workspace_init(ws)
+    prepared = []
+    for c in range(2):
+        heads = [dict(h=h, gamma=torch.from_numpy(hd["gamma"]).cuda(), beta=torch.from_numpy(hd["beta"]).cuda(),
+                      W=bf16(hd["W"]), tau=taus[k]) for k, hd in enumerate(cfg["heads"])]
+        prepared.append(ee.PreparedCascade(heads, 1e-5, workspace=ws))
+    for i in range(6):
+        prepared[i % 2]()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for i in range(calls):
+        prepared[i % 2]()
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / calls
+    out = {k: v.cpu().numpy() for k, v in prepared[(calls - 1) % 2].out.items()}
+    c0 = time.perf_counter()
+    ref = oracle.cascade([cfg["h"]] * 3, cfg["heads"], taus)
+    cpu_s = time.perf_counter() - c0
+    same = int((out["exit_head"] == ref["exit_head"]).sum())
+    w_bytes = 3 * 2.0 * cfg["V"] * cfg["d"]
+    gbs = w_bytes / (us * 1e-6) / 1e9
+    return dict(M=M, heads=3, taus=[1.0, 1.0, "inf"], us_per_call=round(us, 2), launches=3 * 3, rows_in=out["rows_in"].tolist(),
+                rows_per_s=M / (us * 1e-6), rows_agreeing_with_oracle=same,
+                roofline=dict(bound="hbm", algorithmic_bytes=w_bytes, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                              frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None),
+                cpu_baseline=dict(value=M / cpu_s, unit="rows/s", seconds=round(cpu_s, 2), kind="oracle", cores=oracle_threads(),
+                                  sample="the same 64 rows through the same three heads"))
+
+
 def oracle_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -557,6 +602,7 @@ def main():
             torch.cuda.empty_cache()
         line["configs"] = extra
         line["calibration"] = measure_calibration(peaks, peak_src)
+        line["cascade"] = measure_cascade(peaks, peak_src)
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):

@@ -342,6 +342,14 @@ def prepare_compact_accept(exit_mask, h, draft_tok, draft_exit_mask, verify_tok,
     return PreparedCall(_lib.load().ee_compact_accept, args, "ee_compact_accept", keep, out)
 
 
+def ee_cascade_workspace_bytes(M: int, d: int, V: int) -> int:
+    return int(_lib.load().ee_cascade_workspace_bytes(int(M), int(d), int(V)))
+
+
+def ee_calibrate_workspace_bytes(n: int) -> int:
+    return int(_lib.load().ee_calibrate_workspace_bytes(int(n)))
+
+
 def _cascade_args(heads, ln_eps, out, workspace):
     n = len(heads)
     arr = (_lib.EEHead * n)()
