@@ -73,3 +73,33 @@ def test_argument_errors_come_back_before_any_launch(lib):
     addr = (ctypes.addressof(buf) + 255) // 256 * 256
     assert lib.ee_workspace_init(ctypes.c_void_p(addr + 8), 512, None) == 3      # EE_ERR_ALIGN
     assert lib.ee_workspace_init(ctypes.c_void_p(addr), 16, None) == 4           # EE_ERR_WORKSPACE
+
+
+def test_argument_errors_of_the_later_entry_points(lib):
+    """ee_compact_accept, ee_exit_head_multi_host, ee_calibrate, ee_cascade: validation returns before any launch."""
+    from paper_2407_21082_b200 import _lib
+    N = None
+    # compaction + accept in one launch: the shape rules of both parts
+    assert lib.ee_compact_accept(N, N, 0, 4, 8, N, N, N, N, N, N, 2, 0, 0, N, N, N, N) == 2          # k < 1
+    assert lib.ee_compact_accept(N, N, 0, 4, 8, N, N, N, N, N, N, 2, 4, 3, N, N, N, N) == 2          # kv < k
+    assert lib.ee_compact_accept(N, N, 0, 4, 8, N, N, N, N, N, N, 2, 4, 4, N, N, N, N) == 1          # kept_count NULL
+    # packed results
+    assert lib.ee_exit_head_results_bytes(3, 64) == 3 * 832 and lib.ee_exit_head_results_bytes(1, 1) == 16
+    assert lib.ee_exit_head_results_bytes(0, 64) == 0 and lib.ee_exit_head_results_bytes(2, -1) == 0
+    heads = (_lib.EEHead * 2)()
+    assert lib.ee_exit_head_multi_host(heads, 2, 1e-5, 8, 500, 100, N, N, N, N, N, 0, N) == 2        # d % 8
+    assert lib.ee_exit_head_multi_host(heads, 2, 1e-5, 8, 512, 100, N, N, N, N, N, 0, N) == 1        # NULL buffers
+    assert lib.ee_exit_head_multi_host(heads, 0, 1e-5, 8, 512, 100, N, N, N, N, N, 0, N) == 0        # no heads: no-op
+    # calibration
+    assert lib.ee_calibrate_workspace_bytes(-1) == 0
+    w0, w1 = lib.ee_calibrate_workspace_bytes(0), lib.ee_calibrate_workspace_bytes(1 << 20)
+    assert w0 >= 2048 and w1 >= 2 * 8 * (1 << 20) and w1 < 3 * 8 * (1 << 20)
+    assert lib.ee_calibrate(N, N, N, -1, 0.5, N, N, N, 0, N) == 2
+    assert lib.ee_calibrate(N, N, N, 4, 1.5, N, N, N, 0, N) == 2                                     # epsilon outside [0, 1]
+    assert lib.ee_calibrate(N, N, N, 4, float("nan"), N, N, N, 0, N) == 2
+    assert lib.ee_calibrate(N, N, N, 4, 0.5, N, N, N, 0, N) == 1
+    # cascade
+    assert lib.ee_cascade_workspace_bytes(8, 500, 100) == 0
+    assert lib.ee_cascade_workspace_bytes(64, 1024, 50304) > lib.ee_exit_head_workspace_bytes(64, 1024, 50304)
+    assert lib.ee_cascade(heads, 0, 1e-5, 8, 512, 100, N, N, N, N, N, 0, N) == 2                     # no heads
+    assert lib.ee_cascade(heads, 2, 1e-5, 8, 512, 100, N, N, N, N, N, 0, N) == 1                     # NULL outputs
