@@ -271,6 +271,15 @@ ee_status ee_calibrate(const float* entropy, const int* argmax_head, const int* 
  */
 ee_status ee_query_async_error(void* workspace, void* stream);
 
+/*
+ * Diagnostic for the error path above (no counterpart in the paper): launches one small kernel whose only wait
+ * is on a barrier that nothing signals.  The wait gives up after about a millisecond, the kernel records the
+ * error word in `workspace`'s control block as the real kernels would and returns normally -- nothing faults,
+ * the context and the workspace stay usable.  The next ee_query_async_error on that workspace returns
+ * EE_ERR_TIMEOUT (and clears the word).  For tests of a caller's error handling.
+ */
+ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -46,6 +46,7 @@ PROTOTYPES = {
     "ee_calibrate_workspace_bytes": (C.c_size_t, [C.c_int]),
     "ee_calibrate": (C.c_int, [_p, _p, _p, C.c_int, C.c_double, _p, _p, _p, C.c_size_t, _p]),
     "ee_query_async_error": (C.c_int, [_p, _p]),
+    "ee_selftest_wait_timeout": (C.c_int, [_p, C.c_size_t, _p]),
 }
 
 

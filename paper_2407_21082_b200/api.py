@@ -350,6 +350,11 @@ def ee_calibrate_workspace_bytes(n: int) -> int:
     return int(_lib.load().ee_calibrate_workspace_bytes(int(n)))
 
 
+def ee_selftest_wait_timeout(workspace) -> None:
+    """Makes one bounded device-side wait give up (see include/eexit.h); ee_query_async_error then reports it."""
+    _check(_lib.load().ee_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream()), "ee_selftest_wait_timeout")
+
+
 def _cascade_args(heads, ln_eps, out, workspace):
     n = len(heads)
     arr = (_lib.EEHead * n)()

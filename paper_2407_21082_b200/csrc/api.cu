@@ -379,6 +379,16 @@ ee_status ee_calibrate(const float* entropy, const int* argmax_head, const int* 
                             static_cast<cudaStream_t>(stream));
 }
 
+ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!workspace) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < (size_t)kCtrlBytes) return EE_ERR_WORKSPACE;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return selftest_wait_timeout_launch(workspace, static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_query_async_error(void* workspace, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -81,6 +81,9 @@ int calibrate_launches(int n);
 ee_status calibrate_launch(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
                            float* tau, int* counts, void* workspace, cudaStream_t stream);
 
+// ---- diagnostic: a bounded wait that is made to give up ----
+ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
+
 // ---- one step of the cascade of heads: rows answered by head k are recorded, the others move on ----
 ee_status cascade_step_launch(const unsigned char* exit_mask, const int* argmax, const float* entropy,
                               const int* idx_in, const int* m_in, int M, int k, int is_last, int n_heads,
