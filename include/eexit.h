@@ -211,6 +211,30 @@ ee_status dssd_accept(const int* draft_tok, const unsigned char* draft_exit_mask
                       int S, int k, int kv, int* draft_len, int* accept_len, int* next_tok, void* stream);
 
 /*
+ * Commit step of one DSSD round for S sequences whose committed tokens live in device buffers (section 4.3.1:
+ * the three stop conditions of the drafting phase and the atomic commit of the verification phase).  For a
+ * sequence with finished[s] == 0:
+ *   draft_len[s]  = leading confident draft slots, at most k (the buffer limit), and not beyond the first
+ *                   drafted token equal to eos_token (that token is the last one drafted); eos_token < 0
+ *                   switches that stop off
+ *   accept_len[s] = leading j < draft_len[s] with draft_tok[s, j] == verify_tok[s, j]
+ *   committed     = the accepted tokens, then verify_tok[s, accept_len[s]] if accept_len[s] < kv and the last
+ *                   accepted token is not eos_token (next_tok[s]; -1 when nothing follows), appended to
+ *                   out_tok[s, seq_len[s] ...] and cut at `capacity`
+ *   seq_len[s] grows by the number appended; finished[s] becomes 1 when eos_token was appended or the buffer
+ *   is full.
+ * A sequence with finished[s] != 0 is left untouched (its draft_len, accept_len = 0, next_tok = -1).
+ * stats int64 [4] accumulates over calls: tokens drafted, accepted, appended, and sequences that took part (the
+ * paper's acceptance rate is accepted / drafted, its wasted tokens drafted - accepted); the caller zeroes it.
+ * draft_tok int32 [S, k], draft_exit_mask uint8 [S, k] or NULL, verify_tok int32 [S, kv], 1 <= k <= 32,
+ * kv >= k; out_tok int32 [S, capacity]; seq_len int32 [S]; finished uint8 [S]; the three outputs int32 [S].
+ */
+ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S,
+                      int k, int kv, int eos_token, int* out_tok, int capacity, int* seq_len,
+                      unsigned char* finished, int* draft_len, int* accept_len, int* next_tok, long long* stats,
+                      void* stream);
+
+/*
  * ee_compact and dssd_accept in one kernel launch, for a decoding step that needs both (section 3.4.2 and
  * section 4.3.1): both read the heads' outputs and write disjoint results, so one launch does the work of two
  * and a step saves a launch boundary.  Arguments, layouts and results are exactly those of the two calls;

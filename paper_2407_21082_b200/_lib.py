@@ -38,6 +38,7 @@ PROTOTYPES = {
                                       _p, _p, _p, _p, _p]),
     "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
+    "dssd_commit": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, C.c_int, _p, C.c_int, _p, _p, _p, _p, _p, _p, _p]),
     "ee_compact_accept": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p,
                                     _p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_cascade_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),

@@ -430,6 +430,23 @@ def prepare_calibrate(entropy, argmax_head, argmax_final, epsilon, *, out=None, 
     return PreparedCall(_lib.load().ee_calibrate, args, "ee_calibrate", keep, out)
 
 
+def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos_token, state: dict, *, out=None) -> dict:
+    """Commit step of a DSSD round (see include/eexit.h).  `state` holds the sequences' device tensors: out_tok
+    int32 [S, capacity], seq_len int32 [S], finished uint8 [S], stats int64 [4]; they are updated in place."""
+    S, k = draft_tok.shape
+    kv = verify_tok.shape[1]
+    dev = draft_tok.device
+    if not (draft_tok.is_contiguous() and verify_tok.is_contiguous() and state["out_tok"].is_contiguous()):
+        raise ValueError("token arrays must be contiguous")
+    if out is None:
+        out = {n: torch.empty(S, dtype=torch.int32, device=dev) for n in ("draft_len", "accept_len", "next_tok")}
+    _check(_lib.load().dssd_commit(_ptr(draft_tok), _ptr(draft_exit_mask), _ptr(verify_tok), S, k, kv, int(eos_token),
+                                   _ptr(state["out_tok"]), state["out_tok"].shape[1], _ptr(state["seq_len"]),
+                                   _ptr(state["finished"]), _ptr(out["draft_len"]), _ptr(out["accept_len"]),
+                                   _ptr(out["next_tok"]), _ptr(state["stats"]), _stream()), "dssd_commit")
+    return out
+
+
 def _accept_args(draft_tok, draft_exit_mask, verify_tok, out):
     S, k = draft_tok.shape
     kv = verify_tok.shape[1]

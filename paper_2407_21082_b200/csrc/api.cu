@@ -379,6 +379,20 @@ ee_status ee_calibrate(const float* entropy, const int* argmax_head, const int* 
                             static_cast<cudaStream_t>(stream));
 }
 
+ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k, int kv,
+                      int eos_token, int* out_tok, int capacity, int* seq_len, unsigned char* finished, int* draft_len,
+                      int* accept_len, int* next_tok, long long* stats, void* stream) {
+    if (S < 0 || k < 1 || k > 32 || kv < k || capacity < 1) return EE_ERR_SHAPE;
+    if (S == 0) return EE_OK;
+    if (!draft_tok || !verify_tok || !out_tok || !seq_len || !finished || !draft_len || !accept_len || !next_tok || !stats)
+        return EE_ERR_NULL;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return dssd_commit_launch(draft_tok, draft_exit_mask, verify_tok, S, k, kv, eos_token, out_tok, capacity, seq_len, finished,
+                              draft_len, accept_len, next_tok, stats, static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     if (!aligned(workspace, 256)) return EE_ERR_ALIGN;

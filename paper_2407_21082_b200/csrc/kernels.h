@@ -81,6 +81,11 @@ int calibrate_launches(int n);
 ee_status calibrate_launch(const float* entropy, const int* argmax_head, const int* argmax_final, int n, double epsilon,
                            float* tau, int* counts, void* workspace, cudaStream_t stream);
 
+// ---- commit step of a DSSD round (k <= 32) ----
+ee_status dssd_commit_launch(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k,
+                             int kv, int eos, int* out_tok, int cap, int* seq_len, unsigned char* finished, int* draft_len,
+                             int* accept_len, int* next_tok, long long* stats, cudaStream_t stream);
+
 // ---- diagnostic: a bounded wait that is made to give up ----
 ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
 
