@@ -14,4 +14,5 @@ from .synth import (  # noqa: F401
     make_dssd_hidden,
     random_token_case,
     make_calibration_set,
+    make_markov_model,
 )

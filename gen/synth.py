@@ -171,3 +171,15 @@ def make_calibration_set(seed: int, n: int, V: int = 50304, ties: bool = False) 
     head = np.where(agree, final, (final + 1 + rng.integers(0, V - 1, size=n)) % V).astype(np.int32)
     return dict(entropy=H, argmax_head=head, argmax_final=final)
 
+
+def make_markov_model(seed: int, V: int, d: int, planting: dict | None, sigma: float = 0.5) -> dict:
+    """A stand-in for the transformer below the heads in a decoding loop: the hidden state of a position depends
+    on the previous token only.  Two tables of bf16 rows [V, d], one read by the draft head and one by the full
+    model's head; row t is a*u + N(0, I) as in make_hidden (with a planting the direction is one of the planted
+    ones, so the heads answer with that direction's token), the draft table = the other + sigma * N(0, I)."""
+    rng = _rng(seed, "markov", V, d)
+    hv, a, j = _hidden_f32(rng, V, d, planting)
+    hv_bits = bf16_bits_from_f32(hv)
+    hd = f32_from_bf16_bits(hv_bits) + np.float32(sigma) * rng.standard_normal((V, d), dtype=np.float32)
+    return dict(E_verify=hv_bits, E_draft=bf16_bits_from_f32(hd), a=a, j=j)
+

@@ -16,4 +16,4 @@ from .exit_head import (  # noqa: F401
 )
 from .calibrate import calibrate_threshold, calibrate_threshold_bruteforce, correctness  # noqa: F401,E402
 from .cascade import cascade  # noqa: F401,E402
-from .dssd_round import dssd_commit  # noqa: F401,E402
+from .dssd_round import dssd_commit, dssd_round  # noqa: F401,E402

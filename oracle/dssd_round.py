@@ -58,3 +58,37 @@ def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos: int, out_tok, seq_l
         draft_len[s], accept_len[s] = n, a
         stats += np.array([n, a, len(commit), 1], dtype=stats.dtype)
     return dict(draft_len=draft_len, accept_len=accept_len, next_tok=next_tok)
+
+
+def dssd_round(E_draft, E_verify, draft_head, verify_head, tau: float, eos: int, k: int, last_tok, out_tok, seq_len,
+               finished, stats) -> dict:
+    """One whole DSSD round (drafting phase, verification phase, commit) for S sequences, with the hidden state of
+    a position given by a table row of the previous token (the tests' stand-in for the transformer).
+
+    Drafting: k steps; step j evaluates the draft head on E_draft[previous token] (the last committed token for
+    j = 0, the token drafted at j - 1 after that); its argmax is the drafted token, its exit decision the
+    confidence.  Verification: the full model's head on E_verify[previous token] for the k draft positions and
+    one bonus position, all at once.  Then dssd_commit.  last_tok is updated to each sequence's last committed
+    token.  Every sequence goes through all k steps (what lies beyond its stop is ignored by the commit)."""
+    from .exit_head import exit_head
+    S = last_tok.size
+    cur = last_tok.astype(np.int64).copy()
+    draft = np.zeros((S, k), np.int32)
+    mask = np.zeros((S, k), np.uint8)
+    steps = []
+    for j in range(k):
+        o = exit_head(E_draft[cur], draft_head["gamma"], draft_head["beta"], draft_head["ln_eps"], draft_head["W"], tau)
+        draft[:, j], mask[:, j] = o["argmax"], o["exit_mask"]
+        cur = o["argmax"].astype(np.int64)
+        steps.append(o)
+    prev_all = np.concatenate([last_tok.astype(np.int64)[:, None], draft.astype(np.int64)], axis=1)      # [S, k + 1]
+    v = exit_head(E_verify[prev_all.reshape(-1)], verify_head["gamma"], verify_head["beta"], verify_head["ln_eps"],
+                  verify_head["W"], np.inf)
+    verify = v["argmax"].reshape(S, k + 1).astype(np.int32)
+    was_finished = finished.copy()
+    r = dssd_commit(draft, mask, verify, eos, out_tok, seq_len, finished, stats)
+    for s in range(S):
+        if not was_finished[s] and seq_len[s] > 0:
+            last_tok[s] = out_tok[s, seq_len[s] - 1]
+    return dict(draft_tok=draft, draft_mask=mask, verify_tok=verify, steps=steps, verify_out=v, **r)
+

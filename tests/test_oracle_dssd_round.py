@@ -72,3 +72,49 @@ def test_rounds_accumulate_and_finished_sequences_are_left_alone():
                 assert fin[s] and row[-1] == eos and (row[:-1] != eos).all()     # nothing after the end of sequence
             assert fin[s] == (eos in row or sl[s] >= cap)
     assert fin.sum() > 0 and st[2] == sl.sum() and st[1] <= st[0]
+
+
+def _model(seed=0, V=400, d=64):
+    cfg = gen.make_config("c1", seed=seed, planted=True, M=4, d=d, V=V, heads=2)
+    planting = gen.make_planting(seed, f"c1/planted/d{d}/V{V}", d, V)
+    mm = gen.make_markov_model(seed, V, d, planting, sigma=0.4)
+    return cfg, mm
+
+
+def _greedy(mm, head, start, n):
+    """Plain autoregressive decoding with the full model's head: token after t = argmax head(E_verify[t])."""
+    out, cur = [], start.astype(np.int64)
+    for _ in range(n):
+        o = oracle.exit_head(mm["E_verify"][cur], head["gamma"], head["beta"], head["ln_eps"], head["W"], np.inf)
+        cur = o["argmax"].astype(np.int64)
+        out.append(cur.copy())
+    return np.stack(out, axis=1)
+
+
+def test_round_reduces_to_greedy_decoding_in_the_two_limits():
+    cfg, mm = _model()
+    S, k, cap = 6, 4, 64
+    start = np.arange(S, dtype=np.int32) * 7 % 400
+    want = _greedy(mm, cfg["heads"][1], start, 12)
+    # (a) the draft head is never confident: every round commits exactly the full model's next token
+    st = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    last = start.copy()
+    for _ in range(5):
+        oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], -1.0, -1, k, last, *st)
+    assert np.array_equal(st[0][:, :5], want[:, :5]) and (st[1] == 5).all() and st[3].tolist() == [0, 0, 5 * S, 5 * S]
+    # (b) the draft is the full model itself and always confident: every round commits k + 1 tokens of the same chain
+    st = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    last = start.copy()
+    for _ in range(2):
+        oracle.dssd_round(mm["E_verify"], mm["E_verify"], cfg["heads"][1], cfg["heads"][1], np.inf, -1, k, last, *st)
+    assert (st[1] == 2 * (k + 1)).all() and np.array_equal(st[0][:, :10], want[:, :10])
+    assert st[3].tolist() == [2 * k * S, 2 * k * S, 2 * (k + 1) * S, 2 * S]
+    # (c) any threshold in between: the committed text is still the full model's greedy chain (speculation never
+    #     changes the output), only the number of rounds needed differs
+    st = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    last = start.copy()
+    for _ in range(3):
+        oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], 1.0, -1, k, last, *st)
+    for s in range(S):
+        assert np.array_equal(st[0][s, :st[1][s]], want[s, :st[1][s]])
+    assert 3 * S <= st[1].sum() <= 3 * (k + 1) * S and st[3][1] <= st[3][0]
