@@ -439,6 +439,73 @@ def measure_cascade(peaks: dict, src: str, M: int = 64, calls: int = 300) -> dic
                                   sample="the same 64 rows through the same three heads"))
 
 
+def measure_dssd_round(peaks: dict, src: str, S: int = 32, k: int = 8, rounds: int = 40) -> dict:
+    """Whole DSSD rounds (k drafting steps, one verification pass, commit) on the c1 shape, with the hidden states
+    coming from a table lookup by the previous token (gen.make_markov_model: the stand-in for the transformer,
+    supplied through the driver's callback and run with torch.index_select).  Timed with CUDA events over
+    `rounds` rounds; the first round is also run by the oracle."""
+    import torch
+    import oracle
+    import paper_2407_21082_b200 as ee
+    spec = gen.CONFIGS["c1"]
+    d, V = spec["d"], spec["V"]
+    cfg = gen.make_config("c1", seed=0, planted=True, M=4, heads=2)
+    planting = gen.make_planting(0, f"c1/planted/d{d}/V{V}", d, V)
+    mm = gen.make_markov_model(0, V, d, planting, sigma=0.4)
+
+    def bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    E = [bf16(mm["E_draft"]), bf16(mm["E_verify"])]
+    heads = [dict(gamma=torch.from_numpy(hd["gamma"]).cuda(), beta=torch.from_numpy(hd["beta"]).cuda(), W=bf16(hd["W"]))
+             for hd in cfg["heads"]]
+    heads[0]["tau"] = 1.0
+    cap = rounds * (k + 1) + 1
+    start = ((np.arange(S, dtype=np.int32) * 1543) % V).astype(np.int32)
+    state = dict(last_tok=torch.from_numpy(start).cuda(), out_tok=torch.full((S, cap), -9, dtype=torch.int32, device="cuda"),
+                 seq_len=torch.zeros(S, dtype=torch.int32, device="cuda"), finished=torch.zeros(S, dtype=torch.uint8, device="cuda"),
+                 stats=torch.zeros(4, dtype=torch.int64, device="cuda"))
+
+    def hidden(tokens, which, h_out):
+        torch.index_select(E[which], 0, tokens.long(), out=h_out)
+
+    rnd = ee.DssdRound(heads[0], heads[1], 1e-5, k, -1, hidden, state)
+    first = {n: v.clone() for n, v in rnd().items()}
+    torch.cuda.synchronize()
+    first_len = state["seq_len"].cpu().numpy().copy()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(rounds - 1):
+        rnd()
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / (rounds - 1)
+    stats = state["stats"].cpu().numpy().tolist()
+    ref_state = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    c0 = time.perf_counter()
+    ref = oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], 1.0, -1, k, start.copy(), *ref_state)
+    cpu_s = time.perf_counter() - c0
+    clean = np.ones(S, bool)
+    for o in ref["steps"]:
+        kp = oracle.decisive_rows(o, 1e-3, 1e-3)
+        clean &= kp["argmax"] & kp["exit_mask"]
+    clean &= oracle.decisive_rows(ref["verify_out"], 1e-3, 1e-3)["argmax"].reshape(S, k + 1).all(axis=1)
+    agree = int((first["accept_len"].cpu().numpy()[clean] == ref["accept_len"][clean]).sum()
+                == clean.sum() and (first_len[clean] == ref_state[1][clean]).all())
+    w_bytes = (k + 1) * 2.0 * V * d                                       # the heads' weights, once per evaluation
+    gbs = w_bytes / (us * 1e-6) / 1e9
+    return dict(S=S, k=k, d=d, V=V, tau=1.0, rounds=rounds, us_per_round=round(us, 1), head_evaluations_per_round=k + 1,
+                tokens_committed_per_round_per_sequence=round(stats[2] / (rounds * S), 3),
+                acceptance_rate=round(stats[1] / max(stats[0], 1), 4), wasted_tokens=stats[0] - stats[1],
+                committed_tokens_per_s=stats[2] / rounds / (us * 1e-6),
+                first_round_matches_oracle_on_decisive_sequences=bool(agree), decisive_sequences=int(clean.sum()),
+                roofline=dict(bound="hbm", algorithmic_bytes=w_bytes, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                              frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None,
+                              note="includes the nine Python callbacks that run the stand-in model"),
+                cpu_baseline=dict(value=float(ref_state[3][2]) / cpu_s, unit="committed tokens/s", seconds=round(cpu_s, 2),
+                                  kind="oracle", cores=oracle_threads(), sample="the first round of the same sequences"))
+
+
 def oracle_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -603,6 +670,7 @@ def main():
         line["configs"] = extra
         line["calibration"] = measure_calibration(peaks, peak_src)
         line["cascade"] = measure_cascade(peaks, peak_src)
+        line["dssd_round"] = measure_dssd_round(peaks, peak_src)
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):

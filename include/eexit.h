@@ -235,6 +235,49 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
                       void* stream);
 
 /*
+ * One whole DSSD round for S sequences (section 4.3.1: drafting phase, verification phase, commit), issued on
+ * the stream without any synchronisation.  The transformer is the caller's: `hidden` is called k times for the
+ * drafting steps (which = 0: n_rows = S tokens, one per sequence, the token each sequence's next position
+ * follows) and once for the verification pass (which = 1: n_rows = S * (k + 1) tokens, row (s, j) = the token
+ * before draft position j, j = k being the bonus position); it must enqueue on `stream` work that writes the
+ * hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING those tokens to h_out, and return 0.
+ * Both pointers it receives are device buffers inside `workspace`.
+ *   drafting step j : draft head (heads' gamma, beta, W; draft_head.tau is the threshold) on the step's hidden
+ *                     states; argmax = drafted token, exit decision = confidence; the token feeds step j + 1
+ *   verification    : verify head (the full model's; its tau is ignored) on all S * (k + 1) rows
+ *   commit          : dssd_commit with kv = k + 1 and the given eos_token; then last_tok[s] = the last token
+ *                     committed, for the sequences that took part
+ * Every sequence goes through all k drafting steps (what lies beyond its stop is ignored by the commit), so
+ * the launch sequence does not depend on device data.  State (device, in/out): last_tok int32 [S], out_tok
+ * int32 [S, capacity], seq_len int32 [S], finished uint8 [S], stats int64 [4]; outputs of the round: draft_len,
+ * accept_len, next_tok int32 [S].  Workspace: dssd_round_workspace_bytes(S, k, d, V), 256-byte aligned,
+ * initialised once with ee_workspace_init.  1 <= k <= 32.
+ */
+typedef int (*ee_hidden_fn)(void* user, const int* tokens, int n_rows, int which, void* h_out, void* stream);
+typedef struct {
+    int S, k, d, V;
+    float ln_eps;
+    int eos_token;
+    ee_head draft_head, verify_head;    /* gamma, beta, W, tau are read; h, ld_h and the outputs are ignored */
+    ee_hidden_fn hidden;
+    void* hidden_user;
+    int* last_tok;
+    int* out_tok;
+    int capacity;
+    int* seq_len;
+    unsigned char* finished;
+    long long* stats;
+    int* draft_len;
+    int* accept_len;
+    int* next_tok;
+    void* workspace;
+    size_t workspace_bytes;
+    void* stream;
+} ee_dssd_round_args;
+size_t    dssd_round_workspace_bytes(int S, int k, int d, int V);     /* host-only, pure; 0 if a size is invalid */
+ee_status dssd_round(const ee_dssd_round_args* args);
+
+/*
  * ee_compact and dssd_accept in one kernel launch, for a decoding step that needs both (section 3.4.2 and
  * section 4.3.1): both read the heads' outputs and write disjoint results, so one launch does the work of two
  * and a step saves a launch boundary.  Arguments, layouts and results are exactly those of the two calls;

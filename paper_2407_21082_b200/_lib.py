@@ -17,6 +17,18 @@ class EEHead(C.Structure):
                 ("tau", C.c_float), ("argmax", _p), ("entropy", _p), ("maxprob", _p), ("exit_mask", _p)]
 
 
+HIDDEN_FN = C.CFUNCTYPE(C.c_int, _p, _p, C.c_int, C.c_int, _p, _p)
+
+
+class EEDssdRoundArgs(C.Structure):
+    """Mirror of `ee_dssd_round_args` in include/eexit.h."""
+    _fields_ = [("S", C.c_int), ("k", C.c_int), ("d", C.c_int), ("V", C.c_int), ("ln_eps", C.c_float), ("eos_token", C.c_int),
+                ("draft_head", EEHead), ("verify_head", EEHead), ("hidden", HIDDEN_FN), ("hidden_user", _p),
+                ("last_tok", _p), ("out_tok", _p), ("capacity", C.c_int), ("seq_len", _p), ("finished", _p), ("stats", _p),
+                ("draft_len", _p), ("accept_len", _p), ("next_tok", _p), ("workspace", _p), ("workspace_bytes", C.c_size_t),
+                ("stream", _p)]
+
+
 PROTOTYPES = {
     "ee_status_string": (C.c_char_p, [C.c_int]),
     "ee_exit_head_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
@@ -39,6 +51,8 @@ PROTOTYPES = {
     "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_commit": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, C.c_int, _p, C.c_int, _p, _p, _p, _p, _p, _p, _p]),
+    "dssd_round_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
+    "dssd_round": (C.c_int, [C.POINTER(EEDssdRoundArgs)]),
     "ee_compact_accept": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p,
                                     _p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_cascade_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),

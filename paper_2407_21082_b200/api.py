@@ -447,6 +447,57 @@ def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos_token, state: dict, 
     return out
 
 
+class DssdRound:
+    """dssd_round (see include/eexit.h) with its argument block built once.
+
+    draft_head / verify_head: dicts with gamma, beta, W (and tau for the draft head).  hidden_fn(tokens, which, h_out)
+    is the caller's model: `tokens` int32 [n_rows] and `h_out` bf16 [n_rows, d] are device tensors (views into the
+    workspace); it must fill h_out on the current stream.  `state`: last_tok, out_tok, seq_len, finished, stats."""
+
+    def __init__(self, draft_head, verify_head, ln_eps, k, eos_token, hidden_fn, state, workspace=None):
+        import ctypes as C
+        S = state["last_tok"].numel()
+        Wd, Wv = _bf16(_dev(draft_head["W"], "W")), _bf16(_dev(verify_head["W"], "W"))
+        V, d = Wd.shape
+        dev = Wd.device
+        if workspace is None:
+            workspace = torch.empty(int(_lib.load().dssd_round_workspace_bytes(S, k, d, V)), dtype=torch.uint8, device=dev)
+            ee_workspace_init(workspace)
+        self.workspace, self.state = workspace, state
+        self.out = {n: torch.empty(S, dtype=torch.int32, device=dev) for n in ("draft_len", "accept_len", "next_tok")}
+        base = workspace.data_ptr()
+
+        def trampoline(user, tokens_ptr, n_rows, which, h_ptr, stream):
+            try:
+                tokens = workspace[tokens_ptr - base:tokens_ptr - base + 4 * n_rows].view(torch.int32)
+                h_out = workspace[h_ptr - base:h_ptr - base + 2 * n_rows * d].view(torch.bfloat16).view(n_rows, d)
+                hidden_fn(tokens, which, h_out)
+                return 0
+            except Exception:                    # an exception must not cross the C boundary
+                import traceback
+                traceback.print_exc()
+                return 1
+
+        self._cb = _lib.HIDDEN_FN(trampoline)
+        a = _lib.EEDssdRoundArgs()
+        a.S, a.k, a.d, a.V, a.ln_eps, a.eos_token = S, int(k), d, V, float(ln_eps), int(eos_token)
+        for dst, src, W in ((a.draft_head, draft_head, Wd), (a.verify_head, verify_head, Wv)):
+            dst.gamma, dst.beta, dst.W, dst.tau = _ptr(src["gamma"]), _ptr(src["beta"]), _ptr(W), float(src.get("tau", 0.0))
+        a.hidden, a.hidden_user = self._cb, None
+        a.last_tok, a.out_tok, a.capacity = _ptr(state["last_tok"]), _ptr(state["out_tok"]), state["out_tok"].shape[1]
+        a.seq_len, a.finished, a.stats = _ptr(state["seq_len"]), _ptr(state["finished"]), _ptr(state["stats"])
+        a.draft_len, a.accept_len, a.next_tok = (_ptr(self.out[n]) for n in ("draft_len", "accept_len", "next_tok"))
+        a.workspace, a.workspace_bytes, a.stream = _ptr(workspace), workspace.numel(), _stream()
+        self._args, self._keep = a, (Wd, Wv, draft_head, verify_head, C)
+
+    def __call__(self):
+        import ctypes as C
+        code = _lib.load().dssd_round(C.byref(self._args))
+        if code:
+            raise EExitError(code, "dssd_round")
+        return self.out
+
+
 def _accept_args(draft_tok, draft_exit_mask, verify_tok, out):
     S, k = draft_tok.shape
     kv = verify_tok.shape[1]

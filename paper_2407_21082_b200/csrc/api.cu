@@ -393,6 +393,37 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
                               draft_len, accept_len, next_tok, stats, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+ee_status round_head_call(const void* h, const ee_head& head, float ln_eps, int M, int d, int V, float tau, int* argmax,
+                          float* entropy, float* maxprob, unsigned char* mask, void* ws, size_t ws_bytes, void* stream) {
+    return ee_exit_head(h, d, head.gamma, head.beta, ln_eps, head.W, M, d, V, nullptr, tau, argmax, entropy, maxprob, mask, ws,
+                        ws_bytes, stream);
+}
+}  // namespace
+
+size_t dssd_round_workspace_bytes(int S, int k, int d, int V) {
+    if (S < 0 || k < 1 || k > 32 || !sizes_ok(S * (k + 1), d, V)) return 0;
+    return dssd_round_layout_bytes(S, k, d, V, workspace_bytes(S * (k + 1), d, V));
+}
+
+ee_status dssd_round(const ee_dssd_round_args* a) {
+    if (!a) return EE_ERR_NULL;
+    if (a->S < 0 || a->k < 1 || a->k > 32 || a->capacity < 1 || !sizes_ok(a->S * (a->k + 1), a->d, a->V)) return EE_ERR_SHAPE;
+    if (a->S == 0) return EE_OK;
+    if (!a->hidden || !a->last_tok || !a->out_tok || !a->seq_len || !a->finished || !a->stats || !a->draft_len ||
+        !a->accept_len || !a->next_tok || !a->workspace)
+        return EE_ERR_NULL;
+    if (!a->draft_head.gamma || !a->draft_head.beta || !a->draft_head.W || !a->verify_head.gamma || !a->verify_head.beta ||
+        !a->verify_head.W)
+        return EE_ERR_NULL;
+    if (!aligned(a->workspace, 256)) return EE_ERR_ALIGN;
+    if (a->workspace_bytes < dssd_round_workspace_bytes(a->S, a->k, a->d, a->V)) return EE_ERR_WORKSPACE;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return dssd_round_run(*a, workspace_bytes(a->S * (a->k + 1), a->d, a->V), round_head_call);
+}
+
 ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     if (!aligned(workspace, 256)) return EE_ERR_ALIGN;

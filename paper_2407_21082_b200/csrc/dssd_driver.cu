@@ -1,0 +1,144 @@
+// One whole DSSD round (paper section 4.3.1) for S sequences, driven from the host without any synchronisation:
+// k drafting steps with the draft head, one verification pass with the full model's head over the k draft
+// positions plus a bonus position, then the commit.  The hidden states come from the caller's model through a
+// callback that is handed device buffers and the stream; everything between the heads (recording the drafted
+// tokens, building the verifier's inputs, the sequences' state) stays on the device.
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ee {
+
+namespace {
+
+// After drafting step j: token and confidence of every sequence go to column j of the draft buffers, and the
+// token becomes the next step's input.
+__global__ void __launch_bounds__(256) record_draft_kernel(const int* __restrict__ argmax,
+                                                           const unsigned char* __restrict__ exit_mask, int S, int j, int k,
+                                                           int* __restrict__ draft_tok, unsigned char* __restrict__ draft_mask,
+                                                           int* __restrict__ cur_tok) {
+    launch_dependents();
+    const int s = blockIdx.x * 256 + threadIdx.x;
+    if (s >= S) return;
+    grid_dependency_wait();
+    const int t = argmax[s];
+    draft_tok[(size_t)s * k + j] = t;
+    draft_mask[(size_t)s * k + j] = exit_mask[s];
+    cur_tok[s] = t;
+}
+
+// The verifier's row (s, j) reads the token before position j: the last committed token for j = 0, the token
+// drafted at j - 1 after that (j = k is the bonus row).
+__global__ void __launch_bounds__(256) verify_inputs_kernel(const int* __restrict__ last_tok,
+                                                            const int* __restrict__ draft_tok, int S, int k,
+                                                            int* __restrict__ prev_all) {
+    launch_dependents();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= S * (k + 1)) return;
+    grid_dependency_wait();
+    const int s = i / (k + 1), j = i - s * (k + 1);
+    prev_all[i] = j == 0 ? last_tok[s] : draft_tok[(size_t)s * k + j - 1];
+}
+
+// Sequences that took part in the round continue from their last committed token.
+__global__ void __launch_bounds__(256) last_token_kernel(const int* __restrict__ out_tok, int cap,
+                                                         const int* __restrict__ seq_len,
+                                                         const unsigned char* __restrict__ was_finished, int S,
+                                                         int* __restrict__ last_tok) {
+    launch_dependents();
+    const int s = blockIdx.x * 256 + threadIdx.x;
+    if (s >= S) return;
+    grid_dependency_wait();
+    if (!was_finished[s] && seq_len[s] > 0) last_tok[s] = out_tok[(size_t)s * cap + seq_len[s] - 1];
+}
+
+__global__ void __launch_bounds__(256) copy_bytes_kernel(const unsigned char* __restrict__ src, int n,
+                                                         unsigned char* __restrict__ dst, const int* __restrict__ src_i,
+                                                         int* __restrict__ dst_i) {
+    launch_dependents();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    grid_dependency_wait();
+    dst[i] = src[i];
+    dst_i[i] = src_i[i];
+}
+
+struct Layout {
+    size_t head_ws, h, outs, draft_tok, draft_mask, prev_all, cur_tok, was_finished, total;
+};
+
+Layout layout(int S, int k, int d, int V, size_t head_ws_bytes) {
+    Layout L;
+    const size_t rows = (size_t)S * (k + 1);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o += align_up(bytes, 256); return at; };
+    L.head_ws = take(head_ws_bytes);
+    L.h = take(rows * d * 2);
+    L.outs = take(4 * align_up(rows * 4, 256));
+    L.draft_tok = take((size_t)S * k * 4);
+    L.draft_mask = take((size_t)S * k);
+    L.prev_all = take(rows * 4);
+    L.cur_tok = take((size_t)S * 4);
+    L.was_finished = take((size_t)S);
+    L.total = o;
+    (void)V;
+    return L;
+}
+
+}  // namespace
+
+size_t dssd_round_layout_bytes(int S, int k, int d, int V, size_t head_ws_bytes) { return layout(S, k, d, V, head_ws_bytes).total; }
+
+ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
+                         ee_status (*head_call)(const void* h, const ee_head& head, float ln_eps, int M, int d, int V, float tau,
+                                                int* argmax, float* entropy, float* maxprob, unsigned char* mask, void* ws,
+                                                size_t ws_bytes, void* stream)) {
+    const int S = a.S, k = a.k, d = a.d, V = a.V;
+    const Layout L = layout(S, k, d, V, head_ws_bytes);
+    unsigned char* ws = static_cast<unsigned char*>(a.workspace);
+    cudaStream_t s = static_cast<cudaStream_t>(a.stream);
+    const size_t rows = (size_t)S * (k + 1);
+    void* h = ws + L.h;
+    const size_t ob = align_up(rows * 4, 256);
+    int* t_argmax = reinterpret_cast<int*>(ws + L.outs);
+    float* t_entropy = reinterpret_cast<float*>(ws + L.outs + ob);
+    float* t_maxprob = reinterpret_cast<float*>(ws + L.outs + 2 * ob);
+    unsigned char* t_mask = ws + L.outs + 3 * ob;
+    int* draft_tok = reinterpret_cast<int*>(ws + L.draft_tok);
+    unsigned char* draft_mask = ws + L.draft_mask;
+    int* prev_all = reinterpret_cast<int*>(ws + L.prev_all);
+    int* cur_tok = reinterpret_cast<int*>(ws + L.cur_tok);
+    unsigned char* was_finished = ws + L.was_finished;
+    const int gs = (S + 255) / 256;
+
+    // the round's inputs: who is still running, and every sequence's last committed token
+    if (launch_pdl(copy_bytes_kernel, gs, 256, 0, s, (const unsigned char*)a.finished, S, was_finished, (const int*)a.last_tok,
+                   cur_tok) != cudaSuccess)
+        return EE_ERR_CUDA;
+    for (int j = 0; j < k; ++j) {
+        if (a.hidden(a.hidden_user, cur_tok, S, 0, h, a.stream) != 0) return EE_ERR_CUDA;
+        ee_status st = head_call(h, a.draft_head, a.ln_eps, S, d, V, a.draft_head.tau, t_argmax, t_entropy, t_maxprob, t_mask,
+                                 ws + L.head_ws, head_ws_bytes, a.stream);
+        if (st != EE_OK) return st;
+        if (launch_pdl(record_draft_kernel, gs, 256, 0, s, (const int*)t_argmax, (const unsigned char*)t_mask, S, j, k, draft_tok,
+                       draft_mask, cur_tok) != cudaSuccess)
+            return EE_ERR_CUDA;
+    }
+    if (launch_pdl(verify_inputs_kernel, (int)((rows + 255) / 256), 256, 0, s, (const int*)a.last_tok, (const int*)draft_tok, S, k,
+                   prev_all) != cudaSuccess)
+        return EE_ERR_CUDA;
+    if (a.hidden(a.hidden_user, prev_all, (int)rows, 1, h, a.stream) != 0) return EE_ERR_CUDA;
+    ee_status st = head_call(h, a.verify_head, a.ln_eps, (int)rows, d, V, HUGE_VALF, t_argmax, t_entropy, t_maxprob, t_mask,
+                             ws + L.head_ws, head_ws_bytes, a.stream);
+    if (st != EE_OK) return st;
+    st = dssd_commit_launch(draft_tok, draft_mask, t_argmax, S, k, k + 1, a.eos_token, a.out_tok, a.capacity, a.seq_len,
+                            a.finished, a.draft_len, a.accept_len, a.next_tok, a.stats, s);
+    if (st != EE_OK) return st;
+    if (launch_pdl(last_token_kernel, gs, 256, 0, s, (const int*)a.out_tok, a.capacity, (const int*)a.seq_len,
+                   (const unsigned char*)was_finished, S, a.last_tok) != cudaSuccess)
+        return EE_ERR_CUDA;
+    return EE_OK;
+}
+
+}  // namespace ee

@@ -86,6 +86,13 @@ ee_status dssd_commit_launch(const int* draft_tok, const unsigned char* draft_ex
                              int kv, int eos, int* out_tok, int cap, int* seq_len, unsigned char* finished, int* draft_len,
                              int* accept_len, int* next_tok, long long* stats, cudaStream_t stream);
 
+// ---- a whole DSSD round driven from the host (drafting steps, verification pass, commit) ----
+size_t dssd_round_layout_bytes(int S, int k, int d, int V, size_t head_ws_bytes);
+ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
+                         ee_status (*head_call)(const void* h, const ee_head& head, float ln_eps, int M, int d, int V, float tau,
+                                                int* argmax, float* entropy, float* maxprob, unsigned char* mask, void* ws,
+                                                size_t ws_bytes, void* stream));
+
 // ---- diagnostic: a bounded wait that is made to give up ----
 ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
 

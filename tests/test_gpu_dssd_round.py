@@ -43,3 +43,58 @@ def test_argument_errors(ee):
     with pytest.raises(ee.EExitError) as e:
         ee.dssd_commit(t, None, t, 0, state)                         # k = 40 > 32
     assert e.value.code == 2
+
+
+def _model(seed, V, d):
+    cfg = gen.make_config("c1", seed=seed, planted=True, M=4, d=d, V=V, heads=2)
+    planting = gen.make_planting(seed, f"c1/planted/d{d}/V{V}", d, V)
+    return cfg, gen.make_markov_model(seed, V, d, planting, sigma=0.4)
+
+
+@pytest.mark.parametrize("S,k,V,d,tau,eos", [(12, 4, 400, 64, 1.0, -1), (40, 8, 1000, 128, 0.7, 5), (3, 1, 300, 64, 5.0, -1),
+                                              (70, 6, 640, 256, 1.5, 17)])
+def test_whole_rounds_match_oracle(ee, S, k, V, d, tau, eos):
+    """Drafting steps, verification pass and commit, several rounds in a row, against the oracle's round.  A
+    sequence drops out of the comparison from the round in which one of its decisions falls inside the tolerance
+    band (near-tied argmax, |H - tau| < 1e-3), because everything it does afterwards may legitimately differ."""
+    from _util import GAP_MIN, MARGIN_MIN, dev_bf16, head_to_dev
+    cfg, mm = _model(S + k, V, d)
+    if eos >= 0:
+        eos = int(gen.make_planting(S + k, f"c1/planted/d{d}/V{V}", d, V)["tokens"][eos % 64])   # a token the chain can reach
+    cap = 3 * (k + 1) + 2
+    start = (np.arange(S, dtype=np.int32) * 13) % V
+    ref_state = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    ref_last = start.copy()
+    state = dict(last_tok=dev(start), out_tok=dev(ref_state[0]), seq_len=dev(ref_state[1]), finished=dev(ref_state[2]),
+                 stats=dev(ref_state[3]))
+    E = [dev_bf16(mm["E_draft"]), dev_bf16(mm["E_verify"])]
+    calls = []
+
+    def hidden(tokens, which, h_out):
+        calls.append((which, tokens.numel()))
+        torch.index_select(E[which], 0, tokens.long(), out=h_out)
+
+    hd, hv = head_to_dev(cfg["heads"][0]), head_to_dev(cfg["heads"][1])
+    rnd = ee.DssdRound(dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=tau), dict(gamma=hv["gamma"], beta=hv["beta"], W=hv["W"]),
+                       1e-5, k, eos, hidden, state)
+    clean = np.ones(S, bool)
+    for r in range(4):
+        ref = oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], tau, eos, k, ref_last, *ref_state)
+        for o in ref["steps"]:
+            keep = oracle.decisive_rows(o, GAP_MIN, MARGIN_MIN)
+            clean &= keep["argmax"] & keep["exit_mask"]
+        clean &= oracle.decisive_rows(ref["verify_out"], GAP_MIN, MARGIN_MIN)["argmax"].reshape(S, k + 1).all(axis=1)
+        got = rnd()
+        torch.cuda.synchronize()
+        assert ee.ee_query_async_error(rnd.workspace) == 0
+        for key in ("draft_len", "accept_len", "next_tok"):
+            assert np.array_equal(got[key].cpu().numpy()[clean], ref[key][clean]), (r, key)
+        assert np.array_equal(state["out_tok"].cpu().numpy()[clean], ref_state[0][clean]), r
+        assert np.array_equal(state["seq_len"].cpu().numpy()[clean], ref_state[1][clean]), r
+        assert np.array_equal(state["finished"].cpu().numpy()[clean], ref_state[2][clean]), r
+        assert np.array_equal(state["last_tok"].cpu().numpy()[clean], ref_last[clean]), r
+        if clean.all():
+            assert state["stats"].cpu().numpy().tolist() == ref_state[3].tolist(), r
+    assert calls[:k + 1] == [(0, S)] * k + [(1, S * (k + 1))] and len(calls) == 4 * (k + 1)
+    assert clean.sum() >= S // 2                        # the case is not dominated by near-ties
+    assert ref_state[1].sum() > 4 * S or tau < 0        # speculation committed more than one token per round somewhere
