@@ -249,7 +249,9 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
     return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"],
                 head_call_us=1e3 * heads_ms / (steps * n_heads),
                 head_call_us_inner_events=1e3 * inner_ms / (n_inner * n_heads),
-                tail_us=1e3 * (t0.elapsed_time(t1) - heads_ms) / steps, clocks=clocks)
+                # step time minus head time; for millisecond-long steps the second region can run slower than the
+                # first (power cap), which would make the difference negative: reported as 0 then
+                tail_us=max(0.0, 1e3 * (t0.elapsed_time(t1) - heads_ms) / steps), clocks=clocks)
 
 
 # DRAM bytes (read + write) one launch of the dominant kernel moved in the ncu captures summarised under
