@@ -80,20 +80,25 @@ def logits(y: np.ndarray, W_bits: np.ndarray) -> np.ndarray:
 
 
 def softmax_stats(z: np.ndarray) -> dict:
-    """A3.  Entropy (nats), max probability, argmax (lowest index), and the top-2 logit gap."""
+    """A3.  Entropy (nats), max probability, argmax (lowest index), the top-2 logit gap, and the difference
+    between the two largest probabilities (the third confidence metric of section 3.4.1, "breaking ties")."""
     m = z.max(axis=1, keepdims=True)
     argmax = np.argmax(z, axis=1).astype(np.int32)           # numpy returns the first maximum
     zc = z - m
     e = np.exp(zc)
     s = e.sum(axis=1)
     t = (e * zc).sum(axis=1)
+    p = e / s[:, None]
     if z.shape[1] > 1:
         top2 = np.partition(z, -2, axis=1)[:, -2:]
         gap = top2[:, 1] - top2[:, 0]
+        top2p = np.partition(p, -2, axis=1)[:, -2:]          # the two largest probabilities (equal maxima count twice)
+        prob_gap = top2p[:, 1] - top2p[:, 0]
     else:
         gap = np.full(z.shape[0], np.inf)
+        prob_gap = p[:, 0].copy()                            # a single class: nothing to subtract
     return dict(argmax=argmax, entropy=np.log(s) - t / s, maxprob=1.0 / s, logZ=m[:, 0] + np.log(s),
-                top2_gap=gap)
+                top2_gap=gap, top2_prob_gap=prob_gap)
 
 
 def exit_decision(entropy: np.ndarray, tau) -> np.ndarray:
@@ -106,7 +111,7 @@ def exit_head(h_bits, gamma, beta, ln_eps, W_bits, tau, rows_per_block: int = 64
     """A1-A4 over all rows.  tau is a scalar or an array [M] (nats)."""
     M = h_bits.shape[0]
     Wd = bf16_decode(W_bits).T.copy()        # [d, V] fp64, decoded once
-    keys = ("argmax", "entropy", "maxprob", "logZ", "top2_gap")
+    keys = ("argmax", "entropy", "maxprob", "logZ", "top2_gap", "top2_prob_gap")
     parts = {k: [] for k in keys}
     for r0 in range(0, M, rows_per_block):
         y = layer_norm(h_bits[r0:r0 + rows_per_block], gamma, beta, ln_eps, round_to_bf16)

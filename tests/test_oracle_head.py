@@ -199,3 +199,30 @@ def test_decisive_rows_lists_near_ties():
     ref = dict(top2_gap=np.array([0.5, 5e-4, 1e-3]), tau_margin=np.array([2e-4, 0.3, 1e-3]))
     keep = oracle.decisive_rows(ref)
     assert keep["argmax"].tolist() == [True, False, True] and keep["exit_mask"].tolist() == [False, True, True]
+
+
+def test_top2_probability_gap_closed_forms_and_brute_force():
+    """Section 3.4.1's third metric: p(1st) - p(2nd)."""
+    import math
+    V = 1000
+    st = oracle.softmax_stats(np.zeros((1, V)))
+    assert st["top2_prob_gap"][0] == 0.0                                        # uniform: no gap
+    a = 3.0
+    z = np.zeros((1, V)); z[0, 17] = a
+    want = (math.exp(a) - 1.0) / (math.exp(a) + V - 1)                          # one raised logit
+    assert abs(oracle.softmax_stats(z)["top2_prob_gap"][0] - want) < 1e-15
+    z[0, 400] = a                                                                # two equal maxima: gap 0
+    assert oracle.softmax_stats(z)["top2_prob_gap"][0] == 0.0
+    z[0, 400] = a - 1.0
+    want = (math.exp(a) - math.exp(a - 1.0)) / (math.exp(a) + math.exp(a - 1.0) + V - 2)
+    assert abs(oracle.softmax_stats(z)["top2_prob_gap"][0] - want) < 1e-15
+    assert oracle.softmax_stats(np.array([[2.5]]))["top2_prob_gap"][0] == 1.0   # a single class
+    rng = np.random.default_rng(5)
+    z = rng.normal(0, 2, size=(7, 50))
+    got = oracle.softmax_stats(z)
+    for i in range(7):
+        p = sorted((math.exp(x - z[i].max()) for x in z[i]), reverse=True)
+        tot = math.fsum(p)
+        assert abs(got["top2_prob_gap"][i] - (p[0] - p[1]) / tot) < 1e-14
+        assert 0.0 <= got["top2_prob_gap"][i] <= got["maxprob"][i]
+    assert np.all(np.diff(np.sort(z, axis=1)[:, -2:], axis=1)[:, 0] == got["top2_gap"])
