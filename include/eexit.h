@@ -90,6 +90,17 @@ ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const 
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * ee_exit_head with the third confidence metric of section 3.4.1 as well: top2gap fp32 [M] = the difference
+ * between the two largest probabilities of each row's distribution ("breaking ties"; 0 when the maximum is
+ * attained twice, p itself when V = 1).  Everything else as in ee_exit_head (same workspace size); the
+ * tensor-core path is used for every size.
+ */
+ee_status ee_exit_head_top2(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau,
+                            int* argmax, float* entropy, float* maxprob, float* top2gap, unsigned char* exit_mask,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Several heads on batches of the same shape in one call -- what the calibration pass of section 3.4.1 does
  * (every head is evaluated on every token of the calibration set) and what a verify step with several
  * heads does.  Equivalent to n_heads calls of ee_exit_head with the same M, d, V, ln_eps and workspace; up to

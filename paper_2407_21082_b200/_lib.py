@@ -36,6 +36,8 @@ PROTOTYPES = {
     "ee_workspace_init": (C.c_int, [_p, C.c_size_t, _p]),
     "ee_exit_head": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                _p, _p, _p, _p, _p, C.c_size_t, _p]),
+    "ee_exit_head_top2": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
+                                    _p, _p, _p, _p, _p, _p, C.c_size_t, _p]),
     "ee_exit_head_multi_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "ee_exit_head_multi_launches": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "ee_exit_head_multi": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, _p, C.c_size_t, _p]),

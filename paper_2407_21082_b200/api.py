@@ -181,6 +181,24 @@ class PreparedMulti:
         return self.out
 
 
+def ee_exit_head_top2(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None) -> dict:
+    """ee_exit_head plus out["top2gap"]: the difference between the two largest probabilities of every row."""
+    h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
+    M, d = h.shape
+    V = W.shape[0]
+    if out is None:
+        out = new_outputs(M, h.device)
+        out["top2gap"] = torch.empty(M, dtype=torch.float32, device=h.device)
+    if workspace is None:
+        workspace = new_workspace(M, d, V, h.device)
+    tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
+    _check(_lib.load().ee_exit_head_top2(
+        _ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W), M, d, V,
+        _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]), _ptr(out["top2gap"]),
+        _ptr(out["exit_mask"]), _ptr(workspace), workspace.numel(), _stream()), "ee_exit_head_top2")
+    return out
+
+
 def ee_exit_head_results_bytes(n_heads: int, M: int) -> int:
     return int(_lib.load().ee_exit_head_results_bytes(n_heads, M))
 

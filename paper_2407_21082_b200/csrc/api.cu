@@ -126,6 +126,28 @@ ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, c
     return gemm_launch(&a, 1);
 }
 
+ee_status ee_exit_head_top2(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
+                            const void* W, int M, int d, int V, const float* tau_per_row, float tau, int* argmax,
+                            float* entropy, float* maxprob, float* top2gap, unsigned char* exit_mask, void* workspace,
+                            size_t workspace_bytes_, void* stream) {
+    if (!sizes_ok(M, d, V)) return EE_ERR_SHAPE;
+    if (M == 0) return EE_OK;
+    if (!h || !gamma || !beta || !W || !argmax || !entropy || !maxprob || !top2gap || !exit_mask || !workspace) return EE_ERR_NULL;
+    if (ld_h < d || (ld_h % 8) != 0) return EE_ERR_SHAPE;
+    if (!aligned(h, 16) || !aligned(W, 16) || !aligned(gamma, 16) || !aligned(beta, 16) || !aligned(workspace, 256))
+        return EE_ERR_ALIGN;
+    if (workspace_bytes_ < workspace_bytes(M, d, V)) return EE_ERR_WORKSPACE;
+    HeadArgs a{};
+    const ee_status dev = current_device(&a.device, &a.num_sms);
+    if (dev != EE_OK) return dev;
+    a.h = h; a.ld_h = ld_h; a.gamma = gamma; a.beta = beta; a.ln_eps = ln_eps; a.W = W;
+    a.M = M; a.d = d; a.V = V; a.tau_per_row = tau_per_row; a.tau = tau;
+    a.argmax = argmax; a.entropy = entropy; a.maxprob = maxprob; a.exit_mask = exit_mask; a.top2gap = top2gap;
+    a.workspace = workspace; a.workspace_bytes = workspace_bytes_;
+    a.stream = static_cast<cudaStream_t>(stream);
+    return gemm_launch(&a, 1);
+}
+
 size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1) return 0;
     size_t need = workspace_bytes(M, d, V);

@@ -26,7 +26,8 @@ constexpr int kGemmThreads = 320;           // producer warp, MMA warp, eight ep
 constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile order
 constexpr int kATileBytes = BM * BK * 2;    // 16 KB
 
-constexpr int kBarBytes = 512 + 2048;          // barriers and flags (512 B), then 128 states exchanged between epilogue warps
+constexpr int kBarBytes = 512 + 2048 + 1024;   // barriers and flags (512 B), then 128 states and 128 (max, second) pairs
+                                               // exchanged between epilogue warps
 constexpr int kGemmMaxHeads = kGemmLaunchMaxHeads;
 constexpr int kMaxGemmStages = 12;
 constexpr size_t kGemmSmemBudget = 226 * 1024;
@@ -55,24 +56,49 @@ struct MergeHeads {
     float* entropy[kGemmMaxHeads];
     float* maxprob[kGemmMaxHeads];
     unsigned char* exit_mask[kGemmMaxHeads];
+    float* top2gap[kGemmMaxHeads];           // NULL unless the caller asked for the top-2 probability gap
 };
+
+// Largest and second-largest value of a multiset kept as a pair (equal maxima count twice).
+__device__ __forceinline__ void top2_merge(float& m1, float& m2, float o1, float o2) {
+    m2 = fmaxf(fmaxf(m2, o2), fminf(m1, o1));
+    m1 = fmaxf(m1, o1);
+}
 
 // One warp: merge of the n_tiles partial states of one row (lane-strided, twelve independent loads at a
 // time -- one round trip for up to 384 tiles -- then the lanes reduce) and the final decision for that row.
-__device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ partials, int n_tiles, int head, int row,
-                                                     const MergeHeads& hs, int lane) {
+// `second` (NULL if not asked for) holds each tile's second-largest logit for this row: with the tiles' maxima
+// it gives the row's second-largest logit z2 and the gap of the two largest probabilities (1 - e^(z2 - m)) / s.
+__device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ partials, const float* __restrict__ second,
+                                                     int n_tiles, int head, int row, const MergeHeads& hs, int lane) {
     constexpr int kBatch = 12;
     State v[kBatch + 1];
     v[kBatch] = state_empty();                                    // running result of this lane
+    float t1 = -CUDART_INF_F, t2 = -CUDART_INF_F;
     for (int n0 = lane; n0 < n_tiles; n0 += 32 * kBatch) {
 #pragma unroll
         for (int i = 0; i < kBatch; ++i) {
             const int n = n0 + 32 * i;
             v[i] = n < n_tiles ? state_load_cg(partials + n) : state_empty();
         }
+        if (second) {
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int n = n0 + 32 * i;
+                if (n < n_tiles) top2_merge(t1, t2, v[i].m, __ldcg(second + n));
+            }
+        }
         v[kBatch] = state_combine<kBatch + 1>(v);
     }
     const State a = state_reduce_lanes<1, 16>(v[kBatch]);
+    if (second) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float o1 = __shfl_xor_sync(0xffffffffu, t1, o), o2 = __shfl_xor_sync(0xffffffffu, t2, o);
+            top2_merge(t1, t2, o1, o2);
+        }
+        if (lane == 0) hs.top2gap[head][row] = (1.f - expf(t2 - t1)) / a.s;
+    }
     if (lane == 0)
         state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
                      hs.maxprob[head], hs.exit_mask[head], row);
@@ -83,6 +109,7 @@ struct GemmParams {
     int m_tiles, n_tiles, k_blocks;
     int n_heads;
     State* partials;       // [head][M][n_tiles]
+    float* second;         // [head][M][n_tiles]: each tile's second-largest logit, or NULL if nobody asked
     Control* ctrl;
     int bn;                // tile width (vocabulary rows per tile), a multiple of 16, <= 256
     int n_stages;          // smem ring depth
@@ -143,7 +170,29 @@ __device__ __forceinline__ void fold_chunk(State& st, const float (&v)[32], int 
     st.t = fmaf(t2, kLn2, st.t);
 }
 
-template <int BN_T>
+// Largest and second-largest of 32 consecutive logits of one row (the first `nvalid` real); equal maxima count twice.
+template <bool kFull>
+__device__ __forceinline__ void chunk_top2(const float (&v)[32], int nvalid, float& c1, float& c2) {
+    c1 = v[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j)
+        if (kFull || j < nvalid) c1 = fmaxf(c1, v[j]);
+    int dup = 0;
+    c2 = -CUDART_INF_F;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (kFull || j < nvalid) {
+            const bool eq = v[j] == c1;
+            dup += eq ? 1 : 0;
+            c2 = fmaxf(c2, eq ? -CUDART_INF_F : v[j]);
+        }
+    }
+    if (dup > 1) c2 = c1;
+}
+
+// kTop2: also track the second-largest logit (for the top-2 probability gap); a separate instantiation, so
+// that the default kernel carries none of its registers or branches.
+template <int BN_T, bool kTop2>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p) {
     using C = Cfg<BN_T>;
@@ -322,6 +371,8 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
         constexpr bool kSplit = BN_T == 0;
         const int half = (warp - 2) >> 2;
         State* xchg = reinterpret_cast<State*>(bar_mem + 512) + quarter * 32 + lane;
+        float2* xchg2 = reinterpret_cast<float2*>(bar_mem + 512 + 2048) + quarter * 32 + lane;
+        constexpr bool want_top2 = kTop2;
         // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in the first 16 lanes of
         // quarter q, the other 16 lanes hold nothing.
         const int row_in_tile = mma_m == 64 ? (lane < 16 ? quarter * 16 + lane : BM) : quarter * 32 + lane;
@@ -342,6 +393,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             const int ncols = min(BN, p.V - n0);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kAccStride);
             State st = state_empty();
+            float z1 = -CUDART_INF_F, z2 = -CUDART_INF_F;     // largest and second-largest logit seen (only if asked for)
             const int row = m_tile * BM + row_in_tile;
             const bool live = row < p.M;                  // padding rows are neither read nor folded
             if (__any_sync(0xffffffffu, live)) {
@@ -353,6 +405,12 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     if (live) {
                         if (nvalid >= 32) fold_chunk<true>(st, v, n0 + c * 32, 32);
                         else fold_chunk<false>(st, v, n0 + c * 32, nvalid);
+                        if constexpr (want_top2) {
+                            float c1, c2;
+                            if (nvalid >= 32) chunk_top2<true>(v, 32, c1, c2);
+                            else chunk_top2<false>(v, nvalid, c1, c2);
+                            top2_merge(z1, z2, c1, c2);
+                        }
                     }
                 }
             }
@@ -361,7 +419,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
             const uint32_t x_phase = (uint32_t)local & 1u;
             if (!kSplit) {
-                if (live) p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                if (live) {
+                    p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                    if constexpr (want_top2) p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
+                }
             } else if (half == 1) {
                 // the slot is free once the partner has read the state of the tile before
                 const bool free_ = local == 0 || ptx::mbar_wait(xfree_bar(quarter), x_phase ^ 1u, abort_flag);
@@ -370,6 +431,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     break;
                 }
                 *xchg = st;
+                if constexpr (want_top2) *xchg2 = make_float2(z1, z2);
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(xfull_bar(quarter));
             } else {
@@ -379,11 +441,17 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     break;
                 }
                 const State other = *xchg;
+                float2 other2 = make_float2(0.f, 0.f);
+                if constexpr (want_top2) other2 = *xchg2;
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(xfree_bar(quarter));
                 if (live) {
                     state_merge(st, other);
                     p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                    if constexpr (want_top2) {
+                        top2_merge(z1, z2, other2.x, other2.y);
+                        p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
+                    }
                 }
             }
         }
@@ -416,7 +484,8 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     int mine = 0;
                     for (int r = first; r < total_rows; r += (int)gridDim.x * 8, ++mine) {
                         const int head = r / p.M, row = r - head * p.M;
-                        merge_row_and_decide(p.partials + (size_t)r * p.n_tiles, p.n_tiles, head, row, p.mg, lane);
+                        merge_row_and_decide(p.partials + (size_t)r * p.n_tiles,
+                                             kTop2 ? p.second + (size_t)r * p.n_tiles : nullptr, p.n_tiles, head, row, p.mg, lane);
                     }
                     if (lane == 0) {
                         const unsigned int old = atomicAdd(&p.ctrl->merge_seen, (unsigned int)mine);
@@ -563,7 +632,8 @@ __global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloa
 // Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
 // blockIdx.y = head.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials_all, int n_tiles, int M,
+__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials_all,
+                                                         const float* __restrict__ second_all, int n_tiles, int M,
                                                          const __grid_constant__ MergeHeads hs) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -572,7 +642,8 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
     if (row >= M) return;
     const State* partials = partials_all + ((size_t)head * M + row) * n_tiles;
     grid_dependency_wait();                              // the partial states come from the GEMM kernel
-    merge_row_and_decide(partials, n_tiles, head, row, hs, lane);
+    merge_row_and_decide(partials, second_all ? second_all + ((size_t)head * M + row) * n_tiles : nullptr, n_tiles, head, row,
+                         hs, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -588,23 +659,24 @@ int stages_for(int bn, int mma_m) {
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
 
-template <int BN_T>
+template <int BN_T, bool kTop2>
 ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int device, cudaStream_t stream) {
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
-        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T, kTop2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kGemmSmemBudget) != cudaSuccess)
             return EE_ERR_CUDA;
         configured[device] = true;
     }
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
                              : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
-    return launch_pdl(exit_head_gemm_kernel<BN_T>, grid, kGemmThreads, smem, stream, maps, p) == cudaSuccess
+    return launch_pdl(exit_head_gemm_kernel<BN_T, kTop2>, grid, kGemmThreads, smem, stream, maps, p) == cudaSuccess
                ? EE_OK
                : EE_ERR_CUDA;
 }
 
 // Upper bound on the partial states of M rows of one head whatever tile width the launch picks.
+size_t second_bytes(int M, int V);
 size_t partials_bytes(int M, int V) {
     const int bn = M > 1024 ? 256 : kMinTileN;
     return align_up((size_t)M * ((V + bn - 1) / bn) * sizeof(State), 256);
@@ -615,6 +687,9 @@ size_t partials_bytes(int M, int V) {
 // faster than a tile it has to fill with zeros itself, and no tile holds another head's rows.
 size_t y_rows(int M, int n_heads) { return (size_t)n_heads * (size_t)((M + BM - 1) / BM) * BM; }
 size_t y_bytes(int M, int d, int n_heads) { return align_up(y_rows(M, n_heads) * d * sizeof(__nv_bfloat16), 256); }
+
+// One float per partial state (the tile's second-largest logit), used when the top-2 probability gap is asked for.
+size_t second_bytes(int M, int V) { return align_up(partials_bytes(M, V) / 4, 256); }
 
 }  // namespace
 
@@ -642,7 +717,7 @@ int gemm_tile_n(int M, int V, int n_heads, int num_sms) {
 int gemm_launches(int M, int n_heads) { return n_heads * M <= kFusedMergeMaxRows ? 2 : 3; }
 
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
-    return (size_t)n_heads * partials_bytes(M, V) + y_bytes(M, d, n_heads);
+    return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads);
 }
 
 ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
@@ -650,7 +725,9 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     const HeadArgs& a = heads[0];
     unsigned char* ws = static_cast<unsigned char*>(a.workspace);
     State* partials = reinterpret_cast<State*>(ws + kCtrlBytes);
-    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + (size_t)n_heads * partials_bytes(a.M, a.V));
+    float* second = reinterpret_cast<float*>(ws + kCtrlBytes + (size_t)n_heads * partials_bytes(a.M, a.V));
+    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes +
+                                                        (size_t)n_heads * (partials_bytes(a.M, a.V) + second_bytes(a.M, a.V)));
     const int bn = gemm_tile_n(a.M, a.V, n_heads, a.num_sms);
 
     LnHeads ln = {};
@@ -666,6 +743,7 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         mg.entropy[k] = heads[k].entropy;
         mg.maxprob[k] = heads[k].maxprob;
         mg.exit_mask[k] = heads[k].exit_mask;
+        mg.top2gap[k] = heads[k].top2gap;
     }
     const dim3 row_grid((a.M + 7) / 8, n_heads);
     const dim3 ln_grid((a.M + BM - 1) / BM * (BM / 8), n_heads);
@@ -698,6 +776,11 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.k_blocks = (a.d + BK - 1) / BK;
     p.n_heads = n_heads;
     p.partials = partials;
+    p.second = nullptr;
+    for (int k = 0; k < n_heads; ++k)
+        if (heads[k].top2gap) p.second = second;
+    for (int k = 0; k < n_heads; ++k)
+        if (p.second && !heads[k].top2gap) return EE_ERR_NULL;        // all heads of a launch or none
     p.ctrl = reinterpret_cast<Control*>(ws);
     p.bn = bn;
     p.mma_m = mma_m;
@@ -706,12 +789,15 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.n_stages = stages_for(bn, mma_m);
     const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
     const int grid = (int)(total < a.num_sms ? total : a.num_sms);
-    const ee_status st = (a.M > 1024) ? launch_gemm<256>(maps, p, grid, a.device, a.stream)
-                                      : launch_gemm<0>(maps, p, grid, a.device, a.stream);
+    const ee_status st = (a.M > 1024) ? (p.second ? launch_gemm<256, true>(maps, p, grid, a.device, a.stream)
+                                                  : launch_gemm<256, false>(maps, p, grid, a.device, a.stream))
+                                      : (p.second ? launch_gemm<0, true>(maps, p, grid, a.device, a.stream)
+                                                  : launch_gemm<0, false>(maps, p, grid, a.device, a.stream));
     if (st != EE_OK) return st;
     if (p.fused_merge) return EE_OK;
 
-    err = launch_pdl(merge_rows_kernel, row_grid, 256, 0, a.stream, (const State*)partials, p.n_tiles, a.M, mg);
+    err = launch_pdl(merge_rows_kernel, row_grid, 256, 0, a.stream, (const State*)partials, (const float*)p.second, p.n_tiles,
+                     a.M, mg);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
 }
 

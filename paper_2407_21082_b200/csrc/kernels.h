@@ -35,6 +35,8 @@ struct HeadArgs {
     // earlier kernels have finished.
     const int* row_idx;
     const int* m_dev;
+    // Optional (tensor-core path): fp32 [M], the difference between the two largest probabilities of each row.
+    float* top2gap;
 };
 
 // ---- streaming kernel (fused LayerNorm + split-V mma.sync GEMV + last-CTA merge; up to four heads per launch) ----

@@ -274,3 +274,32 @@ def test_multi_head_host_call_matches_oracle(ee):
             for key in out[k]:
                 assert torch.equal(out[k][key], call.out_dev[k][key].cpu()), (k, key)
     assert ee.ee_query_async_error(ws) == 0
+
+
+@pytest.mark.parametrize("M,d,V", [(1, 64, 1), (5, 72, 257), (64, 128, 400), (130, 256, 2049), (600, 64, 300), (1100, 64, 520),
+                                   (8, 512, 50304)])
+def test_top2_probability_gap_matches_oracle(ee, M, d, V):
+    """The third confidence metric, p(1st) - p(2nd), from the tensor-core path; the other outputs unchanged."""
+    for planted in (False, True):
+        cfg = gen.make_config("c0", seed=21, planted=planted, M=M, d=d, V=V)
+        hd = head_to_dev(cfg["heads"][0])
+        h = dev_bf16(cfg["h"])
+        out = ee.ee_exit_head_top2(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0)
+        plain = ee.ee_exit_head(h, hd["gamma"], hd["beta"], 1e-5, hd["W"], 1.0, path=ee.EE_PATH_TCGEN05)
+        torch.cuda.synchronize()
+        ref = oracle_head(cfg["h"], cfg["heads"][0], 1.0)
+        assert_head_matches({k: out[k] for k in plain}, ref, label=f"top2 M={M} V={V} planted={planted}")
+        for k in plain:
+            assert torch.equal(out[k], plain[k]), k
+        got = out["top2gap"].cpu().numpy().astype(np.float64)
+        assert np.abs(got - ref["top2_prob_gap"]).max() <= 2e-3, np.abs(got - ref["top2_prob_gap"]).max()
+        assert np.all(got >= -1e-6) and np.all(got <= out["maxprob"].cpu().numpy() + 1e-6)
+
+
+def test_top2_gap_is_zero_when_the_maximum_is_attained_twice(ee):
+    d, V, M = 64, 300, 3
+    x = np.tile([1.0, -1.0], d // 2)[None, :].repeat(M, 0)
+    Wv = np.zeros((V, d)); Wv[7, 0] = 1.0; Wv[250, 0] = 1.0; Wv[100, 0] = 0.5          # tokens 7 and 250 tie, in different tiles
+    out = ee.ee_exit_head_top2(dev_bf16(gen.bf16_bits_from_f32(x.astype(np.float32))), dev(np.ones(d, np.float32)),
+                               dev(np.zeros(d, np.float32)), 1e-5, dev_bf16(gen.bf16_bits_from_f32(Wv.astype(np.float32))), 1.0)
+    assert torch.all(out["top2gap"] == 0) and out["argmax"].cpu().tolist() == [7, 7, 7]
