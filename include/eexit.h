@@ -320,6 +320,24 @@ ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int
                      void* stream);
 
 /*
+ * Forward pass of a head's self-supervised training objective (section 3.3, paragraph "Losses":
+ * L_KL(y_hat || f_theta) with y_hat the head's distribution and f_theta the main model's).  For each of M tokens
+ * the head's logits come from its hidden states (h_head, LayerNorm gamma_head / beta_head, W_head) and the
+ * teacher's from the final hidden states and the main model's head, both exactly as in ee_exit_head; neither
+ * M x V logit matrix is ever stored.
+ *   kl   fp32 [M]: sum_v p_head(v) (log p_head(v) - log p_teacher(v)), nats
+ *   loss fp32 [1]: their mean (summed in a fixed order: bit-identical from run to run); may be NULL
+ * h_* bf16 [M, d] (row strides ld_* elements), gamma_*, beta_* fp32 [d], W_* bf16 [V, d]; alignment as in
+ * ee_exit_head.  Workspace: ee_head_kl_workspace_bytes(M, d, V), 256-byte aligned, initialised once with
+ * ee_workspace_init.  M = 0 is a no-op.
+ */
+size_t    ee_head_kl_workspace_bytes(int M, int d, int V);      /* host-only, pure; 0 if a size is invalid */
+ee_status ee_head_kl(const void* h_head, long long ld_head, const float* gamma_head, const float* beta_head,
+                     const void* W_head, const void* h_teacher, long long ld_teacher, const float* gamma_teacher,
+                     const float* beta_teacher, const void* W_teacher, float ln_eps, int M, int d, int V,
+                     float* kl, float* loss, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Calibration of one head's threshold from a calibration set (section 3.4.1, "Calibration of Confidence
  * Thresholds": Eq. 3 and the two equations that define the index j-hat and tau_k = c_{k, j-hat}), with the
  * entropy as the confidence metric.  Over n calibration tokens:

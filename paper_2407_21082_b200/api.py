@@ -368,6 +368,42 @@ def ee_calibrate_workspace_bytes(n: int) -> int:
     return int(_lib.load().ee_calibrate_workspace_bytes(int(n)))
 
 
+def _head_kl_args(head, teacher, ln_eps, out, workspace):
+    hh, Wh = _bf16(_dev(head["h"], "h")), _bf16(_dev(head["W"], "W"))
+    ht, Wt = _bf16(_dev(teacher["h"], "h")), _bf16(_dev(teacher["W"], "W"))
+    M, d = hh.shape
+    V = Wh.shape[0]
+    if ht.shape != (M, d) or Wt.shape != (V, d) or not (Wh.is_contiguous() and Wt.is_contiguous()):
+        raise ValueError("head and teacher must share M, d, V; W contiguous [V, d]")
+    dev = hh.device
+    if out is None:
+        out = dict(kl=torch.empty(M, dtype=torch.float32, device=dev), loss=torch.empty(1, dtype=torch.float32, device=dev))
+    if workspace is None:
+        workspace = torch.empty(int(_lib.load().ee_head_kl_workspace_bytes(M, d, V)), dtype=torch.uint8, device=dev)
+        ee_workspace_init(workspace)
+
+    def ld(h):
+        return h.stride(0) if M > 1 else max(h.stride(0), d)
+
+    args = (_ptr(hh), ld(hh), _ptr(head["gamma"]), _ptr(head["beta"]), _ptr(Wh), _ptr(ht), ld(ht), _ptr(teacher["gamma"]),
+            _ptr(teacher["beta"]), _ptr(Wt), float(ln_eps), M, d, V, _ptr(out["kl"]), _ptr(out.get("loss")), _ptr(workspace),
+            workspace.numel(), _stream())
+    return args, out, (hh, Wh, ht, Wt, head, teacher, workspace, out)
+
+
+def ee_head_kl(head, teacher, ln_eps, *, out=None, workspace=None) -> dict:
+    """KL divergence of a head's distribution from the teacher's, per token and mean (see include/eexit.h).
+    head / teacher: dicts with h, gamma, beta, W."""
+    args, out, _ = _head_kl_args(head, teacher, ln_eps, out, workspace)
+    _check(_lib.load().ee_head_kl(*args), "ee_head_kl")
+    return out
+
+
+def prepare_head_kl(head, teacher, ln_eps, *, out=None, workspace=None) -> PreparedCall:
+    args, out, keep = _head_kl_args(head, teacher, ln_eps, out, workspace)
+    return PreparedCall(_lib.load().ee_head_kl, args, "ee_head_kl", keep, out)
+
+
 def ee_selftest_wait_timeout(workspace) -> None:
     """Makes one bounded device-side wait give up (see include/eexit.h); ee_query_async_error then reports it."""
     _check(_lib.load().ee_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream()), "ee_selftest_wait_timeout")

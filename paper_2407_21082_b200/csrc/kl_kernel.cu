@@ -1,0 +1,533 @@
+// Forward pass of a head's self-supervised training objective (paper section 3.3, "Losses"):
+//     kl_i = sum_v p_head(v) (log p_head(v) - log p_teacher(v))       loss = mean_i kl_i
+// for M tokens, from the head's hidden states and weights and the main model's final hidden states and head,
+// without ever writing either M x V logit matrix.
+//
+// With z = head logits, w = teacher logits:  kl = -H(p_head) + logZ(w) - E_{p_head}[w], so next to the head's
+// mergeable state (m, s, t, idx) a row carries the teacher's (m_w, s_w) and the cross sum u = sum e^{z - m} w.
+//
+// Three kernels chained by programmatic dependent launch:
+//   LayerNorm of both inputs (warp per row) into one bf16 buffer, rows padded to whole 128-row tiles with zeros;
+//   a persistent TMA + tcgen05 kernel, one CTA per SM: every tile of (128 rows x BN vocabulary rows) is computed
+//   twice in a row -- head operands into TMEM buffer 0, teacher operands into buffer 1 -- and the eight
+//   epilogue warps then read both buffers column chunk by column chunk and fold the joint statistics (so the
+//   epilogue of a tile pair does not overlap the next pair's MMAs; the roles and the bounded waits are those
+//   of the inference kernel);
+//   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
+#include "common.cuh"
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+#include "tensor_map.h"
+
+namespace ee {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kThreads = 320;                   // producer warp, MMA warp, eight epilogue warps
+constexpr int kGroupM = 16;
+constexpr int kATileBytes = BM * BK * 2;
+constexpr int kBarBytes = 512 + 2048 + 2048;    // barriers, then 128 head states and 128 teacher/cross states exchanged
+constexpr size_t kSmemBudget = 226 * 1024;
+constexpr int kMaxStages = 12;
+constexpr int kAccStride = 256;
+constexpr int kTmemCols = 512;
+
+struct KlMaps {
+    CUtensorMap y;         // [2 * m_pad, d]: the head's rows, then the teacher's
+    CUtensorMap w[2];      // head weights, teacher weights, each [V, d]
+};
+
+// Teacher side and cross term of a row restricted to some vocabulary range.
+struct Cross {
+    float mw, sw;          // running maximum of the teacher logits and sum of e^{w - mw}
+    float u;               // sum of e^{z - m} w, m being the head state's maximum
+    float pad;
+};
+static_assert(sizeof(Cross) == 16, "one 16-byte store per (row, tile)");
+
+struct KlParams {
+    int M, V, d;
+    int m_tiles, n_tiles, k_blocks, m_pad;
+    int bn, n_stages;
+    State* head_part;      // [M][n_tiles]
+    Cross* cross_part;     // [M][n_tiles]
+    Control* ctrl;
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
+    const int per_group = kGroupM * n_tiles;
+    const int grp = tile / per_group;
+    const int within = tile - grp * per_group;
+    const int rows_in_group = min(kGroupM, m_tiles - grp * kGroupM);
+    n_tile = within / rows_in_group;
+    m_tile = grp * kGroupM + (within - n_tile * rows_in_group);
+}
+
+__device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abort_flag, unsigned role, unsigned stage,
+                                               unsigned tile) {
+    if (atomicCAS(&ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
+        ctrl->error_info = (role << 24) | ((stage & 0xffu) << 16) | (tile & 0xffffu);
+    *abort_flag = 1;
+    __threadfence_block();
+}
+
+// Fold 32 consecutive columns of one row: head logits z, teacher logits w (the first `nvalid` real).
+template <bool kFull>
+__device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)[32], const float (&w)[32], int col0,
+                                          int nvalid) {
+    float cm = z[0], cw = w[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j)
+        if (kFull || j < nvalid) { cm = fmaxf(cm, z[j]); cw = fmaxf(cw, w[j]); }
+    if (cm > st.m) {
+        int j0 = 0;
+#pragma unroll
+        for (int j = 31; j >= 0; --j)
+            if ((kFull || j < nvalid) && z[j] == cm) j0 = j;
+        const float dl = st.m - cm;
+        const bool was_empty = (st.s == 0.f);
+        const float al = was_empty ? 0.f : ex2(dl * kLog2e);
+        st.t = was_empty ? 0.f : al * fmaf(dl, st.s, st.t);
+        st.s = al * st.s;
+        cr.u = al * cr.u;                                   // the cross sum is scaled like s
+        st.m = cm;
+        st.idx = col0 + j0;
+    }
+    if (cw > cr.mw) {
+        cr.sw = (cr.sw == 0.f) ? 0.f : cr.sw * ex2((cr.mw - cw) * kLog2e);
+        cr.mw = cw;
+    }
+    const float neg_m2 = -st.m * kLog2e, neg_w2 = -cr.mw * kLog2e;
+    float s = 0.f, t2 = 0.f, u = 0.f, sw = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (kFull || j < nvalid) {
+            const float a = fmaf(z[j], kLog2e, neg_m2);      // (z - m) * log2(e)
+            const float e = ex2(a);
+            s += e;
+            t2 = fmaf(e, a, t2);
+            u = fmaf(e, w[j], u);
+            sw += ex2(fmaf(w[j], kLog2e, neg_w2));
+        }
+    }
+    st.s += s;
+    st.t = fmaf(t2, kLn2, st.t);
+    cr.u += u;
+    cr.sw += sw;
+}
+
+// (st, cr) <- merge with (so, co): two vocabulary ranges of the same row.
+__device__ __forceinline__ void merge_pair(State& st, Cross& cr, const State& so, const Cross& co) {
+    if (so.s != 0.f) {
+        if (st.s == 0.f) {
+            cr.u = co.u;
+        } else {
+            const float m = fmaxf(st.m, so.m);
+            cr.u = ex2((st.m - m) * kLog2e) * cr.u + ex2((so.m - m) * kLog2e) * co.u;
+        }
+    }
+    state_merge(st, so);
+    if (co.sw != 0.f) {
+        if (cr.sw == 0.f) {
+            cr.mw = co.mw;
+            cr.sw = co.sw;
+        } else {
+            const float mw = fmaxf(cr.mw, co.mw);
+            cr.sw = ex2((cr.mw - mw) * kLog2e) * cr.sw + ex2((co.mw - mw) * kLog2e) * co.sw;
+            cr.mw = mw;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
+    const int BN = p.bn, S = p.n_stages;
+    const int b_tile_bytes = BN * BK * 2;
+    const int stage_bytes = kATileBytes + b_tile_bytes;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+    const uint32_t a_base = ptx::smem_addr(smem);
+    const uint32_t b_base = a_base + S * kATileBytes;
+    unsigned char* bar_mem = smem + S * stage_bytes;
+    const uint32_t bar_base = ptx::smem_addr(bar_mem);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * S + 4);
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_mem + 8 * (2 * S + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 5) + 4);
+    auto xfull_bar = [&](int q) { return bar_base + 8u * (2 * S + 6 + q); };
+    auto xfree_bar = [&](int q) { return bar_base + 8u * (2 * S + 10 + q); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull_bar(b), 1);
+            ptx::mbar_init(tempty_bar(b), 8);
+        }
+        for (int q = 0; q < 4; ++q) {
+            ptx::mbar_init(xfull_bar(q), 1);
+            ptx::mbar_init(xfree_bar(q), 1);
+        }
+        ptx::mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&maps.y);
+        ptx::prefetch_tensormap(&maps.w[0]);
+        ptx::prefetch_tensormap(&maps.w[1]);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+    const int total_tiles = p.m_tiles * p.n_tiles;           // each tile is computed for the head and for the teacher
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, armed = 0, armed_parity = 0;
+            bool ok = true;
+            int n_pre = 0;
+            if ((int)blockIdx.x < total_tiles) {              // head weights of the first stages before the wait
+                int m_tile, n_tile;
+                tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                n_pre = min(S, p.k_blocks);
+                for (int kb = 0; kb < n_pre; ++kb) {
+                    ptx::mbar_arrive_expect_tx(full_bar(kb), stage_bytes);
+                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &maps.w[0], kb * BK, n_tile * BN, full_bar(kb));
+                    armed |= 1u << kb;
+                }
+            }
+            grid_dependency_wait();
+            int issued = 0;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                int m_tile, n_tile;
+                tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                for (int which = 0; ok && which < 2; ++which) {
+                    const int y_row = which * p.m_pad + m_tile * BM;
+                    for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
+                        if (issued < n_pre) {
+                            ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                            if (++stage == S) { stage = 0; phase ^= 1u; }
+                            continue;
+                        }
+                        if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+                            record_failure(p.ctrl, abort_flag, 1, stage, tile);
+                            ok = false;
+                            break;
+                        }
+                        ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
+                        ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                        ptx::tma_load_2d(b_base + stage * b_tile_bytes, &maps.w[which], kb * BK, n_tile * BN, full_bar(stage));
+                        armed |= 1u << stage;
+                        armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (*abort_flag) {
+                for (int s = 0; s < S; ++s)
+                    if (armed & (1u << s)) {
+                        const uint32_t par = (armed_parity >> s) & 1u;
+                        for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
+                    }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer: buffer 0 = head, 1 = teacher
+        if (lane == 0) {
+            const uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+                const uint32_t acc_phase = (uint32_t)local & 1u;
+                for (int which = 0; ok && which < 2; ++which) {
+                    if (!ptx::mbar_wait(tempty_bar(which), acc_phase ^ 1u, abort_flag)) {
+                        record_failure(p.ctrl, abort_flag, 2, 0x80 | which, tile);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(which * kAccStride);
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
+                            record_failure(p.ctrl, abort_flag, 2, stage, tile);
+                            ok = false;
+                            break;
+                        }
+                        ptx::tc_fence_after_sync();
+                        const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
+                        const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        ptx::mma_commit(empty_bar(stage));
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) ptx::mma_commit(tfull_bar(which));
+                }
+            }
+            if (*abort_flag) {
+                ptx::mma_commit(drain_bar);
+                for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;                   // even / odd 32-column chunks
+        State* xchg = reinterpret_cast<State*>(bar_mem + 512) + quarter * 32 + lane;
+        Cross* xchg_c = reinterpret_cast<Cross*>(bar_mem + 512 + 2048) + quarter * 32 + lane;
+        const int row_in_tile = quarter * 32 + lane;
+        int local = 0;
+        grid_dependency_wait();
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+            int m_tile, n_tile;
+            tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+            const uint32_t acc_phase = (uint32_t)local & 1u;
+            const bool landed = ptx::mbar_wait(tfull_bar(0), acc_phase, abort_flag) &&
+                                ptx::mbar_wait(tfull_bar(1), acc_phase, abort_flag);
+            if (!__all_sync(0xffffffffu, landed)) {
+                if (lane == 0) record_failure(p.ctrl, abort_flag, 3, 0, tile);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int n0 = n_tile * BN;
+            const int ncols = min(BN, p.V - n0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            State st = state_empty();
+            Cross cr = {-CUDART_INF_F, 0.f, 0.f, 0.f};
+            const int row = m_tile * BM + row_in_tile;
+            const bool live = row < p.M;
+            if (__any_sync(0xffffffffu, live)) {
+                for (int c = half; c * 32 < ncols; c += 2) {
+                    float z[32], w[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, z);
+                    ptx::tmem_ld_32x32(taddr + kAccStride + c * 32, w);
+                    ptx::tmem_ld_wait();
+                    const int nvalid = ncols - c * 32;
+                    if (live) {
+                        if (nvalid >= 32) fold_pair<true>(st, cr, z, w, n0 + c * 32, 32);
+                        else fold_pair<false>(st, cr, z, w, n0 + c * 32, nvalid);
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive(tempty_bar(0));
+                ptx::mbar_arrive(tempty_bar(1));
+            }
+            const uint32_t x_phase = (uint32_t)local & 1u;
+            if (half == 1) {
+                const bool free_ = local == 0 || ptx::mbar_wait(xfree_bar(quarter), x_phase ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, free_)) {
+                    if (lane == 0) record_failure(p.ctrl, abort_flag, 5, quarter, tile);
+                    break;
+                }
+                *xchg = st;
+                *xchg_c = cr;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(xfull_bar(quarter));
+            } else {
+                const bool there = ptx::mbar_wait(xfull_bar(quarter), x_phase, abort_flag);
+                if (!__all_sync(0xffffffffu, there)) {
+                    if (lane == 0) record_failure(p.ctrl, abort_flag, 6, quarter, tile);
+                    break;
+                }
+                const State so = *xchg;
+                const Cross co = *xchg_c;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(xfree_bar(quarter));
+                if (live) {
+                    merge_pair(st, cr, so, co);
+                    p.head_part[(size_t)row * p.n_tiles + n_tile] = st;
+                    p.cross_part[(size_t)row * p.n_tiles + n_tile] = cr;
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// LayerNorm of the head's rows (blockIdx.y = 0) and the teacher's (1) into y [2][m_pad][d]; zero rows above M.
+struct KlLnArgs {
+    const __nv_bfloat16* h[2];
+    long long ld_h[2];
+    const float* gamma[2];
+    const float* beta[2];
+    float ln_eps[2];
+};
+
+__global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constant__ KlLnArgs a, __nv_bfloat16* __restrict__ y,
+                                                            int M, int m_pad, int d) {
+    launch_dependents();
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int which = blockIdx.y;
+    if (row >= m_pad) return;
+    const int nvec = d >> 3;
+    uint4* yrow = reinterpret_cast<uint4*>(y + ((size_t)which * m_pad + row) * d);
+    grid_dependency_wait();
+    if (row >= M) {
+        for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const uint4* hrow = reinterpret_cast<const uint4*>(a.h[which] + (size_t)row * a.ld_h[which]);
+    const float inv_d = 1.f / (float)d;
+    float sum = 0.f;
+    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
+    const float mu = warp_sum(sum) * inv_d;
+    float sq = 0.f;
+    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
+    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + a.ln_eps[which]);
+    for (int c = lane; c < nvec; c += 32)
+        yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, a.gamma[which], a.beta[which], c);
+}
+
+// One warp per row: the tiles' states in vocabulary order -> kl.
+__global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__ head_part, const Cross* __restrict__ cross_part,
+                                                       int n_tiles, int M, float* __restrict__ kl) {
+    launch_dependents();
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    grid_dependency_wait();
+    State st = state_empty();
+    Cross cr = {-CUDART_INF_F, 0.f, 0.f, 0.f};
+    for (int n = lane; n < n_tiles; n += 32) {
+        const State so = state_load_cg(head_part + (size_t)row * n_tiles + n);
+        const float4 c4 = __ldcg(reinterpret_cast<const float4*>(cross_part + (size_t)row * n_tiles + n));
+        merge_pair(st, cr, so, Cross{c4.x, c4.y, c4.z, 0.f});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const State so = state_shfl_xor(st, o);
+        Cross co;
+        co.mw = __shfl_xor_sync(0xffffffffu, cr.mw, o);
+        co.sw = __shfl_xor_sync(0xffffffffu, cr.sw, o);
+        co.u = __shfl_xor_sync(0xffffffffu, cr.u, o);
+        co.pad = 0.f;
+        // both lanes of a pair must end with the same bits: merge in a fixed (lower lane first) order
+        State a = (lane & o) ? so : st, b = (lane & o) ? st : so;
+        Cross ca = (lane & o) ? co : cr, cb = (lane & o) ? cr : co;
+        merge_pair(a, ca, b, cb);
+        st = a;
+        cr = ca;
+    }
+    if (lane == 0) {
+        const float entropy = logf(st.s) - st.t / st.s;                 // H(p_head)
+        const float log_z_teacher = cr.mw + logf(cr.sw);
+        kl[row] = -entropy + log_z_teacher - cr.u / st.s;
+    }
+}
+
+// loss = mean of kl, one CTA, fixed summation order (bit-identical from run to run).
+__global__ void __launch_bounds__(256) kl_mean_kernel(const float* __restrict__ kl, int M, float* __restrict__ loss) {
+    __shared__ float part[256];
+    launch_dependents();
+    grid_dependency_wait();
+    float s = 0.f;
+    for (int i = threadIdx.x; i < M; i += 256) s += kl[i];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *loss = part[0] / (float)M;
+}
+
+int stages_for(int bn) {
+    const size_t stage = kATileBytes + (size_t)bn * BK * 2;
+    const size_t n = (kSmemBudget - kBarBytes - 1024) / stage;
+    return (int)(n < (size_t)kMaxStages ? n : (size_t)kMaxStages);
+}
+
+int m_pad_of(int M) { return (M + BM - 1) / BM * BM; }
+size_t part_bytes(int M, int V) { return align_up((size_t)M * ((V + 63) / 64) * sizeof(State), 256); }
+
+}  // namespace
+
+size_t kl_workspace_bytes(int M, int d, int V) {
+    return kCtrlBytes + 2 * part_bytes(M, V) + align_up((size_t)2 * m_pad_of(M) * d * sizeof(__nv_bfloat16), 256);
+}
+
+ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, float* kl, float* loss) {
+    const int M = head.M, d = head.d, V = head.V;
+    unsigned char* ws = static_cast<unsigned char*>(head.workspace);
+    State* head_part = reinterpret_cast<State*>(ws + kCtrlBytes);
+    Cross* cross_part = reinterpret_cast<Cross*>(ws + kCtrlBytes + part_bytes(M, V));
+    __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + 2 * part_bytes(M, V));
+    const int m_pad = m_pad_of(M);
+    const int bn = gemm_tile_n(M, V, 1, head.num_sms);
+
+    KlLnArgs ln;
+    const HeadArgs* both[2] = {&head, &teacher};
+    for (int k = 0; k < 2; ++k) {
+        ln.h[k] = static_cast<const __nv_bfloat16*>(both[k]->h);
+        ln.ld_h[k] = both[k]->ld_h;
+        ln.gamma[k] = both[k]->gamma;
+        ln.beta[k] = both[k]->beta;
+        ln.ln_eps[k] = both[k]->ln_eps;
+    }
+    if (launch_pdl(kl_layer_norm_kernel, dim3(m_pad / 8, 2), 256, 0, head.stream, ln, y, M, m_pad, d) != cudaSuccess)
+        return EE_ERR_CUDA;
+
+    KlMaps maps;
+    const CUtensorMapL2promotion promo = M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+    if (!make_tile_map(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map(&maps.w[0], head.W, V, d, bn, promo) ||
+        !make_tile_map(&maps.w[1], teacher.W, V, d, bn, promo))
+        return EE_ERR_CUDA;
+    KlParams p;
+    p.M = M; p.V = V; p.d = d;
+    p.m_tiles = m_pad / BM;
+    p.n_tiles = (V + bn - 1) / bn;
+    p.k_blocks = (d + BK - 1) / BK;
+    p.m_pad = m_pad;
+    p.bn = bn;
+    p.n_stages = stages_for(bn);
+    p.head_part = head_part;
+    p.cross_part = cross_part;
+    p.ctrl = reinterpret_cast<Control*>(ws);
+    static bool configured[kMaxDevices] = {};
+    if (!configured[head.device]) {
+        if (cudaFuncSetAttribute(kl_pair_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+            return EE_ERR_CUDA;
+        configured[head.device] = true;
+    }
+    const long long total = (long long)p.m_tiles * p.n_tiles;
+    const int grid = (int)(total < head.num_sms ? total : head.num_sms);
+    const size_t smem = (size_t)p.n_stages * (kATileBytes + (size_t)bn * BK * 2) + kBarBytes + 1024;
+    if (launch_pdl(kl_pair_gemm_kernel, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
+    if (launch_pdl(kl_merge_kernel, (M + 7) / 8, 256, 0, head.stream, (const State*)head_part, (const Cross*)cross_part, p.n_tiles,
+                   M, kl) != cudaSuccess)
+        return EE_ERR_CUDA;
+    if (loss && launch_pdl(kl_mean_kernel, 1, 256, 0, head.stream, (const float*)kl, M, loss) != cudaSuccess) return EE_ERR_CUDA;
+    return EE_OK;
+}
+
+}  // namespace ee

@@ -1,0 +1,59 @@
+"""ee_head_kl against the oracle: per-token KL of the head's distribution from the teacher's, and their mean."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from _util import dev_bf16, head_to_dev
+
+pytestmark = pytest.mark.gpu
+KL_TOL = 2e-3          # absolute, nats: the tolerance of the entropy it contains
+
+
+@pytest.fixture(scope="module")
+def ee():
+    import paper_2407_21082_b200 as ee
+    return ee
+
+
+def _run(ee, cfg, h_head, h_teacher):
+    hd, tc = head_to_dev(cfg["heads"][0]), head_to_dev(cfg["heads"][1])
+    out = ee.ee_head_kl(dict(h=dev_bf16(h_head), gamma=hd["gamma"], beta=hd["beta"], W=hd["W"]),
+                        dict(h=dev_bf16(h_teacher), gamma=tc["gamma"], beta=tc["beta"], W=tc["W"]), 1e-5)
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("M,d,V", [(1, 64, 1), (5, 72, 257), (64, 128, 400), (129, 320, 515), (300, 64, 2049), (16, 1024, 50304)])
+def test_kl_matches_oracle(ee, M, d, V):
+    for planted in (False, True):
+        cfg = gen.make_config("c1", seed=31, planted=planted, M=M, d=d, V=V, heads=2)
+        rng = np.random.default_rng(M)
+        h_t = gen.bf16_bits_from_f32(gen.f32_from_bf16_bits(cfg["h"]) + rng.normal(0, 0.5, cfg["h"].shape).astype(np.float32))
+        ref = oracle.kl_to_teacher(cfg["h"], cfg["heads"][0], h_t, cfg["heads"][1])
+        out = _run(ee, cfg, cfg["h"], h_t)
+        again = _run(ee, cfg, cfg["h"], h_t)
+        kl = out["kl"].cpu().numpy().astype(np.float64)
+        assert np.isfinite(kl).all()
+        assert np.abs(kl - ref["kl"]).max() <= KL_TOL, (planted, np.abs(kl - ref["kl"]).max())
+        assert abs(float(out["loss"].item()) - ref["loss"]) <= KL_TOL
+        assert torch.equal(out["kl"], again["kl"]) and torch.equal(out["loss"], again["loss"])     # fixed reduction order
+        assert (kl > -1e-4).all()
+
+
+def test_kl_of_a_model_from_itself_is_zero(ee):
+    cfg = gen.make_config("c1", seed=3, planted=True, M=40, d=128, V=900, heads=2)
+    cfg["heads"][1] = cfg["heads"][0]
+    out = _run(ee, cfg, cfg["h"], cfg["h"])
+    assert float(out["kl"].abs().max()) <= 1e-5 and abs(float(out["loss"].item())) <= 1e-5
+
+
+def test_kl_argument_errors(ee):
+    cfg = gen.make_config("c1", seed=3, planted=False, M=4, d=64, V=100, heads=2)
+    hd = head_to_dev(cfg["heads"][0])
+    h = dev_bf16(cfg["h"])
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_head_kl(dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"]), dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"]),
+                      1e-5, workspace=torch.zeros(512, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == 4
