@@ -508,6 +508,57 @@ def measure_dssd_round(peaks: dict, src: str, S: int = 32, k: int = 8, rounds: i
                                   kind="oracle", cores=oracle_threads(), sample="the first round of the same sequences"))
 
 
+def measure_kl(peaks: dict, src: str, M: int, calls: int = 100) -> dict:
+    """ee_head_kl on the c1 shape (one head against the teacher head, M tokens); two copies of both weight
+    matrices in rotation (cold L2); the oracle on a sample of the rows."""
+    import torch
+    import oracle
+    import paper_2407_21082_b200 as ee
+    cfg = gen.make_config("c1", seed=0, planted=True, M=M, heads=2)
+    d, V = cfg["d"], cfg["V"]
+    rng = np.random.default_rng(0)
+    h_t = gen.bf16_bits_from_f32(gen.f32_from_bf16_bits(cfg["h"]) + rng.normal(0, 0.5, cfg["h"].shape).astype(np.float32))
+
+    def bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    ws = torch.empty(ee.ee_head_kl_workspace_bytes(M, d, V), dtype=torch.uint8, device="cuda")
+    ee.ee_workspace_init(ws)
+    hh, ht = bf16(cfg["h"]), bf16(h_t)
+    prepared = []
+    for c in range(2):
+        sides = [dict(h=h, gamma=torch.from_numpy(hd["gamma"]).cuda(), beta=torch.from_numpy(hd["beta"]).cuda(), W=bf16(hd["W"]))
+                 for h, hd in zip((hh, ht), cfg["heads"])]
+        prepared.append(ee.prepare_head_kl(sides[0], sides[1], 1e-5, workspace=ws))
+    calls = max(10, calls if M <= 256 else calls // 5)
+    for i in range(4):
+        prepared[i % 2]()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for i in range(calls):
+        prepared[i % 2]()
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / calls
+    got = prepared[(calls - 1) % 2].out["kl"].cpu().numpy()
+    rows = min(M, 32)
+    c0 = time.perf_counter()
+    ref = oracle.kl_to_teacher(cfg["h"][:rows], cfg["heads"][0], h_t[:rows], cfg["heads"][1])
+    cpu_s = time.perf_counter() - c0
+    nbytes = 2 * (2.0 * V * d + 2.0 * M * d) + 4.0 * M
+    flops = 2 * 2.0 * M * V * d
+    gbs, tfs = nbytes / (us * 1e-6) / 1e9, flops / (us * 1e-6) / 1e12
+    hbm_bound = nbytes / (peaks["hbm_gbs"] * 1e9) >= flops / (peaks["bf16_tflops"] * 1e12)
+    roof = (dict(bound="hbm", achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s", frac=round(gbs / peaks["hbm_gbs"], 4)) if hbm_bound
+            else dict(bound="tensor", achieved=round(tfs, 1), peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=round(tfs / peaks["bf16_tflops"], 4)))
+    roof.update(peak_source=f"of {src}", traffic=None, algorithmic_bytes=nbytes, flops=flops)
+    return dict(M=M, d=d, V=V, us_per_call=round(us, 2), launches=4, tokens_per_s=M / (us * 1e-6), roofline=roof,
+                max_abs_error_vs_oracle=float(np.abs(got[:rows] - ref["kl"]).max()), loss=float(prepared[(calls - 1) % 2].out["loss"].item()),
+                cpu_baseline=dict(value=rows / cpu_s, unit="tokens/s", seconds=round(cpu_s, 2), kind="oracle", cores=oracle_threads(),
+                                  sample=f"the first {rows} tokens"))
+
+
 def oracle_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -673,6 +724,7 @@ def main():
         line["calibration"] = measure_calibration(peaks, peak_src)
         line["cascade"] = measure_cascade(peaks, peak_src)
         line["dssd_round"] = measure_dssd_round(peaks, peak_src)
+        line["kl_loss"] = [measure_kl(peaks, peak_src, M) for M in (64, 4096)]
         if args.sweep:
             sweep = {}
             for rows in (1, 8, 16, 32, 64):

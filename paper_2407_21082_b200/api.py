@@ -368,6 +368,10 @@ def ee_calibrate_workspace_bytes(n: int) -> int:
     return int(_lib.load().ee_calibrate_workspace_bytes(int(n)))
 
 
+def ee_head_kl_workspace_bytes(M: int, d: int, V: int) -> int:
+    return int(_lib.load().ee_head_kl_workspace_bytes(int(M), int(d), int(V)))
+
+
 def _head_kl_args(head, teacher, ln_eps, out, workspace):
     hh, Wh = _bf16(_dev(head["h"], "h")), _bf16(_dev(head["W"], "W"))
     ht, Wt = _bf16(_dev(teacher["h"], "h")), _bf16(_dev(teacher["W"], "W"))
