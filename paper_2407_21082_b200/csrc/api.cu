@@ -45,6 +45,11 @@ bool sizes_ok(int M, int d, int V) { return M >= 0 && V >= 1 && d >= 8 && d <= 8
 // d = 512 M = 1 and 41.8 against 56.7 us at d = 2048 M = 16; the other two kernels stay selectable.)
 int auto_path(int, int) { return EE_PATH_TCGEN05; }
 
+// Heads one launch (sequence) of any of the three kernels takes.
+constexpr int kHeadsPerLaunch = 4;
+static_assert(kStreamMaxHeads == kHeadsPerLaunch && kSkinnyMaxHeads == kHeadsPerLaunch && kGemmLaunchMaxHeads == kHeadsPerLaunch,
+              "the multi-head entry point cuts its heads into groups every kernel accepts");
+
 size_t workspace_bytes(int M, int d, int V) {
     size_t need = gemm_workspace_bytes(M, d, V, 1);
     const size_t s = stream_workspace_bytes(1);
@@ -151,7 +156,7 @@ ee_status ee_exit_head_top2(const void* h, long long ld_h, const float* gamma, c
 size_t ee_exit_head_multi_workspace_bytes(int n_heads, int M, int d, int V) {
     if (!sizes_ok(M, d, V) || n_heads < 1) return 0;
     size_t need = workspace_bytes(M, d, V);
-    const int per_launch = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
+    const int per_launch = n_heads < kHeadsPerLaunch ? n_heads : kHeadsPerLaunch;
     if (kCtrlBytes + skinny_workspace_bytes(per_launch) > need) need = kCtrlBytes + skinny_workspace_bytes(per_launch);
     if (kCtrlBytes + stream_workspace_bytes(per_launch) > need) need = kCtrlBytes + stream_workspace_bytes(per_launch);
     if (kCtrlBytes + gemm_workspace_bytes(M, d, V, per_launch) > need) need = kCtrlBytes + gemm_workspace_bytes(M, d, V, per_launch);
@@ -186,7 +191,7 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     // EE_MULTI_KERNEL=stream | skinny | gemm | none overrides the choice (for A/B timing; a kernel that does
     // not take the shape leaves the default).
     enum { kNone, kStream, kSkinny, kGemm } mode = kGemm;
-    const int chunk = n_heads < kSkinnyMaxHeads ? n_heads : kSkinnyMaxHeads;
+    const int chunk = n_heads < kHeadsPerLaunch ? n_heads : kHeadsPerLaunch;
     const bool stream_ok = stream_slab_rows(d, chunk) >= M;
     if (const char* force = getenv("EE_MULTI_KERNEL")) {
         if (!strcmp(force, "stream") && stream_ok) mode = kStream;
@@ -194,9 +199,9 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
         else if (!strcmp(force, "gemm")) mode = kGemm;
         else if (!strcmp(force, "none")) mode = kNone;
     }
-    for (int k0 = 0; k0 < n_heads; k0 += kSkinnyMaxHeads) {
-        HeadArgs a[kSkinnyMaxHeads];
-        const int n = n_heads - k0 < kSkinnyMaxHeads ? n_heads - k0 : kSkinnyMaxHeads;
+    for (int k0 = 0; k0 < n_heads; k0 += kHeadsPerLaunch) {
+        HeadArgs a[kHeadsPerLaunch];
+        const int n = n_heads - k0 < kHeadsPerLaunch ? n_heads - k0 : kHeadsPerLaunch;
         for (int k = 0; k < n; ++k) {
             const ee_head& e = heads[k0 + k];
             a[k] = base;

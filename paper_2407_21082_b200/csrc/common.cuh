@@ -353,20 +353,4 @@ __device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem,
                                   maxprob, exit_mask);
 }
 
-// Whole-CTA variant: `scratch` is shared memory the partials are first copied to with independent loads, if it
-// is large enough.
-template <int THREADS>
-__device__ void merge_partials_and_decide(const State* partials, int n_cta, int np, int M, State* scratch,
-                                          size_t scratch_bytes, const float* tau_per_row, float tau, int* argmax,
-                                          float* entropy, float* maxprob, unsigned char* exit_mask) {
-    const int n_part = n_cta * np;
-    const bool via_smem = (size_t)n_part * sizeof(State) <= scratch_bytes;
-    if (via_smem) {
-        for (int i = threadIdx.x; i < n_part; i += THREADS) scratch[i] = state_load_cg(partials + i);
-        __syncthreads();
-    }
-    merge_tokens(via_smem ? scratch : partials, via_smem, n_cta, np, M, threadIdx.x >> 5, THREADS / 32, threadIdx.x & 31,
-                 tau_per_row, tau, argmax, entropy, maxprob, exit_mask);
-}
-
 }  // namespace ee
