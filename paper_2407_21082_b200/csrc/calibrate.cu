@@ -18,9 +18,9 @@ namespace ee {
 namespace {
 
 constexpr int kSortThreads = 256;
-constexpr int kItems = 16;                              // words per thread
-constexpr int kTile = kSortThreads * kItems;            // 4096 words per CTA
-constexpr int kWarpChunk = 32 * kItems;                 // 512 consecutive words per warp
+constexpr int kItems = 8;                               // words per thread
+constexpr int kTile = kSortThreads * kItems;            // 2048 words per CTA
+constexpr int kWarpChunk = 32 * kItems;                 // 256 consecutive words per warp
 constexpr int kDigits = 256;
 constexpr int kPasses = 4;                              // the 32 key bits; bit 0 (t) is carried, not sorted on
 
@@ -104,18 +104,17 @@ __global__ void __launch_bounds__(1024) calib_scan_kernel(unsigned int* __restri
     if (threadIdx.x == 0) digit_total[blockIdx.x] = s_carry;
 }
 
-// Stable scatter of one tile.  Warp w owns words [512 w, 512 w + 512) of the tile and walks them 32 at a time,
+// Stable scatter of one tile.  Warp w owns a run of 32 * kItems consecutive words of the tile and walks them 32 at a time,
 // so the order of equal digits inside the tile is (warp, round, lane) = their order in memory.  The tile is
 // first put in output order in shared memory, so that consecutive threads then write consecutive words of a
 // digit's run to global memory.
-__global__ void __launch_bounds__(kSortThreads, 3) calib_scatter_kernel(const u64* __restrict__ src, u64* __restrict__ dst,
+__global__ void __launch_bounds__(kSortThreads, 4) calib_scatter_kernel(const u64* __restrict__ src, u64* __restrict__ dst,
                                                                      int n, int shift,
                                                                      const unsigned int* __restrict__ tile_start,
                                                                      const unsigned int* __restrict__ digit_total,
                                                                      int n_tiles) {
     __shared__ unsigned int cnt[kSortThreads / 32][kDigits];
-    __shared__ unsigned int local_start[kDigits];      // where the digit's words start inside the sorted tile
-    __shared__ unsigned int global_start[kDigits];     // where this tile's words of the digit start in the output
+    __shared__ unsigned int out_shift[kDigits];        // output position minus position inside the sorted tile, per digit
     __shared__ unsigned int warp_part[kSortThreads / 32];
     __shared__ u64 staged[kTile];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -163,8 +162,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) calib_scatter_kernel(const u6
         unsigned int gbase = 0;
         for (int w = 0; w < warp; ++w) gbase += warp_part[w];
         const unsigned int lstart = lbase + incl - mine;
-        local_start[d] = lstart;
-        global_start[d] = gbase + gincl - total + tile_start[(size_t)d * n_tiles + blockIdx.x];
+        out_shift[d] = gbase + gincl - total + tile_start[(size_t)d * n_tiles + blockIdx.x] - lstart;
         unsigned int run = lstart;
 #pragma unroll
         for (int w = 0; w < kSortThreads / 32; ++w) {
@@ -184,7 +182,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) calib_scatter_kernel(const u6
     for (int k = threadIdx.x; k < in_tile; k += kSortThreads) {
         const u64 w = staged[k];
         const unsigned int d = (unsigned int)(w >> shift) & 255u;
-        dst[global_start[d] + ((unsigned int)k - local_start[d])] = w;
+        dst[out_shift[d] + (unsigned int)k] = w;
     }
 }
 
@@ -210,7 +208,7 @@ __global__ void __launch_bounds__(kSortThreads) calib_tile_sum_kernel(const u64*
 }
 
 // Position i (0-based, surest first) closes a group when the next word has another key.  There the set of the
-// i + 1 surest tokens is tested; the largest qualifying set wins.  Warp w walks positions [512 w, 512 w + 512)
+// i + 1 surest tokens is tested; the largest qualifying set wins.  Warp w walks its run of 32 * kItems positions
 // of the tile 32 at a time (held in registers), after the warps have exchanged their counts.
 __global__ void __launch_bounds__(kSortThreads) calib_select_kernel(const u64* __restrict__ sorted, int n,
                                                                     const unsigned int* __restrict__ tile_sum,
