@@ -554,7 +554,7 @@ def measure_kl(peaks: dict, src: str, M: int, calls: int = 100) -> dict:
             else dict(bound="tensor", achieved=round(tfs, 1), peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=round(tfs / peaks["bf16_tflops"], 4)))
     roof.update(peak_source=f"of {src}", traffic=None, algorithmic_bytes=nbytes, flops=flops)
     return dict(M=M, d=d, V=V, us_per_call=round(us, 2), launches=4, tokens_per_s=M / (us * 1e-6), roofline=roof,
-                max_abs_error_vs_oracle=float(np.abs(got[:rows] - ref["kl"]).max()), loss=float(prepared[(calls - 1) % 2].out["loss"].item()),
+                max_abs_error_vs_oracle=float(np.abs(got[:rows] - ref["kl"]).max()), loss=float(prepared[(calls - 1) % 2].out["loss"][0].item()),
                 cpu_baseline=dict(value=rows / cpu_s, unit="tokens/s", seconds=round(cpu_s, 2), kind="oracle", cores=oracle_threads(),
                                   sample=f"the first {rows} tokens"))
 

@@ -326,7 +326,10 @@ ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int
  * teacher's from the final hidden states and the main model's head, both exactly as in ee_exit_head; neither
  * M x V logit matrix is ever stored.
  *   kl   fp32 [M]: sum_v p_head(v) (log p_head(v) - log p_teacher(v)), nats
- *   loss fp32 [1]: their mean (summed in a fixed order: bit-identical from run to run); may be NULL
+ *   ce   fp32 [M]: -log p_head(labels[i]), the supervised objective L_CE of the same paragraph; ce and labels
+ *                  (int32 [M], 0 <= label < V) are given together or both NULL
+ *   loss fp32 [2]: the means of kl and (when asked for) of ce, each summed in a fixed order (bit-identical from
+ *                  run to run); may be NULL.  The hybrid objective is alpha * loss[1] + (1 - alpha) * loss[0].
  * h_* bf16 [M, d] (row strides ld_* elements), gamma_*, beta_* fp32 [d], W_* bf16 [V, d]; alignment as in
  * ee_exit_head.  Workspace: ee_head_kl_workspace_bytes(M, d, V), 256-byte aligned, initialised once with
  * ee_workspace_init.  M = 0 is a no-op.
@@ -335,7 +338,8 @@ size_t    ee_head_kl_workspace_bytes(int M, int d, int V);      /* host-only, pu
 ee_status ee_head_kl(const void* h_head, long long ld_head, const float* gamma_head, const float* beta_head,
                      const void* W_head, const void* h_teacher, long long ld_teacher, const float* gamma_teacher,
                      const float* beta_teacher, const void* W_teacher, float ln_eps, int M, int d, int V,
-                     float* kl, float* loss, void* workspace, size_t workspace_bytes, void* stream);
+                     const int* labels, float* kl, float* ce, float* loss, void* workspace, size_t workspace_bytes,
+                     void* stream);
 
 /*
  * Calibration of one head's threshold from a calibration set (section 3.4.1, "Calibration of Confidence

@@ -27,15 +27,30 @@ def kl_from_logits(z_head: np.ndarray, z_teacher: np.ndarray) -> np.ndarray:
     return (np.exp(lp) * (lp - lq)).sum(axis=1)
 
 
-def kl_to_teacher(h_head_bits, head, h_teacher_bits, teacher, rows_per_block: int = 64) -> dict:
-    """kl [M] per token and their mean (the loss).  head / teacher: dict(gamma, beta, ln_eps, W)."""
+def ce_from_logits(z_head: np.ndarray, labels: np.ndarray) -> np.ndarray:
+    """Per row: -log softmax(z_head)[label] (the supervised objective L_CE of the same paragraph)."""
+    m = z_head.max(axis=1)
+    log_z = m + np.log(np.exp(z_head - m[:, None]).sum(axis=1))
+    return log_z - z_head[np.arange(z_head.shape[0]), labels]
+
+
+def kl_to_teacher(h_head_bits, head, h_teacher_bits, teacher, rows_per_block: int = 64, labels=None) -> dict:
+    """kl [M] per token and their mean (the loss); with labels also ce [M] and its mean (the hybrid objective is
+    alpha * ce_loss + (1 - alpha) * loss).  head / teacher: dict(gamma, beta, ln_eps, W)."""
     M = h_head_bits.shape[0]
     Wh = bf16_decode(head["W"]).T.copy()
     Wt = bf16_decode(teacher["W"]).T.copy()
-    parts = []
+    parts, ce_parts = [], []
     for r0 in range(0, M, rows_per_block):
         yh = layer_norm(h_head_bits[r0:r0 + rows_per_block], head["gamma"], head["beta"], head["ln_eps"], True)
         yt = layer_norm(h_teacher_bits[r0:r0 + rows_per_block], teacher["gamma"], teacher["beta"], teacher["ln_eps"], True)
-        parts.append(kl_from_logits(yh @ Wh, yt @ Wt))
+        zh = yh @ Wh
+        parts.append(kl_from_logits(zh, yt @ Wt))
+        if labels is not None:
+            ce_parts.append(ce_from_logits(zh, np.asarray(labels)[r0:r0 + rows_per_block]))
     kl = np.concatenate(parts) if parts else np.zeros(0)
-    return dict(kl=kl, loss=float(kl.mean()) if M else 0.0)
+    out = dict(kl=kl, loss=float(kl.mean()) if M else 0.0)
+    if labels is not None:
+        ce = np.concatenate(ce_parts) if ce_parts else np.zeros(0)
+        out.update(ce=ce, ce_loss=float(ce.mean()) if M else 0.0)
+    return out

@@ -59,7 +59,7 @@ PROTOTYPES = {
                                     _p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_head_kl_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
     "ee_head_kl": (C.c_int, [_p, C.c_longlong, _p, _p, _p, _p, C.c_longlong, _p, _p, _p, C.c_float, C.c_int, C.c_int, C.c_int,
-                             _p, _p, _p, C.c_size_t, _p]),
+                             _p, _p, _p, _p, _p, C.c_size_t, _p]),
     "ee_cascade_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
     "ee_cascade": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p,
                              _p, C.c_size_t, _p]),

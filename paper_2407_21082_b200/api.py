@@ -372,7 +372,7 @@ def ee_head_kl_workspace_bytes(M: int, d: int, V: int) -> int:
     return int(_lib.load().ee_head_kl_workspace_bytes(int(M), int(d), int(V)))
 
 
-def _head_kl_args(head, teacher, ln_eps, out, workspace):
+def _head_kl_args(head, teacher, ln_eps, out, workspace, labels=None):
     hh, Wh = _bf16(_dev(head["h"], "h")), _bf16(_dev(head["W"], "W"))
     ht, Wt = _bf16(_dev(teacher["h"], "h")), _bf16(_dev(teacher["W"], "W"))
     M, d = hh.shape
@@ -381,7 +381,11 @@ def _head_kl_args(head, teacher, ln_eps, out, workspace):
         raise ValueError("head and teacher must share M, d, V; W contiguous [V, d]")
     dev = hh.device
     if out is None:
-        out = dict(kl=torch.empty(M, dtype=torch.float32, device=dev), loss=torch.empty(1, dtype=torch.float32, device=dev))
+        out = dict(kl=torch.empty(M, dtype=torch.float32, device=dev), loss=torch.zeros(2, dtype=torch.float32, device=dev))
+        if labels is not None:
+            out["ce"] = torch.empty(M, dtype=torch.float32, device=dev)
+    if labels is not None and (labels.dtype != torch.int32 or not labels.is_contiguous() or labels.numel() != M):
+        raise TypeError("labels must be a contiguous int32 tensor [M]")
     if workspace is None:
         workspace = torch.empty(int(_lib.load().ee_head_kl_workspace_bytes(M, d, V)), dtype=torch.uint8, device=dev)
         ee_workspace_init(workspace)
@@ -390,21 +394,22 @@ def _head_kl_args(head, teacher, ln_eps, out, workspace):
         return h.stride(0) if M > 1 else max(h.stride(0), d)
 
     args = (_ptr(hh), ld(hh), _ptr(head["gamma"]), _ptr(head["beta"]), _ptr(Wh), _ptr(ht), ld(ht), _ptr(teacher["gamma"]),
-            _ptr(teacher["beta"]), _ptr(Wt), float(ln_eps), M, d, V, _ptr(out["kl"]), _ptr(out.get("loss")), _ptr(workspace),
-            workspace.numel(), _stream())
-    return args, out, (hh, Wh, ht, Wt, head, teacher, workspace, out)
+            _ptr(teacher["beta"]), _ptr(Wt), float(ln_eps), M, d, V, _ptr(labels), _ptr(out["kl"]),
+            _ptr(out.get("ce")) if labels is not None else None, _ptr(out.get("loss")), _ptr(workspace), workspace.numel(), _stream())
+    return args, out, (hh, Wh, ht, Wt, head, teacher, workspace, out, labels)
 
 
-def ee_head_kl(head, teacher, ln_eps, *, out=None, workspace=None) -> dict:
-    """KL divergence of a head's distribution from the teacher's, per token and mean (see include/eexit.h).
+def ee_head_kl(head, teacher, ln_eps, *, labels=None, out=None, workspace=None) -> dict:
+    """KL divergence of a head's distribution from the teacher's, per token and mean (see include/eexit.h); with
+    `labels` also the cross-entropy per token (out["ce"]) and its mean (out["loss"][1]).
     head / teacher: dicts with h, gamma, beta, W."""
-    args, out, _ = _head_kl_args(head, teacher, ln_eps, out, workspace)
+    args, out, _ = _head_kl_args(head, teacher, ln_eps, out, workspace, labels)
     _check(_lib.load().ee_head_kl(*args), "ee_head_kl")
     return out
 
 
-def prepare_head_kl(head, teacher, ln_eps, *, out=None, workspace=None) -> PreparedCall:
-    args, out, keep = _head_kl_args(head, teacher, ln_eps, out, workspace)
+def prepare_head_kl(head, teacher, ln_eps, *, labels=None, out=None, workspace=None) -> PreparedCall:
+    args, out, keep = _head_kl_args(head, teacher, ln_eps, out, workspace, labels)
     return PreparedCall(_lib.load().ee_head_kl, args, "ee_head_kl", keep, out)
 
 

@@ -458,13 +458,15 @@ size_t ee_head_kl_workspace_bytes(int M, int d, int V) {
 
 ee_status ee_head_kl(const void* h_head, long long ld_head, const float* gamma_head, const float* beta_head,
                      const void* W_head, const void* h_teacher, long long ld_teacher, const float* gamma_teacher,
-                     const float* beta_teacher, const void* W_teacher, float ln_eps, int M, int d, int V, float* kl,
-                     float* loss, void* workspace, size_t workspace_bytes_, void* stream) {
+                     const float* beta_teacher, const void* W_teacher, float ln_eps, int M, int d, int V,
+                     const int* labels, float* kl, float* ce, float* loss, void* workspace, size_t workspace_bytes_,
+                     void* stream) {
     if (!sizes_ok(M, d, V)) return EE_ERR_SHAPE;
     if (M == 0) return EE_OK;
     if (!h_head || !gamma_head || !beta_head || !W_head || !h_teacher || !gamma_teacher || !beta_teacher || !W_teacher || !kl ||
         !workspace)
         return EE_ERR_NULL;
+    if ((ce != nullptr) != (labels != nullptr)) return EE_ERR_NULL;      // the cross-entropy needs labels, and only it does
     if (ld_head < d || (ld_head % 8) != 0 || ld_teacher < d || (ld_teacher % 8) != 0) return EE_ERR_SHAPE;
     if (!aligned(h_head, 16) || !aligned(W_head, 16) || !aligned(gamma_head, 16) || !aligned(beta_head, 16) ||
         !aligned(h_teacher, 16) || !aligned(W_teacher, 16) || !aligned(gamma_teacher, 16) || !aligned(beta_teacher, 16) ||
@@ -479,7 +481,7 @@ ee_status ee_head_kl(const void* h_head, long long ld_head, const float* gamma_h
     a.stream = static_cast<cudaStream_t>(stream);
     t = a;
     t.h = h_teacher; t.ld_h = ld_teacher; t.gamma = gamma_teacher; t.beta = beta_teacher; t.W = W_teacher;
-    return kl_launch(a, t, kl, loss);
+    return kl_launch(a, t, labels, kl, ce, loss);
 }
 
 ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, void* stream) {

@@ -85,7 +85,7 @@ ee_status calibrate_launch(const float* entropy, const int* argmax_head, const i
 
 // ---- KL divergence of a head's distribution from the teacher's, per token and mean (both logit sets fused) ----
 size_t kl_workspace_bytes(int M, int d, int V);
-ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, float* kl, float* loss);
+ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* labels, float* kl, float* ce, float* loss);
 
 // ---- commit step of a DSSD round (k <= 32) ----
 ee_status dssd_commit_launch(const int* draft_tok, const unsigned char* draft_exit_mask, const int* verify_tok, int S, int k,

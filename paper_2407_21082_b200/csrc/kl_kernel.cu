@@ -5,6 +5,8 @@
 //
 // With z = head logits, w = teacher logits:  kl = -H(p_head) + logZ(w) - E_{p_head}[w], so next to the head's
 // mergeable state (m, s, t, idx) a row carries the teacher's (m_w, s_w) and the cross sum u = sum e^{z - m} w.
+// With labels the same pass also gives the supervised objective of that paragraph, ce_i = -log p_head(label_i)
+// = logZ(z) - z[label_i]: the epilogue keeps the head's logit at the label's column.
 //
 // Three kernels chained by programmatic dependent launch:
 //   LayerNorm of both inputs (warp per row) into one bf16 buffer, rows padded to whole 128-row tiles with zeros;
@@ -43,7 +45,7 @@ struct KlMaps {
 struct Cross {
     float mw, sw;          // running maximum of the teacher logits and sum of e^{w - mw}
     float u;               // sum of e^{z - m} w, m being the head state's maximum
-    float pad;
+    float zl;              // the head's logit at the row's label, -inf while the label's column has not been seen
 };
 static_assert(sizeof(Cross) == 16, "one 16-byte store per (row, tile)");
 
@@ -54,6 +56,7 @@ struct KlParams {
     State* head_part;      // [M][n_tiles]
     Cross* cross_part;     // [M][n_tiles]
     Control* ctrl;
+    const int* labels;     // [M] or NULL (no cross-entropy asked for)
 };
 
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
@@ -76,7 +79,7 @@ __device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abor
 // Fold 32 consecutive columns of one row: head logits z, teacher logits w (the first `nvalid` real).
 template <bool kFull>
 __device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)[32], const float (&w)[32], int col0,
-                                          int nvalid) {
+                                          int nvalid, int label) {
     float cm = z[0], cw = w[0];
 #pragma unroll
     for (int j = 1; j < 32; ++j)
@@ -110,6 +113,7 @@ __device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)
             t2 = fmaf(e, a, t2);
             u = fmaf(e, w[j], u);
             sw += ex2(fmaf(w[j], kLog2e, neg_w2));
+            cr.zl = (col0 + j == label) ? z[j] : cr.zl;
         }
     }
     st.s += s;
@@ -129,6 +133,7 @@ __device__ __forceinline__ void merge_pair(State& st, Cross& cr, const State& so
         }
     }
     state_merge(st, so);
+    cr.zl = fmaxf(cr.zl, co.zl);                            // at most one range holds the label's column
     if (co.sw != 0.f) {
         if (cr.sw == 0.f) {
             cr.mw = co.mw;
@@ -312,9 +317,10 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             const int ncols = min(BN, p.V - n0);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
             State st = state_empty();
-            Cross cr = {-CUDART_INF_F, 0.f, 0.f, 0.f};
+            Cross cr = {-CUDART_INF_F, 0.f, 0.f, -CUDART_INF_F};
             const int row = m_tile * BM + row_in_tile;
             const bool live = row < p.M;
+            const int label = (live && p.labels) ? p.labels[row] : -1;
             if (__any_sync(0xffffffffu, live)) {
                 for (int c = half; c * 32 < ncols; c += 2) {
                     float z[32], w[32];
@@ -323,8 +329,8 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     ptx::tmem_ld_wait();
                     const int nvalid = ncols - c * 32;
                     if (live) {
-                        if (nvalid >= 32) fold_pair<true>(st, cr, z, w, n0 + c * 32, 32);
-                        else fold_pair<false>(st, cr, z, w, n0 + c * 32, nvalid);
+                        if (nvalid >= 32) fold_pair<true>(st, cr, z, w, n0 + c * 32, 32, label);
+                        else fold_pair<false>(st, cr, z, w, n0 + c * 32, nvalid, label);
                     }
                 }
             }
@@ -410,18 +416,18 @@ __global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constan
 
 // One warp per row: the tiles' states in vocabulary order -> kl.
 __global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__ head_part, const Cross* __restrict__ cross_part,
-                                                       int n_tiles, int M, float* __restrict__ kl) {
+                                                       int n_tiles, int M, float* __restrict__ kl, float* __restrict__ ce) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
     grid_dependency_wait();
     State st = state_empty();
-    Cross cr = {-CUDART_INF_F, 0.f, 0.f, 0.f};
+    Cross cr = {-CUDART_INF_F, 0.f, 0.f, -CUDART_INF_F};
     for (int n = lane; n < n_tiles; n += 32) {
         const State so = state_load_cg(head_part + (size_t)row * n_tiles + n);
         const float4 c4 = __ldcg(reinterpret_cast<const float4*>(cross_part + (size_t)row * n_tiles + n));
-        merge_pair(st, cr, so, Cross{c4.x, c4.y, c4.z, 0.f});
+        merge_pair(st, cr, so, Cross{c4.x, c4.y, c4.z, c4.w});
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -430,7 +436,7 @@ __global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__
         co.mw = __shfl_xor_sync(0xffffffffu, cr.mw, o);
         co.sw = __shfl_xor_sync(0xffffffffu, cr.sw, o);
         co.u = __shfl_xor_sync(0xffffffffu, cr.u, o);
-        co.pad = 0.f;
+        co.zl = __shfl_xor_sync(0xffffffffu, cr.zl, o);
         // both lanes of a pair must end with the same bits: merge in a fixed (lower lane first) order
         State a = (lane & o) ? so : st, b = (lane & o) ? st : so;
         Cross ca = (lane & o) ? co : cr, cb = (lane & o) ? cr : co;
@@ -442,23 +448,27 @@ __global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__
         const float entropy = logf(st.s) - st.t / st.s;                 // H(p_head)
         const float log_z_teacher = cr.mw + logf(cr.sw);
         kl[row] = -entropy + log_z_teacher - cr.u / st.s;
+        if (ce) ce[row] = st.m + logf(st.s) - cr.zl;                    // -log p_head(label)
     }
 }
 
-// loss = mean of kl, one CTA, fixed summation order (bit-identical from run to run).
-__global__ void __launch_bounds__(256) kl_mean_kernel(const float* __restrict__ kl, int M, float* __restrict__ loss) {
+// loss[0] = mean of kl, loss[1] = mean of ce (if there is one); CTA b sums array b in a fixed order
+// (bit-identical from run to run).
+__global__ void __launch_bounds__(256) kl_mean_kernel(const float* __restrict__ kl, const float* __restrict__ ce, int M,
+                                                      float* __restrict__ loss) {
     __shared__ float part[256];
     launch_dependents();
     grid_dependency_wait();
+    const float* src = blockIdx.x == 0 ? kl : ce;
     float s = 0.f;
-    for (int i = threadIdx.x; i < M; i += 256) s += kl[i];
+    for (int i = threadIdx.x; i < M; i += 256) s += src[i];
     part[threadIdx.x] = s;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
         if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
         __syncthreads();
     }
-    if (threadIdx.x == 0) *loss = part[0] / (float)M;
+    if (threadIdx.x == 0) loss[blockIdx.x] = part[0] / (float)M;
 }
 
 int stages_for(int bn) {
@@ -476,7 +486,7 @@ size_t kl_workspace_bytes(int M, int d, int V) {
     return kCtrlBytes + 2 * part_bytes(M, V) + align_up((size_t)2 * m_pad_of(M) * d * sizeof(__nv_bfloat16), 256);
 }
 
-ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, float* kl, float* loss) {
+ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* labels, float* kl, float* ce, float* loss) {
     const int M = head.M, d = head.d, V = head.V;
     unsigned char* ws = static_cast<unsigned char*>(head.workspace);
     State* head_part = reinterpret_cast<State*>(ws + kCtrlBytes);
@@ -513,6 +523,7 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, float* kl, fl
     p.head_part = head_part;
     p.cross_part = cross_part;
     p.ctrl = reinterpret_cast<Control*>(ws);
+    p.labels = ce ? labels : nullptr;
     static bool configured[kMaxDevices] = {};
     if (!configured[head.device]) {
         if (cudaFuncSetAttribute(kl_pair_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
@@ -524,9 +535,11 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, float* kl, fl
     const size_t smem = (size_t)p.n_stages * (kATileBytes + (size_t)bn * BK * 2) + kBarBytes + 1024;
     if (launch_pdl(kl_pair_gemm_kernel, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
     if (launch_pdl(kl_merge_kernel, (M + 7) / 8, 256, 0, head.stream, (const State*)head_part, (const Cross*)cross_part, p.n_tiles,
-                   M, kl) != cudaSuccess)
+                   M, kl, ce) != cudaSuccess)
         return EE_ERR_CUDA;
-    if (loss && launch_pdl(kl_mean_kernel, 1, 256, 0, head.stream, (const float*)kl, M, loss) != cudaSuccess) return EE_ERR_CUDA;
+    if (loss && launch_pdl(kl_mean_kernel, ce ? 2 : 1, 256, 0, head.stream, (const float*)kl, (const float*)ce, M, loss) !=
+                    cudaSuccess)
+        return EE_ERR_CUDA;
     return EE_OK;
 }
 

@@ -17,10 +17,11 @@ def ee():
     return ee
 
 
-def _run(ee, cfg, h_head, h_teacher):
+def _run(ee, cfg, h_head, h_teacher, labels=None):
     hd, tc = head_to_dev(cfg["heads"][0]), head_to_dev(cfg["heads"][1])
     out = ee.ee_head_kl(dict(h=dev_bf16(h_head), gamma=hd["gamma"], beta=hd["beta"], W=hd["W"]),
-                        dict(h=dev_bf16(h_teacher), gamma=tc["gamma"], beta=tc["beta"], W=tc["W"]), 1e-5)
+                        dict(h=dev_bf16(h_teacher), gamma=tc["gamma"], beta=tc["beta"], W=tc["W"]), 1e-5,
+                        labels=None if labels is None else torch.from_numpy(labels).cuda())
     torch.cuda.synchronize()
     return out
 
@@ -31,13 +32,21 @@ def test_kl_matches_oracle(ee, M, d, V):
         cfg = gen.make_config("c1", seed=31, planted=planted, M=M, d=d, V=V, heads=2)
         rng = np.random.default_rng(M)
         h_t = gen.bf16_bits_from_f32(gen.f32_from_bf16_bits(cfg["h"]) + rng.normal(0, 0.5, cfg["h"].shape).astype(np.float32))
-        ref = oracle.kl_to_teacher(cfg["h"], cfg["heads"][0], h_t, cfg["heads"][1])
-        out = _run(ee, cfg, cfg["h"], h_t)
-        again = _run(ee, cfg, cfg["h"], h_t)
+        labels = rng.integers(0, V, size=M).astype(np.int32)
+        labels[0] = V - 1                                               # the last column of the ragged last tile
+        ref = oracle.kl_to_teacher(cfg["h"], cfg["heads"][0], h_t, cfg["heads"][1], labels=labels)
+        out = _run(ee, cfg, cfg["h"], h_t, labels)
+        again = _run(ee, cfg, cfg["h"], h_t, labels)
+        ce = out["ce"].cpu().numpy().astype(np.float64)
+        assert np.abs(ce - ref["ce"]).max() <= KL_TOL, (planted, np.abs(ce - ref["ce"]).max())
+        assert abs(float(out["loss"][1].item()) - ref["ce_loss"]) <= KL_TOL
+        assert torch.equal(out["ce"], again["ce"])
+        no_labels = _run(ee, cfg, cfg["h"], h_t)
+        assert torch.equal(no_labels["kl"], out["kl"]) and "ce" not in no_labels
         kl = out["kl"].cpu().numpy().astype(np.float64)
         assert np.isfinite(kl).all()
         assert np.abs(kl - ref["kl"]).max() <= KL_TOL, (planted, np.abs(kl - ref["kl"]).max())
-        assert abs(float(out["loss"].item()) - ref["loss"]) <= KL_TOL
+        assert abs(float(out["loss"][0].item()) - ref["loss"]) <= KL_TOL
         assert torch.equal(out["kl"], again["kl"]) and torch.equal(out["loss"], again["loss"])     # fixed reduction order
         assert (kl > -1e-4).all()
 
@@ -46,7 +55,7 @@ def test_kl_of_a_model_from_itself_is_zero(ee):
     cfg = gen.make_config("c1", seed=3, planted=True, M=40, d=128, V=900, heads=2)
     cfg["heads"][1] = cfg["heads"][0]
     out = _run(ee, cfg, cfg["h"], cfg["h"])
-    assert float(out["kl"].abs().max()) <= 1e-5 and abs(float(out["loss"].item())) <= 1e-5
+    assert float(out["kl"].abs().max()) <= 1e-5 and abs(float(out["loss"][0].item())) <= 1e-5
 
 
 def test_kl_argument_errors(ee):

@@ -45,3 +45,24 @@ def test_whole_path_is_zero_for_identical_models_and_positive_otherwise():
     zh, zt = yh @ oracle.bf16_decode(cfg["heads"][0]["W"]).T, yt @ oracle.bf16_decode(cfg["heads"][1]["W"]).T
     ph = np.exp(zh - out_h["logZ"][:, None])
     assert np.abs(diff["kl"] - (-out_h["entropy"] + out_t["logZ"] - (ph * zt).sum(axis=1))).max() < 1e-11
+
+
+def test_cross_entropy_closed_forms():
+    V = 500
+    assert abs(oracle.ce_from_logits(np.zeros((1, V)), np.array([7]))[0] - math.log(V)) < 1e-14          # uniform
+    z = np.zeros((1, V)); z[0, 3] = 4.0
+    assert abs(oracle.ce_from_logits(z, np.array([3]))[0] - (math.log(math.exp(4.0) + V - 1) - 4.0)) < 1e-13
+    assert abs(oracle.ce_from_logits(z, np.array([9]))[0] - math.log(math.exp(4.0) + V - 1)) < 1e-13
+    rng = np.random.default_rng(2)
+    z = rng.normal(0, 3, (5, 30)); lab = rng.integers(0, 30, 5)
+    got = oracle.ce_from_logits(z, lab)
+    for i in range(5):
+        p = np.exp(z[i] - z[i].max()); p /= math.fsum(p)
+        assert abs(got[i] + math.log(p[lab[i]])) < 1e-13
+    assert np.allclose(oracle.ce_from_logits(z + 11.0, lab), got, atol=1e-13)                            # shift invariance
+    cfg = gen.make_config("c1", seed=2, planted=True, M=6, d=64, V=300, heads=2)
+    out = oracle.kl_to_teacher(cfg["h"], cfg["heads"][0], cfg["h"], cfg["heads"][1], labels=np.arange(6) * 7)
+    full = oracle.exit_head(cfg["h"], cfg["heads"][0]["gamma"], cfg["heads"][0]["beta"], 1e-5, cfg["heads"][0]["W"], 1.0)
+    own = oracle.kl_to_teacher(cfg["h"], cfg["heads"][0], cfg["h"], cfg["heads"][1], labels=full["argmax"])
+    assert np.abs(own["ce"] + np.log(full["maxprob"])).max() < 1e-12      # CE at the head's own prediction = -log p_max
+    assert abs(out["ce_loss"] - out["ce"].mean()) < 1e-15 and (out["ce"] >= own["ce"] - 1e-12).all()
