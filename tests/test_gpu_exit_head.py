@@ -303,3 +303,29 @@ def test_top2_gap_is_zero_when_the_maximum_is_attained_twice(ee):
     out = ee.ee_exit_head_top2(dev_bf16(gen.bf16_bits_from_f32(x.astype(np.float32))), dev(np.ones(d, np.float32)),
                                dev(np.zeros(d, np.float32)), 1e-5, dev_bf16(gen.bf16_bits_from_f32(Wv.astype(np.float32))), 1.0)
     assert torch.all(out["top2gap"] == 0) and out["argmax"].cpu().tolist() == [7, 7, 7]
+
+
+def test_calls_on_a_side_stream_interleaved_with_other_kernels(ee):
+    """The library's kernels are chained by programmatic dependent launch; work of other libraries before,
+    between and after them on a non-default stream must still be ordered as the stream says."""
+    cfg = gen.make_config("c1", seed=41, planted=True, M=48, d=256, V=3000, heads=2)
+    hds = [head_to_dev(cfg["heads"][k]) for k in range(2)]
+    base = dev_bf16(cfg["h"])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        outs = []
+        for rep in range(3):
+            h = base.clone()                                         # produced by a kernel right before the call
+            h.add_(0)                                                # and touched once more
+            o = ee.ee_exit_head_multi([dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=1.0) for hd in hds], 1e-5)
+            kept = ee.ee_compact(o[0]["exit_mask"], h)
+            total = o[0]["exit_mask"].to(torch.int32).sum() + kept["kept_count"][0]        # consumed by a kernel right after
+            outs.append((o, kept, total, h))
+        side.synchronize()
+    for o, kept, total, h in outs:
+        assert int(total.item()) == 48
+        for k in range(2):
+            assert_head_matches(o[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"side stream head {k}")
+            for key in o[k]:
+                assert torch.equal(o[k][key], outs[0][0][k][key])
