@@ -91,7 +91,7 @@ ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const 
 
 /*
  * ee_exit_head with the third confidence metric of section 3.4.1 as well: top2gap fp32 [M] = the difference
- * between the two largest probabilities of each row's distribution ("breaking ties"; 0 when the maximum is
+ * between the two largest probabilities of each row's distribution (the paper's tie-breaking metric; 0 when the maximum is
  * attained twice, p itself when V = 1).  Everything else as in ee_exit_head (same workspace size); the
  * tensor-core path is used for every size.
  */

@@ -11,8 +11,9 @@ the head answers when c >= tau.
 
 With the entropy H as the metric, c = -H: "c >= tau_c" is "H <= tau" with tau = -tau_c, the entropy at j-hat.
 Readings where the text is silent:
-  * ties: the suffix condition is evaluated on whole groups of equal confidence ("all samples with higher
-    (or equal) metric values"), so the result does not depend on how a sort orders equal values;
+  * ties: the suffix condition is evaluated on whole groups of equal confidence (the paper's prose counts every
+    sample whose metric is at least the candidate value), so the result does not depend on how a sort orders
+    equal values;
   * no index qualifies (the surest group is already below epsilon): the head never answers, tau = -inf;
   * the threshold returned is the paper's (a sample AT the threshold is inside the set); a caller whose rule
     is the strict H < tau passes the next float above it.

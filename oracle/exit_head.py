@@ -81,7 +81,7 @@ def logits(y: np.ndarray, W_bits: np.ndarray) -> np.ndarray:
 
 def softmax_stats(z: np.ndarray) -> dict:
     """A3.  Entropy (nats), max probability, argmax (lowest index), the top-2 logit gap, and the difference
-    between the two largest probabilities (the third confidence metric of section 3.4.1, "breaking ties")."""
+    between the two largest probabilities (the third confidence metric of section 3.4.1, the tie-breaking one)."""
     m = z.max(axis=1, keepdims=True)
     argmax = np.argmax(z, axis=1).astype(np.int32)           # numpy returns the first maximum
     zc = z - m
