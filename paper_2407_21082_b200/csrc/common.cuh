@@ -294,6 +294,32 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int block, si
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// The same with the grid grouped into clusters of two CTAs (grid.x even).
+inline void pair_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute (&attr)[2], dim3 grid, int block, size_t smem,
+                               cudaStream_t stream) {
+    cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+}
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, int block, size_t smem, cudaStream_t stream,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    pair_launch_config(cfg, attr, grid, block, smem, stream);
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Completion ticket and final merge shared by the one-launch kernels.
 // ---------------------------------------------------------------------------------------------

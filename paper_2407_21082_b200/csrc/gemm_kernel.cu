@@ -37,6 +37,7 @@ constexpr size_t kGemmSmemBudget = 226 * 1024;
 template <int BN_T>
 struct Cfg {
     static constexpr int kStages = 4;
+    static constexpr int kPairStages = 6;                             // a CTA of a pair stages half of the W tile
     static constexpr int kBTileBytes = 256 * BK * 2;
     static constexpr int kStageBytes = kATileBytes + kBTileBytes;
     static constexpr int kTmemCols = 512;                             // two accumulator buffers of 256 columns
@@ -192,13 +193,21 @@ __device__ __forceinline__ void chunk_top2(const float (&v)[32], int nvalid, flo
 
 // kTop2: also track the second-largest logit (for the top-2 probability gap); a separate instantiation, so
 // that the default kernel carries none of its registers or branches.
-template <int BN_T, bool kTop2>
+// kPair: the grid is made of clusters of two CTAs and each pair works on 256-row tiles (row tiles 2u and 2u + 1 of
+// a head): each CTA stages its own 128 rows of y and half of the W tile's rows, rank 0 issues 256 x BN MMAs
+// that read both CTAs' shared memory, and every CTA folds its own 128 rows out of its own tensor memory.  A W
+// tile then crosses L2 -> shared memory once per 256 rows instead of once per 128.
+template <int BN_T, bool kTop2, bool kPair>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p) {
     using C = Cfg<BN_T>;
     const int BN = BN_T ? BN_T : p.bn;
-    const int S = BN_T ? C::kStages : p.n_stages;
-    const int b_tile_bytes = BN * BK * 2;
+    const int S = BN_T ? (kPair ? C::kPairStages : C::kStages) : p.n_stages;
+    const uint32_t rank = kPair ? ptx::cluster_cta_rank() : 0u;
+    const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;        // tiles go round the CTAs / the pairs
+    const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int b_rows = kPair ? BN / 2 : BN;                                     // rows of W this CTA stages per k-block
+    const int b_tile_bytes = b_rows * BK * 2;
     // With at most 64 rows per head the MMA is issued with M = 64: half the tensor work (and power) of a
     // 128-row MMA whose lower half would be padding, and an 8 KB instead of a 16 KB y tile per stage.
     const int mma_m = BN_T ? BM : p.mma_m;
@@ -238,7 +247,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), BN_T ? 4 : 8);
+            ptx::mbar_init(tempty_bar(b), (BN_T ? 4 : 8) * (kPair ? 2 : 1));   // a pair's epilogue warps all report to rank 0
         }
         for (int q = 0; q < 4; ++q) {
             ptx::mbar_init(xfull_bar(q), 1);
@@ -251,21 +260,36 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
         for (int k = 0; k < p.n_heads; ++k) ptx::prefetch_tensormap(&maps.w[k]);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), C::kTmemCols);
-        ptx::tmem_relinquish();
+        if (kPair) {
+            ptx::tmem_alloc_pair(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), C::kTmemCols);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), C::kTmemCols);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();                   // the partner's barriers exist before anything signals them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
 
-    const int tiles_per_head = p.m_tiles * p.n_tiles;
+    const int m_units = kPair ? p.m_tiles >> 1 : p.m_tiles;     // row tiles, or pairs of row tiles
+    const int tiles_per_head = m_units * p.n_tiles;
     const int total_tiles = p.n_heads * tiles_per_head;
     // tile -> (head, m_tile, n_tile); within a head the order keeps concurrent CTAs on the same W tiles
     auto locate = [&](int tile, int& head, int& m_tile, int& n_tile) {
         head = tile / tiles_per_head;
-        tile_coords(tile - head * tiles_per_head, p.m_tiles, p.n_tiles, m_tile, n_tile);
+        tile_coords(tile - head * tiles_per_head, m_units, p.n_tiles, m_tile, n_tile);
+        if (kPair) m_tile = 2 * m_tile + (int)rank;
     };
+    // Where a stage's loads report their bytes (rank 0's barrier) and how they are issued.
+    auto load_full_bar = [&](int s) { return kPair ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s); };
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
+        if (kPair) ptx::tma_load_2d_pair(dst, m, c0, c1, bar);
+        else ptx::tma_load_2d(dst, m, c0, c1, bar);
+    };
+    const uint32_t arm_bytes = (uint32_t)stage_bytes * (kPair ? 2u : 1u);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -276,26 +300,27 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             // The weights do not depend on earlier kernels of the stream: the W tiles of the first stages are
             // requested before the dependency wait, the y tiles (written by the LayerNorm kernel) after it.
             int n_pre = 0;
-            if ((int)blockIdx.x < total_tiles) {
+            if (worker < total_tiles) {
                 int head, m_tile, n_tile;
-                locate(blockIdx.x, head, m_tile, n_tile);
+                locate(worker, head, m_tile, n_tile);
                 n_pre = min(S, p.k_blocks);
                 for (int kb = 0; kb < n_pre; ++kb) {
-                    ptx::mbar_arrive_expect_tx(full_bar(kb), stage_bytes);
-                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN, full_bar(kb));
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(kb), arm_bytes);
+                    load_tile(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
+                              load_full_bar(kb));
                     armed |= 1u << kb;
                 }
             }
             grid_dependency_wait();
             int issued = 0;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
                 int head, m_tile, n_tile;
                 locate(tile, head, m_tile, n_tile);
                 const int y_row = (head * p.m_tiles + m_tile) * BM;   // each head's rows are padded to whole tiles
-                if (BN_T != 0 && tile + (int)gridDim.x >= total_tiles) launch_dependents();
+                if (BN_T != 0 && tile + n_workers >= total_tiles) launch_dependents();
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
-                        ptx::tma_load_2d(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                        load_tile(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                         continue;
                     }
@@ -304,32 +329,39 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                         ok = false;
                         break;
                     }
-                    ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
-                    ptx::tma_load_2d(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, full_bar(stage));
-                    ptx::tma_load_2d(b_base + stage * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN, full_bar(stage));
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), arm_bytes);
+                    load_tile(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
+                    load_tile(b_base + stage * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
+                              load_full_bar(stage));
                     armed |= 1u << stage;
                     armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
             if (*abort_flag) {
-                // Let the copies still in flight land before the CTA gives its shared memory back.
-                for (int s = 0; s < S; ++s)
-                    if (armed & (1u << s)) {
-                        const uint32_t par = (armed_parity >> s) & 1u;
-                        for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
-                    }
+                // Let the copies still in flight land before the CTA gives its shared memory back.  (Rank 1 of a
+                // pair cannot poll the barrier its copies report to: it waits out a fixed time instead.)
+                if (rank != 0) {
+                    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+                } else {
+                    for (int s = 0; s < S; ++s)
+                        if (armed & (1u << s)) {
+                            const uint32_t par = (armed_parity >> s) & 1u;
+                            for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i)
+                                __nanosleep(100);
+                        }
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = ptx::idesc_bf16_f32(mma_m, BN);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = ptx::idesc_bf16_f32(kPair ? 2 * BM : mma_m, BN);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers, ++local) {
                 const int buf = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1u;
                 if (!ptx::mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag)) {
@@ -348,16 +380,24 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * a_tile_bytes);
                     const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes = 2 descriptor units per step
-                        ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    ptx::mma_commit(empty_bar(stage));    // frees the smem stage when these MMAs are done
+                    for (int k = 0; k < BK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor units per step
+                        if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        else ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    // frees the smem stage (in both CTAs of a pair) when these MMAs are done
+                    if (kPair) ptx::mma_commit_pair(empty_bar(stage), 3);
+                    else ptx::mma_commit(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) ptx::mma_commit(tfull_bar(buf));  // accumulator complete
+                if (ok) {                                 // accumulator complete
+                    if (kPair) ptx::mma_commit_pair(tfull_bar(buf), 3);
+                    else ptx::mma_commit(tfull_bar(buf));
+                }
             }
             if (*abort_flag) {
                 // Make sure no MMA is still writing TMEM when it is released.
-                ptx::mma_commit(drain_bar);
+                if (kPair) ptx::mma_commit_pair(drain_bar, 1);
+                else ptx::mma_commit(drain_bar);
                 for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
             }
         }
@@ -378,7 +418,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
         const int row_in_tile = mma_m == 64 ? (lane < 16 ? quarter * 16 + lane : BM) : quarter * 32 + lane;
         int local = 0;
         grid_dependency_wait();                           // the partial states may still be read by an earlier merge
-        for (int tile = blockIdx.x; (kSplit || half == 0) && tile < total_tiles; tile += gridDim.x, ++local) {
+        for (int tile = worker; (kSplit || half == 0) && tile < total_tiles; tile += n_workers, ++local) {
             int head, m_tile, n_tile;
             locate(tile, head, m_tile, n_tile);
             const int buf = local & 1;
@@ -416,7 +456,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
+            if (lane == 0) {
+                if (kPair) ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(buf), 0));
+                else ptx::mbar_arrive(tempty_bar(buf));
+            }
             const uint32_t x_phase = (uint32_t)local & 1u;
             if (!kSplit) {
                 if (live) {
@@ -501,10 +544,14 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
 
     ptx::tc_fence_before_sync();
     __syncthreads();
+    // Neither CTA of a pair leaves, or gives its tensor memory back, while the other may still signal its
+    // barriers, read its shared memory or write its accumulators.
+    if (kPair) ptx::cluster_sync_all();
     if (warp == 1) {
         __syncwarp();
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+        if (kPair) ptx::tmem_dealloc_pair(tmem_base, C::kTmemCols);
+        else ptx::tmem_dealloc(tmem_base, C::kTmemCols);
     }
 }
 
@@ -652,27 +699,67 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 constexpr int kMinTileN = 64;
 constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
 
-// Ring depth for a runtime tile width.
-int stages_for(int bn, int mma_m) {
-    const size_t stage = (size_t)mma_m * BK * 2 + (size_t)bn * BK * 2;
+// Ring depth for a runtime tile width; b_rows = rows of W one CTA stages per k-block.
+int stages_for(int b_rows, int mma_m) {
+    const size_t stage = (size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2;
     const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
 
-template <int BN_T, bool kTop2>
-ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int device, cudaStream_t stream) {
+template <int BN_T, bool kTop2, bool kPair>
+ee_status configure_gemm(int device) {
     static bool configured[kMaxDevices] = {};
     if (!configured[device]) {
-        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T, kTop2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(exit_head_gemm_kernel<BN_T, kTop2, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kGemmSmemBudget) != cudaSuccess)
             return EE_ERR_CUDA;
         configured[device] = true;
     }
+    return EE_OK;
+}
+
+template <int BN_T, bool kTop2, bool kPair>
+ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int device, cudaStream_t stream) {
+    if (configure_gemm<BN_T, kTop2, kPair>(device) != EE_OK) return EE_ERR_CUDA;
+    const int b_rows = kPair ? p.bn / 2 : p.bn;
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
-                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)p.bn * BK * 2) + kBarBytes + 1024;
-    return launch_pdl(exit_head_gemm_kernel<BN_T, kTop2>, grid, kGemmThreads, smem, stream, maps, p) == cudaSuccess
-               ? EE_OK
-               : EE_ERR_CUDA;
+                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
+    const cudaError_t err = kPair ? launch_pdl_pairs(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p)
+                                  : launch_pdl(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p);
+    return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+// How many two-CTA clusters of the GEMM kernel the device runs at once (0: none, or the query failed); asked
+// once per device.  All instantiations have the same footprint (one CTA per SM, the whole shared memory).
+int resident_pairs(int device) {
+    static int pairs[kMaxDevices];
+    static bool asked[kMaxDevices] = {};
+    if (!asked[device]) {
+        pairs[device] = 0;
+        if (configure_gemm<0, false, true>(device) == EE_OK) {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[2];
+            pair_launch_config(cfg, attr, dim3(2), kGemmThreads, kGemmSmemBudget, nullptr);
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, exit_head_gemm_kernel<0, false, true>, &cfg) == cudaSuccess && n > 0)
+                pairs[device] = n;
+            else
+                (void)cudaGetLastError();
+        }
+        asked[device] = true;
+    }
+    return pairs[device];
+}
+
+// Pairs of CTAs work on 256-row tiles when a head has an even number of 128-row tiles; EE_GEMM_PAIRS=0 in the
+// environment keeps every CTA on its own 128-row tiles (for comparisons).
+bool pairs_enabled() {
+    static int enabled = -1;
+    if (enabled < 0) {
+        const char* e = getenv("EE_GEMM_PAIRS");
+        enabled = (e && e[0] == '0') ? 0 : 1;
+    }
+    return enabled != 0;
 }
 
 // Upper bound on the partial states of M rows of one head whatever tile width the launch picks.
@@ -696,9 +783,13 @@ size_t second_bytes(int M, int V) { return align_up(partials_bytes(M, V) / 4, 25
 // Large M: 256, the widest accumulator (two fit in tensor memory), which maximises the reuse of each y tile.
 // Up to 1024 rows the weights are read about once and the launch is bound by HBM and by how evenly the
 // tiles fill the SMs: the width in 64..256 (multiple of 16) that minimises waves x (width + fixed cost).
+static int tile_n_for(long long m_units, int V, int n_heads, int num_sms);
 int gemm_tile_n(int M, int V, int n_heads, int num_sms) {
     if (M > 1024) return 256;
-    const long long m_tiles = (M + BM - 1) / BM;
+    return tile_n_for((M + BM - 1) / BM, V, n_heads, num_sms);
+}
+// m_units row tiles (or pairs of row tiles) per head, num_sms CTAs (or pairs of CTAs) to spread the tiles over.
+static int tile_n_for(long long m_tiles, int V, int n_heads, int num_sms) {
     int best = 128;
     long long best_cost = -1;
     for (int bn = kMinTileN; bn <= 256; bn += 16) {
@@ -728,7 +819,11 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     float* second = reinterpret_cast<float*>(ws + kCtrlBytes + (size_t)n_heads * partials_bytes(a.M, a.V));
     __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes +
                                                         (size_t)n_heads * (partials_bytes(a.M, a.V) + second_bytes(a.M, a.V)));
-    const int bn = gemm_tile_n(a.M, a.V, n_heads, a.num_sms);
+    const int m_tiles = (a.M + BM - 1) / BM;
+    const int n_pairs = (m_tiles % 2 == 0 && pairs_enabled()) ? resident_pairs(a.device) : 0;
+    const bool pair = n_pairs > 0;
+    const int bn = !pair ? gemm_tile_n(a.M, a.V, n_heads, a.num_sms)
+                         : (a.M > 1024 ? 256 : tile_n_for(m_tiles / 2, a.V, n_heads, n_pairs));
 
     LnHeads ln = {};
     MergeHeads mg = {};
@@ -765,7 +860,7 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     const int mma_m = a.M <= 64 ? 64 : BM;
     if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)) return EE_ERR_CUDA;
     for (int k = 0; k < kGemmMaxHeads; ++k)
-        if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, bn, promo)) return EE_ERR_CUDA;
+        if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, pair ? bn / 2 : bn, promo)) return EE_ERR_CUDA;
 
     GemmParams p;
     p.M = a.M;
@@ -786,13 +881,23 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
     p.mg = mg;
-    p.n_stages = stages_for(bn, mma_m);
-    const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
-    const int grid = (int)(total < a.num_sms ? total : a.num_sms);
-    const ee_status st = (a.M > 1024) ? (p.second ? launch_gemm<256, true>(maps, p, grid, a.device, a.stream)
-                                                  : launch_gemm<256, false>(maps, p, grid, a.device, a.stream))
-                                      : (p.second ? launch_gemm<0, true>(maps, p, grid, a.device, a.stream)
-                                                  : launch_gemm<0, false>(maps, p, grid, a.device, a.stream));
+    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
+    ee_status st;
+    if (pair) {
+        const long long total = (long long)n_heads * (p.m_tiles / 2) * p.n_tiles;
+        const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
+        st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, true>(maps, p, grid, a.device, a.stream)
+                                      : launch_gemm<256, false, true>(maps, p, grid, a.device, a.stream))
+                          : (p.second ? launch_gemm<0, true, true>(maps, p, grid, a.device, a.stream)
+                                      : launch_gemm<0, false, true>(maps, p, grid, a.device, a.stream));
+    } else {
+        const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
+        const int grid = (int)(total < a.num_sms ? total : a.num_sms);
+        st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, false>(maps, p, grid, a.device, a.stream)
+                                      : launch_gemm<256, false, false>(maps, p, grid, a.device, a.stream))
+                          : (p.second ? launch_gemm<0, true, false>(maps, p, grid, a.device, a.stream)
+                                      : launch_gemm<0, false, false>(maps, p, grid, a.device, a.stream));
+    }
     if (st != EE_OK) return st;
     if (p.fused_merge) return EE_OK;
 

@@ -38,6 +38,10 @@ SMALL = [
     ("v2", 2, 8, 2), ("v127", 3, 64, 127), ("v128", 127, 64, 128), ("v129", 1, 64, 129),
     ("m64", 64, 128, 400), ("m65", 65, 128, 400), ("m512", 512, 64, 300), ("m513", 513, 64, 300),
     ("m1024", 1024, 64, 300), ("m1025", 1025, 64, 520),
+    # an even number of 128-row tiles: two CTAs share each 256-row tile (runtime-width and 256-wide variants,
+    # ragged last vocabulary tiles, row counts that are not multiples of 128)
+    ("pair_m256", 256, 136, 700), ("pair_ragged", 200, 256, 3001), ("pair_m768", 768, 192, 2049),
+    ("pair_m1280", 1280, 128, 1500), ("pair_m2000", 2000, 72, 260),
 ]
 
 
@@ -214,6 +218,8 @@ def test_device_side_argument_errors(ee):
     ("odd_width", 40, 72, 500, 3),                # d % 64 != 0: the tensor-core path's ragged last k-block
     ("two_m_tiles", 150, 128, 1000, 3),           # stacked LayerNorm outputs: a 128-row tile reaches into the next head
     ("one_row", 1, 512, 777, 4),
+    ("paired_tiles", 256, 256, 3000, 3),          # 256-row tiles shared by two CTAs, merge kernel (768 rows)
+    ("paired_fused", 160, 128, 1200, 2),          # the same with the merge inside the GEMM kernel (320 rows)
 ])
 @pytest.mark.parametrize("kernel", ["auto", "stream", "skinny", "gemm", "none"])
 def test_multi_head_call_matches_oracle(ee, monkeypatch, name, M, d, V, n_heads, kernel):
