@@ -259,15 +259,15 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
 # while the SHA-256 of those sources still matches and as null afterwards.
 CSRC = os.path.join(ROOT, "paper_2407_21082_b200", "csrc")
 TRAFFIC = {
-    ("c1", 64): dict(bytes=309864960 + 3899392, heads_per_launch=3, kernel="exit_head_gemm_kernel<0>",
+    ("c1", 64): dict(bytes=309865728 + 3677696, heads_per_launch=3, kernel="exit_head_gemm_kernel<0>",
                      sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                     sha256="45cd14cadadc3bd078fe03378754e8b2d0d0d28a19a84d2b15654dce0cc59320", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
-    ("c2", 256): dict(bytes=207637760 + 4094976, heads_per_launch=1, kernel="exit_head_gemm_kernel<0>",
+                     sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
+    ("c2", 256): dict(bytes=207750656 + 4271744, heads_per_launch=1, kernel="exit_head_gemm_kernel<0> (CTA pairs)",
                       sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                      sha256="45cd14cadadc3bd078fe03378754e8b2d0d0d28a19a84d2b15654dce0cc59320", profile="profiles/exit_head_gemm_kernel_c2.md"),
-    ("c4", 16384): dict(bytes=2145157120 + 53726208, heads_per_launch=1, kernel="exit_head_gemm_kernel<256>",
+                      sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c2.md"),
+    ("c4", 16384): dict(bytes=1616886272 + 61617152, heads_per_launch=1, kernel="exit_head_gemm_kernel<256> (CTA pairs)",
                         sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                        sha256="45cd14cadadc3bd078fe03378754e8b2d0d0d28a19a84d2b15654dce0cc59320", profile="profiles/exit_head_gemm_kernel_c4.md"),
+                        sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c4.md"),
 }
 
 
