@@ -309,55 +309,112 @@ def roofline(wl: Workload, head_call_us: float, peaks: dict, src: str) -> dict:
 # --------------------------------------------------------------------------------------------- e2e and CPU baseline
 
 
+class E2ESlot:
+    """Everything one in-flight step of the host-buffer loop owns: a stream, pinned input rows, staging and result
+    buffers, a workspace, and the marshalled calls (one per copy of the weights)."""
+
+    def __init__(self, wl: Workload, stream):
+        torch, ee = wl.torch, wl.ee
+        S, k = wl.S, wl.k
+        self.torch = torch
+        self.stream = stream
+        self.done = torch.cuda.Event()
+        with torch.cuda.stream(stream):       # the binding binds a prepared call to the stream current at its creation
+            self.h_host = torch.stack([h.cpu() for h in wl.h]).pin_memory()             # [n_heads, M, d]
+            self.ws = torch.empty_like(wl.ws)
+            ee.ee_workspace_init(self.ws)
+            self.calls = [ee.PreparedMultiHost([dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"][c], tau=wl.tau) for hd in wl.heads],
+                                               1e-5, self.h_host, self.ws) for c in range(wl.n_copies)]
+            self.small_dev = torch.zeros(1 + 3 * max(S, 1), dtype=torch.int32, device="cuda")   # kept_count | draft_len | accept_len | next_tok
+            self.small_host = torch.zeros_like(self.small_dev, device="cpu").pin_memory()
+            comp = dict(kept_idx=torch.empty_like(wl.comp["kept_idx"]), kept_count=self.small_dev[0:1],
+                        h_out=torch.empty_like(wl.comp["h_out"]))
+            acc = {n: self.small_dev[1 + i * max(S, 1):1 + (i + 1) * max(S, 1)]
+                   for i, n in enumerate(("draft_len", "accept_len", "next_tok"))}
+            self.tails = []
+            for call in self.calls:
+                o = call.out_dev
+                if S == 0:
+                    self.tails.append(ee.prepare_compact(o[0]["exit_mask"], call.h_dev[0], out=comp))
+                else:
+                    n = S * k
+                    self.tails.append(ee.prepare_compact_accept(o[0]["exit_mask"], call.h_dev[0], o[0]["argmax"][:n].view(S, k),
+                                                                o[0]["exit_mask"][:n].view(S, k), o[-1]["argmax"][:n].view(S, k),
+                                                                out=dict(compact=comp, accept=acc)))
+        stream.synchronize()
+
+    def enqueue(self, c: int):
+        """One step: inputs host -> device, the heads, results device -> host, compaction + accept, their counts
+        device -> host; all asynchronous on this slot's stream."""
+        with self.torch.cuda.stream(self.stream):
+            self.calls[c]()
+            self.tails[c]()
+            self.small_host.copy_(self.small_dev, non_blocking=True)
+            self.done.record()
+
+    def read(self) -> int:
+        """The caller's read of a finished step: waits for it and touches the results on the host."""
+        self.done.synchronize()
+        return int(self.small_host[0])
+
+    def error(self, ee) -> int:
+        return ee.ee_query_async_error(self.ws)
+
+
+def run_e2e_loop(wl: Workload, slots, steps: int, warmup: int):
+    """steps + warmup steps round-robin over the slots.  With one slot every step is read before the next is
+    issued; with two, step i is issued, then step i - 1 is read, so that the host's share of a step (issuing,
+    waiting, reading) and its copies overlap the other batch's kernels."""
+    torch = wl.torch
+    n = len(slots)
+    checksum = 0
+
+    def run(count):
+        nonlocal checksum
+        for it in range(count):
+            c = wl.calls % wl.n_copies
+            wl.calls += 1
+            slots[it % n].enqueue(c)
+            if n == 1:
+                checksum += slots[0].read()
+            elif it >= 1:
+                checksum += slots[(it - 1) % n].read()
+        if n > 1 and count >= 1:
+            checksum += slots[(count - 1) % n].read()
+
+    run(warmup)
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    run(steps)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    for sl in slots:
+        code = sl.error(wl.ee)
+        if code != 0:
+            raise RuntimeError(f"device-side wait timed out in the end-to-end loop of workload {wl.name} (ee_status {code})")
+    return wall, checksum
+
+
 def measure_e2e(wl: Workload, steps: int, warmup: int) -> dict:
     """The same step through the host-buffer API: every step copies the heads' input rows from pinned host
     memory (one copy), evaluates the heads (ee_exit_head_multi_host), copies the packed results back (one
-    copy), runs compaction + accept on the device results, copies their counts back and synchronises,
-    because the caller reads its results every step.  Wall-clock around the loop."""
-    torch, ee = wl.torch, wl.ee
-    n_heads, S, k = len(wl.heads), wl.S, wl.k
-    h_host = torch.stack([h.cpu() for h in wl.h]).pin_memory()                  # [n_heads, M, d]
-    calls = [ee.PreparedMultiHost([dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"][c], tau=wl.tau) for hd in wl.heads],
-                                  1e-5, h_host, wl.ws) for c in range(wl.n_copies)]
-    small_dev = torch.zeros(1 + 3 * max(S, 1), dtype=torch.int32, device="cuda")  # kept_count | draft_len | accept_len | next_tok
-    small_host = torch.zeros_like(small_dev, device="cpu").pin_memory()
-    comp = dict(kept_idx=wl.comp["kept_idx"], kept_count=small_dev[0:1], h_out=wl.comp["h_out"])
-    acc = {n: small_dev[1 + i * max(S, 1):1 + (i + 1) * max(S, 1)] for i, n in enumerate(("draft_len", "accept_len", "next_tok"))}
-    tails = []
-    for call in calls:
-        o = call.out_dev
-        if S == 0:
-            tails.append(ee.prepare_compact(o[0]["exit_mask"], call.h_dev[0], out=comp))
-        else:
-            n = S * k
-            tails.append(ee.prepare_compact_accept(o[0]["exit_mask"], call.h_dev[0], o[0]["argmax"][:n].view(S, k),
-                                                   o[0]["exit_mask"][:n].view(S, k), o[-1]["argmax"][:n].view(S, k),
-                                                   out=dict(compact=comp, accept=acc)))
-
-    def step():
-        c = wl.calls % wl.n_copies
-        wl.calls += 1
-        calls[c]()
-        tails[c]()
-        small_host.copy_(small_dev, non_blocking=True)
-        torch.cuda.synchronize()          # the caller reads its results every step
-
-    for _ in range(warmup):
-        step()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    wall0 = time.perf_counter()
-    t0.record()
-    for _ in range(steps):
-        step()
-    t1.record()
-    torch.cuda.synchronize()
-    wall = time.perf_counter() - wall0
-    wl.check()
-    return dict(value=n_heads * wl.M * steps / wall, unit=UNIT, h2d_bytes_per_step=calls[0].h2d_bytes,
-                d2h_bytes_per_step=calls[0].d2h_bytes + small_host.numel() * 4,
-                ms_per_step=1e3 * wall / steps, device_ms_per_step=t0.elapsed_time(t1) / steps,
-                api="ee_exit_head_multi_host + ee_compact_accept, three copies and one synchronise per step")
+    copy), runs compaction + accept on the device results, copies their counts back, and the host waits for
+    the step and reads its results.  Wall-clock around the loop.  `value` is measured with two independent
+    batches in flight (each with its own stream, pinned buffers and workspace; a step's results are read before
+    its buffers are used again), `one_batch` with a single batch, where every step is read before the next starts."""
+    torch = wl.torch
+    n_heads = len(wl.heads)
+    slots = [E2ESlot(wl, torch.cuda.Stream()) for _ in range(2)]
+    wall1, _ = run_e2e_loop(wl, slots[:1], steps, warmup)
+    wall2, _ = run_e2e_loop(wl, slots, steps, warmup)
+    call = slots[0].calls[0]
+    return dict(value=n_heads * wl.M * steps / wall2, unit=UNIT, h2d_bytes_per_step=call.h2d_bytes,
+                d2h_bytes_per_step=call.d2h_bytes + slots[0].small_host.numel() * 4,
+                ms_per_step=1e3 * wall2 / steps, batches_in_flight=2,
+                one_batch=dict(value=n_heads * wl.M * steps / wall1, ms_per_step=1e3 * wall1 / steps),
+                api="ee_exit_head_multi_host + ee_compact_accept per step (three copies), the host waits for each step "
+                    "and reads its counts; two independent batches alternate on two streams (their kernels may overlap on the GPU, "
+                    "which also fills one batch's dependent-launch bubbles with the other's work)")
 
 
 def measure_calibration(peaks: dict, src: str, n: int = 1 << 22, calls: int = 30) -> dict:
