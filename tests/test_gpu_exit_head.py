@@ -335,3 +335,37 @@ def test_calls_on_a_side_stream_interleaved_with_other_kernels(ee):
             assert_head_matches(o[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"side stream head {k}")
             for key in o[k]:
                 assert torch.equal(o[k][key], outs[0][0][k][key])
+
+
+@pytest.mark.parametrize("M,d,V,n_heads", [(64, 256, 6000, 3), (256, 128, 9000, 2)])
+def test_two_calls_in_flight_on_two_streams(ee, M, d, V, n_heads):
+    """Two calls with workspaces of their own may overlap on the GPU (the documented limit): their results equal
+    the ones of the same calls run one after the other, and no bounded wait gives up."""
+    cfgs = [gen.make_config("c1", seed=51 + i, planted=True, M=M, d=d, V=V, heads=n_heads) for i in range(2)]
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    calls, refs = [], []
+    for cfg in cfgs:
+        hds = [head_to_dev(hd) for hd in cfg["heads"]]
+        h = dev_bf16(cfg["h"])
+        heads = [dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=1.0) for hd in hds]
+        refs.append([{k: v.clone() for k, v in o.items()} for o in ee.ee_exit_head_multi(heads, 1e-5)])
+        calls.append(heads)
+    torch.cuda.synchronize()
+    prepared = []
+    for heads, stream in zip(calls, streams):
+        with torch.cuda.stream(stream):                              # a prepared call is bound to the stream current here
+            ws = torch.empty(ee.ee_exit_head_multi_workspace_bytes(n_heads, M, d, V), dtype=torch.uint8, device="cuda")
+            ee.ee_workspace_init(ws)
+            outs = [ee.new_outputs(M) for _ in range(n_heads)]
+            prepared.append((ee.PreparedMulti([dict(hd, out=o) for hd, o in zip(heads, outs)], 1e-5, ws), outs, ws))
+    torch.cuda.synchronize()
+    for rep in range(40):
+        for call, _, _ in prepared:
+            call()
+    torch.cuda.synchronize()
+    for (call, outs, ws), ref, cfg in zip(prepared, refs, cfgs):
+        assert ee.ee_query_async_error(ws) == 0
+        for k in range(n_heads):
+            for key in ref[k]:
+                assert torch.equal(outs[k][key], ref[k][key]), (k, key)
+            assert_head_matches(outs[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"two streams head {k}")
