@@ -14,7 +14,8 @@
 //   twice in a row -- head operands into TMEM buffer 0, teacher operands into buffer 1 -- and the eight
 //   epilogue warps then read both buffers column chunk by column chunk and fold the joint statistics (so the
 //   epilogue of a tile pair does not overlap the next pair's MMAs; the roles and the bounded waits are those
-//   of the inference kernel);
+//   of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
+//   staging half of every W tile (cta_group::2 MMAs), as in the inference kernel;
 //   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
 #include "common.cuh"
 #include "kernels.h"
@@ -146,10 +147,18 @@ __device__ __forceinline__ void merge_pair(State& st, Cross& cr, const State& so
     }
 }
 
+// kPair: clusters of two CTAs share 256-row tiles (row tiles 2u and 2u + 1): each CTA stages its own 128 rows
+// of y and half of the W tile's rows, rank 0 issues 256 x BN MMAs over both CTAs' shared memory, each CTA folds its
+// own rows out of its own tensor memory (the protocol of the inference kernel's pair mode).
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
     const int BN = p.bn, S = p.n_stages;
-    const int b_tile_bytes = BN * BK * 2;
+    const uint32_t rank = kPair ? ptx::cluster_cta_rank() : 0u;
+    const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int b_rows = kPair ? BN / 2 : BN;
+    const int b_tile_bytes = b_rows * BK * 2;
     const int stage_bytes = kATileBytes + b_tile_bytes;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -177,7 +186,7 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 8);
+            ptx::mbar_init(tempty_bar(b), kPair ? 16 : 8);
         }
         for (int q = 0; q < 4; ++q) {
             ptx::mbar_init(xfull_bar(q), 1);
@@ -191,14 +200,31 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
         ptx::prefetch_tensormap(&maps.w[1]);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
-        ptx::tmem_relinquish();
+        if (kPair) {
+            ptx::tmem_alloc_pair(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();                      // the partner's barriers exist before anything signals them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
-    const int total_tiles = p.m_tiles * p.n_tiles;           // each tile is computed for the head and for the teacher
+    const int m_units = kPair ? p.m_tiles >> 1 : p.m_tiles;
+    const int total_tiles = m_units * p.n_tiles;             // each tile is computed for the head and for the teacher
+    auto locate = [&](int tile, int& m_tile, int& n_tile) {
+        tile_coords(tile, m_units, p.n_tiles, m_tile, n_tile);
+        if (kPair) m_tile = 2 * m_tile + (int)rank;
+    };
+    auto load_full_bar = [&](int s) { return kPair ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s); };
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
+        if (kPair) ptx::tma_load_2d_pair(dst, m, c0, c1, bar);
+        else ptx::tma_load_2d(dst, m, c0, c1, bar);
+    };
+    const uint32_t arm_bytes = (uint32_t)stage_bytes * (kPair ? 2u : 1u);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -207,26 +233,26 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             uint32_t phase = 0, armed = 0, armed_parity = 0;
             bool ok = true;
             int n_pre = 0;
-            if ((int)blockIdx.x < total_tiles) {              // head weights of the first stages before the wait
+            if (worker < total_tiles) {                       // head weights of the first stages before the wait
                 int m_tile, n_tile;
-                tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                locate(worker, m_tile, n_tile);
                 n_pre = min(S, p.k_blocks);
                 for (int kb = 0; kb < n_pre; ++kb) {
-                    ptx::mbar_arrive_expect_tx(full_bar(kb), stage_bytes);
-                    ptx::tma_load_2d(b_base + kb * b_tile_bytes, &maps.w[0], kb * BK, n_tile * BN, full_bar(kb));
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(kb), arm_bytes);
+                    load_tile(b_base + kb * b_tile_bytes, &maps.w[0], kb * BK, n_tile * BN + (int)rank * b_rows, load_full_bar(kb));
                     armed |= 1u << kb;
                 }
             }
             grid_dependency_wait();
             int issued = 0;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
                 int m_tile, n_tile;
-                tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+                locate(tile, m_tile, n_tile);
                 for (int which = 0; ok && which < 2; ++which) {
                     const int y_row = which * p.m_pad + m_tile * BM;
                     for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
                         if (issued < n_pre) {
-                            ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
+                            load_tile(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                             continue;
                         }
@@ -235,9 +261,10 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                             ok = false;
                             break;
                         }
-                        ptx::mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
-                        ptx::tma_load_2d(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, full_bar(stage));
-                        ptx::tma_load_2d(b_base + stage * b_tile_bytes, &maps.w[which], kb * BK, n_tile * BN, full_bar(stage));
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), arm_bytes);
+                        load_tile(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
+                        load_tile(b_base + stage * b_tile_bytes, &maps.w[which], kb * BK, n_tile * BN + (int)rank * b_rows,
+                                  load_full_bar(stage));
                         armed |= 1u << stage;
                         armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
                         if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -245,22 +272,28 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                 }
             }
             if (*abort_flag) {
-                for (int s = 0; s < S; ++s)
-                    if (armed & (1u << s)) {
-                        const uint32_t par = (armed_parity >> s) & 1u;
-                        for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
-                    }
+                // copies in flight land before the shared memory is given back (rank 1 of a pair cannot poll the
+                // barrier its copies report to and waits out a fixed time)
+                if (rank != 0) {
+                    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+                } else {
+                    for (int s = 0; s < S; ++s)
+                        if (armed & (1u << s)) {
+                            const uint32_t par = (armed_parity >> s) & 1u;
+                            for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
+                        }
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer: buffer 0 = head, 1 = teacher
-        if (lane == 0) {
-            const uint32_t idesc = ptx::idesc_bf16_f32(BM, BN);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = ptx::idesc_bf16_f32(kPair ? 2 * BM : BM, BN);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++local) {
+            for (int tile = worker; ok && tile < total_tiles; tile += n_workers, ++local) {
                 const uint32_t acc_phase = (uint32_t)local & 1u;
                 for (int which = 0; ok && which < 2; ++which) {
                     if (!ptx::mbar_wait(tempty_bar(which), acc_phase ^ 1u, abort_flag)) {
@@ -280,16 +313,23 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                         const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
                         const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                        ptx::mma_commit(empty_bar(stage));
+                        for (int k = 0; k < BK / 16; ++k) {
+                            if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            else ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
+                        if (kPair) ptx::mma_commit_pair(empty_bar(stage), 3);
+                        else ptx::mma_commit(empty_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok) ptx::mma_commit(tfull_bar(which));
+                    if (ok) {
+                        if (kPair) ptx::mma_commit_pair(tfull_bar(which), 3);
+                        else ptx::mma_commit(tfull_bar(which));
+                    }
                 }
             }
             if (*abort_flag) {
-                ptx::mma_commit(drain_bar);
+                if (kPair) ptx::mma_commit_pair(drain_bar, 1);
+                else ptx::mma_commit(drain_bar);
                 for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
             }
         }
@@ -302,9 +342,9 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
         const int row_in_tile = quarter * 32 + lane;
         int local = 0;
         grid_dependency_wait();
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local) {
+        for (int tile = worker; tile < total_tiles; tile += n_workers, ++local) {
             int m_tile, n_tile;
-            tile_coords(tile, p.m_tiles, p.n_tiles, m_tile, n_tile);
+            locate(tile, m_tile, n_tile);
             const uint32_t acc_phase = (uint32_t)local & 1u;
             const bool landed = ptx::mbar_wait(tfull_bar(0), acc_phase, abort_flag) &&
                                 ptx::mbar_wait(tfull_bar(1), acc_phase, abort_flag);
@@ -337,8 +377,13 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                ptx::mbar_arrive(tempty_bar(0));
-                ptx::mbar_arrive(tempty_bar(1));
+                if (kPair) {
+                    ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(0), 0));
+                    ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(1), 0));
+                } else {
+                    ptx::mbar_arrive(tempty_bar(0));
+                    ptx::mbar_arrive(tempty_bar(1));
+                }
             }
             const uint32_t x_phase = (uint32_t)local & 1u;
             if (half == 1) {
@@ -372,10 +417,12 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
 
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (kPair) ptx::cluster_sync_all();       // neither CTA leaves while the other may still signal it or write its accumulators
     if (warp == 1) {
         __syncwarp();
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if (kPair) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+        else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -471,10 +518,50 @@ __global__ void __launch_bounds__(256) kl_mean_kernel(const float* __restrict__ 
     if (threadIdx.x == 0) loss[blockIdx.x] = part[0] / (float)M;
 }
 
-int stages_for(int bn) {
-    const size_t stage = kATileBytes + (size_t)bn * BK * 2;
+int stages_for(int b_rows) {
+    const size_t stage = kATileBytes + (size_t)b_rows * BK * 2;
     const size_t n = (kSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxStages ? n : (size_t)kMaxStages);
+}
+
+// How many two-CTA clusters of the pair kernel the device runs at once; 0 if the query fails or EE_GEMM_PAIRS=0
+// in the environment switches pairs off.  Asked once per device.
+int resident_pairs(int device) {
+    static int pairs[kMaxDevices];
+    static bool asked[kMaxDevices] = {};
+    if (!asked[device]) {
+        pairs[device] = 0;
+        const char* e = getenv("EE_GEMM_PAIRS");
+        if (!(e && e[0] == '0') &&
+            cudaFuncSetAttribute(kl_pair_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) == cudaSuccess) {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[2];
+            pair_launch_config(cfg, attr, dim3(2), kThreads, kSmemBudget, nullptr);
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kl_pair_gemm_kernel<true>, &cfg) == cudaSuccess && n > 0) pairs[device] = n;
+            else (void)cudaGetLastError();
+        }
+        asked[device] = true;
+    }
+    return pairs[device];
+}
+
+// Tile width for m_units pairs of row tiles spread over n_pairs pairs of CTAs: 256 for many rows, else the multiple
+// of 16 in 64..256 that minimises waves x (width + 16).
+int pair_tile_n(int m_units, int V, int n_pairs) {
+    if (m_units > 4) return 256;
+    int best = 128;
+    long long best_cost = -1;
+    for (int bn = 64; bn <= 256; bn += 16) {
+        const long long tiles = (long long)m_units * ((V + bn - 1) / bn);
+        const long long waves = (tiles + n_pairs - 1) / n_pairs;
+        const long long cost = waves * (bn + 16);
+        if (best_cost < 0 || cost < best_cost || (cost == best_cost && bn > best)) {
+            best = bn;
+            best_cost = cost;
+        }
+    }
+    return best;
 }
 
 int m_pad_of(int M) { return (M + BM - 1) / BM * BM; }
@@ -493,7 +580,10 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
     Cross* cross_part = reinterpret_cast<Cross*>(ws + kCtrlBytes + part_bytes(M, V));
     __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(ws + kCtrlBytes + 2 * part_bytes(M, V));
     const int m_pad = m_pad_of(M);
-    const int bn = gemm_tile_n(M, V, 1, head.num_sms);
+    const int n_pairs = ((m_pad / BM) % 2 == 0) ? resident_pairs(head.device) : 0;     // 0: pairs switched off or unavailable
+    const bool pair = n_pairs > 0;
+    const int bn = pair ? pair_tile_n(m_pad / BM / 2, V, n_pairs) : gemm_tile_n(M, V, 1, head.num_sms);
+    const int b_rows = pair ? bn / 2 : bn;
 
     KlLnArgs ln;
     const HeadArgs* both[2] = {&head, &teacher};
@@ -509,8 +599,8 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
 
     KlMaps maps;
     const CUtensorMapL2promotion promo = M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
-    if (!make_tile_map(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map(&maps.w[0], head.W, V, d, bn, promo) ||
-        !make_tile_map(&maps.w[1], teacher.W, V, d, bn, promo))
+    if (!make_tile_map(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map(&maps.w[0], head.W, V, d, b_rows, promo) ||
+        !make_tile_map(&maps.w[1], teacher.W, V, d, b_rows, promo))
         return EE_ERR_CUDA;
     KlParams p;
     p.M = M; p.V = V; p.d = d;
@@ -519,21 +609,28 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
     p.k_blocks = (d + BK - 1) / BK;
     p.m_pad = m_pad;
     p.bn = bn;
-    p.n_stages = stages_for(bn);
+    p.n_stages = stages_for(b_rows);
     p.head_part = head_part;
     p.cross_part = cross_part;
     p.ctrl = reinterpret_cast<Control*>(ws);
     p.labels = ce ? labels : nullptr;
     static bool configured[kMaxDevices] = {};
     if (!configured[head.device]) {
-        if (cudaFuncSetAttribute(kl_pair_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+        if (cudaFuncSetAttribute(kl_pair_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+            cudaFuncSetAttribute(kl_pair_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
             return EE_ERR_CUDA;
         configured[head.device] = true;
     }
-    const long long total = (long long)p.m_tiles * p.n_tiles;
-    const int grid = (int)(total < head.num_sms ? total : head.num_sms);
-    const size_t smem = (size_t)p.n_stages * (kATileBytes + (size_t)bn * BK * 2) + kBarBytes + 1024;
-    if (launch_pdl(kl_pair_gemm_kernel, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
+    const size_t smem = (size_t)p.n_stages * (kATileBytes + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
+    if (pair) {
+        const long long total = (long long)(p.m_tiles / 2) * p.n_tiles;
+        const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
+        if (launch_pdl_pairs(kl_pair_gemm_kernel<true>, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
+    } else {
+        const long long total = (long long)p.m_tiles * p.n_tiles;
+        const int grid = (int)(total < head.num_sms ? total : head.num_sms);
+        if (launch_pdl(kl_pair_gemm_kernel<false>, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
+    }
     if (launch_pdl(kl_merge_kernel, (M + 7) / 8, 256, 0, head.stream, (const State*)head_part, (const Cross*)cross_part, p.n_tiles,
                    M, kl, ce) != cudaSuccess)
         return EE_ERR_CUDA;
