@@ -692,6 +692,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "stream", "tcgen05", "skinny"], help="force a kernel")
     ap.add_argument("--sweep", action="store_true", help="time every kernel that accepts the size, for c1 at several M")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-config table and the CPU baseline")
+    ap.add_argument("--only", default=None, choices=["calibration", "cascade", "dssd_round", "kl_loss"],
+                    help="run that entry of the table alone and print its JSON (for profiling one kernel family)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -726,6 +728,17 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks, peak_src = load_peaks()
+    if args.only is not None:
+        if rank == 0:
+            rows = [args.rows] if args.rows is not None else [64, 4096]
+            entry = {"calibration": lambda: measure_calibration(peaks, peak_src),
+                     "cascade": lambda: measure_cascade(peaks, peak_src),
+                     "dssd_round": lambda: measure_dssd_round(peaks, peak_src),
+                     "kl_loss": lambda: [measure_kl(peaks, peak_src, m) for m in rows]}[args.only]()
+            print(json.dumps({args.only: entry}))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     n_copies = {"c0": 8, "c1": 2}.get(args.workload, 2)
     path = dict(auto=0, stream=1, tcgen05=2, skinny=3)[args.path]
