@@ -12,9 +12,9 @@
 //   LayerNorm of both inputs (warp per row) into one bf16 buffer, rows padded to whole 128-row tiles with zeros;
 //   a persistent TMA + tcgen05 kernel, one CTA per SM: every tile of (128 rows x BN vocabulary rows) is computed
 //   twice in a row -- head operands into TMEM buffer 0, teacher operands into buffer 1 -- and the eight
-//   epilogue warps then read both buffers column chunk by column chunk and fold the joint statistics (so the
-//   epilogue of a tile pair does not overlap the next pair's MMAs; the roles and the bounded waits are those
-//   of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
+//   epilogue warps fold the head's statistics out of buffer 0 while the teacher's MMAs still run, then read both
+//   buffers column chunk by column chunk for the cross sum and the teacher's state (only this second pass does
+//   not overlap MMAs; the roles and the bounded waits are those of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
 //   staging half of every W tile (cta_group::2 MMAs), as in the inference kernel;
 //   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
 #include "common.cuh"
@@ -77,14 +77,14 @@ __device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abor
     __threadfence_block();
 }
 
-// Fold 32 consecutive columns of one row: head logits z, teacher logits w (the first `nvalid` real).
+// Fold 32 consecutive head logits of one row (the first `nvalid` real) into (m, s, t, idx); the logit at the
+// row's label is picked up on the way.
 template <bool kFull>
-__device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)[32], const float (&w)[32], int col0,
-                                          int nvalid, int label) {
-    float cm = z[0], cw = w[0];
+__device__ __forceinline__ void fold_head(State& st, float& zl, const float (&z)[32], int col0, int nvalid, int label) {
+    float cm = z[0];
 #pragma unroll
     for (int j = 1; j < 32; ++j)
-        if (kFull || j < nvalid) { cm = fmaxf(cm, z[j]); cw = fmaxf(cw, w[j]); }
+        if (kFull || j < nvalid) cm = fmaxf(cm, z[j]);
     if (cm > st.m) {
         int j0 = 0;
 #pragma unroll
@@ -95,16 +95,11 @@ __device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)
         const float al = was_empty ? 0.f : ex2(dl * kLog2e);
         st.t = was_empty ? 0.f : al * fmaf(dl, st.s, st.t);
         st.s = al * st.s;
-        cr.u = al * cr.u;                                   // the cross sum is scaled like s
         st.m = cm;
         st.idx = col0 + j0;
     }
-    if (cw > cr.mw) {
-        cr.sw = (cr.sw == 0.f) ? 0.f : cr.sw * ex2((cr.mw - cw) * kLog2e);
-        cr.mw = cw;
-    }
-    const float neg_m2 = -st.m * kLog2e, neg_w2 = -cr.mw * kLog2e;
-    float s = 0.f, t2 = 0.f, u = 0.f, sw = 0.f;
+    const float neg_m2 = -st.m * kLog2e;
+    float s = 0.f, t2 = 0.f;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         if (kFull || j < nvalid) {
@@ -112,13 +107,37 @@ __device__ __forceinline__ void fold_pair(State& st, Cross& cr, const float (&z)
             const float e = ex2(a);
             s += e;
             t2 = fmaf(e, a, t2);
-            u = fmaf(e, w[j], u);
-            sw += ex2(fmaf(w[j], kLog2e, neg_w2));
-            cr.zl = (col0 + j == label) ? z[j] : cr.zl;
         }
     }
     st.s += s;
     st.t = fmaf(t2, kLn2, st.t);
+    if ((unsigned)(label - col0) < (unsigned)nvalid) {       // one chunk of a row at most; columns past nvalid are the next tile's
+#pragma unroll
+        for (int j = 0; j < 32; ++j) zl = (col0 + j == label) ? z[j] : zl;
+    }
+}
+
+// Teacher state (mw, sw) and cross sum u over the same 32 columns, once the maximum of the head logits this
+// thread folds is final (neg_m2 = -m * log2(e)): no rescaling of u is left.
+template <bool kFull>
+__device__ __forceinline__ void fold_cross(Cross& cr, float neg_m2, const float (&z)[32], const float (&w)[32], int nvalid) {
+    float cw = w[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j)
+        if (kFull || j < nvalid) cw = fmaxf(cw, w[j]);
+    if (cw > cr.mw) {
+        cr.sw = (cr.sw == 0.f) ? 0.f : cr.sw * ex2((cr.mw - cw) * kLog2e);
+        cr.mw = cw;
+    }
+    const float neg_w2 = -cr.mw * kLog2e;
+    float u = 0.f, sw = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (kFull || j < nvalid) {
+            u = fmaf(ex2(fmaf(z[j], kLog2e, neg_m2)), w[j], u);
+            sw += ex2(fmaf(w[j], kLog2e, neg_w2));
+        }
+    }
     cr.u += u;
     cr.sw += sw;
 }
@@ -346,9 +365,8 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             int m_tile, n_tile;
             locate(tile, m_tile, n_tile);
             const uint32_t acc_phase = (uint32_t)local & 1u;
-            const bool landed = ptx::mbar_wait(tfull_bar(0), acc_phase, abort_flag) &&
-                                ptx::mbar_wait(tfull_bar(1), acc_phase, abort_flag);
-            if (!__all_sync(0xffffffffu, landed)) {
+            // the head's statistics are folded while the teacher's MMAs of the same tile still run
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(tfull_bar(0), acc_phase, abort_flag))) {
                 if (lane == 0) record_failure(p.ctrl, abort_flag, 3, 0, tile);
                 break;
             }
@@ -360,8 +378,28 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             Cross cr = {-CUDART_INF_F, 0.f, 0.f, -CUDART_INF_F};
             const int row = m_tile * BM + row_in_tile;
             const bool live = row < p.M;
+            const bool any_live = __any_sync(0xffffffffu, live);
             const int label = (live && p.labels) ? p.labels[row] : -1;
-            if (__any_sync(0xffffffffu, live)) {
+            if (any_live) {
+                for (int c = half; c * 32 < ncols; c += 2) {
+                    float z[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, z);
+                    ptx::tmem_ld_wait();
+                    const int nvalid = ncols - c * 32;
+                    if (live) {
+                        if (nvalid >= 32) fold_head<true>(st, cr.zl, z, n0 + c * 32, 32, label);
+                        else fold_head<false>(st, cr.zl, z, n0 + c * 32, nvalid, label);
+                    }
+                }
+            }
+            // second pass over both accumulators: the cross sum against the now final maximum, and the teacher's state
+            if (!__all_sync(0xffffffffu, ptx::mbar_wait(tfull_bar(1), acc_phase, abort_flag))) {
+                if (lane == 0) record_failure(p.ctrl, abort_flag, 3, 1, tile);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            if (any_live) {
+                const float neg_m2 = -st.m * kLog2e;
                 for (int c = half; c * 32 < ncols; c += 2) {
                     float z[32], w[32];
                     ptx::tmem_ld_32x32(taddr + c * 32, z);
@@ -369,8 +407,8 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     ptx::tmem_ld_wait();
                     const int nvalid = ncols - c * 32;
                     if (live) {
-                        if (nvalid >= 32) fold_pair<true>(st, cr, z, w, n0 + c * 32, 32, label);
-                        else fold_pair<false>(st, cr, z, w, n0 + c * 32, nvalid, label);
+                        if (nvalid >= 32) fold_cross<true>(cr, neg_m2, z, w, 32);
+                        else fold_cross<false>(cr, neg_m2, z, w, nvalid);
                     }
                 }
             }
