@@ -13,8 +13,9 @@
 //   a persistent TMA + tcgen05 kernel, one CTA per SM: every tile of (128 rows x BN vocabulary rows) is computed
 //   twice in a row -- head operands into TMEM buffer 0, teacher operands into buffer 1 -- and the eight
 //   epilogue warps fold the head's statistics out of buffer 0 while the teacher's MMAs still run, then read both
-//   buffers column chunk by column chunk for the cross sum and the teacher's state (only this second pass does
-//   not overlap MMAs; the roles and the bounded waits are those of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
+//   buffers column chunk by column chunk for the cross sum and the teacher's maximum, give buffer 0 back, and
+//   sum the teacher's exponentials out of buffer 1 while the next tile's head MMAs run (only the second pass
+//   does not overlap MMAs; the roles and the bounded waits are those of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
 //   staging half of every W tile (cta_group::2 MMAs), as in the inference kernel;
 //   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
 #include "common.cuh"
@@ -117,29 +118,31 @@ __device__ __forceinline__ void fold_head(State& st, float& zl, const float (&z)
     }
 }
 
-// Teacher state (mw, sw) and cross sum u over the same 32 columns, once the maximum of the head logits this
-// thread folds is final (neg_m2 = -m * log2(e)): no rescaling of u is left.
+// Cross sum u over 32 columns once the maximum of the head logits this thread folds is final (neg_m2 =
+// -m * log2(e); no rescaling of u is left), and the running maximum of the teacher logits.
 template <bool kFull>
-__device__ __forceinline__ void fold_cross(Cross& cr, float neg_m2, const float (&z)[32], const float (&w)[32], int nvalid) {
-    float cw = w[0];
-#pragma unroll
-    for (int j = 1; j < 32; ++j)
-        if (kFull || j < nvalid) cw = fmaxf(cw, w[j]);
-    if (cw > cr.mw) {
-        cr.sw = (cr.sw == 0.f) ? 0.f : cr.sw * ex2((cr.mw - cw) * kLog2e);
-        cr.mw = cw;
-    }
-    const float neg_w2 = -cr.mw * kLog2e;
-    float u = 0.f, sw = 0.f;
+__device__ __forceinline__ void fold_cross(float& u_acc, float& mw, float neg_m2, const float (&z)[32], const float (&w)[32],
+                                           int nvalid) {
+    float u = 0.f, cw = w[0];
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         if (kFull || j < nvalid) {
             u = fmaf(ex2(fmaf(z[j], kLog2e, neg_m2)), w[j], u);
-            sw += ex2(fmaf(w[j], kLog2e, neg_w2));
+            cw = fmaxf(cw, w[j]);
         }
     }
-    cr.u += u;
-    cr.sw += sw;
+    u_acc += u;
+    mw = fmaxf(mw, cw);
+}
+
+// sum of e^{w - mw} over 32 teacher logits, mw being final (neg_w2 = -mw * log2(e)).
+template <bool kFull>
+__device__ __forceinline__ float fold_teacher(float neg_w2, const float (&w)[32], int nvalid) {
+    float sw = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        if (kFull || j < nvalid) sw += ex2(fmaf(w[j], kLog2e, neg_w2));
+    return sw;
 }
 
 // (st, cr) <- merge with (so, co): two vocabulary ranges of the same row.
@@ -392,7 +395,8 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     }
                 }
             }
-            // second pass over both accumulators: the cross sum against the now final maximum, and the teacher's state
+            // second pass over both accumulators: the cross sum against the now final maximum and the teacher's
+            // maximum; the head's accumulator is then free for the next tile's MMAs
             if (!__all_sync(0xffffffffu, ptx::mbar_wait(tfull_bar(1), acc_phase, abort_flag))) {
                 if (lane == 0) record_failure(p.ctrl, abort_flag, 3, 1, tile);
                 break;
@@ -407,21 +411,33 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     ptx::tmem_ld_wait();
                     const int nvalid = ncols - c * 32;
                     if (live) {
-                        if (nvalid >= 32) fold_cross<true>(cr, neg_m2, z, w, 32);
-                        else fold_cross<false>(cr, neg_m2, z, w, nvalid);
+                        if (nvalid >= 32) fold_cross<true>(cr.u, cr.mw, neg_m2, z, w, 32);
+                        else fold_cross<false>(cr.u, cr.mw, neg_m2, z, w, nvalid);
                     }
                 }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                if (kPair) {
-                    ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(0), 0));
-                    ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(1), 0));
-                } else {
-                    ptx::mbar_arrive(tempty_bar(0));
-                    ptx::mbar_arrive(tempty_bar(1));
+                if (kPair) ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(0), 0));
+                else ptx::mbar_arrive(tempty_bar(0));
+            }
+            // third pass, over the teacher's accumulator alone (the next tile's head MMAs may run meanwhile)
+            if (any_live) {
+                const float neg_w2 = -cr.mw * kLog2e;
+                for (int c = half; c * 32 < ncols; c += 2) {
+                    float w[32];
+                    ptx::tmem_ld_32x32(taddr + kAccStride + c * 32, w);
+                    ptx::tmem_ld_wait();
+                    const int nvalid = ncols - c * 32;
+                    if (live) cr.sw += nvalid >= 32 ? fold_teacher<true>(neg_w2, w, 32) : fold_teacher<false>(neg_w2, w, nvalid);
                 }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                if (kPair) ptx::mbar_arrive_remote(ptx::map_to_cta(tempty_bar(1), 0));
+                else ptx::mbar_arrive(tempty_bar(1));
             }
             const uint32_t x_phase = (uint32_t)local & 1u;
             if (half == 1) {
