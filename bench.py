@@ -490,7 +490,7 @@ def measure_cascade(peaks: dict, src: str, M: int = 64, calls: int = 300) -> dic
     same = int((out["exit_head"] == ref["exit_head"]).sum())
     w_bytes = 3 * 2.0 * cfg["V"] * cfg["d"]
     gbs = w_bytes / (us * 1e-6) / 1e9
-    return dict(M=M, heads=3, taus=[1.0, 1.0, "inf"], us_per_call=round(us, 2), launches=3 * 3, rows_in=out["rows_in"].tolist(),
+    return dict(M=M, heads=3, taus=[1.0, 1.0, "inf"], us_per_call=round(us, 2), launches=3 if M <= 128 else 3 * 3, rows_in=out["rows_in"].tolist(),
                 rows_per_s=M / (us * 1e-6), rows_agreeing_with_oracle=same,
                 roofline=dict(bound="hbm", algorithmic_bytes=w_bytes, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
                               frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None),

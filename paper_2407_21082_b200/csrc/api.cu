@@ -338,11 +338,18 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
 namespace {
 size_t cascade_head_ws(int M, int d, int V) { return align_up(kCtrlBytes + gemm_workspace_bytes(M, d, V, 1), 256); }
 size_t cascade_rows_bytes(int M) { return align_up((size_t)M * 4, 256); }
+// small batches: up to four heads per launch on all rows, four result arrays per head
+size_t cascade_group_ws(int M, int d, int V) {
+    return align_up(kCtrlBytes + gemm_workspace_bytes(M, d, V, kHeadsPerLaunch), 256);
+}
 }  // namespace
 
 size_t ee_cascade_workspace_bytes(int M, int d, int V) {
     if (!sizes_ok(M, d, V)) return 0;
-    return cascade_head_ws(M, d, V) + 6 * cascade_rows_bytes(M) + 256;
+    const size_t by_step = cascade_head_ws(M, d, V) + 6 * cascade_rows_bytes(M) + 256;
+    if (M > cascade_select_max_rows()) return by_step;
+    const size_t by_group = cascade_group_ws(M, d, V) + 4 * kHeadsPerLaunch * cascade_rows_bytes(M);
+    return by_group > by_step ? by_group : by_step;
 }
 
 ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V, int* exit_head, int* token,
@@ -365,8 +372,33 @@ ee_status ee_cascade(const ee_head* heads, int n_heads, float ln_eps, int M, int
     const ee_status dev = current_device(&a.device, &a.num_sms);
     if (dev != EE_OK) return dev;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
-    unsigned char* p = ws + cascade_head_ws(M, d, V);
     const size_t rb = cascade_rows_bytes(M);
+    if (M <= cascade_select_max_rows()) {
+        // One row tile: evaluating a head on all rows costs what evaluating it on the open rows costs, so the
+        // heads go through the batched launch four at a time and a one-CTA kernel picks each row's first answer.
+        unsigned char* q = ws + cascade_group_ws(M, d, V);
+        for (int k0 = 0; k0 < n_heads; k0 += kHeadsPerLaunch) {
+            HeadArgs g[kHeadsPerLaunch];
+            const int n = n_heads - k0 < kHeadsPerLaunch ? n_heads - k0 : kHeadsPerLaunch;
+            for (int k = 0; k < n; ++k) {
+                const ee_head& e = heads[k0 + k];
+                g[k] = a;
+                g[k].h = e.h; g[k].ld_h = e.ld_h; g[k].gamma = e.gamma; g[k].beta = e.beta; g[k].ln_eps = ln_eps; g[k].W = e.W;
+                g[k].M = M; g[k].d = d; g[k].V = V; g[k].tau_per_row = nullptr; g[k].tau = e.tau;
+                unsigned char* r = q + (size_t)k * 4 * rb;
+                g[k].argmax = reinterpret_cast<int*>(r); g[k].entropy = reinterpret_cast<float*>(r + rb);
+                g[k].maxprob = reinterpret_cast<float*>(r + 2 * rb); g[k].exit_mask = r + 3 * rb;
+                g[k].workspace = workspace; g[k].workspace_bytes = cascade_group_ws(M, d, V); g[k].stream = s;
+            }
+            ee_status st = gemm_launch(g, n);
+            if (st != EE_OK) return st;
+            st = cascade_select_launch(q + 3 * rb, reinterpret_cast<const int*>(q), reinterpret_cast<const float*>(q + rb), 4 * rb,
+                                       M, k0, n, n_heads, exit_head, token, entropy, rows_in, s);
+            if (st != EE_OK) return st;
+        }
+        return EE_OK;
+    }
+    unsigned char* p = ws + cascade_head_ws(M, d, V);
     int* t_argmax = reinterpret_cast<int*>(p);
     float* t_entropy = reinterpret_cast<float*>(p + rb);
     float* t_maxprob = reinterpret_cast<float*>(p + 2 * rb);

@@ -66,7 +66,56 @@ __global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsign
     if (lane == 0 && row0 < max(m, 1) && row0 + kStepRows >= m) *m_out = base + __popc(ballot);
 }
 
+// Small batches (M <= kSelectThreads): up to four heads have been evaluated on EVERY row of the batch (a head's
+// weights are streamed once whatever the number of rows, and one 128-row tile costs the tensor pipe the same
+// full or not), and this kernel walks them in order for each row: a row still open takes the first head of the
+// group that answers it.  Between groups the state of a row is its exit_head entry (n_heads = still open).
+// One CTA, thread = row; head k of the group has its results at argmax0 / entropy0 / mask0 + k * stride bytes.
+constexpr int kSelectThreads = 128;
+
+__global__ void __launch_bounds__(kSelectThreads) cascade_select_kernel(const unsigned char* __restrict__ mask0,
+                                                                        const unsigned char* __restrict__ argmax0,
+                                                                        const unsigned char* __restrict__ entropy0,
+                                                                        size_t stride, int M, int k0, int n, int n_heads,
+                                                                        int* __restrict__ exit_head, int* __restrict__ token,
+                                                                        float* __restrict__ entropy_out,
+                                                                        int* __restrict__ rows_in) {
+    launch_dependents();
+    grid_dependency_wait();
+    const int i = threadIdx.x;
+    const bool in = i < M;
+    bool open = in && (k0 == 0 || exit_head[i] == n_heads);
+    for (int k = 0; k < n; ++k) {
+        const int cnt = __syncthreads_count(open);
+        if (i == 0) rows_in[k0 + k] = cnt;
+        if (open && (mask0 + k * stride)[i] != 0) {
+            exit_head[i] = k0 + k;
+            token[i] = reinterpret_cast<const int*>(argmax0 + k * stride)[i];
+            entropy_out[i] = reinterpret_cast<const float*>(entropy0 + k * stride)[i];
+            open = false;
+        }
+    }
+    if (open && k0 == 0) {                                              // stays so unless a later group answers
+        exit_head[i] = n_heads;
+        token[i] = -1;
+        entropy_out[i] = __int_as_float(0x7fc00000);
+    }
+}
+
 }  // namespace
+
+int cascade_select_max_rows() { return kSelectThreads; }
+
+ee_status cascade_select_launch(const unsigned char* mask0, const int* argmax0, const float* entropy0, size_t stride, int M,
+                                int k0, int n, int n_heads, int* exit_head, int* token, float* entropy_out, int* rows_in,
+                                cudaStream_t stream) {
+    if (M > kSelectThreads) return EE_ERR_SHAPE;
+    return launch_pdl(cascade_select_kernel, 1, kSelectThreads, 0, stream, mask0, reinterpret_cast<const unsigned char*>(argmax0),
+                      reinterpret_cast<const unsigned char*>(entropy0), stride, M, k0, n, n_heads, exit_head, token,
+                      entropy_out, rows_in) == cudaSuccess
+               ? EE_OK
+               : EE_ERR_CUDA;
+}
 
 ee_status cascade_step_launch(const unsigned char* exit_mask, const int* argmax, const float* entropy,
                               const int* idx_in, const int* m_in, int M, int k, int is_last, int n_heads,

@@ -103,6 +103,10 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
 ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
 
 // ---- one step of the cascade of heads: rows answered by head k are recorded, the others move on ----
+int cascade_select_max_rows();
+ee_status cascade_select_launch(const unsigned char* mask0, const int* argmax0, const float* entropy0, size_t stride, int M,
+                                int k0, int n, int n_heads, int* exit_head, int* token, float* entropy_out, int* rows_in,
+                                cudaStream_t stream);
 ee_status cascade_step_launch(const unsigned char* exit_mask, const int* argmax, const float* entropy,
                               const int* idx_in, const int* m_in, int M, int k, int is_last, int n_heads,
                               int* exit_head, int* token, float* entropy_out, int* idx_out, int* m_out, int* rows_in,

@@ -39,7 +39,8 @@ def _fragile_rows(ref, taus):
     return margin_bad, token_bad
 
 
-@pytest.mark.parametrize("M,d,V,K", [(24, 64, 300, 3), (1, 64, 129, 2), (100, 256, 1000, 4), (600, 128, 700, 3), (1100, 64, 520, 2)])
+@pytest.mark.parametrize("M,d,V,K", [(24, 64, 300, 3), (1, 64, 129, 2), (100, 256, 1000, 4), (600, 128, 700, 3), (1100, 64, 520, 2),
+                                     (128, 64, 700, 6), (37, 128, 515, 9), (129, 64, 300, 5)])   # groups of four heads below 129 rows
 def test_cascade_matches_oracle(ee, M, d, V, K):
     cfg, h_list = _case(3 + M, M, d, V, K)
     taus = [0.6 + 0.7 * k for k in range(K)]
