@@ -55,6 +55,29 @@ def test_kl_matches_oracle(ee, M, d, V):
         assert (kl > -1e-4).all()
 
 
+def test_kl_full_size_on_a_row_sample(ee):
+    """The benchmark's training-sized call (c1 shape, M = 4096: CTA pairs on 256-row tiles, 256 columns wide): the
+    oracle checks two rows of every 128-row tile plus the tiles' edges; properties that hold for every row."""
+    M, d, V = 4096, 1024, 50304
+    cfg = gen.make_config("c1", seed=0, planted=False, M=M, heads=2)
+    rng = np.random.default_rng(0)
+    h_t = gen.bf16_bits_from_f32(gen.f32_from_bf16_bits(cfg["h"]) + rng.normal(0, 0.5, cfg["h"].shape).astype(np.float32))
+    labels = rng.integers(0, V, size=M).astype(np.int32)
+    labels[:4] = [0, 255, 256, V - 1]                                   # tile edges of the vocabulary
+    out = _run(ee, cfg, cfg["h"], h_t, labels)
+    rows = np.unique(np.concatenate([[0, 1, 2, 3, 127, 128, 255, 256, 4095],
+                                     [t * 128 + (37 * t + 64 * i) % 128 for t in range(32) for i in range(2)]]))
+    ref = oracle.kl_to_teacher(cfg["h"][rows], cfg["heads"][0], h_t[rows], cfg["heads"][1], labels=labels[rows])
+    kl = out["kl"].cpu().numpy().astype(np.float64)
+    ce = out["ce"].cpu().numpy().astype(np.float64)
+    assert np.abs(kl[rows] - ref["kl"]).max() <= KL_TOL
+    assert np.abs(ce[rows] - ref["ce"]).max() <= KL_TOL
+    assert len(set(rows // 128)) == 32
+    assert np.isfinite(kl).all() and (kl > -1e-4).all()                 # a divergence
+    assert np.isfinite(ce).all() and (ce > 0).all()                     # -log of a probability below one
+    assert abs(float(out["loss"][0].item()) - kl.mean()) <= 1e-4 and abs(float(out["loss"][1].item()) - ce.mean()) <= 1e-4
+
+
 def test_kl_of_a_model_from_itself_is_zero(ee):
     cfg = gen.make_config("c1", seed=3, planted=True, M=40, d=128, V=900, heads=2)
     cfg["heads"][1] = cfg["heads"][0]
