@@ -490,12 +490,12 @@ def measure_cascade(peaks: dict, src: str, M: int = 64, calls: int = 300) -> dic
     same = int((out["exit_head"] == ref["exit_head"]).sum())
     w_bytes = 3 * 2.0 * cfg["V"] * cfg["d"]
     gbs = w_bytes / (us * 1e-6) / 1e9
-    return dict(M=M, heads=3, taus=[1.0, 1.0, "inf"], us_per_call=round(us, 2), launches=3 if M <= 128 else 3 * 3, rows_in=out["rows_in"].tolist(),
+    return dict(M=M, heads=3, taus=[1.0, 1.0, "inf"], us_per_call=round(us, 2), launches=3 if M <= 512 else 3 * 3, rows_in=out["rows_in"].tolist(),
                 rows_per_s=M / (us * 1e-6), rows_agreeing_with_oracle=same,
                 roofline=dict(bound="hbm", algorithmic_bytes=w_bytes, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
                               frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None),
                 cpu_baseline=dict(value=M / cpu_s, unit="rows/s", seconds=round(cpu_s, 2), kind="oracle", cores=oracle_threads(),
-                                  sample="the same 64 rows through the same three heads"))
+                                  sample=f"the same {M} rows through the same three heads"))
 
 
 def measure_dssd_round(peaks: dict, src: str, S: int = 32, k: int = 8, rounds: int = 40) -> dict:
@@ -734,7 +734,7 @@ def main():
         if rank == 0:
             rows = [args.rows] if args.rows is not None else [64, 4096]
             entry = {"calibration": lambda: measure_calibration(peaks, peak_src),
-                     "cascade": lambda: measure_cascade(peaks, peak_src),
+                     "cascade": lambda: measure_cascade(peaks, peak_src, M=args.rows or 64),
                      "dssd_round": lambda: measure_dssd_round(peaks, peak_src),
                      "kl_loss": lambda: [measure_kl(peaks, peak_src, m) for m in rows]}[args.only]()
             print(json.dumps({args.only: entry}))

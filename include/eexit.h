@@ -313,11 +313,11 @@ ee_status ee_compact_accept(const unsigned char* exit_mask, const void* h, long 
  * head's argmax, -1 if none; entropy fp32 [M] = that head's entropy, NaN if none; rows_in int32 [n_heads] =
  * the number of rows each head was evaluated on (head usage = rows_in[k] - rows_in[k+1]).
  * Of each ee_head the output pointers are ignored and tau_per_row must be NULL.  The row counts stay on the
- * device: no synchronisation between heads; head k's weights are streamed once whatever the count.  Above 128
- * rows its LayerNorm and statistics run on the surviving rows only (three launches per head).  With at most 128
- * rows (one row tile, where open rows and all rows cost the same) the heads are evaluated on every row, four
- * heads per launch, and a row takes the first head that answers it: same results, two launches plus one small
- * one per four heads.  Workspace: ee_cascade_workspace_bytes(M, d, V), 256-byte aligned, initialised once with
+ * device: no synchronisation between heads; head k's weights are streamed once whatever the count.  Above 512
+ * rows its LayerNorm and statistics run on the surviving rows only (three launches per head).  With at most 512
+ * rows (where the weight stream and the chain of launches, not the rows, set the time) the heads are evaluated
+ * on every row, four heads per launch, and a row takes the first head that answers it: same results, two
+ * launches plus one small one per four heads.  Workspace: ee_cascade_workspace_bytes(M, d, V), 256-byte aligned, initialised once with
  * ee_workspace_init.  M = 0 writes rows_in = 0.
  */
 size_t    ee_cascade_workspace_bytes(int M, int d, int V);      /* host-only, pure; 0 if a size is invalid */

@@ -67,11 +67,11 @@ __global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsign
 }
 
 // Small batches (M <= kSelectThreads): up to four heads have been evaluated on EVERY row of the batch (a head's
-// weights are streamed once whatever the number of rows, and one 128-row tile costs the tensor pipe the same
-// full or not), and this kernel walks them in order for each row: a row still open takes the first head of the
-// group that answers it.  Between groups the state of a row is its exit_head entry (n_heads = still open).
-// One CTA, thread = row; head k of the group has its results at argmax0 / entropy0 / mask0 + k * stride bytes.
-constexpr int kSelectThreads = 128;
+// weights are streamed once whatever the number of rows), and this kernel walks them in order for each row: a
+// row still open takes the first head of the group that answers it.  Between groups the state of a row is its
+// exit_head entry (n_heads = still open).  One CTA of M threads rounded up to whole warps, thread = row; head k
+// of the group has its results at argmax0 / entropy0 / mask0 + k * stride bytes.
+constexpr int kSelectThreads = 1024;
 
 __global__ void __launch_bounds__(kSelectThreads) cascade_select_kernel(const unsigned char* __restrict__ mask0,
                                                                         const unsigned char* __restrict__ argmax0,
@@ -110,7 +110,7 @@ ee_status cascade_select_launch(const unsigned char* mask0, const int* argmax0, 
                                 int k0, int n, int n_heads, int* exit_head, int* token, float* entropy_out, int* rows_in,
                                 cudaStream_t stream) {
     if (M > kSelectThreads) return EE_ERR_SHAPE;
-    return launch_pdl(cascade_select_kernel, 1, kSelectThreads, 0, stream, mask0, reinterpret_cast<const unsigned char*>(argmax0),
+    return launch_pdl(cascade_select_kernel, 1, (M + 31) / 32 * 32, 0, stream, mask0, reinterpret_cast<const unsigned char*>(argmax0),
                       reinterpret_cast<const unsigned char*>(entropy0), stride, M, k0, n, n_heads, exit_head, token,
                       entropy_out, rows_in) == cudaSuccess
                ? EE_OK

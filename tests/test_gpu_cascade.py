@@ -40,7 +40,8 @@ def _fragile_rows(ref, taus):
 
 
 @pytest.mark.parametrize("M,d,V,K", [(24, 64, 300, 3), (1, 64, 129, 2), (100, 256, 1000, 4), (600, 128, 700, 3), (1100, 64, 520, 2),
-                                     (128, 64, 700, 6), (37, 128, 515, 9), (129, 64, 300, 5)])   # groups of four heads below 129 rows
+                                     (128, 64, 700, 6), (37, 128, 515, 9), (129, 64, 300, 5), (512, 64, 520, 5), (513, 64, 520, 3)])
+# up to 512 rows: every head on every row, in groups of four; above: head by head on the open rows
 def test_cascade_matches_oracle(ee, M, d, V, K):
     cfg, h_list = _case(3 + M, M, d, V, K)
     taus = [0.6 + 0.7 * k for k in range(K)]
