@@ -306,6 +306,32 @@ def roofline(wl: Workload, head_call_us: float, peaks: dict, src: str) -> dict:
                 frac_of_sustained=round(tfs / peaks["bf16_tflops_sustained"], 4), hbm_frac=round(gbs / peaks["hbm_gbs"], 4))
 
 
+def measure_read_stream(peaks: dict, src: str, gib: float = 1.0, calls: int = 20) -> dict:
+    """Rate of a read-only stream over a buffer larger than L2 with the kernels' own weight-streaming mechanism
+    (ee_selftest_read_stream), to set beside the copy figure the fractions are quoted against."""
+    import torch
+    import paper_2407_21082_b200 as ee
+    nbytes = int(gib * (1 << 30))
+    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    buf.fill_(1)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        ee.ee_selftest_read_stream(buf, ws)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(calls):
+        ee.ee_selftest_read_stream(buf, ws)
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / calls
+    status = ee.ee_query_async_error(ws)
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return dict(bytes=nbytes, us_per_pass=round(us, 2), gbs=round(gbs, 1), of_copy_peak=round(gbs / peaks["hbm_gbs"], 4),
+                peak_source=f"of {src}", status=status,
+                note="read-only, one CTA per SM, 12 x 16 KB bulk copies in flight per SM, back-to-back passes over a buffer larger than L2")
+
+
 # --------------------------------------------------------------------------------------------- e2e and CPU baseline
 
 
@@ -694,7 +720,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "stream", "tcgen05", "skinny"], help="force a kernel")
     ap.add_argument("--sweep", action="store_true", help="time every kernel that accepts the size, for c1 at several M")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-config table and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["calibration", "cascade", "dssd_round", "kl_loss"],
+    ap.add_argument("--only", default=None, choices=["calibration", "cascade", "dssd_round", "kl_loss", "read_stream"],
                     help="run that entry of the table alone and print its JSON (for profiling one kernel family)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -736,6 +762,7 @@ def main():
             entry = {"calibration": lambda: measure_calibration(peaks, peak_src),
                      "cascade": lambda: measure_cascade(peaks, peak_src, M=args.rows or 64),
                      "dssd_round": lambda: measure_dssd_round(peaks, peak_src),
+                     "read_stream": lambda: measure_read_stream(peaks, peak_src),
                      "kl_loss": lambda: [measure_kl(peaks, peak_src, m) for m in rows]}[args.only]()
             print(json.dumps({args.only: entry}))
         if dist is not None:
@@ -793,6 +820,7 @@ def main():
             del w
             torch.cuda.empty_cache()
         line["configs"] = extra
+        line["roofline"]["read_stream"] = measure_read_stream(peaks, peak_src)
         line["calibration"] = measure_calibration(peaks, peak_src)
         line["cascade"] = measure_cascade(peaks, peak_src)
         line["dssd_round"] = measure_dssd_round(peaks, peak_src)

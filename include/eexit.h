@@ -386,6 +386,18 @@ ee_status ee_query_async_error(void* workspace, void* stream);
  */
 ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Diagnostic for the roofline (no counterpart in the paper): reads `bytes` bytes (rounded down to whole 16 KB
+ * stages; at least one) of the device buffer `buffer` (16-byte aligned) once, with the mechanism the kernels
+ * stream weights with -- one CTA per SM, contiguous bulk asynchronous copies into a shared-memory ring -- and
+ * looks at none of them.  Timed by the caller over a buffer larger than L2 it gives the rate a read-only
+ * stream reaches on this device, to set beside the copy figure the roofline fractions are quoted against.
+ * Writes nothing but the error word of `workspace`'s control block if a bounded wait gives up
+ * (ee_query_async_error reports it).  Asynchronous on `stream`.
+ */
+ee_status ee_selftest_read_stream(const void* buffer, size_t bytes, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -67,6 +67,7 @@ PROTOTYPES = {
     "ee_calibrate": (C.c_int, [_p, _p, _p, C.c_int, C.c_double, _p, _p, _p, C.c_size_t, _p]),
     "ee_query_async_error": (C.c_int, [_p, _p]),
     "ee_selftest_wait_timeout": (C.c_int, [_p, C.c_size_t, _p]),
+    "ee_selftest_read_stream": (C.c_int, [_p, C.c_size_t, _p, C.c_size_t, _p]),
 }
 
 

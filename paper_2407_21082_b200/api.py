@@ -418,6 +418,13 @@ def ee_selftest_wait_timeout(workspace) -> None:
     _check(_lib.load().ee_selftest_wait_timeout(_ptr(workspace), workspace.numel(), _stream()), "ee_selftest_wait_timeout")
 
 
+def ee_selftest_read_stream(buffer, workspace) -> None:
+    """Reads `buffer` (a device tensor) once with the kernels' weight-streaming mechanism (see include/eexit.h);
+    the caller times it."""
+    _check(_lib.load().ee_selftest_read_stream(_ptr(buffer), buffer.numel() * buffer.element_size(), _ptr(workspace),
+                                               workspace.numel(), _stream()), "ee_selftest_read_stream")
+
+
 def _cascade_args(heads, ln_eps, out, workspace):
     n = len(heads)
     arr = (_lib.EEHead * n)()

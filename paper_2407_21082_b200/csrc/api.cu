@@ -541,6 +541,17 @@ ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, voi
     return selftest_wait_timeout_launch(workspace, static_cast<cudaStream_t>(stream));
 }
 
+ee_status ee_selftest_read_stream(const void* buffer, size_t bytes, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!buffer || !workspace) return EE_ERR_NULL;
+    if (!aligned(buffer, 16) || !aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (bytes < 16384) return EE_ERR_SHAPE;
+    if (workspace_bytes_ < (size_t)kCtrlBytes) return EE_ERR_WORKSPACE;
+    int device, num_sms;
+    const ee_status dev = current_device(&device, &num_sms);
+    if (dev != EE_OK) return dev;
+    return selftest_read_stream_launch(buffer, bytes, workspace, num_sms, static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_query_async_error(void* workspace, void* stream) {
     if (!workspace) return EE_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

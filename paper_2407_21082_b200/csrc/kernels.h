@@ -101,6 +101,7 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
 
 // ---- diagnostic: a bounded wait that is made to give up ----
 ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
+ee_status selftest_read_stream_launch(const void* src, size_t bytes, void* workspace, int num_sms, cudaStream_t stream);
 
 // ---- one step of the cascade of heads: rows answered by head k are recorded, the others move on ----
 int cascade_select_max_rows();

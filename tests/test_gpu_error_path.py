@@ -34,3 +34,19 @@ def test_a_wait_that_runs_out_is_reported_and_nothing_else_breaks():
     with pytest.raises(ee.EExitError) as e:
         ee.ee_selftest_wait_timeout(torch.zeros(64, dtype=torch.uint8, device="cuda"))
     assert e.value.code == 4
+
+
+def test_read_stream_diagnostic_runs_clean_and_checks_its_arguments():
+    import paper_2407_21082_b200 as ee
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    for nbytes in (16384, 16384 * 148 + 5000, 64 << 20):      # one stage, a ragged split over the SMs, larger than the rings
+        buf = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        ee.ee_selftest_read_stream(buf, ws)
+        ee.ee_selftest_read_stream(buf, ws)
+        assert ee.ee_query_async_error(ws) == 0
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_selftest_read_stream(torch.zeros(1000, dtype=torch.uint8, device="cuda"), ws)
+    assert e.value.code == 2
+    with pytest.raises(ee.EExitError) as e:
+        ee.ee_selftest_read_stream(torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")[8:], ws)
+    assert e.value.code == 3
