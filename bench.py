@@ -259,6 +259,12 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
 # while the SHA-256 of those sources still matches and as null afterwards.
 CSRC = os.path.join(ROOT, "paper_2407_21082_b200", "csrc")
 TRAFFIC = {
+    ("c0", 8): dict(bytes=51654144 + 5632, heads_per_launch=1, kernel="exit_head_gemm_kernel<0>",
+                    sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
+                    sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c0_c3.md"),
+    ("c3", 256): dict(bytes=521996032 + 4496128, heads_per_launch=2, kernel="exit_head_gemm_kernel<0> (CTA pairs)",
+                      sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
+                      sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c0_c3.md"),
     ("c1", 64): dict(bytes=309865728 + 3677696, heads_per_launch=3, kernel="exit_head_gemm_kernel<0>",
                      sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
                      sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
