@@ -820,9 +820,11 @@ def main():
             w = Workload(name, rows, seed=0, n_copies=copies)
             r = measure(w, steps, 5)
             key = name if rows is None else f"{name}_M{rows}"
+            roof = roofline(w, r["head_call_us"], peaks, peak_src)
+            roof["traffic"], roof["traffic_note"] = measured_traffic(w)      # per launch, like the headline's
             extra[key] = dict(M=w.M, d=w.d, heads=len(w.heads), head_call_us=round(r["head_call_us"], 2),
                               tail_us=round(r["tail_us"], 2), tokens_per_s=w.M / (r["head_call_us"] * 1e-6),
-                              roofline=roofline(w, r["head_call_us"], peaks, peak_src), launches_per_head=w.head_launches)
+                              roofline=roof, launches_per_head=w.head_launches)
             del w
             torch.cuda.empty_cache()
         line["configs"] = extra
