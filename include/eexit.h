@@ -255,7 +255,9 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
  * follows) and once for the verification pass (which = 1: n_rows = S * (k + 1) tokens, row (s, j) = the token
  * before draft position j, j = k being the bonus position); it must enqueue on `stream` work that writes the
  * hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING those tokens to h_out, and return 0.
- * Both pointers it receives are device buffers inside `workspace`.
+ * Both pointers it receives are device buffers inside `workspace`.  The work it enqueues must be ordinary stream
+ * work (kernels launched without programmatic stream serialization that do not trigger their dependents early):
+ * the round's own kernels rely on the model's work starting after, and finishing before, its neighbours.
  *   drafting step j : draft head (heads' gamma, beta, W; draft_head.tau is the threshold) on the step's hidden
  *                     states; argmax = drafted token, exit decision = confidence; the token feeds step j + 1
  *   verification    : verify head (the full model's; its tau is ignored) on all S * (k + 1) rows
@@ -290,6 +292,20 @@ typedef struct {
 } ee_dssd_round_args;
 size_t    dssd_round_workspace_bytes(int S, int k, int d, int V);     /* host-only, pure; 0 if a size is invalid */
 ee_status dssd_round(const ee_dssd_round_args* args);
+
+/*
+ * A ready-made ee_hidden_fn for tests and benchmarks (no counterpart in the paper; the transformer is the
+ * caller's): the hidden state of a row is row `token` of a table, table[0] for the drafting steps (which = 0)
+ * and table[1] for the verification pass (which = 1), each bf16 [V, d] on the device, contiguous, 16-byte
+ * aligned; a token outside [0, V) gives a zero row.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a
+ * pointer to an ee_hidden_tables (host memory that outlives the call) as `hidden_user`.  One kernel launch on
+ * `stream` per call; returns 0, or 1 if an argument is unusable or the launch failed.
+ */
+typedef struct {
+    const void* table[2];
+    int d, V;
+} ee_hidden_tables;
+int ee_hidden_from_tables(void* user, const int* tokens, int n_rows, int which, void* h_out, void* stream);
 
 /*
  * ee_compact and dssd_accept in one kernel launch, for a decoding step that needs both (section 3.4.2 and

@@ -29,6 +29,11 @@ class EEDssdRoundArgs(C.Structure):
                 ("stream", _p)]
 
 
+class EEHiddenTables(C.Structure):
+    """Mirror of `ee_hidden_tables` in include/eexit.h."""
+    _fields_ = [("table", _p * 2), ("d", C.c_int), ("V", C.c_int)]
+
+
 PROTOTYPES = {
     "ee_status_string": (C.c_char_p, [C.c_int]),
     "ee_exit_head_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
@@ -55,6 +60,7 @@ PROTOTYPES = {
     "dssd_commit": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, C.c_int, _p, C.c_int, _p, _p, _p, _p, _p, _p, _p]),
     "dssd_round_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "dssd_round": (C.c_int, [C.POINTER(EEDssdRoundArgs)]),
+    "ee_hidden_from_tables": (C.c_int, [_p, _p, C.c_int, C.c_int, _p, _p]),
     "ee_compact_accept": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p,
                                     _p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "ee_head_kl_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),

@@ -517,6 +517,21 @@ def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos_token, state: dict, 
     return out
 
 
+class TableModel:
+    """Stand-in model for dssd_round served by the library itself (ee_hidden_from_tables in include/eexit.h): the
+    hidden state after a token is that token's row of `draft_table` (drafting steps) or `verify_table`
+    (verification pass), bf16 [V, d] device tensors.  Pass it to DssdRound as `hidden_fn`."""
+
+    def __init__(self, draft_table, verify_table):
+        self.tables = (_bf16(_dev(draft_table, "draft_table")), _bf16(_dev(verify_table, "verify_table")))
+        if self.tables[0].shape != self.tables[1].shape or not all(t.is_contiguous() for t in self.tables):
+            raise ValueError("tables must be contiguous and of one shape [V, d]")
+        V, d = self.tables[0].shape
+        self.struct = _lib.EEHiddenTables()
+        self.struct.table[0], self.struct.table[1] = _ptr(self.tables[0]), _ptr(self.tables[1])
+        self.struct.d, self.struct.V = d, V
+
+
 class DssdRound:
     """dssd_round (see include/eexit.h) with its argument block built once.
 
@@ -548,17 +563,20 @@ class DssdRound:
                 traceback.print_exc()
                 return 1
 
-        self._cb = _lib.HIDDEN_FN(trampoline)
+        native = isinstance(hidden_fn, TableModel)
+        if native and hidden_fn.tables[0].shape != (V, d):
+            raise ValueError("the table model's tables must be [V, d]")
+        self._cb = C.cast(_lib.load().ee_hidden_from_tables, _lib.HIDDEN_FN) if native else _lib.HIDDEN_FN(trampoline)
         a = _lib.EEDssdRoundArgs()
         a.S, a.k, a.d, a.V, a.ln_eps, a.eos_token = S, int(k), d, V, float(ln_eps), int(eos_token)
         for dst, src, W in ((a.draft_head, draft_head, Wd), (a.verify_head, verify_head, Wv)):
             dst.gamma, dst.beta, dst.W, dst.tau = _ptr(src["gamma"]), _ptr(src["beta"]), _ptr(W), float(src.get("tau", 0.0))
-        a.hidden, a.hidden_user = self._cb, None
+        a.hidden, a.hidden_user = self._cb, (C.cast(C.pointer(hidden_fn.struct), C.c_void_p) if native else None)
         a.last_tok, a.out_tok, a.capacity = _ptr(state["last_tok"]), _ptr(state["out_tok"]), state["out_tok"].shape[1]
         a.seq_len, a.finished, a.stats = _ptr(state["seq_len"]), _ptr(state["finished"]), _ptr(state["stats"])
         a.draft_len, a.accept_len, a.next_tok = (_ptr(self.out[n]) for n in ("draft_len", "accept_len", "next_tok"))
         a.workspace, a.workspace_bytes, a.stream = _ptr(workspace), workspace.numel(), _stream()
-        self._args, self._keep = a, (Wd, Wv, draft_head, verify_head, C)
+        self._args, self._keep = a, (Wd, Wv, draft_head, verify_head, C, hidden_fn)
 
     def __call__(self):
         import ctypes as C

@@ -541,6 +541,11 @@ ee_status ee_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, voi
     return selftest_wait_timeout_launch(workspace, static_cast<cudaStream_t>(stream));
 }
 
+int ee_hidden_from_tables(void* user, const int* tokens, int n_rows, int which, void* h_out, void* stream) {
+    return hidden_from_tables(static_cast<const ee_hidden_tables*>(user), tokens, n_rows, which, h_out,
+                              static_cast<cudaStream_t>(stream));
+}
+
 ee_status ee_selftest_read_stream(const void* buffer, size_t bytes, void* workspace, size_t workspace_bytes_, void* stream) {
     if (!buffer || !workspace) return EE_ERR_NULL;
     if (!aligned(buffer, 16) || !aligned(workspace, 256)) return EE_ERR_ALIGN;

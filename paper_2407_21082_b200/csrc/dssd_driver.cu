@@ -141,4 +141,30 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
     return EE_OK;
 }
 
+// Stand-in for the caller's model: the hidden state of a row is row `token` of a table (a token outside the
+// table gives a zero row).  Warp per row, 16-byte vectors.
+namespace {
+__global__ void __launch_bounds__(256) hidden_from_table_kernel(const uint4* __restrict__ table, int V, int nvec,
+                                                                const int* __restrict__ tokens, int n_rows,
+                                                                uint4* __restrict__ h_out) {
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= n_rows) return;
+    const int t = tokens[r];
+    const bool in = t >= 0 && t < V;
+    for (int c = lane; c < nvec; c += 32) h_out[(size_t)r * nvec + c] = in ? __ldg(table + (size_t)t * nvec + c) : make_uint4(0, 0, 0, 0);
+}
+}  // namespace
+
+int hidden_from_tables(const ee_hidden_tables* m, const int* tokens, int n_rows, int which, void* h_out, cudaStream_t stream) {
+    if (!m || !tokens || !h_out || which < 0 || which > 1 || !m->table[which]) return 1;
+    if (m->d < 8 || (m->d % 8) != 0 || m->V < 1 || n_rows < 0) return 1;
+    if ((reinterpret_cast<uintptr_t>(m->table[which]) & 15) != 0) return 1;
+    if (n_rows == 0) return 0;
+    // An ordinary launch, like any kernel of a caller's model: it starts when everything before it in the stream
+    // has finished and what follows starts when it has.
+    hidden_from_table_kernel<<<(n_rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(m->table[which]), m->V, m->d / 8,
+                                                                  tokens, n_rows, static_cast<uint4*>(h_out));
+    return cudaGetLastError() == cudaSuccess ? 0 : 1;
+}
+
 }  // namespace ee

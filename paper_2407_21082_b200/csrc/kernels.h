@@ -100,6 +100,7 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
                                                 size_t ws_bytes, void* stream));
 
 // ---- diagnostic: a bounded wait that is made to give up ----
+int hidden_from_tables(const ee_hidden_tables* m, const int* tokens, int n_rows, int which, void* h_out, cudaStream_t stream);
 ee_status selftest_wait_timeout_launch(void* workspace, cudaStream_t stream);
 ee_status selftest_read_stream_launch(const void* src, size_t bytes, void* workspace, int num_sms, cudaStream_t stream);
 
