@@ -172,11 +172,29 @@ ee_status ee_exit_head_host(const void* h_host, void* h_dev, const float* gamma,
  *   - All calls on a device share the one array, which keeps the previous call's contents; the kernel
  *     rewrites what it reads and leaves the control block zeroed.  Calls that overlap on the GPU (two
  *     streams, two host threads) therefore race: order them on one stream or with events.
+ *   - A bounded device-side wait that gives up is recorded in the array's control block, which the caller
+ *     cannot address: ee_exit_head_static_query_error reads it (ee_query_async_error needs a workspace pointer
+ *     and does not apply here).
  */
 #define EE_STATIC_MAX_ROWS 32
 ee_status ee_exit_head_static(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
                               const void* W, int M, int d, int V, const float* tau_per_row, float tau,
                               int* argmax, float* entropy, float* maxprob, unsigned char* exit_mask, void* stream);
+
+/*
+ * ee_query_async_error for the built-in array of ee_exit_head_static on the current device (no counterpart in the
+ * paper): synchronises `stream`, returns EE_OK if no wait gave up since the last query, else EE_ERR_TIMEOUT -- the
+ * outputs of that call are undefined -- after zeroing the array's whole control block on `stream`, which is the
+ * recovery step: the next ee_exit_head_static call starts from a clean state.  Allocates nothing.
+ */
+ee_status ee_exit_head_static_query_error(void* stream);
+
+/*
+ * ee_selftest_wait_timeout aimed at the built-in array (diagnostic, no counterpart in the paper): one small kernel
+ * whose only wait runs out after about a millisecond and records the error word there; nothing faults.  The next
+ * ee_exit_head_static_query_error returns EE_ERR_TIMEOUT.  For tests of a caller's error handling.
+ */
+ee_status ee_exit_head_static_selftest_timeout(void* stream);
 
 /*
  * ee_exit_head_multi for a caller whose activations and results live in HOST memory: one copy in, the heads,
@@ -255,9 +273,12 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
  * follows) and once for the verification pass (which = 1: n_rows = S * (k + 1) tokens, row (s, j) = the token
  * before draft position j, j = k being the bonus position); it must enqueue on `stream` work that writes the
  * hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING those tokens to h_out, and return 0.
- * Both pointers it receives are device buffers inside `workspace`.  The work it enqueues must be ordinary stream
- * work (kernels launched without programmatic stream serialization that do not trigger their dependents early):
- * the round's own kernels rely on the model's work starting after, and finishing before, its neighbours.
+ * Both pointers it receives are device buffers inside `workspace`.  The work it enqueues may be ordinary stream
+ * work, or kernels launched with programmatic stream serialization that trigger their dependents early -- the
+ * round's own kernels are chained that way -- provided every such kernel executes griddepcontrol.wait before it
+ * reads `tokens` or writes `h_out`, and reads `tokens` through L2 (ld.global.cg or an equivalent coherent load,
+ * not the read-only path): the token buffer is rewritten by a kernel that may still be running when the model's
+ * kernel becomes resident.
  *   drafting step j : draft head (heads' gamma, beta, W; draft_head.tau is the threshold) on the step's hidden
  *                     states; argmax = drafted token, exit decision = confidence; the token feeds step j + 1
  *   verification    : verify head (the full model's; its tau is ignored) on all S * (k + 1) rows
@@ -299,11 +320,14 @@ ee_status dssd_round(const ee_dssd_round_args* args);
  * and table[1] for the verification pass (which = 1), each bf16 [V, d] on the device, contiguous, 16-byte
  * aligned; a token outside [0, V) gives a zero row.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a
  * pointer to an ee_hidden_tables (host memory that outlives the call) as `hidden_user`.  One kernel launch on
- * `stream` per call; returns 0, or 1 if an argument is unusable or the launch failed.
+ * `stream` per call; returns 0, or 1 if an argument is unusable or the launch failed.  chained = 0: an ordinary
+ * launch; chained != 0: the kernel is launched with programmatic stream serialization, lets its dependents start
+ * at once and waits for its predecessors before it touches the tokens, like the library's own kernels.
  */
 typedef struct {
     const void* table[2];
     int d, V;
+    int chained;
 } ee_hidden_tables;
 int ee_hidden_from_tables(void* user, const int* tokens, int n_rows, int which, void* h_out, void* stream);
 

@@ -31,7 +31,7 @@ class EEDssdRoundArgs(C.Structure):
 
 class EEHiddenTables(C.Structure):
     """Mirror of `ee_hidden_tables` in include/eexit.h."""
-    _fields_ = [("table", _p * 2), ("d", C.c_int), ("V", C.c_int)]
+    _fields_ = [("table", _p * 2), ("d", C.c_int), ("V", C.c_int), ("chained", C.c_int)]
 
 
 PROTOTYPES = {
@@ -55,6 +55,8 @@ PROTOTYPES = {
                                           _p, _p, _p, _p, _p, C.c_size_t, _p]),
     "ee_exit_head_static": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                       _p, _p, _p, _p, _p]),
+    "ee_exit_head_static_query_error": (C.c_int, [_p]),
+    "ee_exit_head_static_selftest_timeout": (C.c_int, [_p]),
     "ee_compact": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_commit": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, C.c_int, _p, C.c_int, _p, _p, _p, _p, _p, _p, _p]),

@@ -77,12 +77,41 @@ def new_outputs(M: int, device="cuda") -> dict:
                 exit_mask=torch.empty(M, dtype=torch.uint8, device=device))
 
 
-def _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path):
+_OUT_DTYPES = dict(argmax=torch.int32, entropy=torch.float32, maxprob=torch.float32, exit_mask=torch.uint8)
+
+
+def _check_head_tensors(h, gamma, beta, W, tau, out=None):
+    """Host-side checks shared by the single-head wrappers: everything the kernels take on trust (shapes, strides,
+    dtypes, devices) is verified here, so that a bad argument raises ValueError instead of reaching the device.
+    Returns h and W as bf16 tensors and (M, d, V)."""
     h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
+    if h.dim() != 2 or W.dim() != 2:
+        raise ValueError("h must be [M, d] and W [V, d]")
     M, d = h.shape
     V = W.shape[0]
-    if W.shape[1] != d or not W.is_contiguous() or h.stride(1) != 1:
+    if W.shape[1] != d or not W.is_contiguous() or (M > 0 and h.stride(1) != 1):
         raise ValueError("W must be contiguous [V, d] and h row-major [M, d]")
+    for name, t in (("gamma", gamma), ("beta", beta)):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.numel() == d):
+            raise ValueError(f"{name} must be a contiguous float32 CUDA tensor of d = {d} elements")
+        if t.device != h.device:
+            raise ValueError(f"{name} is on {t.device}, h on {h.device}")
+    if W.device != h.device:
+        raise ValueError(f"W is on {W.device}, h on {h.device}")
+    if isinstance(tau, torch.Tensor):
+        if not (tau.is_cuda and tau.device == h.device and tau.dtype == torch.float32 and tau.is_contiguous() and tau.numel() == M):
+            raise ValueError(f"a per-row tau must be a contiguous float32 CUDA tensor of M = {M} elements")
+    if out is not None:
+        for name, dtype in _OUT_DTYPES.items():
+            t = out.get(name)
+            if not (isinstance(t, torch.Tensor) and t.is_cuda and t.device == h.device and t.dtype == dtype and
+                    t.is_contiguous() and t.numel() >= M):
+                raise ValueError(f"out[{name!r}] must be a contiguous {dtype} CUDA tensor of at least M = {M} elements")
+    return h, W, (M, d, V)
+
+
+def _exit_head_args(h, gamma, beta, ln_eps, W, tau, out, workspace, path):
+    h, W, (M, d, V) = _check_head_tensors(h, gamma, beta, W, tau, out)
     out = out if out is not None else new_outputs(M, h.device)
     workspace = workspace if workspace is not None else new_workspace(M, d, V, h.device)
     tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
@@ -183,9 +212,7 @@ class PreparedMulti:
 
 def ee_exit_head_top2(h, gamma, beta, ln_eps, W, tau, *, out=None, workspace=None) -> dict:
     """ee_exit_head plus out["top2gap"]: the difference between the two largest probabilities of every row."""
-    h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
-    M, d = h.shape
-    V = W.shape[0]
+    h, W, (M, d, V) = _check_head_tensors(h, gamma, beta, W, tau, out)
     if out is None:
         out = new_outputs(M, h.device)
         out["top2gap"] = torch.empty(M, dtype=torch.float32, device=h.device)
@@ -268,14 +295,24 @@ def ee_exit_head_static(h, gamma, beta, ln_eps, W, tau, *, out: dict) -> dict:
     The library's built-in scratch array is used, so nothing is allocated by the call.  `out` must be given
     (see new_outputs) -- this wrapper creates no tensors either.  Calls sharing a GPU must not overlap.
     """
-    h, W = _bf16(_dev(h, "h")), _bf16(_dev(W, "W"))
-    M, d = h.shape
+    h, W, (M, d, V) = _check_head_tensors(h, gamma, beta, W, tau, out)
     tau_t, tau_f = (tau, 0.0) if isinstance(tau, torch.Tensor) else (None, float(tau))
     _check(_lib.load().ee_exit_head_static(
         _ptr(h), h.stride(0) if M > 1 else max(h.stride(0), d), _ptr(gamma), _ptr(beta), float(ln_eps), _ptr(W),
-        M, d, W.shape[0], _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
+        M, d, V, _ptr(tau_t), tau_f, _ptr(out["argmax"]), _ptr(out["entropy"]), _ptr(out["maxprob"]),
         _ptr(out["exit_mask"]), _stream()), "ee_exit_head_static")
     return out
+
+
+def ee_exit_head_static_query_error() -> int:
+    """ee_query_async_error for the built-in array of ee_exit_head_static: synchronises the current stream; 0, or
+    EE_ERR_TIMEOUT after putting the array's control block back to its initial state."""
+    return int(_lib.load().ee_exit_head_static_query_error(_stream()))
+
+
+def ee_exit_head_static_selftest_timeout() -> None:
+    """Makes one bounded wait give up against the built-in array (see include/eexit.h)."""
+    _check(_lib.load().ee_exit_head_static_selftest_timeout(_stream()), "ee_exit_head_static_selftest_timeout")
 
 
 def _exit_head_host_args(h_host, h_dev, gamma, beta, ln_eps, W, tau, out_host, out_dev, workspace):
@@ -520,16 +557,17 @@ def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos_token, state: dict, 
 class TableModel:
     """Stand-in model for dssd_round served by the library itself (ee_hidden_from_tables in include/eexit.h): the
     hidden state after a token is that token's row of `draft_table` (drafting steps) or `verify_table`
-    (verification pass), bf16 [V, d] device tensors.  Pass it to DssdRound as `hidden_fn`."""
+    (verification pass), bf16 [V, d] device tensors.  Pass it to DssdRound as `hidden_fn`.  chained=True launches
+    its kernel with programmatic stream serialization (early trigger, wait before the tokens are read)."""
 
-    def __init__(self, draft_table, verify_table):
+    def __init__(self, draft_table, verify_table, chained: bool = False):
         self.tables = (_bf16(_dev(draft_table, "draft_table")), _bf16(_dev(verify_table, "verify_table")))
         if self.tables[0].shape != self.tables[1].shape or not all(t.is_contiguous() for t in self.tables):
             raise ValueError("tables must be contiguous and of one shape [V, d]")
         V, d = self.tables[0].shape
         self.struct = _lib.EEHiddenTables()
         self.struct.table[0], self.struct.table[1] = _ptr(self.tables[0]), _ptr(self.tables[1])
-        self.struct.d, self.struct.V = d, V
+        self.struct.d, self.struct.V, self.struct.chained = d, V, int(bool(chained))
 
 
 class DssdRound:

@@ -14,26 +14,26 @@ constexpr int kStepRows = 32;             // one ballot's worth of rows per CTA
 // Row j < m of this step is row idx_in[j] of the batch (j itself when idx_in is NULL).  CTA b owns rows
 // [32 b, 32 b + 32): it counts the survivors before its rows itself from the mask (L2-resident), so no CTA
 // waits for another.  Rows the last head leaves unanswered are marked with exit_head = n_heads.
-__global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsigned char* __restrict__ exit_mask,
-                                                                    const int* __restrict__ argmax,
-                                                                    const float* __restrict__ entropy,
-                                                                    const int* __restrict__ idx_in,
-                                                                    const int* __restrict__ m_in, int M, int k,
+__global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsigned char* exit_mask,
+                                                                    const int* argmax,
+                                                                    const float* entropy,
+                                                                    const int* idx_in,
+                                                                    const int* m_in, int M, int k,
                                                                     int is_last, int n_heads,
-                                                                    int* __restrict__ exit_head, int* __restrict__ token,
-                                                                    float* __restrict__ entropy_out,
-                                                                    int* __restrict__ idx_out, int* __restrict__ m_out,
-                                                                    int* __restrict__ rows_in) {
+                                                                    int* exit_head, int* token,
+                                                                    float* entropy_out,
+                                                                    int* idx_out, int* m_out,
+                                                                    int* rows_in) {
     __shared__ int s_warp_cnt[kStepThreads / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     launch_dependents();
     grid_dependency_wait();
-    const int m = m_in ? min(max(*m_in, 0), M) : M;
+    const int m = m_in ? min(max(ld_dep(m_in), 0), M) : M;
     const int row0 = blockIdx.x * kStepRows;
     if (blockIdx.x == 0 && threadIdx.x == 0) rows_in[k] = m;
     int cnt = 0;
     const int upto = min(row0, m);
-    for (int i = threadIdx.x; i < upto; i += kStepThreads) cnt += (exit_mask[i] == 0);
+    for (int i = threadIdx.x; i < upto; i += kStepThreads) cnt += (ld_dep(exit_mask + i) == 0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     if (lane == 0) s_warp_cnt[warp] = cnt;
@@ -44,14 +44,14 @@ __global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsign
     for (int w = 0; w < kStepThreads / 32; ++w) base += s_warp_cnt[w];
     const int j = row0 + lane;
     const bool in = j < m;
-    const bool answered = in && exit_mask[j] != 0;
+    const bool answered = in && ld_dep(exit_mask + (in ? j : 0)) != 0;
     const bool moves_on = in && !answered;
     const unsigned int ballot = __ballot_sync(0xffffffffu, moves_on);
-    const int orig = in ? (idx_in ? idx_in[j] : j) : 0;
+    const int orig = in ? (idx_in ? ld_dep(idx_in + j) : j) : 0;
     if (answered) {
         exit_head[orig] = k;
-        token[orig] = argmax[j];
-        entropy_out[orig] = entropy[j];
+        token[orig] = ld_dep(argmax + j);
+        entropy_out[orig] = ld_dep(entropy + j);
     }
     if (moves_on) {
         if (is_last) {
@@ -73,25 +73,25 @@ __global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsign
 // of the group has its results at argmax0 / entropy0 / mask0 + k * stride bytes.
 constexpr int kSelectThreads = 1024;
 
-__global__ void __launch_bounds__(kSelectThreads) cascade_select_kernel(const unsigned char* __restrict__ mask0,
-                                                                        const unsigned char* __restrict__ argmax0,
-                                                                        const unsigned char* __restrict__ entropy0,
+__global__ void __launch_bounds__(kSelectThreads) cascade_select_kernel(const unsigned char* mask0,
+                                                                        const unsigned char* argmax0,
+                                                                        const unsigned char* entropy0,
                                                                         size_t stride, int M, int k0, int n, int n_heads,
-                                                                        int* __restrict__ exit_head, int* __restrict__ token,
-                                                                        float* __restrict__ entropy_out,
-                                                                        int* __restrict__ rows_in) {
+                                                                        int* exit_head, int* token,
+                                                                        float* entropy_out,
+                                                                        int* rows_in) {
     launch_dependents();
     grid_dependency_wait();
     const int i = threadIdx.x;
     const bool in = i < M;
-    bool open = in && (k0 == 0 || exit_head[i] == n_heads);
+    bool open = in && (k0 == 0 || ld_dep(exit_head + (in ? i : 0)) == n_heads);
     for (int k = 0; k < n; ++k) {
         const int cnt = __syncthreads_count(open);
         if (i == 0) rows_in[k0 + k] = cnt;
-        if (open && (mask0 + k * stride)[i] != 0) {
+        if (open && ld_dep(mask0 + k * stride + i) != 0) {
             exit_head[i] = k0 + k;
-            token[i] = reinterpret_cast<const int*>(argmax0 + k * stride)[i];
-            entropy_out[i] = reinterpret_cast<const float*>(entropy0 + k * stride)[i];
+            token[i] = ld_dep(reinterpret_cast<const int*>(argmax0 + k * stride) + i);
+            entropy_out[i] = ld_dep(reinterpret_cast<const float*>(entropy0 + k * stride) + i);
             open = false;
         }
     }

@@ -148,8 +148,10 @@ struct Control {
     unsigned int error_info;  // where it gave up (role << 24 | stage << 16 | low bits of the tile index)
     unsigned int pad0;
     unsigned int head_ticket[8];   // completion counters of the heads of a multi-head launch; return to 0 as well
-    unsigned int merge_seen;  // tensor-core kernel, in-kernel merge: rows merged so far; returns to 0 as well
-    unsigned int pad[51];
+    unsigned int merge_seen;  // unused (kept so that the layout of the words above stays as it was)
+    unsigned int group_ticket[16];   // tensor-core kernel, in-kernel merge: CTAs of each group of 16 that have published
+    unsigned int top_ticket;         // ... and groups whose partial states have been combined; both return to 0
+    unsigned int pad[34];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -160,13 +162,15 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // ---------------------------------------------------------------------------------------------
 // Loads, packing, warp reductions
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
+// Reads of data that an earlier kernel of the stream produced (activations, masks, tokens, counts, partial
+// states).  Under programmatic dependent launch a kernel is resident -- possibly next to the previous launch of
+// itself on the same SM -- before its producer has finished, so such data is not read-only for the kernel's
+// lifetime: the non-coherent path (ld.global.nc, which the compiler also picks for const __restrict__
+// parameters) may return a line an earlier co-resident kernel left in the SM's L1.  These loads go to L2, the
+// point of coherence; the parameters they read through carry no __restrict__.  Weights and LayerNorm
+// parameters, which no kernel of the stream writes, keep the read-only path.
+template <class T>
+__device__ __forceinline__ T ld_dep(const T* p) { return __ldcg(p); }
 
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
@@ -180,92 +184,6 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
-}
-
-// LayerNorm of eight consecutive elements (one 16-byte vector of bf16) -> eight bf16, given the row's
-// mean and reciprocal standard deviation and the eight gammas / betas of these columns.
-__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, float4 g0, float4 g1, float4 b0,
-                                                 float4 b1) {
-    uint4 o;
-    o.x = pack_bf16(fmaf((bf16_lo(v.x) - mu) * rstd, g0.x, b0.x), fmaf((bf16_hi(v.x) - mu) * rstd, g0.y, b0.y));
-    o.y = pack_bf16(fmaf((bf16_lo(v.y) - mu) * rstd, g0.z, b0.z), fmaf((bf16_hi(v.y) - mu) * rstd, g0.w, b0.w));
-    o.z = pack_bf16(fmaf((bf16_lo(v.z) - mu) * rstd, g1.x, b1.x), fmaf((bf16_hi(v.z) - mu) * rstd, g1.y, b1.y));
-    o.w = pack_bf16(fmaf((bf16_lo(v.w) - mu) * rstd, g1.z, b1.z), fmaf((bf16_hi(v.w) - mu) * rstd, g1.w, b1.w));
-    return o;
-}
-
-// Same, reading gamma and beta of vector c (columns 8c .. 8c+7) from global memory.
-__device__ __forceinline__ uint4 layer_norm_vec8(uint4 v, float mu, float rstd, const float* gamma,
-                                                 const float* beta, int c) {
-    const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
-    const float4 g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
-    const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
-    const float4 b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
-    return layer_norm_vec8(v, mu, rstd, g0, g1, b0, b1);
-}
-
-__device__ __forceinline__ float vec8_sum(uint4 v) {
-    return ((bf16_lo(v.x) + bf16_hi(v.x)) + (bf16_lo(v.y) + bf16_hi(v.y))) +
-           ((bf16_lo(v.z) + bf16_hi(v.z)) + (bf16_lo(v.w) + bf16_hi(v.w)));
-}
-
-__device__ __forceinline__ float vec8_sqdev(uint4 v, float mu, float acc) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float a = bf16_lo(w[i]) - mu, b = bf16_hi(w[i]) - mu;
-        acc = fmaf(a, a, acc);
-        acc = fmaf(b, b, acc);
-    }
-    return acc;
-}
-
-// ---------------------------------------------------------------------------------------------
-// LayerNorm of rows that already sit in shared memory as raw bf16 (16-byte vectors reached through
-// vec(row, c)), in place.  A warp keeps R whole rows in registers (up to VPL vectors per lane), so each row is
-// read once and the R dependency chains (two warp reductions each) overlap.  Requires nvec <= 32 * VPL.
-// ---------------------------------------------------------------------------------------------
-template <int R, int VPL, class VecFn>
-__device__ __forceinline__ void layer_norm_rows_in_regs(VecFn vec, const int (&rows)[R], int n_rows, int nvec, float inv_d,
-                                                        float ln_eps, const float* gamma_s, const float* beta_s,
-                                                        int lane) {
-    uint4 x[R][VPL];
-    float mu[R], rstd[R];
-#pragma unroll
-    for (int i = 0; i < R; ++i) {
-        float sum = 0.f;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int c = lane + 32 * k;
-            x[i][k] = (i < n_rows && c < nvec) ? *vec(rows[i], c) : make_uint4(0, 0, 0, 0);
-            sum += vec8_sum(x[i][k]);
-        }
-        mu[i] = sum;
-    }
-#pragma unroll
-    for (int i = 0; i < R; ++i) mu[i] = warp_sum(mu[i]) * inv_d;
-#pragma unroll
-    for (int i = 0; i < R; ++i) {
-        float sq = 0.f;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k)
-            if (lane + 32 * k < nvec) sq = vec8_sqdev(x[i][k], mu[i], sq);
-        rstd[i] = sq;
-    }
-#pragma unroll
-    for (int i = 0; i < R; ++i) rstd[i] = 1.f / sqrtf(warp_sum(rstd[i]) * inv_d + ln_eps);
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-        const int c = lane + 32 * k;
-        if (c < nvec) {
-            const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
-            const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-            const float4 g0 = g4[0], g1 = g4[1], b0 = b4[0], b1 = b4[1];
-#pragma unroll
-            for (int i = 0; i < R; ++i)
-                if (i < n_rows) *vec(rows[i], c) = layer_norm_vec8(x[i][k], mu[i], rstd[i], g0, g1, b0, b1);
-        }
-    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -362,7 +280,7 @@ __device__ __forceinline__ void merge_token_batches(const State* src, bool src_i
         }
         if (lane < TB && tok0 + lane < M) {
             const int tok = tok0 + lane;
-            state_finish(mine, tau_per_row ? tau_per_row[tok] : tau, argmax, entropy, maxprob, exit_mask, tok);
+            state_finish(mine, tau_per_row ? ld_dep(tau_per_row + tok) : tau, argmax, entropy, maxprob, exit_mask, tok);
         }
     }
 }

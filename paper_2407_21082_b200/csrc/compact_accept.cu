@@ -12,10 +12,10 @@ constexpr int kRowsPerCta = 32;           // one ballot's worth of rows per CTA
 
 // CTA b owns rows [32b, 32b + 32).  Its output offset is the number of surviving rows before 32b, which it
 // counts itself from the mask (M bytes at most, L2-resident), so no CTA waits for another.
-__device__ __forceinline__ void compact_body(int cta, const unsigned char* __restrict__ exit_mask,
-                                             const __nv_bfloat16* __restrict__ h, long long ld_h, int M, int d,
-                                             int* __restrict__ kept_idx, int* __restrict__ kept_count,
-                                             __nv_bfloat16* __restrict__ h_out) {
+__device__ __forceinline__ void compact_body(int cta, const unsigned char* exit_mask,
+                                             const __nv_bfloat16* h, long long ld_h, int M, int d,
+                                             int* kept_idx, int* kept_count,
+                                             __nv_bfloat16* h_out) {
     __shared__ int s_warp_cnt[kCompactThreads / 32];
     __shared__ int s_src[kRowsPerCta];
     __shared__ int s_base, s_n;
@@ -23,7 +23,7 @@ __device__ __forceinline__ void compact_body(int cta, const unsigned char* __res
     const int row0 = cta * kRowsPerCta;
 
     int cnt = 0;
-    for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (exit_mask[i] == 0);
+    for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (ld_dep(exit_mask + i) == 0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     if (lane == 0) s_warp_cnt[warp] = cnt;
@@ -33,7 +33,7 @@ __device__ __forceinline__ void compact_body(int cta, const unsigned char* __res
 #pragma unroll
         for (int w = 0; w < kCompactThreads / 32; ++w) base += s_warp_cnt[w];
         const int row = row0 + lane;
-        const bool keep = (row < M) && (exit_mask[row] == 0);
+        const bool keep = (row < M) && (ld_dep(exit_mask + min(row, M - 1)) == 0);
         const unsigned int ballot = __ballot_sync(0xffffffffu, keep);
         const int rank = __popc(ballot & ((1u << lane) - 1u));
         if (keep) {
@@ -52,33 +52,33 @@ __device__ __forceinline__ void compact_body(int cta, const unsigned char* __res
     for (int r = warp; r < s_n; r += kCompactThreads / 32) {
         const uint4* src = reinterpret_cast<const uint4*>(h + (size_t)s_src[r] * ld_h);
         uint4* dst = reinterpret_cast<uint4*>(h_out + (size_t)(s_base + r) * d);
-        for (int c = lane; c < nvec; c += 32) dst[c] = __ldg(src + c);
+        for (int c = lane; c < nvec; c += 32) dst[c] = ld_dep(src + c);
     }
 }
 
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned char* __restrict__ exit_mask,
-                                                                  const __nv_bfloat16* __restrict__ h, long long ld_h,
-                                                                  int M, int d, int* __restrict__ kept_idx,
-                                                                  int* __restrict__ kept_count,
-                                                                  __nv_bfloat16* __restrict__ h_out) {
+__global__ void __launch_bounds__(kCompactThreads) compact_kernel(const unsigned char* exit_mask,
+                                                                  const __nv_bfloat16* h, long long ld_h,
+                                                                  int M, int d, int* kept_idx,
+                                                                  int* kept_count,
+                                                                  __nv_bfloat16* h_out) {
     launch_dependents();
     grid_dependency_wait();                              // the mask and h come from earlier kernels of the stream
     compact_body(blockIdx.x, exit_mask, h, ld_h, M, d, kept_idx, kept_count, h_out);
 }
 
 // One warp per sequence s; lane j looks at draft slot j (slots beyond 32 in further rounds).
-__device__ __forceinline__ void accept_body(int s, int lane, const int* __restrict__ draft_tok,
-                                            const unsigned char* __restrict__ draft_exit_mask,
-                                            const int* __restrict__ verify_tok, int k, int kv,
-                                            int* __restrict__ draft_len, int* __restrict__ accept_len,
-                                            int* __restrict__ next_tok) {
+__device__ __forceinline__ void accept_body(int s, int lane, const int* draft_tok,
+                                            const unsigned char* draft_exit_mask,
+                                            const int* verify_tok, int k, int kv,
+                                            int* draft_len, int* accept_len,
+                                            int* next_tok) {
     int n = k;             // first slot that is not confident (draft length)
     int first_mis = k;     // first slot whose drafted token differs from the verifier's
     for (int base = 0; base < k; base += 32) {
         const int j = base + lane;
         const bool in = j < k;
-        const bool conf = in && (draft_exit_mask == nullptr || draft_exit_mask[(size_t)s * k + j] != 0);
-        const bool same = in && (draft_tok[(size_t)s * k + j] == verify_tok[(size_t)s * kv + j]);
+        const bool conf = in && (draft_exit_mask == nullptr || ld_dep(draft_exit_mask + (size_t)s * k + j) != 0);
+        const bool same = in && (ld_dep(draft_tok + (size_t)s * k + j) == ld_dep(verify_tok + (size_t)s * kv + j));
         const unsigned int stop_b = __ballot_sync(0xffffffffu, in && !conf);
         const unsigned int mis_b = __ballot_sync(0xffffffffu, in && !same);
         if (first_mis == k && mis_b) first_mis = base + __ffs(mis_b) - 1;
@@ -88,15 +88,15 @@ __device__ __forceinline__ void accept_body(int s, int lane, const int* __restri
     if (lane == 0) {
         draft_len[s] = n;
         accept_len[s] = a;
-        next_tok[s] = (a < kv) ? verify_tok[(size_t)s * kv + a] : -1;
+        next_tok[s] = (a < kv) ? ld_dep(verify_tok + (size_t)s * kv + a) : -1;
     }
 }
 
-__global__ void __launch_bounds__(128) accept_kernel(const int* __restrict__ draft_tok,
-                                                     const unsigned char* __restrict__ draft_exit_mask,
-                                                     const int* __restrict__ verify_tok, int S, int k, int kv,
-                                                     int* __restrict__ draft_len, int* __restrict__ accept_len,
-                                                     int* __restrict__ next_tok) {
+__global__ void __launch_bounds__(128) accept_kernel(const int* draft_tok,
+                                                     const unsigned char* draft_exit_mask,
+                                                     const int* verify_tok, int S, int k, int kv,
+                                                     int* draft_len, int* accept_len,
+                                                     int* next_tok) {
     const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
     launch_dependents();
     if (s >= S) return;

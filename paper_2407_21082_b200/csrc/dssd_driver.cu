@@ -14,54 +14,55 @@ namespace {
 
 // After drafting step j: token and confidence of every sequence go to column j of the draft buffers, and the
 // token becomes the next step's input.
-__global__ void __launch_bounds__(256) record_draft_kernel(const int* __restrict__ argmax,
-                                                           const unsigned char* __restrict__ exit_mask, int S, int j, int k,
-                                                           int* __restrict__ draft_tok, unsigned char* __restrict__ draft_mask,
-                                                           int* __restrict__ cur_tok) {
+__global__ void __launch_bounds__(256) record_draft_kernel(const int* argmax,
+                                                           const unsigned char* exit_mask, int S, int j, int k,
+                                                           int* draft_tok, unsigned char* draft_mask,
+                                                           int* cur_tok) {
     launch_dependents();
     const int s = blockIdx.x * 256 + threadIdx.x;
     if (s >= S) return;
     grid_dependency_wait();
-    const int t = argmax[s];
+    const int t = ld_dep(argmax + s);
     draft_tok[(size_t)s * k + j] = t;
-    draft_mask[(size_t)s * k + j] = exit_mask[s];
+    draft_mask[(size_t)s * k + j] = ld_dep(exit_mask + s);
     cur_tok[s] = t;
 }
 
 // The verifier's row (s, j) reads the token before position j: the last committed token for j = 0, the token
 // drafted at j - 1 after that (j = k is the bonus row).
-__global__ void __launch_bounds__(256) verify_inputs_kernel(const int* __restrict__ last_tok,
-                                                            const int* __restrict__ draft_tok, int S, int k,
-                                                            int* __restrict__ prev_all) {
+__global__ void __launch_bounds__(256) verify_inputs_kernel(const int* last_tok,
+                                                            const int* draft_tok, int S, int k,
+                                                            int* prev_all) {
     launch_dependents();
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i >= S * (k + 1)) return;
     grid_dependency_wait();
     const int s = i / (k + 1), j = i - s * (k + 1);
-    prev_all[i] = j == 0 ? last_tok[s] : draft_tok[(size_t)s * k + j - 1];
+    prev_all[i] = j == 0 ? ld_dep(last_tok + s) : ld_dep(draft_tok + (size_t)s * k + j - 1);
 }
 
 // Sequences that took part in the round continue from their last committed token.
-__global__ void __launch_bounds__(256) last_token_kernel(const int* __restrict__ out_tok, int cap,
-                                                         const int* __restrict__ seq_len,
-                                                         const unsigned char* __restrict__ was_finished, int S,
-                                                         int* __restrict__ last_tok) {
+__global__ void __launch_bounds__(256) last_token_kernel(const int* out_tok, int cap,
+                                                         const int* seq_len,
+                                                         const unsigned char* was_finished, int S,
+                                                         int* last_tok) {
     launch_dependents();
     const int s = blockIdx.x * 256 + threadIdx.x;
     if (s >= S) return;
     grid_dependency_wait();
-    if (!was_finished[s] && seq_len[s] > 0) last_tok[s] = out_tok[(size_t)s * cap + seq_len[s] - 1];
+    const int len = ld_dep(seq_len + s);
+    if (!ld_dep(was_finished + s) && len > 0) last_tok[s] = ld_dep(out_tok + (size_t)s * cap + len - 1);
 }
 
-__global__ void __launch_bounds__(256) copy_bytes_kernel(const unsigned char* __restrict__ src, int n,
-                                                         unsigned char* __restrict__ dst, const int* __restrict__ src_i,
-                                                         int* __restrict__ dst_i) {
+__global__ void __launch_bounds__(256) copy_bytes_kernel(const unsigned char* src, int n,
+                                                         unsigned char* dst, const int* src_i,
+                                                         int* dst_i) {
     launch_dependents();
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i >= n) return;
     grid_dependency_wait();
-    dst[i] = src[i];
-    dst_i[i] = src_i[i];
+    dst[i] = ld_dep(src + i);
+    dst_i[i] = ld_dep(src_i + i);
 }
 
 struct Layout {
@@ -142,14 +143,17 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
 }
 
 // Stand-in for the caller's model: the hidden state of a row is row `token` of a table (a token outside the
-// table gives a zero row).  Warp per row, 16-byte vectors.
+// table gives a zero row).  Warp per row, 16-byte vectors.  With `chained` the kernel takes part in the chain of
+// programmatic dependent launches like the library's own kernels: it lets its dependents start at once and waits
+// for its predecessors before it reads the tokens or writes a hidden state.
 namespace {
 __global__ void __launch_bounds__(256) hidden_from_table_kernel(const uint4* __restrict__ table, int V, int nvec,
-                                                                const int* __restrict__ tokens, int n_rows,
-                                                                uint4* __restrict__ h_out) {
+                                                                const int* tokens, int n_rows, uint4* h_out, int chained) {
+    if (chained) launch_dependents();
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= n_rows) return;
-    const int t = tokens[r];
+    if (chained) grid_dependency_wait();
+    const int t = ld_dep(tokens + r);
     const bool in = t >= 0 && t < V;
     for (int c = lane; c < nvec; c += 32) h_out[(size_t)r * nvec + c] = in ? __ldg(table + (size_t)t * nvec + c) : make_uint4(0, 0, 0, 0);
 }
@@ -160,10 +164,13 @@ int hidden_from_tables(const ee_hidden_tables* m, const int* tokens, int n_rows,
     if (m->d < 8 || (m->d % 8) != 0 || m->V < 1 || n_rows < 0) return 1;
     if ((reinterpret_cast<uintptr_t>(m->table[which]) & 15) != 0) return 1;
     if (n_rows == 0) return 0;
+    if (m->chained)
+        return launch_pdl(hidden_from_table_kernel, (n_rows + 7) / 8, 256, 0, stream, static_cast<const uint4*>(m->table[which]),
+                          m->V, m->d / 8, tokens, n_rows, static_cast<uint4*>(h_out), 1) == cudaSuccess ? 0 : 1;
     // An ordinary launch, like any kernel of a caller's model: it starts when everything before it in the stream
     // has finished and what follows starts when it has.
     hidden_from_table_kernel<<<(n_rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(m->table[which]), m->V, m->d / 8,
-                                                                  tokens, n_rows, static_cast<uint4*>(h_out));
+                                                                  tokens, n_rows, static_cast<uint4*>(h_out), 0);
     return cudaGetLastError() == cudaSuccess ? 0 : 1;
 }
 

@@ -9,27 +9,32 @@ namespace ee {
 
 namespace {
 
-__global__ void __launch_bounds__(128) dssd_commit_kernel(const int* __restrict__ draft_tok,
-                                                          const unsigned char* __restrict__ draft_exit_mask,
-                                                          const int* __restrict__ verify_tok, int S, int k, int kv, int eos,
-                                                          int* __restrict__ out_tok, int cap, int* __restrict__ seq_len,
-                                                          unsigned char* __restrict__ finished,
-                                                          int* __restrict__ draft_len, int* __restrict__ accept_len,
-                                                          int* __restrict__ next_tok,
-                                                          unsigned long long* __restrict__ stats) {
+__global__ void __launch_bounds__(128) dssd_commit_kernel(const int* draft_tok,
+                                                          const unsigned char* draft_exit_mask,
+                                                          const int* verify_tok, int S, int k, int kv, int eos,
+                                                          int* out_tok, int cap, int* seq_len,
+                                                          unsigned char* finished,
+                                                          int* draft_len, int* accept_len,
+                                                          int* next_tok,
+                                                          unsigned long long* stats) {
     const int s = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     launch_dependents();
     if (s >= S) return;
     grid_dependency_wait();                              // tokens, masks and the sequences' state come from earlier kernels
-    if (finished[s]) {                                   // a finished sequence takes no part in the round
+    // Lane 0 rewrites finished[s] and seq_len[s] at the end: every lane reads both here, and the warp meets again
+    // before those stores, so no lane can see this round's values.
+    const bool was_finished = ld_dep(finished + s) != 0;
+    const int have = ld_dep(seq_len + s);
+    __syncwarp();
+    if (was_finished) {                                  // a finished sequence takes no part in the round
         if (lane == 0) { draft_len[s] = 0; accept_len[s] = 0; next_tok[s] = -1; }
         return;
     }
     const bool in = lane < k;
-    const int d = in ? draft_tok[(size_t)s * k + lane] : 0;
-    const int v = in ? verify_tok[(size_t)s * kv + lane] : 0;
-    const bool conf = in && (draft_exit_mask == nullptr || draft_exit_mask[(size_t)s * k + lane] != 0);
+    const int d = in ? ld_dep(draft_tok + (size_t)s * k + lane) : 0;
+    const int v = in ? ld_dep(verify_tok + (size_t)s * kv + lane) : 0;
+    const bool conf = in && (draft_exit_mask == nullptr || ld_dep(draft_exit_mask + (size_t)s * k + lane) != 0);
     const unsigned int stop_b = __ballot_sync(0xffffffffu, in && !conf);               // slots the head is not sure of
     const unsigned int eos_b = __ballot_sync(0xffffffffu, in && eos >= 0 && d == eos);   // end-of-sequence drafted
     const unsigned int mis_b = __ballot_sync(0xffffffffu, in && d != v);
@@ -38,12 +43,12 @@ __global__ void __launch_bounds__(128) dssd_commit_kernel(const int* __restrict_
     const int first_mis = mis_b ? __ffs(mis_b) - 1 : k;
     const int a = min(first_mis, n);
     const bool ended = a > 0 && eos >= 0 && __shfl_sync(0xffffffffu, d, a - 1) == eos;
-    const int nxt = (!ended && a < kv) ? verify_tok[(size_t)s * kv + a] : -1;
-    const int have = seq_len[s];
+    const int nxt = (!ended && a < kv) ? ld_dep(verify_tok + (size_t)s * kv + a) : -1;
     const int want = a + ((!ended && a < kv) ? 1 : 0);
     const int count = min(want, cap - have);
     int* row = out_tok + (size_t)s * cap + have;
     if (lane < count) row[lane] = lane < a ? d : nxt;     // count <= k + 1 <= 33: lane 31 may have one more below
+    __syncwarp();
     if (lane == 0) {
         if (count == 33) row[32] = nxt;
         const bool eos_committed = eos >= 0 && ((ended && count >= a) || (nxt == eos && count == want && want > a));

@@ -11,8 +11,11 @@
 //                      one 16-byte partial state per (row, vocabulary tile)
 // All mbarrier waits are bounded; a wait that gives up records an error word, raises the CTA's abort
 // flag, and every role drains to the common exit where TMEM is released.
+#include <algorithm>
+
 #include "common.cuh"
 #include "kernels.h"
+#include "layer_norm.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.h"
 
@@ -70,7 +73,7 @@ __device__ __forceinline__ void top2_merge(float& m1, float& m2, float o1, float
 // time -- one round trip for up to 384 tiles -- then the lanes reduce) and the final decision for that row.
 // `second` (NULL if not asked for) holds each tile's second-largest logit for this row: with the tiles' maxima
 // it gives the row's second-largest logit z2 and the gap of the two largest probabilities (1 - e^(z2 - m)) / s.
-__device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ partials, const float* __restrict__ second,
+__device__ __forceinline__ void merge_row_and_decide(const State* partials, const float* second,
                                                      int n_tiles, int head, int row, const MergeHeads& hs, int lane) {
     constexpr int kBatch = 12;
     State v[kBatch + 1];
@@ -101,7 +104,7 @@ __device__ __forceinline__ void merge_row_and_decide(const State* __restrict__ p
         if (lane == 0) hs.top2gap[head][row] = (1.f - expf(t2 - t1)) / a.s;
     }
     if (lane == 0)
-        state_finish(a, hs.tau_per_row[head] ? hs.tau_per_row[head][row] : hs.tau[head], hs.argmax[head], hs.entropy[head],
+        state_finish(a, hs.tau_per_row[head] ? ld_dep(hs.tau_per_row[head] + row) : hs.tau[head], hs.argmax[head], hs.entropy[head],
                      hs.maxprob[head], hs.exit_mask[head], row);
 }
 
@@ -116,6 +119,8 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
+    State* cta_part;       // fused merge: [grid][n_heads * M] one state per CTA and row, then [groups][n_heads * M]
+    float2* cta_top2;      // fused merge, top-2 gap asked for: the two largest logits, same two tables
     MergeHeads mg;
 };
 
@@ -233,7 +238,19 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     auto xfull_bar = [&](int q) { return bar_base + 8u * (2 * S + 6 + q); };
     auto xfree_bar = [&](int q) { return bar_base + 8u * (2 * S + 10 + q); };
 
+    // Fused merge: this CTA's running state of every row of the launch (16 bytes each, then 8 bytes each for the
+    // two largest logits if they are asked for), folded over the CTA's tiles.
+    const int total_rows = p.n_heads * p.M;
+    State* acc = reinterpret_cast<State*>(bar_mem + kBarBytes);
+    float2* acc2 = reinterpret_cast<float2*>(acc + total_rows);
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (BN_T == 0 && p.fused_merge) {
+        for (int r = threadIdx.x; r < total_rows; r += kGemmThreads) {
+            acc[r] = state_empty();
+            if (kTop2) acc2[r] = make_float2(-CUDART_INF_F, -CUDART_INF_F);
+        }
+    }
     // The runtime-width variant (launches of tens of microseconds) lets its dependents start at once; their few
     // CTAs wait beside this one.  The 256-wide variant runs for milliseconds and its merge has thousands of
     // CTAs: resident and waiting they cost it about a tenth of its speed, so it triggers them only when a CTA
@@ -490,53 +507,100 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 if (lane == 0) ptx::mbar_arrive(xfree_bar(quarter));
                 if (live) {
                     state_merge(st, other);
-                    p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
-                    if constexpr (want_top2) {
-                        top2_merge(z1, z2, other2.x, other2.y);
-                        p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
+                    if constexpr (want_top2) top2_merge(z1, z2, other2.x, other2.y);
+                    if (p.fused_merge) {
+                        // A row of a head is always folded by the same thread of the CTA: no other thread touches
+                        // its entry, and the CTA's tiles arrive in a fixed order.
+                        State* mine = acc + head * p.M + row;
+                        State cur = *mine;
+                        state_merge(cur, st);
+                        *mine = cur;
+                        if constexpr (want_top2) {
+                            float2 c2 = acc2[head * p.M + row];
+                            top2_merge(c2.x, c2.y, z1, z2);
+                            acc2[head * p.M + row] = c2;
+                        }
+                    } else {
+                        p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                        if constexpr (want_top2) p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
                     }
                 }
             }
         }
         if (kSplit && p.fused_merge) {
             // With few rows the merge runs here instead of in a kernel of its own (one launch boundary less per
-            // call).  Every CTA publishes its partial states with a ticket; epilogue warp w of CTA c owns rows
-            // 8c + w, 8c + w + 8 * grid, ..: a warp that owns a row waits, bounded, until all CTAs have
-            // published, then merges and decides.  CTAs without rows leave at once.  The warp that finishes
-            // the last row returns both counters to zero.
-            // The barrier orders the epilogue threads' stores before thread 64's release, which is cumulative:
-            // a warp that acquires the full ticket count sees every CTA's partial states.
+            // call), and no CTA ever waits for another: a CTA stores its per-row states, takes a ticket of its group
+            // of 16 CTAs and leaves -- unless it is the group's last arriver, which combines the group's states
+            // (thread = row, sixteen independent loads) and takes a ticket among the groups; the last of those
+            // combines the groups' states, decides, writes the outputs and returns the counters to zero.  The
+            // combination order is fixed by CTA and group number, so results are bit-identical from run to run.
+            // Each barrier orders the epilogue threads' stores before one thread's acquire-release ticket, which is
+            // cumulative: a last arriver sees every state published before it.  A CTA whose roles gave up still
+            // takes its tickets (its outputs are undefined, the error word says so), so the counters always return.
+            constexpr int kGroup = 16, kEpi = 256;
+            const int et = (warp - 2) * 32 + lane;
+            const int grid = (int)gridDim.x;
+            const int n_groups = (grid + kGroup - 1) / kGroup;
+            const int grp = (int)blockIdx.x / kGroup;
+            const int grp_size = min(kGroup, grid - grp * kGroup);
+            State* grp_part = p.cta_part + (size_t)grid * total_rows;
+            float2* grp_top2 = kTop2 ? p.cta_top2 + (size_t)grid * total_rows : nullptr;
+            volatile int* last_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 14));
             asm volatile("bar.sync 1, 256;" ::: "memory");            // the eight epilogue warps, whatever path they took
-            if (warp == 2 && lane == 0)
-                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&p.ctrl->ticket) : "memory");
-            const int total_rows = p.n_heads * p.M;
-            const int first = (int)blockIdx.x * 8 + (warp - 2);
-            if (first < total_rows) {
-                bool there = false;
-                for (uint32_t i = 0; i < ptx::kWaitPolls; ++i) {
-                    unsigned int v;
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(&p.ctrl->ticket) : "memory");
-                    if (v >= gridDim.x) { there = true; break; }
-                    if (*abort_flag) break;
-                    __nanosleep(i < 4096 ? 40 : 400);
-                }
-                there = __all_sync(0xffffffffu, there);
-                if (!there) {
-                    if (lane == 0) record_failure(p.ctrl, abort_flag, 7, 0, blockIdx.x);
-                } else {
-                    int mine = 0;
-                    for (int r = first; r < total_rows; r += (int)gridDim.x * 8, ++mine) {
-                        const int head = r / p.M, row = r - head * p.M;
-                        merge_row_and_decide(p.partials + (size_t)r * p.n_tiles,
-                                             kTop2 ? p.second + (size_t)r * p.n_tiles : nullptr, p.n_tiles, head, row, p.mg, lane);
-                    }
-                    if (lane == 0) {
-                        const unsigned int old = atomicAdd(&p.ctrl->merge_seen, (unsigned int)mine);
-                        if (old + (unsigned int)mine == (unsigned int)total_rows) {
-                            p.ctrl->ticket = 0;
-                            p.ctrl->merge_seen = 0;
+            for (int r = et; r < total_rows; r += kEpi) {
+                p.cta_part[(size_t)blockIdx.x * total_rows + r] = acc[r];
+                if constexpr (kTop2) p.cta_top2[(size_t)blockIdx.x * total_rows + r] = acc2[r];
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (et == 0) *last_flag = ticket_arrive_is_last(&p.ctrl->group_ticket[grp], (unsigned)grp_size) ? 1 : 0;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (*last_flag) {
+                for (int r = et; r < total_rows; r += kEpi) {
+                    State v[kGroup];
+                    float z1 = -CUDART_INF_F, z2 = -CUDART_INF_F;
+#pragma unroll
+                    for (int i = 0; i < kGroup; ++i)
+                        v[i] = i < grp_size ? state_load_cg(p.cta_part + (size_t)(grp * kGroup + i) * total_rows + r) : state_empty();
+                    if constexpr (kTop2) {
+#pragma unroll
+                        for (int i = 0; i < kGroup; ++i) {
+                            if (i < grp_size) {
+                                const float2 o = __ldcg(p.cta_top2 + (size_t)(grp * kGroup + i) * total_rows + r);
+                                top2_merge(z1, z2, o.x, o.y);
+                            }
                         }
+                        grp_top2[(size_t)grp * total_rows + r] = make_float2(z1, z2);
                     }
+                    grp_part[(size_t)grp * total_rows + r] = state_combine<kGroup>(v);
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (et == 0) *last_flag = ticket_arrive_is_last(&p.ctrl->top_ticket, (unsigned)n_groups) ? 1 : 0;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (*last_flag) {
+                    for (int r = et; r < total_rows; r += kEpi) {
+                        State v[kGroup];
+                        float z1 = -CUDART_INF_F, z2 = -CUDART_INF_F;
+#pragma unroll
+                        for (int i = 0; i < kGroup; ++i)
+                            v[i] = i < n_groups ? state_load_cg(grp_part + (size_t)i * total_rows + r) : state_empty();
+                        if constexpr (kTop2) {
+#pragma unroll
+                            for (int i = 0; i < kGroup; ++i) {
+                                if (i < n_groups) {
+                                    const float2 o = __ldcg(grp_top2 + (size_t)i * total_rows + r);
+                                    top2_merge(z1, z2, o.x, o.y);
+                                }
+                            }
+                        }
+                        const State a = state_combine<kGroup>(v);
+                        const int head = r / p.M, row = r - head * p.M;
+                        const MergeHeads& hs = p.mg;
+                        if constexpr (kTop2) hs.top2gap[head][row] = (1.f - expf(z2 - z1)) / a.s;
+                        state_finish(a, hs.tau_per_row[head] ? ld_dep(hs.tau_per_row[head] + row) : hs.tau[head], hs.argmax[head],
+                                     hs.entropy[head], hs.maxprob[head], hs.exit_mask[head], row);
+                    }
+                    if (et < n_groups) p.ctrl->group_ticket[et] = 0;      // every CTA has taken its tickets by now
+                    if (et == 0) p.ctrl->top_ticket = 0;
                 }
             }
         }
@@ -587,18 +651,22 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
     const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
     const float* gamma = hs.gamma[head];
     const float* beta = hs.beta[head];
-    const float inv_d = 1.f / (float)d;
+    const double inv_d = 1.0 / (double)d;
     if constexpr (VPL > 0) {
-        // The LayerNorm parameters are weights, not results of an earlier kernel: fetched before the wait.
-        float4 g[VPL][2], b[VPL][2];
+        // The LayerNorm parameters are weights, not results of an earlier kernel: narrow rows fetch them before the
+        // wait (wide rows would spend too many registers on them and read them through L1 afterwards).
+        constexpr bool kParamsEarly = VPL <= 4;
+        float4 g[kParamsEarly ? VPL : 1][2], b[kParamsEarly ? VPL : 1][2];
+        if constexpr (kParamsEarly) {
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int c = lane + 32 * k;
-            if (c < nvec) {
-                g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
-                g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
-                b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
-                b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+            for (int k = 0; k < VPL; ++k) {
+                const int c = lane + 32 * k;
+                if (c < nvec) {
+                    g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+                    g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+                    b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+                    b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+                }
             }
         }
         // h may be an earlier kernel's output, so it is read after the wait; asking L2 for its lines before
@@ -610,46 +678,43 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
         }
         grid_dependency_wait();                          // y may still be read by the GEMM of the call before
         uint4 x[VPL];
-        float sum = 0.f;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
-            x[k] = c < nvec ? ld_stream_v4(hrow + c) : make_uint4(0, 0, 0, 0);
+            x[k] = c < nvec ? ld_dep(hrow + c) : make_uint4(0, 0, 0, 0);
         }
+        double s0 = 0.0, s1 = 0.0;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) sum += vec8_sum(x[k]);
-        const float mu = warp_sum(sum) * inv_d;
-        float sq = 0.f;
+        for (int k = 0; k < VPL; ++k) vec8_sum_d(x[k], s0, s1);          // vectors beyond the row are zero
+        const double mu = warp_sum_d(s0 + s1) * inv_d;
+        double q0 = 0.0, q1 = 0.0;
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
-            if (lane + 32 * k < nvec) sq = vec8_sqdev(x[k], mu, sq);
-        const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
+            if (lane + 32 * k < nvec) vec8_sqdev_d(x[k], mu, q0, q1);
+        const RowStats st = row_stats(mu, warp_sum_d(q0 + q1), inv_d, ln_eps);
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
-            if (c < nvec) yrow[c] = layer_norm_vec8(x[k], mu, rstd, g[k][0], g[k][1], b[k][0], b[k][1]);
+            if (c < nvec) {
+                if constexpr (kParamsEarly) yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
+                else yrow[c] = layer_norm_vec8(x[k], st, gamma, beta, c);
+            }
         }
     } else {
         grid_dependency_wait();
-        float sum = 0.f;
-        for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
-        const float mu = warp_sum(sum) * inv_d;
-        float sq = 0.f;
-        for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
-        const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
-        for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+        const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, inv_d, ln_eps, lane);
+        for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, gamma, beta, c);
     }
 }
 
 // LayerNorm of a gathered subset of one head's rows: output row j = LayerNorm(h[row_idx[j]]) for j < *m_dev,
 // zeros from there to the end of the padded tile rows.  The list and the count come from an earlier kernel of
 // the stream (the cascade of heads), so everything is read after the dependency wait.  Warp per row.
-__global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloat16* __restrict__ h, long long ld_h,
+__global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloat16* h, long long ld_h,
                                                                 const float* __restrict__ gamma,
                                                                 const float* __restrict__ beta, float ln_eps,
-                                                                const int* __restrict__ row_idx,
-                                                                const int* __restrict__ m_dev,
-                                                                __nv_bfloat16* __restrict__ y, int M, int d) {
+                                                                const int* row_idx, const int* m_dev,
+                                                                __nv_bfloat16* y, int M, int d) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -658,29 +723,22 @@ __global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloa
     const int nvec = d >> 3;
     uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
     grid_dependency_wait();
-    const int m_live = m_dev ? min(max(*m_dev, 0), M) : M;
+    const int m_live = m_dev ? min(max(ld_dep(m_dev), 0), M) : M;
     if (row >= m_live) {
         for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
         return;
     }
-    const int src = row_idx ? row_idx[row] : row;
+    const int src = row_idx ? ld_dep(row_idx + row) : row;
     const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)src * ld_h);
-    const float inv_d = 1.f / (float)d;
-    float sum = 0.f;
-    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
-    const float mu = warp_sum(sum) * inv_d;
-    float sq = 0.f;
-    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
-    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + ln_eps);
-    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, gamma, beta, c);
+    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, 1.0 / (double)d, ln_eps, lane);
+    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, gamma, beta, c);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Merge of the per-tile partial states, one warp per row, in vocabulary order; final decision.
 // blockIdx.y = head.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict__ partials_all,
-                                                         const float* __restrict__ second_all, int n_tiles, int M,
+__global__ void __launch_bounds__(256) merge_rows_kernel(const State* partials_all, const float* second_all, int n_tiles, int M,
                                                          const __grid_constant__ MergeHeads hs) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -698,11 +756,24 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* __restrict
 // ---------------------------------------------------------------------------------------------
 constexpr int kMinTileN = 64;
 constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
+constexpr int kGemmMaxCtas = 192;          // bound on the grid of a launch that merges itself (a B200 has 148 SMs)
+constexpr int kMergeGroup = 16;            // CTAs per group of the in-kernel merge
+
+// Shared memory of the in-kernel merge: one running state per row of the launch, and the two largest logits.
+size_t fused_smem_bytes(int total_rows) {
+    return total_rows <= kFusedMergeMaxRows ? align_up((size_t)total_rows * (sizeof(State) + sizeof(float2)), 16) : 0;
+}
+// Its global scratch: one state (and one pair of logits) per CTA and row, then per group and row.
+size_t fused_scratch_bytes(int total_rows) {
+    if (total_rows > kFusedMergeMaxRows) return 0;
+    const size_t entries = (size_t)(kGemmMaxCtas + kGemmMaxCtas / kMergeGroup) * total_rows;
+    return align_up(entries * sizeof(State), 256) + align_up(entries * sizeof(float2), 256);
+}
 
 // Ring depth for a runtime tile width; b_rows = rows of W one CTA stages per k-block.
-int stages_for(int b_rows, int mma_m) {
+int stages_for(int b_rows, int mma_m, size_t extra) {
     const size_t stage = (size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2;
-    const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
+    const size_t n = (kGemmSmemBudget - kBarBytes - extra - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
 
@@ -723,7 +794,8 @@ ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int d
     if (configure_gemm<BN_T, kTop2, kPair>(device) != EE_OK) return EE_ERR_CUDA;
     const int b_rows = kPair ? p.bn / 2 : p.bn;
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
-                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
+                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes +
+                                   (p.fused_merge ? fused_smem_bytes(p.n_heads * p.M) : 0) + 1024;
     const cudaError_t err = kPair ? launch_pdl_pairs(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p)
                                   : launch_pdl(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
@@ -808,7 +880,8 @@ static int tile_n_for(long long m_tiles, int V, int n_heads, int num_sms) {
 int gemm_launches(int M, int n_heads) { return n_heads * M <= kFusedMergeMaxRows ? 2 : 3; }
 
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
-    return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads);
+    return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads) +
+           fused_scratch_bytes(n_heads * M);
 }
 
 ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
@@ -847,8 +920,10 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         if (n_heads != 1) return EE_ERR_SHAPE;
         err = launch_pdl(layer_norm_gather_kernel, dim3(ln_grid.x), 256, 0, a.stream, ln.h[0], a.ld_h, a.gamma, a.beta,
                          a.ln_eps, a.row_idx, a.m_dev, y, a.M, a.d);
-    } else if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    } else if (a.d <= 512) err = launch_pdl(layer_norm_rows_kernel<2>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+    else if (a.d <= 2560) err = launch_pdl(layer_norm_rows_kernel<10>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     else err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
     if (err != cudaSuccess) return EE_ERR_CUDA;
 
@@ -880,19 +955,26 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.bn = bn;
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
+    {
+        unsigned char* scratch = reinterpret_cast<unsigned char*>(y) + y_bytes(a.M, a.d, n_heads);
+        const size_t entries = (size_t)(kGemmMaxCtas + kGemmMaxCtas / kMergeGroup) * n_heads * a.M;
+        p.cta_part = reinterpret_cast<State*>(scratch);
+        p.cta_top2 = reinterpret_cast<float2*>(scratch + align_up(entries * sizeof(State), 256));
+    }
     p.mg = mg;
-    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
+    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m, p.fused_merge ? fused_smem_bytes(n_heads * a.M) : 0);
+    const int max_ctas = p.fused_merge ? kGemmMaxCtas : (1 << 30);
     ee_status st;
     if (pair) {
         const long long total = (long long)n_heads * (p.m_tiles / 2) * p.n_tiles;
-        const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
+        const int grid = 2 * (int)std::min<long long>(std::min<long long>(total, n_pairs), max_ctas / 2);
         st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, true>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<256, false, true>(maps, p, grid, a.device, a.stream))
                           : (p.second ? launch_gemm<0, true, true>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<0, false, true>(maps, p, grid, a.device, a.stream));
     } else {
         const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
-        const int grid = (int)(total < a.num_sms ? total : a.num_sms);
+        const int grid = (int)std::min<long long>(std::min<long long>(total, a.num_sms), max_ctas);
         st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, false>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<256, false, false>(maps, p, grid, a.device, a.stream))
                           : (p.second ? launch_gemm<0, true, false>(maps, p, grid, a.device, a.stream)

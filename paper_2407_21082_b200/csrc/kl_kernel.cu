@@ -19,6 +19,7 @@
 //   staging half of every W tile (cta_group::2 MMAs), as in the inference kernel;
 //   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
 #include "common.cuh"
+#include "layer_norm.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 #include "tensor_map.h"
@@ -382,7 +383,7 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             const int row = m_tile * BM + row_in_tile;
             const bool live = row < p.M;
             const bool any_live = __any_sync(0xffffffffu, live);
-            const int label = (live && p.labels) ? p.labels[row] : -1;
+            const int label = (live && p.labels) ? ld_dep(p.labels + row) : -1;
             if (any_live) {
                 for (int c = half; c * 32 < ncols; c += 2) {
                     float z[32];
@@ -489,7 +490,7 @@ struct KlLnArgs {
     float ln_eps[2];
 };
 
-__global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constant__ KlLnArgs a, __nv_bfloat16* __restrict__ y,
+__global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constant__ KlLnArgs a, __nv_bfloat16* y,
                                                             int M, int m_pad, int d) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -504,20 +505,13 @@ __global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constan
         return;
     }
     const uint4* hrow = reinterpret_cast<const uint4*>(a.h[which] + (size_t)row * a.ld_h[which]);
-    const float inv_d = 1.f / (float)d;
-    float sum = 0.f;
-    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(__ldg(hrow + c));
-    const float mu = warp_sum(sum) * inv_d;
-    float sq = 0.f;
-    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(__ldg(hrow + c), mu, sq);
-    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + a.ln_eps[which]);
-    for (int c = lane; c < nvec; c += 32)
-        yrow[c] = layer_norm_vec8(__ldg(hrow + c), mu, rstd, a.gamma[which], a.beta[which], c);
+    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, 1.0 / (double)d, a.ln_eps[which], lane);
+    for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, a.gamma[which], a.beta[which], c);
 }
 
 // One warp per row: the tiles' states in vocabulary order -> kl.
-__global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__ head_part, const Cross* __restrict__ cross_part,
-                                                       int n_tiles, int M, float* __restrict__ kl, float* __restrict__ ce) {
+__global__ void __launch_bounds__(256) kl_merge_kernel(const State* head_part, const Cross* cross_part,
+                                                       int n_tiles, int M, float* kl, float* ce) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -555,14 +549,14 @@ __global__ void __launch_bounds__(256) kl_merge_kernel(const State* __restrict__
 
 // loss[0] = mean of kl, loss[1] = mean of ce (if there is one); CTA b sums array b in a fixed order
 // (bit-identical from run to run).
-__global__ void __launch_bounds__(256) kl_mean_kernel(const float* __restrict__ kl, const float* __restrict__ ce, int M,
-                                                      float* __restrict__ loss) {
+__global__ void __launch_bounds__(256) kl_mean_kernel(const float* kl, const float* ce, int M,
+                                                      float* loss) {
     __shared__ float part[256];
     launch_dependents();
     grid_dependency_wait();
     const float* src = blockIdx.x == 0 ? kl : ce;
     float s = 0.f;
-    for (int i = threadIdx.x; i < M; i += 256) s += src[i];
+    for (int i = threadIdx.x; i < M; i += 256) s += ld_dep(src + i);
     part[threadIdx.x] = s;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {

@@ -17,6 +17,7 @@
 // normalise the next head's activations (into a second buffer when shared memory allows, so that the tensor
 // core never waits).  Waits between warps use mbarriers with bounded polling; nothing spins on another CTA.
 #include "common.cuh"
+#include "layer_norm.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 #include "tensor_map.h"
@@ -98,7 +99,6 @@ __device__ __forceinline__ bool fill_activations(const SkinnyParams& p, const Sk
     }
     sk_cp_async_wait_all();
     if (!sync()) return false;
-    const float inv_d = 1.f / (float)p.d;
     auto vec = [&](int r, int c) { return y_vec<N>(y_tiles, r, c); };
     for (int r = p.M + w; r < N; r += n_warps)                    // padding rows
         for (int c = lane; c < nvec; c += 32) *vec(r, c) = make_uint4(0, 0, 0, 0);
@@ -107,27 +107,22 @@ __device__ __forceinline__ bool fill_activations(const SkinnyParams& p, const Sk
         if (nvec <= 128) {
             for (int r = w; r < p.M; r += 2 * n_warps) {
                 const int rows[2] = {r, r + n_warps};
-                layer_norm_rows_in_regs<2, 4>(vec, rows, 1 + (rows[1] < p.M), nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+                layer_norm_rows_in_regs<2, 4>(vec, rows, 1 + (rows[1] < p.M), nvec, p.ln_eps, gamma_s, beta_s, lane);
             }
         } else {
             for (int r = w; r < p.M; r += n_warps) {
                 const int rows[1] = {r};
-                layer_norm_rows_in_regs<1, 8>(vec, rows, 1, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+                layer_norm_rows_in_regs<1, 8>(vec, rows, 1, nvec, p.ln_eps, gamma_s, beta_s, lane);
             }
         }
     } else {
         for (int r = w; r < p.M; r += n_warps) {
-            float sum = 0.f;
-            for (int c = lane; c < nvec; c += 32) sum += vec8_sum(*vec(r, c));
-            const float mu = warp_sum(sum) * inv_d;
-            float sq = 0.f;
-            for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(*vec(r, c), mu, sq);
-            const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
+            const RowStats st = row_stats_strided([&](int c) { return *vec(r, c); }, nvec, 1.0 / (double)p.d, p.ln_eps, lane);
             for (int c = lane; c < nvec; c += 32) {
                 const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
                 const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
                 uint4* v = vec(r, c);
-                *v = layer_norm_vec8(*v, mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+                *v = layer_norm_vec8(*v, st, g4[0], g4[1], b4[0], b4[1]);
             }
         }
     }

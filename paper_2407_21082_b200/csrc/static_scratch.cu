@@ -71,3 +71,36 @@ extern "C" ee_status ee_exit_head_static(const void* h, long long ld_h, const fl
     a.workspace_bytes = kStaticScratchBytes;
     return stream_launch(&a, 1);
 }
+
+namespace {
+// Device checks and the array's address for the two small calls below.
+ee_status static_scratch_here(cudaStream_t stream, void** scratch) {
+    int device = 0, major = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return EE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return EE_ERR_CUDA;
+    if (major != 10) return EE_ERR_ARCH;
+    return scratch_for_device(device, stream, scratch);
+}
+}  // namespace
+
+extern "C" ee_status ee_exit_head_static_query_error(void* stream) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void* scratch = nullptr;
+    const ee_status st = static_scratch_here(s, &scratch);
+    if (st != EE_OK) return st;
+    unsigned int words[3] = {0, 0, 0};
+    if (cudaMemcpyAsync(words, scratch, sizeof(words), cudaMemcpyDeviceToHost, s) != cudaSuccess) return EE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EE_ERR_CUDA;
+    if (words[1] == 0) return EE_OK;
+    // A wait gave up: put the whole control block (error word, completion counters) back to its initial state.
+    if (cudaMemsetAsync(scratch, 0, kCtrlBytes, s) != cudaSuccess) return EE_ERR_CUDA;
+    return EE_ERR_TIMEOUT;
+}
+
+extern "C" ee_status ee_exit_head_static_selftest_timeout(void* stream) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void* scratch = nullptr;
+    const ee_status st = static_scratch_here(s, &scratch);
+    if (st != EE_OK) return st;
+    return selftest_wait_timeout_launch(scratch, s);
+}

@@ -18,6 +18,7 @@
 // ticket, final merge in the last CTA) as soon as the workers are through with it, so that only the last head's
 // merge is not hidden behind the stream.
 #include "common.cuh"
+#include "layer_norm.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -117,29 +118,23 @@ __device__ void layer_norm_in_smem(const StreamParams& p, __nv_bfloat16* y_s, co
     constexpr int MPAD = 8 * NT;
     const int nvec = p.d >> 3;                                   // 16-byte vectors per row
     const int svec = p.y_stride >> 3;
-    const float inv_d = 1.f / (float)p.d;
     auto vec = [&](int r, int c) { return reinterpret_cast<uint4*>(y_s + (size_t)r * p.y_stride) + c; };
     for (int r0 = w; r0 < MPAD; r0 += 2 * nw) {
         const int rows[2] = {r0, r0 + nw};
         const int live = (rows[0] < p.M) + (rows[1] < MPAD && rows[1] < p.M);
         if (live > 0) {
             if (nvec <= 128) {
-                layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+                layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, p.ln_eps, gamma_s, beta_s, lane);
             } else if (nvec <= 256) {
-                layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, inv_d, p.ln_eps, gamma_s, beta_s, lane);
+                layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, p.ln_eps, gamma_s, beta_s, lane);
             } else {
                 for (int i = 0; i < live; ++i) {
                     uint4* yrow = vec(rows[i], 0);
-                    float sum = 0.f;
-                    for (int c = lane; c < nvec; c += 32) sum += vec8_sum(yrow[c]);
-                    const float mu = warp_sum(sum) * inv_d;
-                    float sq = 0.f;
-                    for (int c = lane; c < nvec; c += 32) sq = vec8_sqdev(yrow[c], mu, sq);
-                    const float rstd = 1.f / sqrtf(warp_sum(sq) * inv_d + p.ln_eps);
+                    const RowStats st = row_stats_strided([&](int c) { return yrow[c]; }, nvec, 1.0 / (double)p.d, p.ln_eps, lane);
                     for (int c = lane; c < nvec; c += 32) {
                         const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
                         const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-                        yrow[c] = layer_norm_vec8(yrow[c], mu, rstd, g4[0], g4[1], b4[0], b4[1]);
+                        yrow[c] = layer_norm_vec8(yrow[c], st, g4[0], g4[1], b4[0], b4[1]);
                     }
                 }
             }
@@ -280,9 +275,14 @@ __global__ void __launch_bounds__(kThreads, 1) exit_head_stream_kernel(const Str
         // The first of these warps then completes each head as soon as the workers are through with it, so that
         // no worker ever leaves its ring waiting.
         if (hw == 0) {
+            bool good = true;
             for (int hk = 0; hk < p.n_heads; ++hk) {
-                const bool done = ptx::mbar_wait(hdone_bar(hk), 0, &s_abort);
-                if (!__all_sync(0xffffffffu, done)) break;        // a worker gave up; it has recorded the error
+                if (good) {
+                    const bool done = ptx::mbar_wait(hdone_bar(hk), 0, &s_abort);
+                    good = __all_sync(0xffffffffu, done);         // false: a worker gave up; it has recorded the error
+                }
+                // After a failure the head's outputs are undefined, but the CTA still takes its ticket, so that the
+                // counters in the control block return to zero whatever happened.
                 finalize_head(hk);
             }
         }

@@ -53,7 +53,7 @@ def _model(seed, V, d):
 
 @pytest.mark.parametrize("S,k,V,d,tau,eos", [(12, 4, 400, 64, 1.0, -1), (40, 8, 1000, 128, 0.7, 5), (3, 1, 300, 64, 5.0, -1),
                                               (70, 6, 640, 256, 1.5, 17)])
-@pytest.mark.parametrize("model", ["python callback", "library table model"])
+@pytest.mark.parametrize("model", ["python callback", "library table model", "chained table model"])
 def test_whole_rounds_match_oracle(ee, S, k, V, d, tau, eos, model):
     """Drafting steps, verification pass and commit, several rounds in a row, against the oracle's round.  A
     sequence drops out of the comparison from the round in which one of its decisions falls inside the tolerance
@@ -77,7 +77,7 @@ def test_whole_rounds_match_oracle(ee, S, k, V, d, tau, eos, model):
 
     hd, hv = head_to_dev(cfg["heads"][0]), head_to_dev(cfg["heads"][1])
     rnd = ee.DssdRound(dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=tau), dict(gamma=hv["gamma"], beta=hv["beta"], W=hv["W"]),
-                       1e-5, k, eos, hidden if model == "python callback" else ee.TableModel(E[0], E[1]), state)
+                       1e-5, k, eos, hidden if model == "python callback" else ee.TableModel(E[0], E[1], chained=model.startswith("chained")), state)
     clean = np.ones(S, bool)
     for r in range(4):
         ref = oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], tau, eos, k, ref_last, *ref_state)
