@@ -197,39 +197,51 @@ class Workload:
             raise RuntimeError(f"device-side wait timed out in workload {self.name} (ee_status {code})")
 
 
-def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSampler | None = None) -> dict:
+def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSampler | None = None,
+            min_seconds: float = 2.0) -> dict:
     """Times `steps` whole steps, then the head evaluations of `steps` steps alone, with CUDA events on the
-    launching stream.
+    launching stream -- and repeats both regions, `steps` steps each, until about `min_seconds` of device time
+    have been spent on each, so that a short region (a few steps run at boost clock before the power cap bites,
+    too short for a clock sample) does not stand alone: the reported time is the median over the repeats, the
+    first repeat is reported beside it, and the clocks are sampled across all of them.
 
     The kernels of a step are chained by programmatic dependent launch, and an event recorded between two
-    launches breaks that chain (measured: about 5 us per event), so neither region has events inside it: the
-    first gives the step time (the metric), the second the duration of the dominant launch for the roofline.
-    A third, shorter region with an event pair around the head evaluation of every step is reported beside
-    them (`head_call_us_inner_events`) to show what the events cost.
+    launches breaks that chain (measured: about 5 us per event), so no region has events inside it: the
+    first kind gives the step time (the metric), the second the duration of the dominant launch for the
+    roofline.  A last, shorter region with an event pair around the head evaluation of every step is reported
+    beside them (`head_call_us_inner_events`) to show what the events cost.
     """
     torch = wl.torch
     for _ in range(warmup):
         wl.step()
     wl.check()
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
+
+    def region(fn):
+        """One timed region: barrier and synchronise on both sides, `steps` calls of fn between two events."""
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(steps):
+            fn()
+        t1.record()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        return t0.elapsed_time(t1)
+
     if sampler:
         sampler.start()
-    t0, t1, t2, t3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
-    t0.record()
-    for _ in range(steps):
-        wl.step()
-    t1.record()
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-        torch.cuda.synchronize()
-    t2.record()
-    for _ in range(steps):
-        wl.run_heads()
-    t3.record()
-    torch.cuda.synchronize()
+    step_ms = [region(wl.step)]
+    repeats = int(min(2000, max(1, np.ceil(min_seconds * 1e3 / max(step_ms[0], 1e-3)))))
+    if dist is not None:                                  # every rank must run the same number of regions
+        r = torch.tensor([repeats], device="cuda")
+        dist.all_reduce(r, op=dist.ReduceOp.MAX)
+        repeats = int(r.item())
+    for _ in range(repeats - 1):
+        step_ms.append(region(wl.step))
+    heads_ms = [region(wl.run_heads) for _ in range(repeats)]
     clocks = sampler.stop() if sampler else None
     n_inner = min(steps, 500)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inner)]
@@ -242,16 +254,24 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
     wl.check()
     from paper_2407_21082_b200 import replicas
     n_heads = len(wl.heads)
-    agg = replicas.aggregate_timing(t0.elapsed_time(t1), float(steps * n_heads * wl.M), dist, device="cuda")
-    total_ms = agg["elapsed_ms"]                     # the slowest rank
-    heads_ms = t2.elapsed_time(t3)
+    # per repeat the time of the slowest rank, then the median over the repeats
+    per_repeat = torch.tensor(step_ms, dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(per_repeat, op=dist.ReduceOp.MAX)
+    total_ms = float(per_repeat.median().item())
+    first_ms = float(per_repeat[0].item())
+    agg = replicas.aggregate_timing(total_ms, float(steps * n_heads * wl.M), dist, device="cuda")   # the time is already the slowest rank's
+    head_ms = float(np.median(heads_ms))
     inner_ms = sum(a.elapsed_time(b) for a, b in ev)
-    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"],
-                head_call_us=1e3 * heads_ms / (steps * n_heads),
+    return dict(total_ms=total_ms, ms_per_step=total_ms / steps, units_per_s=agg["units_per_s"], repeats=repeats,
+                ms_per_step_first_repeat=first_ms / steps, ms_per_step_min=float(per_repeat.min().item()) / steps,
+                ms_per_step_max=float(per_repeat.max().item()) / steps,
+                head_call_us=1e3 * head_ms / (steps * n_heads),
+                head_call_us_first_repeat=1e3 * heads_ms[0] / (steps * n_heads),
                 head_call_us_inner_events=1e3 * inner_ms / (n_inner * n_heads),
-                # step time minus head time; for millisecond-long steps the second region can run slower than the
-                # first (power cap), which would make the difference negative: reported as 0 then
-                tail_us=max(0.0, 1e3 * (t0.elapsed_time(t1) - heads_ms) / steps), clocks=clocks)
+                # step time minus head time; for millisecond-long steps the head-only regions can run slower than the
+                # whole steps (power cap), which would make the difference negative: reported as 0 then
+                tail_us=max(0.0, 1e3 * (float(np.median(step_ms)) - head_ms) / steps), clocks=clocks)
 
 
 # DRAM bytes (read + write) one launch of the dominant kernel moved in the ncu captures summarised under
@@ -713,7 +733,10 @@ def parity_report(gpu_outs: list, ref_outs: list) -> dict:
 
 
 def cpu_baseline(cfg: dict, steps: int = 1, warmup: int = 0, keep: list | None = None) -> dict:
-    """Times the oracle, as it stands, on the host cores on a bounded sample of the headline workload."""
+    """Times the oracle, as it stands, on the host cores on a bounded sample of the headline workload.  The oracle
+    decodes a head's bf16 weights to fp64 inside every call; what share of the time that is, is timed separately
+    and reported, so that the figure can be read either way."""
+    import oracle
     rows, heads = min(cfg["M"], 64), len(cfg["heads"])
     for _ in range(warmup):
         oracle_step(cfg, rows, heads)
@@ -722,8 +745,15 @@ def cpu_baseline(cfg: dict, steps: int = 1, warmup: int = 0, keep: list | None =
     for i in range(steps):
         done += oracle_step(cfg, rows, heads, keep if i == 0 else None)
     dt = time.perf_counter() - t0
+    t1 = time.perf_counter()
+    for hd in cfg["heads"][:heads]:
+        oracle.bf16_decode(hd["W"]).T.copy()
+    decode = (time.perf_counter() - t1) * steps
+    share = min(1.0, decode / dt) if dt > 0 else 0.0
     return dict(value=done / dt, unit=UNIT, cores=oracle_threads(), kind="oracle", seconds=round(dt, 2),
-                sample=f"{steps} step(s) of all {rows} rows x {heads} heads of the workload (fp64 numpy, weights decoded per call)")
+                weight_decode_share=round(share, 3), value_without_weight_decode=done / max(dt - decode, 1e-9),
+                sample=f"{steps} step(s) of all {rows} rows x {heads} heads of the workload (fp64 numpy; the oracle decodes "
+                       f"each head's weights from bf16 per call, {100 * share:.0f} % of the time here)")
 
 
 # --------------------------------------------------------------------------------------------- main
@@ -803,9 +833,14 @@ def main():
     config["parallelism"] = f"replicas x{world} (independent batches, no collective)"
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
-                data="synthetic", config=config, clocks=res["clocks"], gpu_launches=wl.launches_per_step * args.steps,
+                data="synthetic", config=config, clocks=res["clocks"],
+                gpu_launches=wl.launches_per_step * args.steps,          # per timed region of `steps` steps
                 head_call_us=res["head_call_us"], head_call_us_inner_events=res["head_call_us_inner_events"],
-                tail_us=res["tail_us"])
+                tail_us=res["tail_us"], repeats=res["repeats"],
+                timing=dict(region="`steps` consecutive steps between two CUDA events, barrier and synchronise on both sides",
+                            repeats=res["repeats"], reported="median over the repeats (max over ranks per repeat)",
+                            ms_per_step_first_repeat=res["ms_per_step_first_repeat"], ms_per_step_min=res["ms_per_step_min"],
+                            ms_per_step_max=res["ms_per_step_max"], head_call_us_first_repeat=res["head_call_us_first_repeat"]))
     line["roofline"] = roofline(wl, res["head_call_us"], peaks, peak_src)
     traffic, traffic_note = measured_traffic(wl)
     heads_per_launch = n_heads if wl.multi else 1
@@ -830,17 +865,30 @@ def main():
         torch.cuda.empty_cache()
         table = [("c0", None, 8, 200), ("c1", 1, 2, 200), ("c1", 4, 2, 200), ("c1", 16, 2, 200), ("c1", 64, 2, 200),
                  ("c2", None, 2, 100), ("c3", None, 2, 100), ("c4", None, 2, 10)]
+        per_config = {}
         for name, rows, copies, steps in table:
             w = Workload(name, rows, seed=0, n_copies=copies)
-            r = measure(w, steps, 5)
+            r = measure(w, steps, 5, min_seconds=0.4)
             key = name if rows is None else f"{name}_M{rows}"
             roof = roofline(w, r["head_call_us"], peaks, peak_src)
             roof["traffic"], roof["traffic_note"] = measured_traffic(w)      # per launch, like the headline's
             extra[key] = dict(M=w.M, d=w.d, heads=len(w.heads), head_call_us=round(r["head_call_us"], 2),
+                              head_call_us_first_repeat=round(r["head_call_us_first_repeat"], 2), repeats=r["repeats"],
                               tail_us=round(r["tail_us"], 2), tokens_per_s=w.M / (r["head_call_us"] * 1e-6),
                               roofline=roof, launches_per_head=w.head_launches)
+            # the same figures in short, inside the roofline object of the line
+            short = dict(us=round(r["head_call_us"], 2), bound=roof["bound"], frac=roof["frac"], achieved=roof["achieved"],
+                         unit=roof["unit"], traffic=roof["traffic"], tokens_per_s=round(w.M / (r["head_call_us"] * 1e-6), 1),
+                         repeats=r["repeats"], steps_per_repeat=steps)
+            for extra_key in ("tensor_frac", "hbm_frac", "frac_of_sustained"):
+                if extra_key in roof:
+                    short[extra_key] = roof[extra_key]
+            per_config[key] = short
             del w
             torch.cuda.empty_cache()
+        line["roofline"]["per_config"] = per_config
+        line["roofline"]["per_config_note"] = ("us = one head evaluation (median over the repeats of a region of steps_per_repeat "
+                                               "consecutive head evaluations, at least 0.4 s in all), frac against the bound named")
         line["configs"] = extra
         line["roofline"]["read_stream"] = measure_read_stream(peaks, peak_src)
         line["calibration"] = measure_calibration(peaks, peak_src)

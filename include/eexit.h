@@ -64,9 +64,8 @@ int ee_exit_head_launches(int M, int d, int V, int path);
  * allocated (and after ee_query_async_error reported EE_ERR_TIMEOUT); every ee_exit_head call leaves
  * the block ready for the next one.  The workspace must be 256-byte aligned.  One workspace serves one
  * call at a time: calls sharing a workspace must be ordered on one stream.  Calls with workspaces of their own
- * may run on different streams at the same time, at most two per GPU: a call of up to 512 rows finishes inside
- * its main kernel, where some CTAs keep their SMs while they wait (bounded) for the launch's other CTAs, and
- * three or more such launches could hold every SM between them until the wait gives up with EE_ERR_TIMEOUT.
+ * may run on different streams at the same time, any number of them: no kernel of the library makes one of its
+ * thread blocks wait for another block to be scheduled.
  */
 ee_status ee_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 

@@ -149,9 +149,10 @@ struct Control {
     unsigned int pad0;
     unsigned int head_ticket[8];   // completion counters of the heads of a multi-head launch; return to 0 as well
     unsigned int merge_seen;  // unused (kept so that the layout of the words above stays as it was)
-    unsigned int group_ticket[16];   // tensor-core kernel, in-kernel merge: CTAs of each group of 16 that have published
-    unsigned int top_ticket;         // ... and groups whose partial states have been combined; both return to 0
-    unsigned int pad[34];
+    unsigned int merge_abandon[2];   // tensor-core kernel, in-kernel merge: one bit per group of rows whose owner gave up
+    unsigned int merge_pair_bits[4]; // ... and two bits per group (owner claims / last arriver takes) for the rare tie;
+                                     // `ticket` and these are zeroed by the LayerNorm kernel of the next call
+    unsigned int pad[45];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 

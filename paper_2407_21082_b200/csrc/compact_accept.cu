@@ -52,7 +52,17 @@ __device__ __forceinline__ void compact_body(int cta, const unsigned char* exit_
     for (int r = warp; r < s_n; r += kCompactThreads / 32) {
         const uint4* src = reinterpret_cast<const uint4*>(h + (size_t)s_src[r] * ld_h);
         uint4* dst = reinterpret_cast<uint4*>(h_out + (size_t)(s_base + r) * d);
-        for (int c = lane; c < nvec; c += 32) dst[c] = ld_dep(src + c);
+        // Four loads in flight per lane before the first store: source and destination may alias as far as the
+        // compiler knows, so it would otherwise finish every store before it starts the next load.
+        for (int c = lane; c < nvec; c += 128) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c + 32 * u < nvec) v[u] = ld_dep(src + c + 32 * u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c + 32 * u < nvec) dst[c + 32 * u] = v[u];
+        }
     }
 }
 

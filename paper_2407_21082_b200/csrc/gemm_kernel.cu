@@ -11,8 +11,6 @@
 //                      one 16-byte partial state per (row, vocabulary tile)
 // All mbarrier waits are bounded; a wait that gives up records an error word, raises the CTA's abort
 // flag, and every role drains to the common exit where TMEM is released.
-#include <algorithm>
-
 #include "common.cuh"
 #include "kernels.h"
 #include "layer_norm.cuh"
@@ -70,15 +68,15 @@ __device__ __forceinline__ void top2_merge(float& m1, float& m2, float o1, float
 }
 
 // One warp: merge of the n_tiles partial states of one row (lane-strided, twelve independent loads at a
-// time -- one round trip for up to 384 tiles -- then the lanes reduce) and the final decision for that row.
-// `second` (NULL if not asked for) holds each tile's second-largest logit for this row: with the tiles' maxima
-// it gives the row's second-largest logit z2 and the gap of the two largest probabilities (1 - e^(z2 - m)) / s.
-__device__ __forceinline__ void merge_row_and_decide(const State* partials, const float* second,
-                                                     int n_tiles, int head, int row, const MergeHeads& hs, int lane) {
+// time -- one round trip for up to 384 tiles -- then the lanes reduce).  `second` (NULL if not asked for) holds each
+// tile's second-largest logit for this row: with the tiles' maxima it gives the row's largest and second-largest
+// logit t1, t2, from which the gap of the two largest probabilities is (1 - e^(t2 - t1)) / s.
+__device__ __forceinline__ State merge_row(const State* partials, const float* second, int n_tiles, int lane, float& t1,
+                                           float& t2) {
     constexpr int kBatch = 12;
     State v[kBatch + 1];
     v[kBatch] = state_empty();                                    // running result of this lane
-    float t1 = -CUDART_INF_F, t2 = -CUDART_INF_F;
+    t1 = t2 = -CUDART_INF_F;
     for (int n0 = lane; n0 < n_tiles; n0 += 32 * kBatch) {
 #pragma unroll
         for (int i = 0; i < kBatch; ++i) {
@@ -101,11 +99,22 @@ __device__ __forceinline__ void merge_row_and_decide(const State* partials, cons
             const float o1 = __shfl_xor_sync(0xffffffffu, t1, o), o2 = __shfl_xor_sync(0xffffffffu, t2, o);
             top2_merge(t1, t2, o1, o2);
         }
-        if (lane == 0) hs.top2gap[head][row] = (1.f - expf(t2 - t1)) / a.s;
     }
-    if (lane == 0)
-        state_finish(a, hs.tau_per_row[head] ? ld_dep(hs.tau_per_row[head] + row) : hs.tau[head], hs.argmax[head], hs.entropy[head],
-                     hs.maxprob[head], hs.exit_mask[head], row);
+    return a;
+}
+// ... and the final decision for that row, written by lane 0.
+__device__ __forceinline__ void decide_row(const State& a, float t1, float t2, bool with_top2, int head, int row,
+                                           const MergeHeads& hs, int lane) {
+    if (lane != 0) return;
+    if (with_top2) hs.top2gap[head][row] = (1.f - expf(t2 - t1)) / a.s;
+    state_finish(a, hs.tau_per_row[head] ? ld_dep(hs.tau_per_row[head] + row) : hs.tau[head], hs.argmax[head], hs.entropy[head],
+                 hs.maxprob[head], hs.exit_mask[head], row);
+}
+__device__ __forceinline__ void merge_row_and_decide(const State* partials, const float* second, int n_tiles, int head, int row,
+                                                     const MergeHeads& hs, int lane) {
+    float t1, t2;
+    const State a = merge_row(partials, second, n_tiles, lane, t1, t2);
+    decide_row(a, t1, t2, second != nullptr, head, row, hs, lane);
 }
 
 struct GemmParams {
@@ -119,8 +128,6 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
-    State* cta_part;       // fused merge: [grid][n_heads * M] one state per CTA and row, then [groups][n_heads * M]
-    float2* cta_top2;      // fused merge, top-2 gap asked for: the two largest logits, same two tables
     MergeHeads mg;
 };
 
@@ -238,19 +245,9 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     auto xfull_bar = [&](int q) { return bar_base + 8u * (2 * S + 6 + q); };
     auto xfree_bar = [&](int q) { return bar_base + 8u * (2 * S + 10 + q); };
 
-    // Fused merge: this CTA's running state of every row of the launch (16 bytes each, then 8 bytes each for the
-    // two largest logits if they are asked for), folded over the CTA's tiles.
     const int total_rows = p.n_heads * p.M;
-    State* acc = reinterpret_cast<State*>(bar_mem + kBarBytes);
-    float2* acc2 = reinterpret_cast<float2*>(acc + total_rows);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (BN_T == 0 && p.fused_merge) {
-        for (int r = threadIdx.x; r < total_rows; r += kGemmThreads) {
-            acc[r] = state_empty();
-            if (kTop2) acc2[r] = make_float2(-CUDART_INF_F, -CUDART_INF_F);
-        }
-    }
     // The runtime-width variant (launches of tens of microseconds) lets its dependents start at once; their few
     // CTAs wait beside this one.  The 256-wide variant runs for milliseconds and its merge has thousands of
     // CTAs: resident and waiting they cost it about a tenth of its speed, so it triggers them only when a CTA
@@ -508,100 +505,99 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 if (live) {
                     state_merge(st, other);
                     if constexpr (want_top2) top2_merge(z1, z2, other2.x, other2.y);
-                    if (p.fused_merge) {
-                        // A row of a head is always folded by the same thread of the CTA: no other thread touches
-                        // its entry, and the CTA's tiles arrive in a fixed order.
-                        State* mine = acc + head * p.M + row;
-                        State cur = *mine;
-                        state_merge(cur, st);
-                        *mine = cur;
-                        if constexpr (want_top2) {
-                            float2 c2 = acc2[head * p.M + row];
-                            top2_merge(c2.x, c2.y, z1, z2);
-                            acc2[head * p.M + row] = c2;
-                        }
-                    } else {
-                        p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
-                        if constexpr (want_top2) p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
-                    }
+                    p.partials[((size_t)head * p.M + row) * p.n_tiles + n_tile] = st;
+                    if constexpr (want_top2) p.second[((size_t)head * p.M + row) * p.n_tiles + n_tile] = z2;
                 }
             }
         }
         if (kSplit && p.fused_merge) {
             // With few rows the merge runs here instead of in a kernel of its own (one launch boundary less per
-            // call), and no CTA ever waits for another: a CTA stores its per-row states, takes a ticket of its group
-            // of 16 CTAs and leaves -- unless it is the group's last arriver, which combines the group's states
-            // (thread = row, sixteen independent loads) and takes a ticket among the groups; the last of those
-            // combines the groups' states, decides, writes the outputs and returns the counters to zero.  The
-            // combination order is fixed by CTA and group number, so results are bit-identical from run to run.
-            // Each barrier orders the epilogue threads' stores before one thread's acquire-release ticket, which is
-            // cumulative: a last arriver sees every state published before it.  A CTA whose roles gave up still
-            // takes its tickets (its outputs are undefined, the error word says so), so the counters always return.
-            constexpr int kGroup = 16, kEpi = 256;
+            // call).  Every CTA has stored its tiles' states and takes a ticket.  The rows are dealt out in groups
+            // (group g: rows 8g + w for epilogue warp w, stepping by 8 * groups) to the first CTAs of the grid, which
+            // also carry the most tiles and so finish among the last.  An owner looks at the ticket for a bounded
+            // time and, once every CTA has published, merges its group: no further atomic on that path.  An owner
+            // whose looks run out says so (a bit in merge_abandon) and leaves; the LAST arriver, whoever it is,
+            // takes and merges every group so marked.  So the call completes whether or not the owners were still
+            // around -- no CTA's progress depends on another CTA being scheduled, and an owner that stops looking
+            // loses nothing but its share of the work.
+            // An owner that gives up just as the last ticket is taken: it sets its bit, fences, and looks once more;
+            // the last arriver takes its ticket, fences, and reads the bits (sequentially consistent fences: at
+            // least one of the two sees the other).  If the owner's last look finds the count full, both may want
+            // the group, and two bits in one word decide: the owner sets CLAIM, the last arriver TAKEN, each with an
+            // atomic OR that shows it the other's bit; whoever finds the other's bit already there leaves the group
+            // to the other.  Ticket and bits are zeroed by the next call's LayerNorm kernel (which starts after
+            // this kernel has completed).
+            // The barrier orders the epilogue threads' stores before one thread's acquire-release ticket, which is
+            // cumulative: whoever sees the full count sees every CTA's states.  A CTA whose roles gave up still
+            // takes its ticket (its tiles' states are missing, the error word says so).
+            constexpr int kMergeLooks = 96;
             const int et = (warp - 2) * 32 + lane;
             const int grid = (int)gridDim.x;
-            const int n_groups = (grid + kGroup - 1) / kGroup;
-            const int grp = (int)blockIdx.x / kGroup;
-            const int grp_size = min(kGroup, grid - grp * kGroup);
-            State* grp_part = p.cta_part + (size_t)grid * total_rows;
-            float2* grp_top2 = kTop2 ? p.cta_top2 + (size_t)grid * total_rows : nullptr;
-            volatile int* last_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 14));
+            const int n_groups = min(grid, (total_rows + 7) >> 3);
+            const int group = (int)blockIdx.x < n_groups ? (int)blockIdx.x : -1;
+            volatile int* slot = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * S + 14));     // three words
+            const bool with_top2 = kTop2 && p.second != nullptr;
+            auto merge_group = [&](int g) {
+                for (int r = g * 8 + (warp - 2); r < total_rows; r += 8 * n_groups) {
+                    const int head = r / p.M;
+                    merge_row_and_decide(p.partials + (size_t)r * p.n_tiles, with_top2 ? p.second + (size_t)r * p.n_tiles : nullptr,
+                                         p.n_tiles, head, r - head * p.M, p.mg, lane);
+                }
+            };
+            auto look = [&]() {
+                unsigned int v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(&p.ctrl->ticket) : "memory");
+                return v >= (unsigned)grid;
+            };
+            auto atom_or = [&](unsigned int* word, unsigned int bits) {
+                unsigned int old;
+                asm volatile("atom.acq_rel.gpu.global.or.b32 %0, [%1], %2;" : "=r"(old) : "l"(word), "r"(bits) : "memory");
+                return old;
+            };
+            constexpr unsigned int kClaim = 1u, kTaken = 2u;          // two bits per group in merge_pair_bits
             asm volatile("bar.sync 1, 256;" ::: "memory");            // the eight epilogue warps, whatever path they took
-            for (int r = et; r < total_rows; r += kEpi) {
-                p.cta_part[(size_t)blockIdx.x * total_rows + r] = acc[r];
-                if constexpr (kTop2) p.cta_top2[(size_t)blockIdx.x * total_rows + r] = acc2[r];
+            unsigned int arrival = 0;                                 // looked at only after the owner's work: the
+            if (et == 0)                                              // ticket's round trip is off the owners' path
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrival) : "l"(&p.ctrl->ticket) : "memory");
+            if (group >= 0) {
+                if (et == 0) {
+                    bool mine = false;
+                    for (int i = 0; !mine && i < kMergeLooks; ++i) {
+                        mine = look();
+                        if (!mine && i >= 8) __nanosleep(i < 32 ? 100 : 1000);
+                    }
+                    if (!mine) {
+                        atom_or(&p.ctrl->merge_abandon[group >> 5], 1u << (group & 31));
+                        asm volatile("fence.sc.gpu;" ::: "memory");
+                        if (look()) {                                 // the last ticket came in meanwhile
+                            const int sh = 2 * (group & 15);
+                            mine = ((atom_or(&p.ctrl->merge_pair_bits[group >> 4], kClaim << sh) >> sh) & kTaken) == 0;
+                        }
+                    }
+                    slot[1] = mine ? 1 : 0;
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (slot[1]) merge_group(group);
             }
+            if (et == 0) slot[2] = arrival == (unsigned)grid - 1u ? 1 : 0;
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (et == 0) *last_flag = ticket_arrive_is_last(&p.ctrl->group_ticket[grp], (unsigned)grp_size) ? 1 : 0;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (*last_flag) {
-                for (int r = et; r < total_rows; r += kEpi) {
-                    State v[kGroup];
-                    float z1 = -CUDART_INF_F, z2 = -CUDART_INF_F;
-#pragma unroll
-                    for (int i = 0; i < kGroup; ++i)
-                        v[i] = i < grp_size ? state_load_cg(p.cta_part + (size_t)(grp * kGroup + i) * total_rows + r) : state_empty();
-                    if constexpr (kTop2) {
-#pragma unroll
-                        for (int i = 0; i < kGroup; ++i) {
-                            if (i < grp_size) {
-                                const float2 o = __ldcg(p.cta_top2 + (size_t)(grp * kGroup + i) * total_rows + r);
-                                top2_merge(z1, z2, o.x, o.y);
-                            }
-                        }
-                        grp_top2[(size_t)grp * total_rows + r] = make_float2(z1, z2);
+            if (slot[2]) {
+                // The last arriver: the groups whose owners have stopped looking.
+                if (et < 2) {
+                    asm volatile("fence.sc.gpu;" ::: "memory");
+                    unsigned int left;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(left) : "l"(&p.ctrl->merge_abandon[et]) : "memory");
+                    unsigned int won = 0;
+                    for (unsigned int rest = left; rest; rest &= rest - 1) {
+                        const int g = 32 * et + __ffs(rest) - 1;
+                        const int sh = 2 * (g & 15);
+                        if (((atom_or(&p.ctrl->merge_pair_bits[g >> 4], kTaken << sh) >> sh) & kClaim) == 0) won |= 1u << (g & 31);
                     }
-                    grp_part[(size_t)grp * total_rows + r] = state_combine<kGroup>(v);
+                    slot[et] = (int)won;
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (et == 0) *last_flag = ticket_arrive_is_last(&p.ctrl->top_ticket, (unsigned)n_groups) ? 1 : 0;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (*last_flag) {
-                    for (int r = et; r < total_rows; r += kEpi) {
-                        State v[kGroup];
-                        float z1 = -CUDART_INF_F, z2 = -CUDART_INF_F;
-#pragma unroll
-                        for (int i = 0; i < kGroup; ++i)
-                            v[i] = i < n_groups ? state_load_cg(grp_part + (size_t)i * total_rows + r) : state_empty();
-                        if constexpr (kTop2) {
-#pragma unroll
-                            for (int i = 0; i < kGroup; ++i) {
-                                if (i < n_groups) {
-                                    const float2 o = __ldcg(grp_top2 + (size_t)i * total_rows + r);
-                                    top2_merge(z1, z2, o.x, o.y);
-                                }
-                            }
-                        }
-                        const State a = state_combine<kGroup>(v);
-                        const int head = r / p.M, row = r - head * p.M;
-                        const MergeHeads& hs = p.mg;
-                        if constexpr (kTop2) hs.top2gap[head][row] = (1.f - expf(z2 - z1)) / a.s;
-                        state_finish(a, hs.tau_per_row[head] ? ld_dep(hs.tau_per_row[head] + row) : hs.tau[head], hs.argmax[head],
-                                     hs.entropy[head], hs.maxprob[head], hs.exit_mask[head], row);
-                    }
-                    if (et < n_groups) p.ctrl->group_ticket[et] = 0;      // every CTA has taken its tickets by now
-                    if (et == 0) p.ctrl->top_ticket = 0;
-                }
+                for (int w2 = 0; w2 < 2; ++w2)
+                    for (unsigned int won = (unsigned int)slot[w2]; won; won &= won - 1) merge_group(32 * w2 + __ffs(won) - 1);
             }
         }
     }
@@ -622,8 +618,20 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
 // ---------------------------------------------------------------------------------------------
 // LayerNorm of every head's input: h_k [M, d] (row stride ld_h) -> y [k][M, d] bf16, one warp per row,
 // blockIdx.y = head.  With VPL > 0 the row stays in registers (VPL 16-byte vectors per lane, d <= 256 * VPL)
-// and is read once; VPL = 0 re-reads it per pass.
+// and is read once; VPL = 0 re-reads it from global memory per pass.  No shared memory and at most 128 registers,
+// so that a CTA fits on an SM beside a CTA of the call before (which holds nearly all of the shared memory) and
+// is resident, its parameters fetched, when that call completes.
 // ---------------------------------------------------------------------------------------------
+// The first kernel of every call zeroes the counters of the in-kernel merge (it passes its dependency wait only
+// after the call before has completed, so nobody is looking at them).
+__device__ __forceinline__ void reset_merge_counters(Control* ctrl) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        ctrl->ticket = 0;
+        ctrl->merge_abandon[0] = ctrl->merge_abandon[1] = 0;
+        ctrl->merge_pair_bits[0] = ctrl->merge_pair_bits[1] = ctrl->merge_pair_bits[2] = ctrl->merge_pair_bits[3] = 0;
+    }
+}
+
 struct LnHeads {
     const __nv_bfloat16* h[kGemmMaxHeads];
     long long ld_h[kGemmMaxHeads];
@@ -631,33 +639,50 @@ struct LnHeads {
     const float* beta[kGemmMaxHeads];
 };
 
+// Threads per CTA: four warps when the rows are held in registers.  With up to 1024 columns a CTA then stays under
+// 24 K registers and uses no shared memory, so it fits on an SM beside a CTA of the GEMM kernel; wider rows stage
+// their parameters in shared memory and take their place as the CTAs of the call before leave.
+__host__ __device__ constexpr int ln_threads(int vpl) { return vpl > 0 ? 128 : 256; }
+
 template <int VPL>
-__global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps,
-                                                              __nv_bfloat16* __restrict__ y_all, int M, int d) {
+__global__ void __launch_bounds__(ln_threads(VPL), VPL >= 8 ? 2 : 3)
+layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bfloat16* __restrict__ y_all, int M, int d,
+                       Control* ctrl) {
     launch_dependents();
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int row = blockIdx.x * (ln_threads(VPL) / 32) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int head = blockIdx.y;
     const int m_pad = (M + BM - 1) / BM * BM;            // a head's rows are padded to whole 128-row tiles
-    if (row >= m_pad) return;
     const int nvec = d >> 3;
+    const float* gamma = hs.gamma[head];
+    const float* beta = hs.beta[head];
+    // The LayerNorm parameters are weights, not results of an earlier kernel: they are fetched before the wait,
+    // because a load from L2 after it costs about a microsecond while the next call's weight stream is running.
+    // Narrow rows keep them in registers (sixteen per vector); wide rows stage them in shared memory
+    // (2 * d * 4 bytes of dynamic shared memory, one copy for the CTA's four rows).
+    constexpr bool kParamsInRegs = VPL > 0 && VPL < 8;
+    extern __shared__ float ln_params[];
+    float4 g[kParamsInRegs ? VPL : 1][2], b[kParamsInRegs ? VPL : 1][2];
+    if constexpr (VPL >= 8) {
+        for (int i = threadIdx.x; i < (d >> 2); i += ln_threads(VPL)) {
+            reinterpret_cast<float4*>(ln_params)[i] = __ldg(reinterpret_cast<const float4*>(gamma) + i);
+            reinterpret_cast<float4*>(ln_params + d)[i] = __ldg(reinterpret_cast<const float4*>(beta) + i);
+        }
+        __syncthreads();
+    }
+    if (row >= m_pad) return;
     uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * m_pad + row) * d);
     if (row >= M) {
         // Padding row: zeros, so that the rows of a tile that carry no token cost the tensor pipe no switching.
         grid_dependency_wait();
+        reset_merge_counters(ctrl);
         for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
         return;
     }
     const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
-    const float* gamma = hs.gamma[head];
-    const float* beta = hs.beta[head];
-    const double inv_d = 1.0 / (double)d;
     if constexpr (VPL > 0) {
-        // The LayerNorm parameters are weights, not results of an earlier kernel: narrow rows fetch them before the
-        // wait (wide rows would spend too many registers on them and read them through L1 afterwards).
-        constexpr bool kParamsEarly = VPL <= 4;
-        float4 g[kParamsEarly ? VPL : 1][2], b[kParamsEarly ? VPL : 1][2];
-        if constexpr (kParamsEarly) {
+        const double dd = (double)d, inv_d = 1.0 / dd;       // a division: some thirty dependent operations, done before the wait
+        if constexpr (kParamsInRegs) {
 #pragma unroll
             for (int k = 0; k < VPL; ++k) {
                 const int c = lane + 32 * k;
@@ -669,6 +694,17 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
                 }
             }
         }
+        // The parameters of vector c (columns 8c .. 8c + 7), wherever they are kept.
+        auto params = [&](int k, int c, float4& g0, float4& g1, float4& b0, float4& b1) {
+            if constexpr (kParamsInRegs) {
+                g0 = g[k][0]; g1 = g[k][1]; b0 = b[k][0]; b1 = b[k][1];
+            } else {
+                g0 = reinterpret_cast<const float4*>(ln_params)[2 * c];
+                g1 = reinterpret_cast<const float4*>(ln_params)[2 * c + 1];
+                b0 = reinterpret_cast<const float4*>(ln_params + d)[2 * c];
+                b1 = reinterpret_cast<const float4*>(ln_params + d)[2 * c + 1];
+            }
+        };
         // h may be an earlier kernel's output, so it is read after the wait; asking L2 for its lines before
         // the wait is harmless (L2 is the point of coherence) and hides a DRAM round trip when h is not cached.
 #pragma unroll
@@ -677,32 +713,55 @@ __global__ void __launch_bounds__(256) layer_norm_rows_kernel(const __grid_const
             if (c < nvec && (c & 7) == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(hrow + c));
         }
         grid_dependency_wait();                          // y may still be read by the GEMM of the call before
+        reset_merge_counters(ctrl);
         uint4 x[VPL];
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
             x[k] = c < nvec ? ld_dep(hrow + c) : make_uint4(0, 0, 0, 0);
         }
-        double s0 = 0.0, s1 = 0.0;
+        Moments m;
+        m.clear();
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) vec8_sum_d(x[k], s0, s1);          // vectors beyond the row are zero
-        const double mu = warp_sum_d(s0 + s1) * inv_d;
-        double q0 = 0.0, q1 = 0.0;
+        for (int k = 0; k < VPL; ++k) m.add(x[k], k);                     // vectors beyond the row are zero
+        double s = m.sum(), q = m.sum_sq();
+        warp_sum2_d(s, q);
+        double mu, var;
+        if (!row_variance_one_pass(s, q, dd, inv_d, mu, var)) {
+            double q0 = 0.0, q1 = 0.0;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k)
-            if (lane + 32 * k < nvec) vec8_sqdev_d(x[k], mu, q0, q1);
-        const RowStats st = row_stats(mu, warp_sum_d(q0 + q1), inv_d, ln_eps);
+            for (int k = 0; k < VPL; ++k)
+                if (lane + 32 * k < nvec) vec8_sqdev_d(x[k], mu, q0, q1);
+            var = warp_sum_d(q0 + q1) * inv_d;
+        }
+        const RowStats st = row_stats(mu, var, ln_eps);
+        uint32_t doubts[VPL];
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
+            doubts[k] = 0;
             if (c < nvec) {
-                if constexpr (kParamsEarly) yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
-                else yrow[c] = layer_norm_vec8(x[k], st, gamma, beta, c);
+                float4 g0, g1, b0, b1;
+                params(k, c, g0, g1, b0, b1);
+                yrow[c] = layer_norm_vec8_fast(x[k], st, g0, g1, b0, b1, doubts[k]);
+            }
+        }
+        // The few elements fp64 has to decide, after the loop: the doubtful elements of a vector are replaced.
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            if (doubts[k]) {
+                float4 g0, g1, b0, b1;
+                params(k, c, g0, g1, b0, b1);
+                uint32_t again;                              // recomputed rather than read back: a load would cost a round trip
+                const uint4 y = layer_norm_vec8_fast(x[k], st, g0, g1, b0, b1, again);
+                yrow[c] = layer_norm_vec8_redo_inline(x[k], y, st.mu, st.rstd, g0, g1, b0, b1, doubts[k]);
             }
         }
     } else {
         grid_dependency_wait();
-        const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, inv_d, ln_eps, lane);
+        reset_merge_counters(ctrl);
+        const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, ln_eps, lane);
         for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, gamma, beta, c);
     }
 }
@@ -714,7 +773,7 @@ __global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloa
                                                                 const float* __restrict__ gamma,
                                                                 const float* __restrict__ beta, float ln_eps,
                                                                 const int* row_idx, const int* m_dev,
-                                                                __nv_bfloat16* y, int M, int d) {
+                                                                __nv_bfloat16* y, int M, int d, Control* ctrl) {
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -723,6 +782,7 @@ __global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloa
     const int nvec = d >> 3;
     uint4* yrow = reinterpret_cast<uint4*>(y + (size_t)row * d);
     grid_dependency_wait();
+        reset_merge_counters(ctrl);
     const int m_live = m_dev ? min(max(ld_dep(m_dev), 0), M) : M;
     if (row >= m_live) {
         for (int c = lane; c < nvec; c += 32) yrow[c] = make_uint4(0, 0, 0, 0);
@@ -730,7 +790,7 @@ __global__ void __launch_bounds__(256) layer_norm_gather_kernel(const __nv_bfloa
     }
     const int src = row_idx ? ld_dep(row_idx + row) : row;
     const uint4* hrow = reinterpret_cast<const uint4*>(h + (size_t)src * ld_h);
-    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, 1.0 / (double)d, ln_eps, lane);
+    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, ln_eps, lane);
     for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, gamma, beta, c);
 }
 
@@ -756,24 +816,12 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* partials_a
 // ---------------------------------------------------------------------------------------------
 constexpr int kMinTileN = 64;
 constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
-constexpr int kGemmMaxCtas = 192;          // bound on the grid of a launch that merges itself (a B200 has 148 SMs)
-constexpr int kMergeGroup = 16;            // CTAs per group of the in-kernel merge
-
-// Shared memory of the in-kernel merge: one running state per row of the launch, and the two largest logits.
-size_t fused_smem_bytes(int total_rows) {
-    return total_rows <= kFusedMergeMaxRows ? align_up((size_t)total_rows * (sizeof(State) + sizeof(float2)), 16) : 0;
-}
-// Its global scratch: one state (and one pair of logits) per CTA and row, then per group and row.
-size_t fused_scratch_bytes(int total_rows) {
-    if (total_rows > kFusedMergeMaxRows) return 0;
-    const size_t entries = (size_t)(kGemmMaxCtas + kGemmMaxCtas / kMergeGroup) * total_rows;
-    return align_up(entries * sizeof(State), 256) + align_up(entries * sizeof(float2), 256);
-}
-
 // Ring depth for a runtime tile width; b_rows = rows of W one CTA stages per k-block.
-int stages_for(int b_rows, int mma_m, size_t extra) {
+// `reserve`: shared memory left free on the SM for a CTA of the next call's LayerNorm kernel, which for rows wider
+// than 1024 columns stages its parameters there; without it that CTA would keep the next GEMM CTA off the SM.
+int stages_for(int b_rows, int mma_m, size_t reserve) {
     const size_t stage = (size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2;
-    const size_t n = (kGemmSmemBudget - kBarBytes - extra - 1024) / stage;
+    const size_t n = (kGemmSmemBudget - reserve - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
 
@@ -794,8 +842,7 @@ ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int d
     if (configure_gemm<BN_T, kTop2, kPair>(device) != EE_OK) return EE_ERR_CUDA;
     const int b_rows = kPair ? p.bn / 2 : p.bn;
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
-                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes +
-                                   (p.fused_merge ? fused_smem_bytes(p.n_heads * p.M) : 0) + 1024;
+                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
     const cudaError_t err = kPair ? launch_pdl_pairs(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p)
                                   : launch_pdl(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
@@ -880,8 +927,7 @@ static int tile_n_for(long long m_tiles, int V, int n_heads, int num_sms) {
 int gemm_launches(int M, int n_heads) { return n_heads * M <= kFusedMergeMaxRows ? 2 : 3; }
 
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
-    return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads) +
-           fused_scratch_bytes(n_heads * M);
+    return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads);
 }
 
 ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
@@ -913,18 +959,25 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         mg.exit_mask[k] = heads[k].exit_mask;
         mg.top2gap[k] = heads[k].top2gap;
     }
+    Control* ctrl = reinterpret_cast<Control*>(ws);
     const dim3 row_grid((a.M + 7) / 8, n_heads);
     const dim3 ln_grid((a.M + BM - 1) / BM * (BM / 8), n_heads);
     cudaError_t err;
     if (a.row_idx || a.m_dev) {
         if (n_heads != 1) return EE_ERR_SHAPE;
         err = launch_pdl(layer_norm_gather_kernel, dim3(ln_grid.x), 256, 0, a.stream, ln.h[0], a.ld_h, a.gamma, a.beta,
-                         a.ln_eps, a.row_idx, a.m_dev, y, a.M, a.d);
-    } else if (a.d <= 512) err = launch_pdl(layer_norm_rows_kernel<2>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else if (a.d <= 1024) err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else if (a.d <= 2048) err = launch_pdl(layer_norm_rows_kernel<8>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else if (a.d <= 2560) err = launch_pdl(layer_norm_rows_kernel<10>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
-    else err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, 256, 0, a.stream, ln, a.ln_eps, y, a.M, a.d);
+                         a.ln_eps, a.row_idx, a.m_dev, y, a.M, a.d, ctrl);
+    } else {
+        const int m_pad = (a.M + BM - 1) / BM * BM;
+        auto launch_ln = [&](auto kernel, int threads, size_t smem) {
+            return launch_pdl(kernel, dim3(m_pad / (threads / 32), n_heads), threads, smem, a.stream, ln, a.ln_eps, y, a.M, a.d, ctrl);
+        };
+        if (a.d <= 512) err = launch_ln(layer_norm_rows_kernel<2>, ln_threads(2), 0);
+        else if (a.d <= 1024) err = launch_ln(layer_norm_rows_kernel<4>, ln_threads(4), 0);
+        else if (a.d <= 2048) err = launch_ln(layer_norm_rows_kernel<8>, ln_threads(8), (size_t)8 * a.d);
+        else if (a.d <= 2560) err = launch_ln(layer_norm_rows_kernel<10>, ln_threads(10), (size_t)8 * a.d);
+        else err = launch_ln(layer_norm_rows_kernel<0>, ln_threads(0), 0);
+    }
     if (err != cudaSuccess) return EE_ERR_CUDA;
 
     // 256-byte L2 promotion for the weights while they are read about once: a tile load touches 128 bytes of
@@ -955,26 +1008,19 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.bn = bn;
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
-    {
-        unsigned char* scratch = reinterpret_cast<unsigned char*>(y) + y_bytes(a.M, a.d, n_heads);
-        const size_t entries = (size_t)(kGemmMaxCtas + kGemmMaxCtas / kMergeGroup) * n_heads * a.M;
-        p.cta_part = reinterpret_cast<State*>(scratch);
-        p.cta_top2 = reinterpret_cast<float2*>(scratch + align_up(entries * sizeof(State), 256));
-    }
     p.mg = mg;
-    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m, p.fused_merge ? fused_smem_bytes(n_heads * a.M) : 0);
-    const int max_ctas = p.fused_merge ? kGemmMaxCtas : (1 << 30);
+    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m, (a.d > 1024 && a.d <= 2560) ? (size_t)8 * a.d + 2048 : 0);
     ee_status st;
     if (pair) {
         const long long total = (long long)n_heads * (p.m_tiles / 2) * p.n_tiles;
-        const int grid = 2 * (int)std::min<long long>(std::min<long long>(total, n_pairs), max_ctas / 2);
+        const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
         st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, true>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<256, false, true>(maps, p, grid, a.device, a.stream))
                           : (p.second ? launch_gemm<0, true, true>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<0, false, true>(maps, p, grid, a.device, a.stream));
     } else {
         const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
-        const int grid = (int)std::min<long long>(std::min<long long>(total, a.num_sms), max_ctas);
+        const int grid = (int)(total < a.num_sms ? total : a.num_sms);
         st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, false>(maps, p, grid, a.device, a.stream)
                                       : launch_gemm<256, false, false>(maps, p, grid, a.device, a.stream))
                           : (p.second ? launch_gemm<0, true, false>(maps, p, grid, a.device, a.stream)

@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constan
         return;
     }
     const uint4* hrow = reinterpret_cast<const uint4*>(a.h[which] + (size_t)row * a.ld_h[which]);
-    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, 1.0 / (double)d, a.ln_eps[which], lane);
+    const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, a.ln_eps[which], lane);
     for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, a.gamma[which], a.beta[which], c);
 }
 

@@ -102,29 +102,9 @@ __device__ __forceinline__ bool fill_activations(const SkinnyParams& p, const Sk
     auto vec = [&](int r, int c) { return y_vec<N>(y_tiles, r, c); };
     for (int r = p.M + w; r < N; r += n_warps)                    // padding rows
         for (int c = lane; c < nvec; c += 32) *vec(r, c) = make_uint4(0, 0, 0, 0);
-    if (nvec <= 256) {
-        // Rows held in registers: one pass over shared memory, two rows at a time.
-        if (nvec <= 128) {
-            for (int r = w; r < p.M; r += 2 * n_warps) {
-                const int rows[2] = {r, r + n_warps};
-                layer_norm_rows_in_regs<2, 4>(vec, rows, 1 + (rows[1] < p.M), nvec, p.ln_eps, gamma_s, beta_s, lane);
-            }
-        } else {
-            for (int r = w; r < p.M; r += n_warps) {
-                const int rows[1] = {r};
-                layer_norm_rows_in_regs<1, 8>(vec, rows, 1, nvec, p.ln_eps, gamma_s, beta_s, lane);
-            }
-        }
-    } else {
-        for (int r = w; r < p.M; r += n_warps) {
-            const RowStats st = row_stats_strided([&](int c) { return *vec(r, c); }, nvec, 1.0 / (double)p.d, p.ln_eps, lane);
-            for (int c = lane; c < nvec; c += 32) {
-                const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
-                const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-                uint4* v = vec(r, c);
-                *v = layer_norm_vec8(*v, st, g4[0], g4[1], b4[0], b4[1]);
-            }
-        }
+    for (int r = w; r < p.M; r += 2 * n_warps) {                  // two rows at a time
+        const int rows[2] = {r, r + n_warps};
+        layer_norm_rows_in_smem<2>(vec, rows, 1 + (rows[1] < p.M), nvec, p.ln_eps, gamma_s, beta_s, lane);
     }
     ptx::fence_proxy_async();                                     // y was written by threads, is read by the MMA
     return true;

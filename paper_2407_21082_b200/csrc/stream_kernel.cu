@@ -122,23 +122,7 @@ __device__ void layer_norm_in_smem(const StreamParams& p, __nv_bfloat16* y_s, co
     for (int r0 = w; r0 < MPAD; r0 += 2 * nw) {
         const int rows[2] = {r0, r0 + nw};
         const int live = (rows[0] < p.M) + (rows[1] < MPAD && rows[1] < p.M);
-        if (live > 0) {
-            if (nvec <= 128) {
-                layer_norm_rows_in_regs<2, 4>(vec, rows, live, nvec, p.ln_eps, gamma_s, beta_s, lane);
-            } else if (nvec <= 256) {
-                layer_norm_rows_in_regs<2, 8>(vec, rows, live, nvec, p.ln_eps, gamma_s, beta_s, lane);
-            } else {
-                for (int i = 0; i < live; ++i) {
-                    uint4* yrow = vec(rows[i], 0);
-                    const RowStats st = row_stats_strided([&](int c) { return yrow[c]; }, nvec, 1.0 / (double)p.d, p.ln_eps, lane);
-                    for (int c = lane; c < nvec; c += 32) {
-                        const float4* g4 = reinterpret_cast<const float4*>(gamma_s) + 2 * c;
-                        const float4* b4 = reinterpret_cast<const float4*>(beta_s) + 2 * c;
-                        yrow[c] = layer_norm_vec8(yrow[c], st, g4[0], g4[1], b4[0], b4[1]);
-                    }
-                }
-            }
-        }
+        if (live > 0) layer_norm_rows_in_smem<2>(vec, rows, live, nvec, p.ln_eps, gamma_s, beta_s, lane);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int r = rows[i];
