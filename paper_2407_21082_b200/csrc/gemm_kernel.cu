@@ -617,10 +617,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
 
 // ---------------------------------------------------------------------------------------------
 // LayerNorm of every head's input: h_k [M, d] (row stride ld_h) -> y [k][M, d] bf16, one warp per row,
-// blockIdx.y = head.  With VPL > 0 the row stays in registers (VPL 16-byte vectors per lane, d <= 256 * VPL)
-// and is read once; VPL = 0 re-reads it from global memory per pass.  No shared memory and at most 128 registers,
-// so that a CTA fits on an SM beside a CTA of the call before (which holds nearly all of the shared memory) and
-// is resident, its parameters fetched, when that call completes.
+// blockIdx.y = head.  With VPL > 0 (rows of up to 1024 columns) the row stays in registers (VPL 16-byte vectors per
+// lane, d <= 256 * VPL) and is read once; VPL = 0 (rows beyond 4096 columns) re-reads it from global memory per
+// pass.  No shared memory and few enough registers that a CTA fits on an SM beside a CTA of the call before (which
+// holds nearly all of the shared memory) and is resident, its parameters fetched, when that call completes.
 // ---------------------------------------------------------------------------------------------
 // The first kernel of every call zeroes the counters of the in-kernel merge (it passes its dependency wait only
 // after the call before has completed, so nobody is looking at them).
@@ -639,13 +639,12 @@ struct LnHeads {
     const float* beta[kGemmMaxHeads];
 };
 
-// Threads per CTA: four warps when the rows are held in registers.  With up to 1024 columns a CTA then stays under
-// 24 K registers and uses no shared memory, so it fits on an SM beside a CTA of the GEMM kernel; wider rows stage
-// their parameters in shared memory and take their place as the CTAs of the call before leave.
+// Threads per CTA: four warps when the rows are held in registers; a CTA then stays under 24 K registers, what an SM
+// has left beside a CTA of the GEMM kernel.
 __host__ __device__ constexpr int ln_threads(int vpl) { return vpl > 0 ? 128 : 256; }
 
 template <int VPL>
-__global__ void __launch_bounds__(ln_threads(VPL), VPL >= 8 ? 2 : 3)
+__global__ void __launch_bounds__(ln_threads(VPL), 3)
 layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bfloat16* __restrict__ y_all, int M, int d,
                        Control* ctrl) {
     launch_dependents();
@@ -656,20 +655,10 @@ layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bf
     const int nvec = d >> 3;
     const float* gamma = hs.gamma[head];
     const float* beta = hs.beta[head];
-    // The LayerNorm parameters are weights, not results of an earlier kernel: they are fetched before the wait,
-    // because a load from L2 after it costs about a microsecond while the next call's weight stream is running.
-    // Narrow rows keep them in registers (sixteen per vector); wide rows stage them in shared memory
-    // (2 * d * 4 bytes of dynamic shared memory, one copy for the CTA's four rows).
-    constexpr bool kParamsInRegs = VPL > 0 && VPL < 8;
-    extern __shared__ float ln_params[];
-    float4 g[kParamsInRegs ? VPL : 1][2], b[kParamsInRegs ? VPL : 1][2];
-    if constexpr (VPL >= 8) {
-        for (int i = threadIdx.x; i < (d >> 2); i += ln_threads(VPL)) {
-            reinterpret_cast<float4*>(ln_params)[i] = __ldg(reinterpret_cast<const float4*>(gamma) + i);
-            reinterpret_cast<float4*>(ln_params + d)[i] = __ldg(reinterpret_cast<const float4*>(beta) + i);
-        }
-        __syncthreads();
-    }
+    // The LayerNorm parameters are weights, not results of an earlier kernel: they are fetched before the wait, into
+    // registers (sixteen per vector), because a load from L2 after it costs about a microsecond while the next
+    // call's weight stream is running.
+    float4 g[VPL > 0 ? VPL : 1][2], b[VPL > 0 ? VPL : 1][2];
     if (row >= m_pad) return;
     uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * m_pad + row) * d);
     if (row >= M) {
@@ -682,29 +671,16 @@ layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bf
     const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
     if constexpr (VPL > 0) {
         const double dd = (double)d, inv_d = 1.0 / dd;       // a division: some thirty dependent operations, done before the wait
-        if constexpr (kParamsInRegs) {
 #pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-                const int c = lane + 32 * k;
-                if (c < nvec) {
-                    g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
-                    g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
-                    b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
-                    b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
-                }
+        for (int k = 0; k < VPL; ++k) {
+            const int c = lane + 32 * k;
+            if (c < nvec) {
+                g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+                g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+                b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+                b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
             }
         }
-        // The parameters of vector c (columns 8c .. 8c + 7), wherever they are kept.
-        auto params = [&](int k, int c, float4& g0, float4& g1, float4& b0, float4& b1) {
-            if constexpr (kParamsInRegs) {
-                g0 = g[k][0]; g1 = g[k][1]; b0 = b[k][0]; b1 = b[k][1];
-            } else {
-                g0 = reinterpret_cast<const float4*>(ln_params)[2 * c];
-                g1 = reinterpret_cast<const float4*>(ln_params)[2 * c + 1];
-                b0 = reinterpret_cast<const float4*>(ln_params + d)[2 * c];
-                b1 = reinterpret_cast<const float4*>(ln_params + d)[2 * c + 1];
-            }
-        };
         // h may be an earlier kernel's output, so it is read after the wait; asking L2 for its lines before
         // the wait is harmless (L2 is the point of coherence) and hides a DRAM round trip when h is not cached.
 #pragma unroll
@@ -735,34 +711,88 @@ layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bf
             var = warp_sum_d(q0 + q1) * inv_d;
         }
         const RowStats st = row_stats(mu, var, ln_eps);
-        uint32_t doubts[VPL];
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             const int c = lane + 32 * k;
-            doubts[k] = 0;
-            if (c < nvec) {
-                float4 g0, g1, b0, b1;
-                params(k, c, g0, g1, b0, b1);
-                yrow[c] = layer_norm_vec8_fast(x[k], st, g0, g1, b0, b1, doubts[k]);
-            }
-        }
-        // The few elements fp64 has to decide, after the loop: the doubtful elements of a vector are replaced.
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int c = lane + 32 * k;
-            if (doubts[k]) {
-                float4 g0, g1, b0, b1;
-                params(k, c, g0, g1, b0, b1);
-                uint32_t again;                              // recomputed rather than read back: a load would cost a round trip
-                const uint4 y = layer_norm_vec8_fast(x[k], st, g0, g1, b0, b1, again);
-                yrow[c] = layer_norm_vec8_redo_inline(x[k], y, st.mu, st.rstd, g0, g1, b0, b1, doubts[k]);
-            }
+            if (c < nvec) yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
         }
     } else {
         grid_dependency_wait();
         reset_merge_counters(ctrl);
         const RowStats st = row_stats_strided([&](int c) { return ld_dep(hrow + c); }, nvec, ln_eps, lane);
         for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, gamma, beta, c);
+    }
+}
+
+// Rows wider than 1024 columns: one CTA of four warps per row, VPL 16-byte vectors per thread (d <= 1024 * VPL), so
+// that a row's work -- 64 and more elements per lane if one warp took it -- is a quarter as long.  The warps' moments
+// meet in shared memory (64 bytes; summed in a fixed order).  Parameters in registers, fetched before the wait.
+template <int VPL>
+__global__ void __launch_bounds__(128, 3)
+layer_norm_wide_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bfloat16* __restrict__ y_all, int M, int d,
+                            Control* ctrl) {
+    __shared__ double part[2][4][2];
+    launch_dependents();
+    const int row = blockIdx.x, head = blockIdx.y;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m_pad = (M + BM - 1) / BM * BM;
+    const int nvec = d >> 3;
+    uint4* yrow = reinterpret_cast<uint4*>(y_all + ((size_t)head * m_pad + row) * d);
+    if (row >= M) {                                      // padding row (the whole CTA)
+        grid_dependency_wait();
+        for (int c = tid; c < nvec; c += 128) yrow[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const uint4* hrow = reinterpret_cast<const uint4*>(hs.h[head] + (size_t)row * hs.ld_h[head]);
+    const float* gamma = hs.gamma[head];
+    const float* beta = hs.beta[head];
+    const double dd = (double)d, inv_d = 1.0 / dd;
+    float4 g[VPL][2], b[VPL][2];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int c = tid + 128 * k;
+        if (c < nvec) {
+            g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
+            g[k][1] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+            b[k][0] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c);
+            b[k][1] = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+            if ((c & 7) == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(hrow + c));
+        }
+    }
+    grid_dependency_wait();                              // y may still be read by the GEMM of the call before
+    reset_merge_counters(ctrl);
+    uint4 x[VPL];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int c = tid + 128 * k;
+        x[k] = c < nvec ? ld_dep(hrow + c) : make_uint4(0, 0, 0, 0);
+    }
+    Moments m;
+    m.clear();
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) m.add(x[k], k);
+    double s = m.sum(), q = m.sum_sq();
+    warp_sum2_d(s, q);
+    if (lane == 0) { part[0][warp][0] = s; part[0][warp][1] = q; }
+    __syncthreads();
+    s = (part[0][0][0] + part[0][1][0]) + (part[0][2][0] + part[0][3][0]);
+    q = (part[0][0][1] + part[0][1][1]) + (part[0][2][1] + part[0][3][1]);
+    double mu, var;
+    if (!row_variance_one_pass(s, q, dd, inv_d, mu, var)) {          // the same decision in every thread of the CTA
+        double q0 = 0.0, q1 = 0.0;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (tid + 128 * k < nvec) vec8_sqdev_d(x[k], mu, q0, q1);
+        q0 = warp_sum_d(q0 + q1);
+        if (lane == 0) part[1][warp][0] = q0;
+        __syncthreads();
+        var = ((part[1][0][0] + part[1][1][0]) + (part[1][2][0] + part[1][3][0])) * inv_d;
+    }
+    const RowStats st = row_stats(mu, var, ln_eps);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int c = tid + 128 * k;
+        if (c < nvec) yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
     }
 }
 
@@ -817,11 +847,9 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* partials_a
 constexpr int kMinTileN = 64;
 constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
 // Ring depth for a runtime tile width; b_rows = rows of W one CTA stages per k-block.
-// `reserve`: shared memory left free on the SM for a CTA of the next call's LayerNorm kernel, which for rows wider
-// than 1024 columns stages its parameters there; without it that CTA would keep the next GEMM CTA off the SM.
-int stages_for(int b_rows, int mma_m, size_t reserve) {
+int stages_for(int b_rows, int mma_m) {
     const size_t stage = (size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2;
-    const size_t n = (kGemmSmemBudget - reserve - kBarBytes - 1024) / stage;
+    const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
 
@@ -972,10 +1000,14 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         auto launch_ln = [&](auto kernel, int threads, size_t smem) {
             return launch_pdl(kernel, dim3(m_pad / (threads / 32), n_heads), threads, smem, a.stream, ln, a.ln_eps, y, a.M, a.d, ctrl);
         };
+        auto launch_wide = [&](auto kernel) {
+            return launch_pdl(kernel, dim3(m_pad, n_heads), 128, 0, a.stream, ln, a.ln_eps, y, a.M, a.d, ctrl);
+        };
         if (a.d <= 512) err = launch_ln(layer_norm_rows_kernel<2>, ln_threads(2), 0);
         else if (a.d <= 1024) err = launch_ln(layer_norm_rows_kernel<4>, ln_threads(4), 0);
-        else if (a.d <= 2048) err = launch_ln(layer_norm_rows_kernel<8>, ln_threads(8), (size_t)8 * a.d);
-        else if (a.d <= 2560) err = launch_ln(layer_norm_rows_kernel<10>, ln_threads(10), (size_t)8 * a.d);
+        else if (a.d <= 2048) err = launch_wide(layer_norm_wide_rows_kernel<2>);
+        else if (a.d <= 3072) err = launch_wide(layer_norm_wide_rows_kernel<3>);
+        else if (a.d <= 4096) err = launch_wide(layer_norm_wide_rows_kernel<4>);
         else err = launch_ln(layer_norm_rows_kernel<0>, ln_threads(0), 0);
     }
     if (err != cudaSuccess) return EE_ERR_CUDA;
@@ -1009,7 +1041,7 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
     p.mg = mg;
-    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m, (a.d > 1024 && a.d <= 2560) ? (size_t)8 * a.d + 2048 : 0);
+    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
     ee_status st;
     if (pair) {
         const long long total = (long long)n_heads * (p.m_tiles / 2) * p.n_tiles;
