@@ -134,7 +134,7 @@ class Workload:
             self.k = 8
             self.S = self.M // self.k
         self.tau = torch.from_numpy(cfg["tau_per_row"]).cuda() if "tau_per_row" in cfg else float(cfg["tau"])
-        self.multi = self.multi and len(self.heads) > 1 and len({hh.data_ptr() for hh in self.h}) >= 1
+        # one prepared plan for all heads of the step (a single head included): a call only launches
         ws_bytes = max(ee.ee_exit_head_workspace_bytes(self.M, self.d, self.V),
                        ee.ee_exit_head_multi_workspace_bytes(len(self.heads), self.M, self.d, self.V))
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
@@ -848,12 +848,12 @@ def main():
                             launch=dict(heads=heads_per_launch, algorithmic_bytes=heads_per_launch * wl.bytes_per_call,
                                         flops=heads_per_launch * wl.flops_per_call,
                                         us=heads_per_launch * res["head_call_us"]))
-    line["roofline"]["kernel"] = (("ee_exit_head_multi: %d heads in one launch; " % n_heads if wl.multi else
+    line["roofline"]["kernel"] = (("ee_exit_head_plan_run: %d head(s) in one launch sequence; " % n_heads if wl.multi else
                                    "one ee_exit_head call (%d launch(es)); " % wl.head_launches) +
                                   "duration = CUDA events around `steps` consecutive head evaluations (no event between launches: "
                                   "one would break their programmatic dependent launch chain), averaged per head; "
                                   "tail_us = step time minus that")
-    config["heads_call"] = "ee_exit_head_multi" if wl.multi else "ee_exit_head per head"
+    config["heads_call"] = ("ee_exit_head_plan_run (plan of all heads, initialised once)" if wl.multi else "ee_exit_head_path per head")
     gpu_outs = [{k: v.cpu().numpy() for k, v in o.items()} for o in wl.outs] if rank == 0 else None
     if rank == 0:
         line["e2e"] = measure_e2e(wl, max(10, args.steps // 4), 3)

@@ -129,6 +129,30 @@ int       ee_exit_head_multi_launches(int n_heads, int M, int d, int V);   /* ke
 ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * ee_exit_head_multi in two steps, for a call that is repeated with the same buffers (a decoding loop): the host
+ * work of a call -- argument checks, tensor maps of the weights, tile width, launch shapes, environment overrides --
+ * is done once by ee_exit_head_plan_init into a caller-owned, fixed-size plan (plain data, no allocation, nothing
+ * to release), and ee_exit_head_plan_run only launches (two or three kernel launches per four heads).  Same
+ * passages, results and workspace as ee_exit_head_multi; up to EE_PLAN_MAX_HEADS heads.  Every pointer given at
+ * initialisation (the heads' inputs, parameters, weights, thresholds, outputs, the workspace) is captured: the
+ * buffers must stay where they are, their CONTENTS may change between runs.  The device that is current at
+ * initialisation must be current at every run; a plan may be run on any stream, one run at a time (it shares its
+ * workspace).  ee_exit_head_plan_run_host is the plan's counterpart of ee_exit_head_multi_host: h_host (h_bytes,
+ * pinned for an asynchronous copy) is copied to h_dev, the plan is run, results_dev (results_bytes) is copied to
+ * results_host; the plan must have been initialised with heads whose h and outputs lie inside h_dev and results_dev.
+ */
+#define EE_PLAN_MAX_HEADS 16
+#define EE_EXIT_HEAD_PLAN_BYTES (64 + (EE_PLAN_MAX_HEADS / 4) * 2048)
+typedef struct {
+    unsigned long long opaque[EE_EXIT_HEAD_PLAN_BYTES / 8];
+} ee_exit_head_plan;
+ee_status ee_exit_head_plan_init(ee_exit_head_plan* plan, const ee_head* heads, int n_heads, float ln_eps, int M, int d,
+                                 int V, void* workspace, size_t workspace_bytes);
+ee_status ee_exit_head_plan_run(const ee_exit_head_plan* plan, void* stream);
+ee_status ee_exit_head_plan_run_host(const ee_exit_head_plan* plan, const void* h_host, void* h_dev, size_t h_bytes,
+                                     void* results_host, const void* results_dev, size_t results_bytes, void* stream);
+
 /* Same operation with the kernel chosen by the caller (`path` is an ee_path); used to cross-check the
  * kernels against each other and to time them separately. */
 ee_status ee_exit_head_path(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,

@@ -16,5 +16,5 @@ from .exit_head import (  # noqa: F401
 )
 from .calibrate import calibrate_threshold, calibrate_threshold_bruteforce, correctness  # noqa: F401,E402
 from .cascade import cascade  # noqa: F401,E402
-from .dssd_round import dssd_commit, dssd_round  # noqa: F401,E402
+from .dssd_round import dssd_commit, dssd_round, dssd_round_multi  # noqa: F401,E402
 from .kl_loss import ce_from_logits, kl_from_logits, kl_to_teacher  # noqa: F401,E402

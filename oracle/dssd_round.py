@@ -92,3 +92,54 @@ def dssd_round(E_draft, E_verify, draft_head, verify_head, tau: float, eos: int,
             last_tok[s] = out_tok[s, seq_len[s] - 1]
     return dict(draft_tok=draft, draft_mask=mask, verify_tok=verify, steps=steps, verify_out=v, **r)
 
+
+
+def dssd_round_multi(E_drafts, E_verify, draft_heads, verify_head, taus, eos: int, k: int, last_tok, out_tok, seq_len,
+                     finished, stats, head_use) -> dict:
+    """One whole DSSD round with K draft heads (paper section 4.3.1, drafting phase: at every position the heads
+    are tried from the shallowest to the deepest and the first one whose entropy is below its threshold supplies
+    the token; a position that no head is sure of ends the draft -- stop (iii), the fallback to the full model).
+
+    E_drafts[h] is the table of hidden states at head h's layer (row = previous token), draft_heads[h] that head,
+    taus[h] its threshold.  Step j runs oracle.cascade on the S rows of the step: a sequence's token and
+    confidence at position j are those of the answering head; where no head answers the slot is not confident and
+    carries the deepest head's argmax (never committed: the draft stopped before it; it only feeds the later,
+    ignored steps).  Verification and commit as in dssd_round.  head_use [K] (int64) accumulates, over the sequences
+    that took part, the positions inside the draft (j < draft_len) supplied by each head: the head-usage figure of
+    the paper's DSSD experiments; the mean exit head is sum(h * head_use[h]) / sum(head_use).
+    """
+    from .cascade import cascade
+    from .exit_head import exit_head
+    K = len(draft_heads)
+    S = last_tok.size
+    cur = last_tok.astype(np.int64).copy()
+    draft = np.zeros((S, k), np.int32)
+    mask = np.zeros((S, k), np.uint8)
+    which = np.full((S, k), K, np.int32)
+    steps = []
+    for j in range(k):
+        c = cascade([E[cur] for E in E_drafts], draft_heads, taus)
+        tok = c["token"].copy()
+        none = c["exit_head"] == K
+        if none.any():                                   # the deepest head saw exactly the rows nobody answered before it
+            last = c["per_head"][K - 1]
+            pos = {int(r): i for i, r in enumerate(last["rows"])}
+            for s in np.flatnonzero(none):
+                tok[s] = last["argmax"][pos[int(s)]]
+        draft[:, j], mask[:, j], which[:, j] = tok, (~none).astype(np.uint8), c["exit_head"]
+        cur = tok.astype(np.int64)
+        steps.append(c)
+    prev_all = np.concatenate([last_tok.astype(np.int64)[:, None], draft.astype(np.int64)], axis=1)
+    v = exit_head(E_verify[prev_all.reshape(-1)], verify_head["gamma"], verify_head["beta"], verify_head["ln_eps"],
+                  verify_head["W"], np.inf)
+    verify = v["argmax"].reshape(S, k + 1).astype(np.int32)
+    was_finished = finished.copy()
+    r = dssd_commit(draft, mask, verify, eos, out_tok, seq_len, finished, stats)
+    for s in range(S):
+        if was_finished[s]:
+            continue
+        if seq_len[s] > 0:
+            last_tok[s] = out_tok[s, seq_len[s] - 1]
+        for j in range(int(r["draft_len"][s])):
+            head_use[which[s, j]] += 1
+    return dict(draft_tok=draft, draft_mask=mask, draft_head=which, verify_tok=verify, steps=steps, verify_out=v, **r)

@@ -29,6 +29,15 @@ class EEDssdRoundArgs(C.Structure):
                 ("stream", _p)]
 
 
+EE_PLAN_MAX_HEADS = 16
+EE_EXIT_HEAD_PLAN_BYTES = 64 + (EE_PLAN_MAX_HEADS // 4) * 2048
+
+
+class EEExitHeadPlan(C.Structure):
+    """Mirror of `ee_exit_head_plan` in include/eexit.h (opaque storage)."""
+    _fields_ = [("opaque", C.c_ulonglong * (EE_EXIT_HEAD_PLAN_BYTES // 8))]
+
+
 class EEHiddenTables(C.Structure):
     """Mirror of `ee_hidden_tables` in include/eexit.h."""
     _fields_ = [("table", _p * 2), ("d", C.c_int), ("V", C.c_int), ("chained", C.c_int)]
@@ -46,6 +55,10 @@ PROTOTYPES = {
     "ee_exit_head_multi_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "ee_exit_head_multi_launches": (C.c_int, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "ee_exit_head_multi": (C.c_int, [C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, _p, C.c_size_t, _p]),
+    "ee_exit_head_plan_init": (C.c_int, [C.POINTER(EEExitHeadPlan), C.POINTER(EEHead), C.c_int, C.c_float, C.c_int, C.c_int, C.c_int,
+                                         _p, C.c_size_t]),
+    "ee_exit_head_plan_run": (C.c_int, [C.POINTER(EEExitHeadPlan), _p]),
+    "ee_exit_head_plan_run_host": (C.c_int, [C.POINTER(EEExitHeadPlan), _p, _p, C.c_size_t, _p, _p, C.c_size_t, _p]),
     "ee_exit_head_path": (C.c_int, [_p, C.c_longlong, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,
                                     _p, _p, _p, _p, _p, C.c_size_t, _p, C.c_int]),
     "ee_exit_head_host": (C.c_int, [_p, _p, _p, _p, C.c_float, _p, C.c_int, C.c_int, C.c_int, _p, C.c_float,

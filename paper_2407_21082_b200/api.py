@@ -197,14 +197,26 @@ def ee_exit_head_multi(heads, ln_eps, *, workspace=None) -> list:
 
 
 class PreparedMulti:
-    """ee_exit_head_multi with its argument block built once (see PreparedCall)."""
-    __slots__ = ("_args", "_keep", "out")
+    """ee_exit_head_multi for a loop that repeats the call: the host work (argument checks, tensor maps, launch shapes)
+    is done once here (ee_exit_head_plan_init) and a call only launches (ee_exit_head_plan_run) on the stream that was
+    current at preparation time.  More heads than a plan takes fall back to ee_exit_head_multi with its argument
+    block built once."""
+    __slots__ = ("_args", "_keep", "out", "_plan", "_stream", "_run")
 
     def __init__(self, heads, ln_eps, workspace=None):
+        import ctypes as C
         self._args, self.out, self._keep = _multi_args(heads, ln_eps, workspace)
+        self._plan = None
+        arr, n, eps, M, d, V, ws, ws_bytes, stream = self._args
+        if 1 <= n <= _lib.EE_PLAN_MAX_HEADS and M >= 1:
+            self._plan = _lib.EEExitHeadPlan()
+            _check(_lib.load().ee_exit_head_plan_init(C.byref(self._plan), arr, n, eps, M, d, V, ws, ws_bytes), "ee_exit_head_plan_init")
+            self._stream = C.c_void_p(stream)
+            self._plan = C.byref(self._plan), self._plan          # the reference passed to C, and the object it refers to
+            self._run = _lib.load().ee_exit_head_plan_run
 
     def __call__(self):
-        code = _lib.load().ee_exit_head_multi(*self._args)
+        code = self._run(self._plan[0], self._stream) if self._plan is not None else _lib.load().ee_exit_head_multi(*self._args)
         if code:
             raise EExitError(code, "ee_exit_head_multi")
         return self.out
@@ -248,7 +260,7 @@ class PreparedMultiHost:
     [n_heads, M, d].  The staging buffers and the pinned result block are created here, once; `out_host`
     and `out_dev` are per-head views into the packed result blocks.
     """
-    __slots__ = ("_args", "_keep", "out_host", "out_dev", "h_dev", "h2d_bytes", "d2h_bytes")
+    __slots__ = ("_args", "_keep", "out_host", "out_dev", "h_dev", "h2d_bytes", "d2h_bytes", "_plan")
 
     def __init__(self, heads, ln_eps, h_host, workspace):
         n, (_, M, d) = len(heads), h_host.shape
@@ -263,6 +275,7 @@ class PreparedMultiHost:
             e = arr[i]
             e.gamma, e.beta, e.W, e.tau_per_row, e.tau = _ptr(hd["gamma"]), _ptr(hd["beta"]), _ptr(W), _ptr(tau_t), tau_f
             keep.append((W, hd["gamma"], hd["beta"], tau_t))
+        import ctypes as C
         nbytes = ee_exit_head_results_bytes(n, M)
         self.h_dev = torch.empty((n, M, d), dtype=torch.bfloat16, device=dev)
         res_dev = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
@@ -272,9 +285,25 @@ class PreparedMultiHost:
         self._args = (arr, n, float(ln_eps), M, d, V, _ptr(h_host), _ptr(self.h_dev), _ptr(res_host), _ptr(res_dev),
                       _ptr(workspace), workspace.numel(), _stream())
         self._keep = (arr, keep, h_host, res_dev, res_host, workspace)
+        self._plan = None
+        if 1 <= n <= _lib.EE_PLAN_MAX_HEADS and M >= 1:
+            # the plan's heads read their rows from the staging buffer and write into the packed device results
+            for i in range(n):
+                e, o = arr[i], self.out_dev[i]
+                e.h, e.ld_h = self.h_dev[i].data_ptr(), d
+                e.argmax, e.entropy, e.maxprob, e.exit_mask = (_ptr(o[k]) for k in ("argmax", "entropy", "maxprob", "exit_mask"))
+            plan = _lib.EEExitHeadPlan()
+            _check(_lib.load().ee_exit_head_plan_init(C.byref(plan), arr, n, float(ln_eps), M, d, V, _ptr(workspace), workspace.numel()),
+                   "ee_exit_head_plan_init")
+            self._plan = (C.byref(plan), plan, C.c_void_p(_ptr(h_host)), C.c_void_p(_ptr(self.h_dev)), C.c_size_t(self.h2d_bytes),
+                          C.c_void_p(_ptr(res_host)), C.c_void_p(_ptr(res_dev)), C.c_size_t(nbytes), C.c_void_p(_stream()))
 
     def __call__(self):
-        code = _lib.load().ee_exit_head_multi_host(*self._args)
+        if self._plan is not None:
+            p = self._plan
+            code = _lib.load().ee_exit_head_plan_run_host(p[0], p[2], p[3], p[4], p[5], p[6], p[7], p[8])
+        else:
+            code = _lib.load().ee_exit_head_multi_host(*self._args)
         if code:
             raise EExitError(code, "ee_exit_head_multi_host")
         return self.out_host

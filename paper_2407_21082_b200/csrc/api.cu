@@ -224,6 +224,76 @@ ee_status ee_exit_head_multi(const ee_head* heads, int n_heads, float ln_eps, in
     return EE_OK;
 }
 
+namespace {
+struct PlanHeader {
+    int n_groups;
+    int device;
+    int pad[14];
+};
+static_assert(sizeof(PlanHeader) == 64, "plan header");
+static_assert(EE_EXIT_HEAD_PLAN_BYTES == 64 + (EE_PLAN_MAX_HEADS / kHeadsPerLaunch) * kGemmPlanBytes, "plan size in eexit.h");
+}  // namespace
+
+ee_status ee_exit_head_plan_init(ee_exit_head_plan* plan, const ee_head* heads, int n_heads, float ln_eps, int M, int d, int V,
+                                 void* workspace, size_t workspace_bytes_) {
+    if (!plan) return EE_ERR_NULL;
+    if (!sizes_ok(M, d, V) || n_heads < 1 || n_heads > EE_PLAN_MAX_HEADS || M < 1) return EE_ERR_SHAPE;
+    if (!heads || !workspace) return EE_ERR_NULL;
+    if (!aligned(workspace, 256)) return EE_ERR_ALIGN;
+    if (workspace_bytes_ < ee_exit_head_multi_workspace_bytes(n_heads, M, d, V)) return EE_ERR_WORKSPACE;
+    for (int k = 0; k < n_heads; ++k) {
+        const ee_head& e = heads[k];
+        if (!e.h || !e.gamma || !e.beta || !e.W || !e.argmax || !e.entropy || !e.maxprob || !e.exit_mask) return EE_ERR_NULL;
+        if (e.ld_h < d || (e.ld_h % 8) != 0) return EE_ERR_SHAPE;
+        if (!aligned(e.h, 16) || !aligned(e.W, 16) || !aligned(e.gamma, 16) || !aligned(e.beta, 16)) return EE_ERR_ALIGN;
+    }
+    HeadArgs base{};
+    const ee_status dev = current_device(&base.device, &base.num_sms);
+    if (dev != EE_OK) return dev;
+    unsigned char* bytes = reinterpret_cast<unsigned char*>(plan->opaque);
+    PlanHeader* hdr = reinterpret_cast<PlanHeader*>(bytes);
+    memset(hdr, 0, sizeof(*hdr));
+    hdr->device = base.device;
+    for (int k0 = 0; k0 < n_heads; k0 += kHeadsPerLaunch) {
+        HeadArgs a[kHeadsPerLaunch];
+        const int n = n_heads - k0 < kHeadsPerLaunch ? n_heads - k0 : kHeadsPerLaunch;
+        for (int k = 0; k < n; ++k) {
+            const ee_head& e = heads[k0 + k];
+            a[k] = base;
+            a[k].h = e.h; a[k].ld_h = e.ld_h; a[k].gamma = e.gamma; a[k].beta = e.beta; a[k].ln_eps = ln_eps; a[k].W = e.W;
+            a[k].M = M; a[k].d = d; a[k].V = V; a[k].tau_per_row = e.tau_per_row; a[k].tau = e.tau;
+            a[k].argmax = e.argmax; a[k].entropy = e.entropy; a[k].maxprob = e.maxprob; a[k].exit_mask = e.exit_mask;
+            a[k].workspace = workspace; a[k].workspace_bytes = workspace_bytes_;
+        }
+        const ee_status st = gemm_plan(a, n, bytes + sizeof(PlanHeader) + (size_t)hdr->n_groups * kGemmPlanBytes);
+        if (st != EE_OK) return st;
+        ++hdr->n_groups;
+    }
+    return EE_OK;
+}
+
+ee_status ee_exit_head_plan_run(const ee_exit_head_plan* plan, void* stream) {
+    if (!plan) return EE_ERR_NULL;
+    const unsigned char* bytes = reinterpret_cast<const unsigned char*>(plan->opaque);
+    const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(bytes);
+    if (hdr->n_groups < 1 || hdr->n_groups > EE_PLAN_MAX_HEADS / kHeadsPerLaunch) return EE_ERR_SHAPE;      // not initialised
+    for (int g = 0; g < hdr->n_groups; ++g) {
+        const ee_status st = gemm_run(bytes + sizeof(PlanHeader) + (size_t)g * kGemmPlanBytes, static_cast<cudaStream_t>(stream));
+        if (st != EE_OK) return st;
+    }
+    return EE_OK;
+}
+
+ee_status ee_exit_head_plan_run_host(const ee_exit_head_plan* plan, const void* h_host, void* h_dev, size_t h_bytes,
+                                     void* results_host, const void* results_dev, size_t results_bytes, void* stream) {
+    if (!plan || !h_host || !h_dev || !results_host || !results_dev) return EE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(h_dev, h_host, h_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return EE_ERR_CUDA;
+    const ee_status st = ee_exit_head_plan_run(plan, stream);
+    if (st != EE_OK) return st;
+    return cudaMemcpyAsync(results_host, results_dev, results_bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
 ee_status ee_exit_head(const void* h, long long ld_h, const float* gamma, const float* beta, float ln_eps,
                        const void* W, int M, int d, int V, const float* tau_per_row, float tau, int* argmax,
                        float* entropy, float* maxprob, unsigned char* exit_mask, void* workspace,

@@ -11,6 +11,8 @@
 //                      one 16-byte partial state per (row, vocabulary tile)
 // All mbarrier waits are bounded; a wait that gives up records an error word, raises the CTA's abort
 // flag, and every role drains to the common exit where TMEM is released.
+#include <string.h>
+
 #include "common.cuh"
 #include "kernels.h"
 #include "layer_norm.cuh"
@@ -128,6 +130,7 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
+    int l2_prefetch;       // k-blocks of W beyond the ring that a CTA asks into L2 before the dependency wait (0: none)
     MergeHeads mg;
 };
 
@@ -323,6 +326,21 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     load_tile(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
                               load_full_bar(kb));
                     armed |= 1u << kb;
+                }
+            }
+            // A head whose weights fit in L2 several times over: what the ring cannot hold of this CTA's weight
+            // tiles is asked into L2 now, while the call before finishes and the LayerNorm runs -- HBM is idle
+            // then -- so that after the wait those tiles come from L2.  Every byte of W still crosses HBM once.
+            if (p.l2_prefetch > 0 && worker < total_tiles) {
+                int left = p.l2_prefetch, skip = n_pre;
+                for (int tile = worker; left > 0 && tile < total_tiles; tile += n_workers) {
+                    int head, m_tile, n_tile;
+                    locate(tile, head, m_tile, n_tile);
+                    for (int kb = 0; left > 0 && kb < p.k_blocks; ++kb) {
+                        if (skip > 0) { --skip; continue; }
+                        ptx::tma_prefetch_2d(&maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows);
+                        --left;
+                    }
                 }
             }
             grid_dependency_wait();
@@ -958,8 +976,33 @@ size_t gemm_workspace_bytes(int M, int d, int V, int n_heads) {
     return (size_t)n_heads * (partials_bytes(M, V) + second_bytes(M, V)) + y_bytes(M, d, n_heads);
 }
 
-ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
+// Everything one call needs but the launches themselves: kernel arguments (tensor maps included), launch shapes and
+// which instantiations to use.  Filled by gemm_plan from the heads' arguments (and, once per process, the
+// environment); gemm_run launches from it on any stream.  Plain data: a caller may keep it in memory of its own.
+namespace {
+struct GemmPlan {
+    LnHeads ln;
+    const int* row_idx;
+    const int* m_dev;
+    unsigned char maps[sizeof(GemmMaps)];      // copied to an aligned object for the launch
+    GemmParams p;
+    __nv_bfloat16* y;
+    float ln_eps;
+    int device;
+    int ln_kind;                               // 2, 4: rows in registers; -2, -3, -4: one CTA per row; 0: re-read; 100: gathered rows
+    int ln_grid_x, ln_threads;
+    int gemm_grid;
+    int pair, wide, top2;                      // GEMM instantiation
+    int merge_grid_x;                          // 0: the GEMM kernel merges itself
+};
+static_assert(sizeof(GemmPlan) <= kGemmPlanBytes, "kGemmPlanBytes in kernels.h is too small");
+static_assert(alignof(GemmPlan) <= 8, "a plan lives in caller memory aligned to 8 bytes");
+}  // namespace
+
+ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     if (n_heads < 1 || n_heads > kGemmMaxHeads) return EE_ERR_SHAPE;
+    GemmPlan& g = *static_cast<GemmPlan*>(storage);
+    memset(&g, 0, sizeof(g));
     const HeadArgs& a = heads[0];
     unsigned char* ws = static_cast<unsigned char*>(a.workspace);
     State* partials = reinterpret_cast<State*>(ws + kCtrlBytes);
@@ -972,13 +1015,12 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     const int bn = !pair ? gemm_tile_n(a.M, a.V, n_heads, a.num_sms)
                          : (a.M > 1024 ? 256 : tile_n_for(m_tiles / 2, a.V, n_heads, n_pairs));
 
-    LnHeads ln = {};
     MergeHeads mg = {};
     for (int k = 0; k < n_heads; ++k) {
-        ln.h[k] = static_cast<const __nv_bfloat16*>(heads[k].h);
-        ln.ld_h[k] = heads[k].ld_h;
-        ln.gamma[k] = heads[k].gamma;
-        ln.beta[k] = heads[k].beta;
+        g.ln.h[k] = static_cast<const __nv_bfloat16*>(heads[k].h);
+        g.ln.ld_h[k] = heads[k].ld_h;
+        g.ln.gamma[k] = heads[k].gamma;
+        g.ln.beta[k] = heads[k].beta;
         mg.tau_per_row[k] = heads[k].tau_per_row;
         mg.tau[k] = heads[k].tau;
         mg.argmax[k] = heads[k].argmax;
@@ -987,30 +1029,22 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
         mg.exit_mask[k] = heads[k].exit_mask;
         mg.top2gap[k] = heads[k].top2gap;
     }
-    Control* ctrl = reinterpret_cast<Control*>(ws);
-    const dim3 row_grid((a.M + 7) / 8, n_heads);
-    const dim3 ln_grid((a.M + BM - 1) / BM * (BM / 8), n_heads);
-    cudaError_t err;
+    g.y = y;
+    g.ln_eps = a.ln_eps;
+    g.device = a.device;
+    g.row_idx = a.row_idx;
+    g.m_dev = a.m_dev;
+    const int m_pad = m_tiles * BM;
     if (a.row_idx || a.m_dev) {
         if (n_heads != 1) return EE_ERR_SHAPE;
-        err = launch_pdl(layer_norm_gather_kernel, dim3(ln_grid.x), 256, 0, a.stream, ln.h[0], a.ld_h, a.gamma, a.beta,
-                         a.ln_eps, a.row_idx, a.m_dev, y, a.M, a.d, ctrl);
+        g.ln_kind = 100; g.ln_threads = 256; g.ln_grid_x = m_pad / 8;
+    } else if (a.d <= 1024) {
+        g.ln_kind = a.d <= 512 ? 2 : 4; g.ln_threads = ln_threads(g.ln_kind); g.ln_grid_x = m_pad / (g.ln_threads / 32);
+    } else if (a.d <= 4096) {
+        g.ln_kind = a.d <= 2048 ? -2 : (a.d <= 3072 ? -3 : -4); g.ln_threads = 128; g.ln_grid_x = m_pad;
     } else {
-        const int m_pad = (a.M + BM - 1) / BM * BM;
-        auto launch_ln = [&](auto kernel, int threads, size_t smem) {
-            return launch_pdl(kernel, dim3(m_pad / (threads / 32), n_heads), threads, smem, a.stream, ln, a.ln_eps, y, a.M, a.d, ctrl);
-        };
-        auto launch_wide = [&](auto kernel) {
-            return launch_pdl(kernel, dim3(m_pad, n_heads), 128, 0, a.stream, ln, a.ln_eps, y, a.M, a.d, ctrl);
-        };
-        if (a.d <= 512) err = launch_ln(layer_norm_rows_kernel<2>, ln_threads(2), 0);
-        else if (a.d <= 1024) err = launch_ln(layer_norm_rows_kernel<4>, ln_threads(4), 0);
-        else if (a.d <= 2048) err = launch_wide(layer_norm_wide_rows_kernel<2>);
-        else if (a.d <= 3072) err = launch_wide(layer_norm_wide_rows_kernel<3>);
-        else if (a.d <= 4096) err = launch_wide(layer_norm_wide_rows_kernel<4>);
-        else err = launch_ln(layer_norm_rows_kernel<0>, ln_threads(0), 0);
+        g.ln_kind = 0; g.ln_threads = ln_threads(0); g.ln_grid_x = m_pad / (g.ln_threads / 32);
     }
-    if (err != cudaSuccess) return EE_ERR_CUDA;
 
     // 256-byte L2 promotion for the weights while they are read about once: a tile load touches 128 bytes of
     // each row, and fetching the neighbouring 128 bytes (the next k-block's) with it lets the row-strided
@@ -1021,12 +1055,13 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)) return EE_ERR_CUDA;
     for (int k = 0; k < kGemmMaxHeads; ++k)
         if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, pair ? bn / 2 : bn, promo)) return EE_ERR_CUDA;
+    memcpy(g.maps, &maps, sizeof(maps));
 
-    GemmParams p;
+    GemmParams& p = g.p;
     p.M = a.M;
     p.V = a.V;
     p.d = a.d;
-    p.m_tiles = (a.M + BM - 1) / BM;
+    p.m_tiles = m_tiles;
     p.n_tiles = (a.V + bn - 1) / bn;
     p.k_blocks = (a.d + BK - 1) / BK;
     p.n_heads = n_heads;
@@ -1040,30 +1075,67 @@ ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
     p.bn = bn;
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
+    // Up to 64 MB of weights per launch (half of L2): the tiles beyond the ring are prefetched into L2.
+    p.l2_prefetch = (a.M <= 1024 && (double)n_heads * a.V * a.d * 2.0 <= 64e6) ? 64 : 0;
     p.mg = mg;
     p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
-    ee_status st;
+    g.pair = pair ? 1 : 0;
+    g.wide = a.M > 1024 ? 1 : 0;
+    g.top2 = p.second ? 1 : 0;
     if (pair) {
         const long long total = (long long)n_heads * (p.m_tiles / 2) * p.n_tiles;
-        const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
-        st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, true>(maps, p, grid, a.device, a.stream)
-                                      : launch_gemm<256, false, true>(maps, p, grid, a.device, a.stream))
-                          : (p.second ? launch_gemm<0, true, true>(maps, p, grid, a.device, a.stream)
-                                      : launch_gemm<0, false, true>(maps, p, grid, a.device, a.stream));
+        g.gemm_grid = 2 * (int)(total < n_pairs ? total : n_pairs);
     } else {
         const long long total = (long long)n_heads * p.m_tiles * p.n_tiles;
-        const int grid = (int)(total < a.num_sms ? total : a.num_sms);
-        st = (a.M > 1024) ? (p.second ? launch_gemm<256, true, false>(maps, p, grid, a.device, a.stream)
-                                      : launch_gemm<256, false, false>(maps, p, grid, a.device, a.stream))
-                          : (p.second ? launch_gemm<0, true, false>(maps, p, grid, a.device, a.stream)
-                                      : launch_gemm<0, false, false>(maps, p, grid, a.device, a.stream));
+        g.gemm_grid = (int)(total < a.num_sms ? total : a.num_sms);
     }
-    if (st != EE_OK) return st;
-    if (p.fused_merge) return EE_OK;
+    g.merge_grid_x = p.fused_merge ? 0 : (a.M + 7) / 8;
+    // the kernels' shared-memory attributes are per device and set once: done here, so that gemm_run only launches
+    ee_status st = EE_OK;
+    if (g.pair) st = g.wide ? (g.top2 ? configure_gemm<256, true, true>(g.device) : configure_gemm<256, false, true>(g.device))
+                            : (g.top2 ? configure_gemm<0, true, true>(g.device) : configure_gemm<0, false, true>(g.device));
+    else st = g.wide ? (g.top2 ? configure_gemm<256, true, false>(g.device) : configure_gemm<256, false, false>(g.device))
+                     : (g.top2 ? configure_gemm<0, true, false>(g.device) : configure_gemm<0, false, false>(g.device));
+    return st;
+}
 
-    err = launch_pdl(merge_rows_kernel, row_grid, 256, 0, a.stream, (const State*)partials, (const float*)p.second, p.n_tiles,
-                     a.M, mg);
+ee_status gemm_run(const void* storage, cudaStream_t stream) {
+    const GemmPlan& g = *static_cast<const GemmPlan*>(storage);
+    const GemmParams& p = g.p;
+    const dim3 ln_grid(g.ln_grid_x, p.n_heads);
+    cudaError_t err;
+    switch (g.ln_kind) {
+        case 100: err = launch_pdl(layer_norm_gather_kernel, dim3(g.ln_grid_x), 256, 0, stream, g.ln.h[0], g.ln.ld_h[0], g.ln.gamma[0],
+                                   g.ln.beta[0], g.ln_eps, g.row_idx, g.m_dev, g.y, p.M, p.d, p.ctrl); break;
+        case 2: err = launch_pdl(layer_norm_rows_kernel<2>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case 4: err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -2: err = launch_pdl(layer_norm_wide_rows_kernel<2>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -3: err = launch_pdl(layer_norm_wide_rows_kernel<3>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -4: err = launch_pdl(layer_norm_wide_rows_kernel<4>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        default: err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+    }
+    if (err != cudaSuccess) return EE_ERR_CUDA;
+    GemmMaps maps;
+    memcpy(&maps, g.maps, sizeof(maps));
+    ee_status st;
+    if (g.pair) st = g.wide ? (g.top2 ? launch_gemm<256, true, true>(maps, p, g.gemm_grid, g.device, stream)
+                                      : launch_gemm<256, false, true>(maps, p, g.gemm_grid, g.device, stream))
+                            : (g.top2 ? launch_gemm<0, true, true>(maps, p, g.gemm_grid, g.device, stream)
+                                      : launch_gemm<0, false, true>(maps, p, g.gemm_grid, g.device, stream));
+    else st = g.wide ? (g.top2 ? launch_gemm<256, true, false>(maps, p, g.gemm_grid, g.device, stream)
+                               : launch_gemm<256, false, false>(maps, p, g.gemm_grid, g.device, stream))
+                     : (g.top2 ? launch_gemm<0, true, false>(maps, p, g.gemm_grid, g.device, stream)
+                               : launch_gemm<0, false, false>(maps, p, g.gemm_grid, g.device, stream));
+    if (st != EE_OK || g.merge_grid_x == 0) return st;
+    err = launch_pdl(merge_rows_kernel, dim3(g.merge_grid_x, p.n_heads), 256, 0, stream, (const State*)p.partials,
+                     (const float*)p.second, p.n_tiles, p.M, p.mg);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
+}
+
+ee_status gemm_launch(const HeadArgs* heads, int n_heads) {
+    alignas(8) unsigned char storage[kGemmPlanBytes];
+    const ee_status st = gemm_plan(heads, n_heads, storage);
+    return st != EE_OK ? st : gemm_run(storage, heads[0].stream);
 }
 
 }  // namespace ee

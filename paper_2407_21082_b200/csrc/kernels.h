@@ -63,6 +63,12 @@ constexpr int kGemmLaunchMaxHeads = 4;
 int gemm_tile_n(int M, int V, int n_heads, int num_sms);   // vocabulary tile width used for M rows on num_sms SMs
 size_t gemm_workspace_bytes(int M, int d, int V, int n_heads);
 ee_status gemm_launch(const HeadArgs* heads, int n_heads);
+// The same in two steps, for calls that are repeated: gemm_plan works out everything but the launches (tensor maps,
+// tile width, launch shapes, instantiations) into `storage` (kGemmPlanBytes bytes, 8-byte aligned, plain data),
+// gemm_run launches from it on `stream`.
+constexpr size_t kGemmPlanBytes = 2048;
+ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage);
+ee_status gemm_run(const void* storage, cudaStream_t stream);
 int gemm_launches(int M, int n_heads);     // kernels one gemm_launch call starts
 
 // ---- compaction and DSSD accept ----

@@ -385,3 +385,38 @@ def test_calls_in_flight_on_several_streams(ee, M, d, V, n_heads, n_streams):
             for key in ref[k]:
                 assert torch.equal(outs[k][key], ref[k][key]), (k, key)
             assert_head_matches(outs[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"{n_streams} streams head {k}")
+
+
+def test_plan_runs_equal_the_one_step_call_and_follow_the_buffers_contents(ee):
+    """ee_exit_head_plan_init / ee_exit_head_plan_run: the same results as ee_exit_head_multi, bit for bit, run after
+    run; the plan captures pointers, not contents, so new rows written into the same buffer give the new rows' results."""
+    import ctypes as C
+    from paper_2407_21082_b200 import _lib
+    for M, d, V, n_heads in ((64, 256, 5000, 3), (300, 136, 3001, 5), (8, 512, 50304, 1), (256, 2048, 4000, 2)):
+        cfg = gen.make_config("c1", seed=61, planted=True, M=M, d=d, V=V, heads=n_heads)
+        other = gen.make_config("c1", seed=62, planted=True, M=M, d=d, V=V, heads=n_heads)
+        hds = [head_to_dev(hd) for hd in cfg["heads"]]
+        h = dev_bf16(cfg["h"])
+        heads = [dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=1.0) for hd in hds]
+        ref = [{k: v.clone() for k, v in o.items()} for o in ee.ee_exit_head_multi(heads, 1e-5)]
+        call = ee.PreparedMulti(heads, 1e-5)
+        assert call._plan is not None
+        for rep in range(3):
+            outs = call()
+            torch.cuda.synchronize()
+            for k in range(n_heads):
+                for key in ref[k]:
+                    assert torch.equal(outs[k][key], ref[k][key]), (M, k, key, rep)
+        h.copy_(dev_bf16(other["h"]))                                 # same buffer, other rows
+        outs = call()
+        torch.cuda.synchronize()
+        for k in range(n_heads):
+            assert_head_matches(outs[k], oracle_head(other["h"], cfg["heads"][k], 1.0), label=f"plan, new rows, head {k}")
+    # argument errors are found at initialisation; a plan that was never initialised does not run
+    plan = _lib.EEExitHeadPlan()
+    lib = _lib.load()
+    assert lib.ee_exit_head_plan_run(C.byref(plan), None) == 2
+    arr = (_lib.EEHead * 17)()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    assert lib.ee_exit_head_plan_init(C.byref(plan), arr, 17, 1e-5, 8, 64, 100, ws.data_ptr(), ws.numel()) == 2      # too many heads
+    assert lib.ee_exit_head_plan_init(C.byref(plan), arr, 1, 1e-5, 8, 64, 100, ws.data_ptr(), ws.numel()) == 1       # NULL pointers

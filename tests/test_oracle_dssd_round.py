@@ -118,3 +118,81 @@ def test_round_reduces_to_greedy_decoding_in_the_two_limits():
     for s in range(S):
         assert np.array_equal(st[0][s, :st[1][s]], want[s, :st[1][s]])
     assert 3 * S <= st[1].sum() <= 3 * (k + 1) * S and st[3][1] <= st[3][0]
+
+
+def _model3(seed=0, V=400, d=64, sigmas=(1.2, 0.6)):
+    """Three heads on three tables: two noisy drafting layers (the shallower one noisier) and the full model."""
+    cfg = gen.make_config("c1", seed=seed, planted=True, M=4, d=d, V=V, heads=3)
+    planting = gen.make_planting(seed, f"c1/planted/d{d}/V{V}", d, V)
+    tables = [gen.make_markov_model(seed + 10 * i, V, d, planting, sigma=sg) for i, sg in enumerate(sigmas)]
+    return cfg, [t["E_draft"] for t in tables], tables[0]["E_verify"], tables
+
+
+def _fresh(S, cap):
+    return (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+
+
+def test_round_with_one_draft_head_is_the_single_head_round():
+    cfg, mm = _model()
+    S, k, cap = 9, 5, 40
+    start = np.arange(S, dtype=np.int32) * 11 % 400
+    a, b = _fresh(S, cap), _fresh(S, cap)
+    la, lb = start.copy(), start.copy()
+    use = np.zeros(1, np.int64)
+    for _ in range(3):
+        ra = oracle.dssd_round(mm["E_draft"], mm["E_verify"], cfg["heads"][0], cfg["heads"][1], 1.0, -1, k, la, *a)
+        rb = oracle.dssd_round_multi([mm["E_draft"]], mm["E_verify"], [cfg["heads"][0]], cfg["heads"][1], [1.0], -1, k, lb, *b, use)
+        for key in ("draft_len", "accept_len", "next_tok", "draft_mask"):
+            assert np.array_equal(ra[key], rb[key]), key
+        live = rb["draft_mask"] != 0                                    # tokens of confident slots are the head's own
+        assert np.array_equal(ra["draft_tok"][live], rb["draft_tok"][live])
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+    assert np.array_equal(la, lb) and use[0] == a[3][0]                 # every drafted position came from the one head
+
+
+def test_multi_head_round_position_by_position_is_the_cascade():
+    cfg, E_drafts, E_verify, _ = _model3()
+    S, k, cap = 24, 4, 40
+    start = (np.arange(S, dtype=np.int32) * 7 + 3) % 400
+    st, last, use = _fresh(S, cap), start.copy(), np.zeros(2, np.int64)
+    taus = [0.5, 1.5]
+    r = oracle.dssd_round_multi(E_drafts, E_verify, cfg["heads"][:2], cfg["heads"][2], taus, -1, k, last, *st, use)
+    cur = start.astype(np.int64)
+    for j in range(k):
+        c = oracle.cascade([E[cur] for E in E_drafts], cfg["heads"][:2], taus)       # the same rows, evaluated independently
+        assert np.array_equal(r["draft_head"][:, j], c["exit_head"])
+        answered = c["exit_head"] < 2
+        assert np.array_equal(r["draft_mask"][:, j], answered.astype(np.uint8))
+        assert np.array_equal(r["draft_tok"][answered, j], c["token"][answered])
+        # first head whose entropy is below its threshold, checked from every head's own evaluation
+        H = [oracle.exit_head(E[cur], hd["gamma"], hd["beta"], hd["ln_eps"], hd["W"], t)["entropy"]
+             for E, hd, t in zip(E_drafts, cfg["heads"][:2], taus)]
+        first = np.where(H[0] < taus[0], 0, np.where(H[1] < taus[1], 1, 2))
+        assert np.array_equal(first, c["exit_head"])
+        cur = r["draft_tok"][:, j].astype(np.int64)
+    # usage counts only positions inside the draft, of sequences that took part
+    want = np.zeros(2, np.int64)
+    for s in range(S):
+        for j in range(r["draft_len"][s]):
+            want[r["draft_head"][s, j]] += 1
+    assert np.array_equal(use, want) and use.sum() == st[3][0] and (r["draft_head"][r["draft_mask"] == 0] == 2).all()
+    assert use[0] > 0 and use[1] > 0                                    # both heads supply tokens in this case
+
+
+def test_multi_head_round_commits_the_full_models_greedy_chain():
+    cfg, E_drafts, E_verify, tables = _model3(seed=2)
+    S, k, cap = 8, 6, 80
+    start = np.arange(S, dtype=np.int32) * 13 % 400
+    want = _greedy(dict(E_verify=E_verify), cfg["heads"][2], start, 30)
+    st, last, use = _fresh(S, cap), start.copy(), np.zeros(2, np.int64)
+    for _ in range(4):
+        oracle.dssd_round_multi(E_drafts, E_verify, cfg["heads"][:2], cfg["heads"][2], [1.0, 2.0], -1, k, last, *st, use)
+    for s in range(S):
+        assert np.array_equal(st[0][s, :st[1][s]], want[s, :st[1][s]])
+    assert st[1].sum() > 4 * S                                          # drafts were accepted somewhere
+    # thresholds that nothing passes: one token per round, no head ever used
+    st, last, use = _fresh(S, cap), start.copy(), np.zeros(2, np.int64)
+    for _ in range(3):
+        oracle.dssd_round_multi(E_drafts, E_verify, cfg["heads"][:2], cfg["heads"][2], [-1.0, -1.0], -1, k, last, *st, use)
+    assert (st[1] == 3).all() and use.sum() == 0 and np.array_equal(st[0][:, :3], want[:, :3])
