@@ -130,7 +130,6 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
-    int l2_prefetch;       // k-blocks of W beyond the ring that a CTA asks into L2 before the dependency wait (0: none)
     MergeHeads mg;
 };
 
@@ -326,21 +325,6 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     load_tile(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
                               load_full_bar(kb));
                     armed |= 1u << kb;
-                }
-            }
-            // A head whose weights fit in L2 several times over: what the ring cannot hold of this CTA's weight
-            // tiles is asked into L2 now, while the call before finishes and the LayerNorm runs -- HBM is idle
-            // then -- so that after the wait those tiles come from L2.  Every byte of W still crosses HBM once.
-            if (p.l2_prefetch > 0 && worker < total_tiles) {
-                int left = p.l2_prefetch, skip = n_pre;
-                for (int tile = worker; left > 0 && tile < total_tiles; tile += n_workers) {
-                    int head, m_tile, n_tile;
-                    locate(tile, head, m_tile, n_tile);
-                    for (int kb = 0; left > 0 && kb < p.k_blocks; ++kb) {
-                        if (skip > 0) { --skip; continue; }
-                        ptx::tma_prefetch_2d(&maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows);
-                        --left;
-                    }
                 }
             }
             grid_dependency_wait();
@@ -1075,8 +1059,6 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     p.bn = bn;
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
-    // Up to 64 MB of weights per launch (half of L2): the tiles beyond the ring are prefetched into L2.
-    p.l2_prefetch = (a.M <= 1024 && (double)n_heads * a.V * a.d * 2.0 <= 64e6) ? 64 : 0;
     p.mg = mg;
     p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
     g.pair = pair ? 1 : 0;
