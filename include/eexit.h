@@ -291,28 +291,40 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
 
 /*
  * One whole DSSD round for S sequences (section 4.3.1: drafting phase, verification phase, commit), issued on
- * the stream without any synchronisation.  The transformer is the caller's: `hidden` is called k times for the
- * drafting steps (which = 0: n_rows = S tokens, one per sequence, the token each sequence's next position
- * follows) and once for the verification pass (which = 1: n_rows = S * (k + 1) tokens, row (s, j) = the token
- * before draft position j, j = k being the bonus position); it must enqueue on `stream` work that writes the
- * hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING those tokens to h_out, and return 0.
+ * the stream without any synchronisation.  Drafting uses K >= 1 draft heads, shallowest first: at every position
+ * the first head whose entropy is below its threshold supplies the token (the paper's per-token head selection);
+ * a position that no head is sure of ends the draft (stop iii, the fallback to the full model).
+ * The transformer is the caller's: `hidden` is called K times per drafting step, k steps (which = h, 0 <= h < K:
+ * n_rows = S tokens, one per sequence, the token each sequence's next position follows; the hidden states AT HEAD
+ * h'S LAYER are wanted) and once for the verification pass (which = K: n_rows = S * (k + 1) tokens, row (s, j) =
+ * the token before draft position j, j = k being the bonus position; the full model's final hidden states); it
+ * must enqueue on `stream` work that writes the hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING
+ * those tokens to h_out, and return 0.
  * Both pointers it receives are device buffers inside `workspace`.  The work it enqueues may be ordinary stream
  * work, or kernels launched with programmatic stream serialization that trigger their dependents early -- the
  * round's own kernels are chained that way -- provided every such kernel executes griddepcontrol.wait before it
  * reads `tokens` or writes `h_out`, and reads `tokens` through L2 (ld.global.cg or an equivalent coherent load,
  * not the read-only path): the token buffer is rewritten by a kernel that may still be running when the model's
  * kernel becomes resident.
- *   drafting step j : draft head (heads' gamma, beta, W; draft_head.tau is the threshold) on the step's hidden
- *                     states; argmax = drafted token, exit decision = confidence; the token feeds step j + 1
+ *   drafting step j : the K draft heads (their gamma, beta, W; tau is each head's threshold) on the step's hidden
+ *                     states, all in one launch sequence; per sequence the first confident head's argmax = drafted
+ *                     token; the token feeds step j + 1
  *   verification    : verify head (the full model's; its tau is ignored) on all S * (k + 1) rows
  *   commit          : dssd_commit with kv = k + 1 and the given eos_token; then last_tok[s] = the last token
  *                     committed, for the sequences that took part
  * Every sequence goes through all k drafting steps (what lies beyond its stop is ignored by the commit), so
  * the launch sequence does not depend on device data.  State (device, in/out): last_tok int32 [S], out_tok
  * int32 [S, capacity], seq_len int32 [S], finished uint8 [S], stats int64 [4]; outputs of the round: draft_len,
- * accept_len, next_tok int32 [S].  Workspace: dssd_round_workspace_bytes(S, k, d, V), 256-byte aligned,
- * initialised once with ee_workspace_init.  1 <= k <= 32.
+ * accept_len, next_tok int32 [S].  n_draft_heads = 0 means one draft head, `draft_head` (then `which` is 0 while
+ * drafting and 1 for the verification pass); otherwise draft_heads is a HOST array of n_draft_heads <=
+ * EE_ROUND_MAX_DRAFT_HEADS heads and `draft_head` is ignored.  head_use (device int64 [K], may be NULL) accumulates
+ * over calls, per head, the drafted positions it supplied -- positions inside a draft (j < draft_len) of sequences
+ * that took part: the head-usage statistic of the paper's DSSD experiments (the mean exit head while drafting is
+ * sum h * head_use[h] / sum head_use[h]); the caller zeroes it.
+ * Workspace: dssd_round_multi_workspace_bytes(S, k, d, V, K) (dssd_round_workspace_bytes = the same with K = 1),
+ * 256-byte aligned, initialised once with ee_workspace_init.  1 <= k <= 32.
  */
+#define EE_ROUND_MAX_DRAFT_HEADS 8
 typedef int (*ee_hidden_fn)(void* user, const int* tokens, int n_rows, int which, void* h_out, void* stream);
 typedef struct {
     int S, k, d, V;
@@ -333,22 +345,26 @@ typedef struct {
     void* workspace;
     size_t workspace_bytes;
     void* stream;
+    int n_draft_heads;
+    const ee_head* draft_heads;
+    long long* head_use;
 } ee_dssd_round_args;
 size_t    dssd_round_workspace_bytes(int S, int k, int d, int V);     /* host-only, pure; 0 if a size is invalid */
+size_t    dssd_round_multi_workspace_bytes(int S, int k, int d, int V, int n_draft_heads);
 ee_status dssd_round(const ee_dssd_round_args* args);
 
 /*
  * A ready-made ee_hidden_fn for tests and benchmarks (no counterpart in the paper; the transformer is the
- * caller's): the hidden state of a row is row `token` of a table, table[0] for the drafting steps (which = 0)
- * and table[1] for the verification pass (which = 1), each bf16 [V, d] on the device, contiguous, 16-byte
- * aligned; a token outside [0, V) gives a zero row.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a
- * pointer to an ee_hidden_tables (host memory that outlives the call) as `hidden_user`.  One kernel launch on
- * `stream` per call; returns 0, or 1 if an argument is unusable or the launch failed.  chained = 0: an ordinary
- * launch; chained != 0: the kernel is launched with programmatic stream serialization, lets its dependents start
- * at once and waits for its predecessors before it touches the tokens, like the library's own kernels.
+ * caller's): the hidden state of a row is row `token` of table[which] -- table[h] for draft head h's layer,
+ * table[K] for the verification pass -- each bf16 [V, d] on the device, contiguous, 16-byte aligned; a token
+ * outside [0, V) gives a zero row.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a pointer to an
+ * ee_hidden_tables (host memory that outlives the call) as `hidden_user`.  One kernel launch on `stream` per call;
+ * returns 0, or 1 if an argument is unusable or the launch failed.  chained = 0: an ordinary launch; chained != 0:
+ * the kernel is launched with programmatic stream serialization, lets its dependents start at once and waits for
+ * its predecessors before it touches the tokens, like the library's own kernels.
  */
 typedef struct {
-    const void* table[2];
+    const void* table[EE_ROUND_MAX_DRAFT_HEADS + 1];
     int d, V;
     int chained;
 } ee_hidden_tables;

@@ -17,6 +17,7 @@ class EEHead(C.Structure):
                 ("tau", C.c_float), ("argmax", _p), ("entropy", _p), ("maxprob", _p), ("exit_mask", _p)]
 
 
+EE_ROUND_MAX_DRAFT_HEADS = 8
 HIDDEN_FN = C.CFUNCTYPE(C.c_int, _p, _p, C.c_int, C.c_int, _p, _p)
 
 
@@ -26,7 +27,7 @@ class EEDssdRoundArgs(C.Structure):
                 ("draft_head", EEHead), ("verify_head", EEHead), ("hidden", HIDDEN_FN), ("hidden_user", _p),
                 ("last_tok", _p), ("out_tok", _p), ("capacity", C.c_int), ("seq_len", _p), ("finished", _p), ("stats", _p),
                 ("draft_len", _p), ("accept_len", _p), ("next_tok", _p), ("workspace", _p), ("workspace_bytes", C.c_size_t),
-                ("stream", _p)]
+                ("stream", _p), ("n_draft_heads", C.c_int), ("draft_heads", C.POINTER(EEHead)), ("head_use", _p)]
 
 
 EE_PLAN_MAX_HEADS = 16
@@ -40,7 +41,7 @@ class EEExitHeadPlan(C.Structure):
 
 class EEHiddenTables(C.Structure):
     """Mirror of `ee_hidden_tables` in include/eexit.h."""
-    _fields_ = [("table", _p * 2), ("d", C.c_int), ("V", C.c_int), ("chained", C.c_int)]
+    _fields_ = [("table", _p * (EE_ROUND_MAX_DRAFT_HEADS + 1)), ("d", C.c_int), ("V", C.c_int), ("chained", C.c_int)]
 
 
 PROTOTYPES = {
@@ -74,6 +75,7 @@ PROTOTYPES = {
     "dssd_accept": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, _p, _p, _p, _p]),
     "dssd_commit": (C.c_int, [_p, _p, _p, C.c_int, C.c_int, C.c_int, C.c_int, _p, C.c_int, _p, _p, _p, _p, _p, _p, _p]),
     "dssd_round_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
+    "dssd_round_multi_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "dssd_round": (C.c_int, [C.POINTER(EEDssdRoundArgs)]),
     "ee_hidden_from_tables": (C.c_int, [_p, _p, C.c_int, C.c_int, _p, _p]),
     "ee_compact_accept": (C.c_int, [_p, _p, C.c_longlong, C.c_int, C.c_int, _p, _p, _p,

@@ -585,38 +585,51 @@ def dssd_commit(draft_tok, draft_exit_mask, verify_tok, eos_token, state: dict, 
 
 class TableModel:
     """Stand-in model for dssd_round served by the library itself (ee_hidden_from_tables in include/eexit.h): the
-    hidden state after a token is that token's row of `draft_table` (drafting steps) or `verify_table`
-    (verification pass), bf16 [V, d] device tensors.  Pass it to DssdRound as `hidden_fn`.  chained=True launches
-    its kernel with programmatic stream serialization (early trigger, wait before the tokens are read)."""
+    hidden state after a token is that token's row of a table, one table per draft head's layer (`draft_table`: a
+    tensor, or a list of K tensors, shallowest first) and `verify_table` for the verification pass, bf16 [V, d]
+    device tensors.  Pass it to DssdRound as `hidden_fn`.  chained=True launches its kernel with programmatic stream
+    serialization (early trigger, wait before the tokens are read)."""
 
     def __init__(self, draft_table, verify_table, chained: bool = False):
-        self.tables = (_bf16(_dev(draft_table, "draft_table")), _bf16(_dev(verify_table, "verify_table")))
-        if self.tables[0].shape != self.tables[1].shape or not all(t.is_contiguous() for t in self.tables):
+        drafts = list(draft_table) if isinstance(draft_table, (list, tuple)) else [draft_table]
+        self.tables = tuple(_bf16(_dev(t, "table")) for t in drafts + [verify_table])
+        if len(drafts) > _lib.EE_ROUND_MAX_DRAFT_HEADS:
+            raise ValueError(f"at most {_lib.EE_ROUND_MAX_DRAFT_HEADS} draft tables")
+        if any(t.shape != self.tables[0].shape for t in self.tables) or not all(t.is_contiguous() for t in self.tables):
             raise ValueError("tables must be contiguous and of one shape [V, d]")
         V, d = self.tables[0].shape
         self.struct = _lib.EEHiddenTables()
-        self.struct.table[0], self.struct.table[1] = _ptr(self.tables[0]), _ptr(self.tables[1])
+        for i, t in enumerate(self.tables):
+            self.struct.table[i] = _ptr(t)
         self.struct.d, self.struct.V, self.struct.chained = d, V, int(bool(chained))
 
 
 class DssdRound:
     """dssd_round (see include/eexit.h) with its argument block built once.
 
-    draft_head / verify_head: dicts with gamma, beta, W (and tau for the draft head).  hidden_fn(tokens, which, h_out)
-    is the caller's model: `tokens` int32 [n_rows] and `h_out` bf16 [n_rows, d] are device tensors (views into the
-    workspace); it must fill h_out on the current stream.  `state`: last_tok, out_tok, seq_len, finished, stats."""
+    draft_head: a dict with gamma, beta, W, tau, or a list of K such dicts (shallowest head first: per position the
+    first confident one supplies the token); verify_head: dict with gamma, beta, W.  hidden_fn(tokens, which, h_out) is
+    the caller's model: `tokens` int32 [n_rows] and `h_out` bf16 [n_rows, d] are device tensors (views into the
+    workspace); it must fill h_out on the current stream with the hidden states at draft head `which`'s layer
+    (which < K) or the full model's (which = K).  `state`: last_tok, out_tok, seq_len, finished, stats.  With a list
+    of heads, self.head_use (int64 [K]) accumulates the positions each head supplied."""
 
     def __init__(self, draft_head, verify_head, ln_eps, k, eos_token, hidden_fn, state, workspace=None):
         import ctypes as C
         S = state["last_tok"].numel()
-        Wd, Wv = _bf16(_dev(draft_head["W"], "W")), _bf16(_dev(verify_head["W"], "W"))
-        V, d = Wd.shape
-        dev = Wd.device
+        multi = isinstance(draft_head, (list, tuple))
+        drafts = list(draft_head) if multi else [draft_head]
+        K = len(drafts)
+        Wd = [_bf16(_dev(h["W"], "W")) for h in drafts]
+        Wv = _bf16(_dev(verify_head["W"], "W"))
+        V, d = Wd[0].shape
+        dev = Wd[0].device
         if workspace is None:
-            workspace = torch.empty(int(_lib.load().dssd_round_workspace_bytes(S, k, d, V)), dtype=torch.uint8, device=dev)
+            workspace = torch.empty(int(_lib.load().dssd_round_multi_workspace_bytes(S, k, d, V, K)), dtype=torch.uint8, device=dev)
             ee_workspace_init(workspace)
         self.workspace, self.state = workspace, state
         self.out = {n: torch.empty(S, dtype=torch.int32, device=dev) for n in ("draft_len", "accept_len", "next_tok")}
+        self.head_use = torch.zeros(K, dtype=torch.int64, device=dev) if multi else None
         base = workspace.data_ptr()
 
         def trampoline(user, tokens_ptr, n_rows, which, h_ptr, stream):
@@ -631,19 +644,22 @@ class DssdRound:
                 return 1
 
         native = isinstance(hidden_fn, TableModel)
-        if native and hidden_fn.tables[0].shape != (V, d):
-            raise ValueError("the table model's tables must be [V, d]")
+        if native and (hidden_fn.tables[0].shape != (V, d) or len(hidden_fn.tables) != K + 1):
+            raise ValueError("the table model needs one [V, d] table per draft head and one for the verification pass")
         self._cb = C.cast(_lib.load().ee_hidden_from_tables, _lib.HIDDEN_FN) if native else _lib.HIDDEN_FN(trampoline)
         a = _lib.EEDssdRoundArgs()
         a.S, a.k, a.d, a.V, a.ln_eps, a.eos_token = S, int(k), d, V, float(ln_eps), int(eos_token)
-        for dst, src, W in ((a.draft_head, draft_head, Wd), (a.verify_head, verify_head, Wv)):
+        arr = (_lib.EEHead * K)()
+        for dst, src, W in [(arr[i], drafts[i], Wd[i]) for i in range(K)] + [(a.draft_head, drafts[0], Wd[0]), (a.verify_head, verify_head, Wv)]:
             dst.gamma, dst.beta, dst.W, dst.tau = _ptr(src["gamma"]), _ptr(src["beta"]), _ptr(W), float(src.get("tau", 0.0))
+        if multi:
+            a.n_draft_heads, a.draft_heads, a.head_use = K, arr, _ptr(self.head_use)
         a.hidden, a.hidden_user = self._cb, (C.cast(C.pointer(hidden_fn.struct), C.c_void_p) if native else None)
         a.last_tok, a.out_tok, a.capacity = _ptr(state["last_tok"]), _ptr(state["out_tok"]), state["out_tok"].shape[1]
         a.seq_len, a.finished, a.stats = _ptr(state["seq_len"]), _ptr(state["finished"]), _ptr(state["stats"])
         a.draft_len, a.accept_len, a.next_tok = (_ptr(self.out[n]) for n in ("draft_len", "accept_len", "next_tok"))
         a.workspace, a.workspace_bytes, a.stream = _ptr(workspace), workspace.numel(), _stream()
-        self._args, self._keep = a, (Wd, Wv, draft_head, verify_head, C, hidden_fn)
+        self._args, self._keep = a, (Wd, Wv, drafts, verify_head, C, hidden_fn, arr)
 
     def __call__(self):
         import ctypes as C

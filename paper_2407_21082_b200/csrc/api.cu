@@ -538,34 +538,43 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
 }
 
 namespace {
-ee_status round_head_call(const void* h, const ee_head& head, float ln_eps, int M, int d, int V, float tau, int* argmax,
-                          float* entropy, float* maxprob, unsigned char* mask, void* ws, size_t ws_bytes, void* stream) {
-    return ee_exit_head(h, d, head.gamma, head.beta, ln_eps, head.W, M, d, V, nullptr, tau, argmax, entropy, maxprob, mask, ws,
-                        ws_bytes, stream);
+// Scratch of the heads inside a round: the verification pass's single head on S (k + 1) rows, or the K draft heads
+// of a step on S rows, whichever needs more.
+size_t round_head_ws(int S, int k, int d, int V, int K) {
+    const size_t verify = workspace_bytes(S * (k + 1), d, V), draft = ee_exit_head_multi_workspace_bytes(K, S, d, V);
+    return verify > draft ? verify : draft;
+}
+bool round_sizes_ok(int S, int k, int d, int V, int K) {
+    return S >= 0 && k >= 1 && k <= 32 && K >= 1 && K <= EE_ROUND_MAX_DRAFT_HEADS && sizes_ok(S * (k + 1), d, V);
 }
 }  // namespace
 
-size_t dssd_round_workspace_bytes(int S, int k, int d, int V) {
-    if (S < 0 || k < 1 || k > 32 || !sizes_ok(S * (k + 1), d, V)) return 0;
-    return dssd_round_layout_bytes(S, k, d, V, workspace_bytes(S * (k + 1), d, V));
+size_t dssd_round_multi_workspace_bytes(int S, int k, int d, int V, int n_draft_heads) {
+    if (!round_sizes_ok(S, k, d, V, n_draft_heads)) return 0;
+    return dssd_round_layout_bytes(S, k, d, n_draft_heads, round_head_ws(S, k, d, V, n_draft_heads));
 }
+
+size_t dssd_round_workspace_bytes(int S, int k, int d, int V) { return dssd_round_multi_workspace_bytes(S, k, d, V, 1); }
 
 ee_status dssd_round(const ee_dssd_round_args* a) {
     if (!a) return EE_ERR_NULL;
-    if (a->S < 0 || a->k < 1 || a->k > 32 || a->capacity < 1 || !sizes_ok(a->S * (a->k + 1), a->d, a->V)) return EE_ERR_SHAPE;
+    if (a->n_draft_heads < 0) return EE_ERR_SHAPE;
+    const int K = a->n_draft_heads ? a->n_draft_heads : 1;
+    const ee_head* draft = a->n_draft_heads ? a->draft_heads : &a->draft_head;
+    if (a->capacity < 1 || !round_sizes_ok(a->S, a->k, a->d, a->V, K)) return EE_ERR_SHAPE;
     if (a->S == 0) return EE_OK;
     if (!a->hidden || !a->last_tok || !a->out_tok || !a->seq_len || !a->finished || !a->stats || !a->draft_len ||
-        !a->accept_len || !a->next_tok || !a->workspace)
+        !a->accept_len || !a->next_tok || !a->workspace || !draft)
         return EE_ERR_NULL;
-    if (!a->draft_head.gamma || !a->draft_head.beta || !a->draft_head.W || !a->verify_head.gamma || !a->verify_head.beta ||
-        !a->verify_head.W)
-        return EE_ERR_NULL;
+    for (int h = 0; h < K; ++h)
+        if (!draft[h].gamma || !draft[h].beta || !draft[h].W) return EE_ERR_NULL;
+    if (!a->verify_head.gamma || !a->verify_head.beta || !a->verify_head.W) return EE_ERR_NULL;
     if (!aligned(a->workspace, 256)) return EE_ERR_ALIGN;
-    if (a->workspace_bytes < dssd_round_workspace_bytes(a->S, a->k, a->d, a->V)) return EE_ERR_WORKSPACE;
+    if (a->workspace_bytes < dssd_round_multi_workspace_bytes(a->S, a->k, a->d, a->V, K)) return EE_ERR_WORKSPACE;
     int device, num_sms;
     const ee_status dev = current_device(&device, &num_sms);
     if (dev != EE_OK) return dev;
-    return dssd_round_run(*a, workspace_bytes(a->S * (a->k + 1), a->d, a->V), round_head_call);
+    return dssd_round_run(*a, draft, K, round_head_ws(a->S, a->k, a->d, a->V, K));
 }
 
 size_t ee_head_kl_workspace_bytes(int M, int d, int V) {

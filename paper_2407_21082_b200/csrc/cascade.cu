@@ -31,9 +31,7 @@ __global__ void __launch_bounds__(kStepThreads) cascade_step_kernel(const unsign
     const int m = m_in ? min(max(ld_dep(m_in), 0), M) : M;
     const int row0 = blockIdx.x * kStepRows;
     if (blockIdx.x == 0 && threadIdx.x == 0) rows_in[k] = m;
-    int cnt = 0;
-    const int upto = min(row0, m);
-    for (int i = threadIdx.x; i < upto; i += kStepThreads) cnt += (ld_dep(exit_mask + i) == 0);
+    int cnt = zero_bytes_share(exit_mask, min(row0, m), threadIdx.x, kStepThreads);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     if (lane == 0) s_warp_cnt[warp] = cnt;

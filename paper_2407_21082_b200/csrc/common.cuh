@@ -173,6 +173,23 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 template <class T>
 __device__ __forceinline__ T ld_dep(const T* p) { return __ldcg(p); }
 
+// This thread's share of the number of zero bytes among mask[0 .. n) (a mask an earlier kernel may have written):
+// sixteen bytes per load once the address is aligned, four bytes per comparison.  The threads' shares add up to
+// the count; used by the kernels that rank surviving rows.
+__device__ __forceinline__ int zero_bytes_share(const unsigned char* mask, int n, int tid, int n_threads) {
+    int cnt = 0;
+    const int head = min(n, (int)((16u - (unsigned)(reinterpret_cast<uintptr_t>(mask) & 15u)) & 15u));
+    for (int i = tid; i < head; i += n_threads) cnt += ld_dep(mask + i) == 0;
+    const int n_vec = (n - head) >> 4;
+    const uint4* v = reinterpret_cast<const uint4*>(mask + head);
+    for (int i = tid; i < n_vec; i += n_threads) {
+        const uint4 w = ld_dep(v + i);
+        cnt += (__popc(__vcmpeq4(w.x, 0u)) + __popc(__vcmpeq4(w.y, 0u)) + __popc(__vcmpeq4(w.z, 0u)) + __popc(__vcmpeq4(w.w, 0u))) >> 3;
+    }
+    for (int i = head + (n_vec << 4) + tid; i < n; i += n_threads) cnt += ld_dep(mask + i) == 0;
+    return cnt;
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 

@@ -11,7 +11,9 @@ constexpr int kCompactThreads = 256;
 constexpr int kRowsPerCta = 32;           // one ballot's worth of rows per CTA
 
 // CTA b owns rows [32b, 32b + 32).  Its output offset is the number of surviving rows before 32b, which it
-// counts itself from the mask (M bytes at most, L2-resident), so no CTA waits for another.
+// counts itself from the mask (M bytes at most, L2-resident, sixteen bytes per load), so no CTA waits for another
+// and the call needs no scratch memory; over all CTAs that is M^2 / 1024 loads -- four megabytes of L2 traffic for
+// 16 K rows, 160 MB for 100 K rows.
 __device__ __forceinline__ void compact_body(int cta, const unsigned char* exit_mask,
                                              const __nv_bfloat16* h, long long ld_h, int M, int d,
                                              int* kept_idx, int* kept_count,
@@ -22,8 +24,7 @@ __device__ __forceinline__ void compact_body(int cta, const unsigned char* exit_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row0 = cta * kRowsPerCta;
 
-    int cnt = 0;
-    for (int i = threadIdx.x; i < row0; i += kCompactThreads) cnt += (ld_dep(exit_mask + i) == 0);
+    int cnt = zero_bytes_share(exit_mask, row0, threadIdx.x, kCompactThreads);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     if (lane == 0) s_warp_cnt[warp] = cnt;

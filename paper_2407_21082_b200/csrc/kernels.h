@@ -99,11 +99,8 @@ ee_status dssd_commit_launch(const int* draft_tok, const unsigned char* draft_ex
                              int* accept_len, int* next_tok, long long* stats, cudaStream_t stream);
 
 // ---- a whole DSSD round driven from the host (drafting steps, verification pass, commit) ----
-size_t dssd_round_layout_bytes(int S, int k, int d, int V, size_t head_ws_bytes);
-ee_status dssd_round_run(const ee_dssd_round_args& a, size_t head_ws_bytes,
-                         ee_status (*head_call)(const void* h, const ee_head& head, float ln_eps, int M, int d, int V, float tau,
-                                                int* argmax, float* entropy, float* maxprob, unsigned char* mask, void* ws,
-                                                size_t ws_bytes, void* stream));
+size_t dssd_round_layout_bytes(int S, int k, int d, int n_draft_heads, size_t head_ws_bytes);
+ee_status dssd_round_run(const ee_dssd_round_args& a, const ee_head* draft_heads, int n_draft_heads, size_t head_ws_bytes);
 
 // ---- diagnostic: a bounded wait that is made to give up ----
 int hidden_from_tables(const ee_hidden_tables* m, const int* tokens, int n_rows, int which, void* h_out, cudaStream_t stream);

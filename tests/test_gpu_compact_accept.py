@@ -30,7 +30,7 @@ def _check_compact(ee, mask, h_bits):
         assert np.array_equal(got, ref["h_out"])
 
 
-@pytest.mark.parametrize("M,d", [(1, 8), (31, 64), (32, 64), (33, 72), (256, 2048), (1000, 40), (5000, 16)])
+@pytest.mark.parametrize("M,d", [(1, 8), (31, 64), (32, 64), (33, 72), (256, 2048), (1000, 40), (5000, 16), (16384, 64), (100000, 8)])
 def test_compact_random_masks(ee, M, d):
     rng = np.random.default_rng(M)
     h = rng.integers(0, 65536, size=(M, d)).astype(np.uint16)
@@ -38,6 +38,15 @@ def test_compact_random_masks(ee, M, d):
         mask = (rng.random(M) < p).astype(np.uint8) * rng.integers(1, 256, size=M).astype(np.uint8)
         _check_compact(ee, mask, h)
     _check_compact(ee, (np.arange(M) % 2).astype(np.uint8), None)
+    if M >= 64:                        # a mask that does not start on a 16-byte boundary (the survivors are counted 16 bytes at a time)
+        for off in (1, 7, 15):
+            big = dev(np.concatenate([np.zeros(off, np.uint8), (rng.random(M - off) < 0.5).astype(np.uint8)]))
+            sub = big[off:]
+            out = ee.ee_compact(sub)
+            torch.cuda.synchronize()
+            ref = oracle.compact(sub.cpu().numpy())
+            n = int(out["kept_count"].item())
+            assert n == ref["kept_count"] and np.array_equal(out["kept_idx"].cpu().numpy()[:n], ref["kept_idx"])
 
 
 def test_compact_hand_masks_and_empty(ee):
