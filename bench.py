@@ -631,6 +631,77 @@ def measure_dssd_round(peaks: dict, src: str, S: int = 32, k: int = 8, rounds: i
                                   kind="oracle", cores=oracle_threads(), sample="the first round of the same sequences"))
 
 
+def measure_dssd_round_multi(peaks: dict, src: str, S: int = 32, k: int = 8, K: int = 3, rounds: int = 30) -> dict:
+    """Whole DSSD rounds with K draft heads (per position the first confident head supplies the token) on the c1
+    shape, the library's table model standing in for the transformer (one table per drafting layer, the shallower
+    the noisier); reports the head usage and the mean exit head while drafting, the statistics of the paper's DSSD
+    experiments (values of this stand-in, not of a trained model).  The first round is also run by the oracle."""
+    import torch
+    import oracle
+    import paper_2407_21082_b200 as ee
+    spec = gen.CONFIGS["c1"]
+    d, V = spec["d"], spec["V"]
+    cfg = gen.make_config("c1", seed=0, planted=True, M=4, heads=K + 1)
+    planting = gen.make_planting(0, f"c1/planted/d{d}/V{V}", d, V)
+    sigmas = np.linspace(1.2, 0.4, K)
+    tables = [gen.make_markov_model(10 * i, V, d, planting, sigma=float(sg)) for i, sg in enumerate(sigmas)]
+    taus = [float(t) for t in np.linspace(0.5, 1.5, K)]
+
+    def bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    E = [bf16(t["E_draft"]) for t in tables] + [bf16(tables[0]["E_verify"])]
+    heads = [dict(gamma=torch.from_numpy(hd["gamma"]).cuda(), beta=torch.from_numpy(hd["beta"]).cuda(), W=bf16(hd["W"]))
+             for hd in cfg["heads"]]
+    for hd, t in zip(heads[:K], taus):
+        hd["tau"] = t
+    cap = rounds * (k + 1) + 1
+    start = ((np.arange(S, dtype=np.int32) * 1543) % V).astype(np.int32)
+    state = dict(last_tok=torch.from_numpy(start).cuda(), out_tok=torch.full((S, cap), -9, dtype=torch.int32, device="cuda"),
+                 seq_len=torch.zeros(S, dtype=torch.int32, device="cuda"), finished=torch.zeros(S, dtype=torch.uint8, device="cuda"),
+                 stats=torch.zeros(4, dtype=torch.int64, device="cuda"))
+    rnd = ee.DssdRound(heads[:K], heads[K], 1e-5, k, -1, ee.TableModel(E[:K], E[K], chained=True), state)
+    first = {n: v.clone() for n, v in rnd().items()}
+    torch.cuda.synchronize()
+    first_len = state["seq_len"].cpu().numpy().copy()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(rounds - 1):
+        rnd()
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / (rounds - 1)
+    status = ee.ee_query_async_error(rnd.workspace)
+    stats = state["stats"].cpu().numpy().tolist()
+    use = rnd.head_use.cpu().numpy().astype(np.int64)
+    ref_state = (np.full((S, cap), -9, np.int32), np.zeros(S, np.int32), np.zeros(S, np.uint8), np.zeros(4, np.int64))
+    ref_use = np.zeros(K, np.int64)
+    c0 = time.perf_counter()
+    ref = oracle.dssd_round_multi([t["E_draft"] for t in tables], tables[0]["E_verify"], cfg["heads"][:K], cfg["heads"][K], taus, -1, k,
+                                  start.copy(), *ref_state, ref_use)
+    cpu_s = time.perf_counter() - c0
+    clean = np.ones(S, bool)
+    for c in ref["steps"]:
+        for o in c["per_head"]:
+            kp = oracle.decisive_rows(o, 1e-3, 1e-3)
+            clean[o["rows"][~(kp["argmax"] & kp["exit_mask"])]] = False
+    clean &= oracle.decisive_rows(ref["verify_out"], 1e-3, 1e-3)["argmax"].reshape(S, k + 1).all(axis=1)
+    agree = bool((first["accept_len"].cpu().numpy()[clean] == ref["accept_len"][clean]).all() and (first_len[clean] == ref_state[1][clean]).all())
+    w_bytes = (k * K + 1) * 2.0 * V * d                                   # the heads' weights, once per evaluation
+    gbs = w_bytes / (us * 1e-6) / 1e9
+    return dict(S=S, k=k, draft_heads=K, taus=taus, d=d, V=V, rounds=rounds, us_per_round=round(us, 1), head_evaluations_per_round=k * K + 1,
+                head_use=use.tolist(), mean_exit_head_while_drafting=round(float((np.arange(K) * use).sum() / max(use.sum(), 1)), 3),
+                tokens_committed_per_round_per_sequence=round(stats[2] / (rounds * S), 3),
+                acceptance_rate=round(stats[1] / max(stats[0], 1), 4), wasted_tokens=stats[0] - stats[1], async_error=status,
+                first_round_matches_oracle_on_decisive_sequences=agree, decisive_sequences=int(clean.sum()),
+                roofline=dict(bound="hbm", algorithmic_bytes=w_bytes, achieved=round(gbs, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                              frac=round(gbs / peaks["hbm_gbs"], 4), peak_source=f"of {src}", traffic=None,
+                              note="K draft heads per drafting step in one launch sequence; the stand-in model is the library's table "
+                                   "lookup, launched in the programmatic chain (one small kernel per layer and step)"),
+                cpu_baseline=dict(value=float(ref_state[3][2]) / cpu_s, unit="committed tokens/s", seconds=round(cpu_s, 2), kind="oracle",
+                                  cores=oracle_threads(), sample="the first round of the same sequences"))
+
+
 def measure_kl(peaks: dict, src: str, M: int, calls: int = 100) -> dict:
     """ee_head_kl on the c1 shape (one head against the teacher head, M tokens); two copies of both weight
     matrices in rotation (cold L2); the oracle on a sample of the rows."""
@@ -770,7 +841,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "stream", "tcgen05", "skinny"], help="force a kernel")
     ap.add_argument("--sweep", action="store_true", help="time every kernel that accepts the size, for c1 at several M")
     ap.add_argument("--no-extra", action="store_true", help="skip the per-config table and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["calibration", "cascade", "dssd_round", "kl_loss", "read_stream"],
+    ap.add_argument("--only", default=None, choices=["calibration", "cascade", "dssd_round", "dssd_round_multi", "kl_loss", "read_stream"],
                     help="run that entry of the table alone and print its JSON (for profiling one kernel family)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -812,6 +883,7 @@ def main():
             entry = {"calibration": lambda: measure_calibration(peaks, peak_src),
                      "cascade": lambda: measure_cascade(peaks, peak_src, M=args.rows or 64),
                      "dssd_round": lambda: measure_dssd_round(peaks, peak_src),
+                     "dssd_round_multi": lambda: measure_dssd_round_multi(peaks, peak_src),
                      "read_stream": lambda: measure_read_stream(peaks, peak_src),
                      "kl_loss": lambda: [measure_kl(peaks, peak_src, m) for m in rows]}[args.only]()
             print(json.dumps({args.only: entry}))
@@ -894,6 +966,7 @@ def main():
         line["calibration"] = measure_calibration(peaks, peak_src)
         line["cascade"] = measure_cascade(peaks, peak_src)
         line["dssd_round"] = measure_dssd_round(peaks, peak_src)
+        line["dssd_round_multi"] = measure_dssd_round_multi(peaks, peak_src)
         line["kl_loss"] = [measure_kl(peaks, peak_src, M) for M in (64, 4096)]
         if args.sweep:
             sweep = {}
