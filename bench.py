@@ -279,21 +279,21 @@ def measure(wl: Workload, steps: int, warmup: int, dist=None, sampler: ClockSamp
 # while the SHA-256 of those sources still matches and as null afterwards.
 CSRC = os.path.join(ROOT, "paper_2407_21082_b200", "csrc")
 TRAFFIC = {
-    ("c0", 8): dict(bytes=51654144 + 5632, heads_per_launch=1, kernel="exit_head_gemm_kernel<0>",
+    ("c0", 8): dict(bytes=51656960 + 1664, heads_per_launch=1, kernel="exit_head_gemm_kernel<0,0,0>",
                     sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                    sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c0_c3.md"),
-    ("c3", 256): dict(bytes=521996032 + 4496128, heads_per_launch=2, kernel="exit_head_gemm_kernel<0> (CTA pairs)",
+                    sha256="28868c65d61667733a51525f40259630d2de274253f26d3abf69ef2a3574bf0d", profile="profiles/exit_head_gemm_kernel_c0_c2_c3.md"),
+    ("c3", 256): dict(bytes=522531712 + 5181056, heads_per_launch=2, kernel="exit_head_gemm_kernel<0,0,1> (CTA pairs)",
                       sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                      sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c0_c3.md"),
-    ("c1", 64): dict(bytes=309865728 + 3677696, heads_per_launch=3, kernel="exit_head_gemm_kernel<0>",
+                      sha256="28868c65d61667733a51525f40259630d2de274253f26d3abf69ef2a3574bf0d", profile="profiles/exit_head_gemm_kernel_c0_c2_c3.md"),
+    ("c1", 64): dict(bytes=309878784 + 4778496, heads_per_launch=3, kernel="exit_head_gemm_kernel<0,0,0>",
                      sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                     sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
-    ("c2", 256): dict(bytes=207750656 + 4271744, heads_per_launch=1, kernel="exit_head_gemm_kernel<0> (CTA pairs)",
+                     sha256="28868c65d61667733a51525f40259630d2de274253f26d3abf69ef2a3574bf0d", profile="profiles/exit_head_gemm_kernel_c1_M64.md"),
+    ("c2", 256): dict(bytes=207645568 + 4119936, heads_per_launch=1, kernel="exit_head_gemm_kernel<0,0,1> (CTA pairs)",
                       sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                      sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c2.md"),
-    ("c4", 16384): dict(bytes=1616886272 + 61617152, heads_per_launch=1, kernel="exit_head_gemm_kernel<256> (CTA pairs)",
+                      sha256="28868c65d61667733a51525f40259630d2de274253f26d3abf69ef2a3574bf0d", profile="profiles/exit_head_gemm_kernel_c0_c2_c3.md"),
+    ("c4", 16384): dict(bytes=1128908288 + 56288768, heads_per_launch=1, kernel="exit_head_gemm_kernel<256,0,1> (CTA pairs)",
                         sources=("gemm_kernel.cu", "common.cuh", "sm100_ptx.cuh", "tensor_map.h"),
-                        sha256="339fce13a05aa7c92dffe3ef330549ff19e90bf5fb51f26f81389a023cf2283f", profile="profiles/exit_head_gemm_kernel_c4.md"),
+                        sha256="28868c65d61667733a51525f40259630d2de274253f26d3abf69ef2a3574bf0d", profile="profiles/exit_head_gemm_kernel_c4.md"),
 }
 
 
@@ -836,6 +836,8 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="repeat the timed regions until about this much device time is spent on each (0: one region, for profiler runs)")
     ap.add_argument("--workload", default="c1")
     ap.add_argument("--rows", type=int, default=None, help="override M of the workload")
     ap.add_argument("--path", default="auto", choices=["auto", "stream", "tcgen05", "skinny"], help="force a kernel")
@@ -897,7 +899,7 @@ def main():
     wl = Workload(args.workload, M, seed=replicas.rank_seed(0, rank), n_copies=n_copies, path=path)
     config["kernel"] = args.path
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    res = measure(wl, args.steps, args.warmup, dist, sampler)
+    res = measure(wl, args.steps, args.warmup, dist, sampler, min_seconds=args.min_seconds)
     n_heads = len(wl.heads)
     value = res["units_per_s"]                       # head evaluations of all ranks / time of the slowest rank
     config["l2"] = (f"inputs larger than L2: the step cycles through {wl.w_bytes_total / 1e6:.0f} MB of head weights "
