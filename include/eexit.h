@@ -8,6 +8,14 @@
  * there is no CPU fallback: a device that is not compute capability 10.x yields EE_ERR_ARCH.
  * Identical inputs give bit-identical outputs (all reductions run in a fixed order).
  *
+ * Constants of the stream.  A head's parameters -- W, gamma, beta of every call, ee_head_kl's teacher
+ * included -- are read while earlier work of the stream may still be running (the kernels request them
+ * ahead of their dependency on that work, through the read-only path).  They must therefore be complete
+ * in memory before the call is issued and must not be written by anything still in flight on `stream`
+ * or on any other stream: after updating weights, synchronise (or wait on an event on the host) before
+ * the next call.  Everything else -- hidden states, thresholds, masks, tokens -- may be produced by
+ * earlier work of the same stream, by ordinary or by programmatic dependent launches.
+ *
  * Notation follows the paper: a head h_k maps the hidden features of a transformer block to a
  * distribution p_k over the vocabulary V (section 3.1 "Early exit heads", section 3.2); the confidence
  * is the entropy of p_k (section 3.4.1); tau_k is the calibrated threshold of head k (section 3.4.1);

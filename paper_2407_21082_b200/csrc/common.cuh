@@ -208,8 +208,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Programmatic dependent launch.  The next kernel of the stream may start once every CTA of this one has
 // passed launch_dependents(); a kernel calls grid_dependency_wait() before it touches anything an earlier
 // kernel of the stream writes or still reads (it returns when those kernels have completed and their stores
-// are visible).  Every kernel of the library is launched through launch_pdl, so completions stay in stream
-// order: a kernel cannot complete before it has passed its own wait.
+// are visible).  Every kernel of the head, compaction, cascade, round and loss calls is launched through
+// launch_pdl and waits before it completes, so completions stay in stream order; the calibration kernels and
+// the diagnostic self-tests are ordinary launches, which wait for everything before them anyway.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
