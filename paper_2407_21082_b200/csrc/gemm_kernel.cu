@@ -729,8 +729,11 @@ layer_norm_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bf
 // Rows wider than 1024 columns: one CTA of four warps per row, VPL 16-byte vectors per thread (d <= 1024 * VPL), so
 // that a row's work -- 64 and more elements per lane if one warp took it -- is a quarter as long.  The warps' moments
 // meet in shared memory (64 bytes; summed in a fixed order).  Parameters in registers, fetched before the wait.
-template <int VPL>
-__global__ void __launch_bounds__(128, 3)
+// kLean (batches of thousands of rows, where the launch is bound by memory and not by a dependent chain): the
+// parameters are read where they are used instead (they stay in L1), which halves the registers and lets six CTAs
+// share an SM (five with four vectors per thread) instead of three -- enough rows in flight to cover the memory latency.
+template <int VPL, bool kLean>
+__global__ void __launch_bounds__(128, kLean ? (VPL == 4 ? 5 : 6) : 3)
 layer_norm_wide_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __nv_bfloat16* __restrict__ y_all, int M, int d,
                             Control* ctrl) {
     __shared__ double part[2][4][2];
@@ -749,9 +752,9 @@ layer_norm_wide_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __
     const float* gamma = hs.gamma[head];
     const float* beta = hs.beta[head];
     const double dd = (double)d, inv_d = 1.0 / dd;
-    float4 g[VPL][2], b[VPL][2];
+    float4 g[kLean ? 1 : VPL][2], b[kLean ? 1 : VPL][2];
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) {
+    for (int k = 0; k < (kLean ? 0 : VPL); ++k) {
         const int c = tid + 128 * k;
         if (c < nvec) {
             g[k][0] = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c);
@@ -794,7 +797,10 @@ layer_norm_wide_rows_kernel(const __grid_constant__ LnHeads hs, float ln_eps, __
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
         const int c = tid + 128 * k;
-        if (c < nvec) yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
+        if (c < nvec) {
+            if constexpr (kLean) yrow[c] = layer_norm_vec8(x[k], st, gamma, beta, c);
+            else yrow[c] = layer_norm_vec8(x[k], st, g[k][0], g[k][1], b[k][0], b[k][1]);
+        }
     }
 }
 
@@ -973,7 +979,7 @@ struct GemmPlan {
     __nv_bfloat16* y;
     float ln_eps;
     int device;
-    int ln_kind;                               // 2, 4: rows in registers; -2, -3, -4: one CTA per row; 0: re-read; 100: gathered rows
+    int ln_kind;                               // 2, 4: rows in registers; -2, -3, -4: one CTA per row (-12 .. -14: lean); 0: re-read; 100: gathered rows
     int ln_grid_x, ln_threads;
     int gemm_grid;
     int pair, wide, top2;                      // GEMM instantiation
@@ -1026,6 +1032,7 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
         g.ln_kind = a.d <= 512 ? 2 : 4; g.ln_threads = ln_threads(g.ln_kind); g.ln_grid_x = m_pad / (g.ln_threads / 32);
     } else if (a.d <= 4096) {
         g.ln_kind = a.d <= 2048 ? -2 : (a.d <= 3072 ? -3 : -4); g.ln_threads = 128; g.ln_grid_x = m_pad;
+        if ((long long)m_pad * n_heads >= 2048) g.ln_kind -= 10;      // memory-bound batch: the lean variant
     } else {
         g.ln_kind = 0; g.ln_threads = ln_threads(0); g.ln_grid_x = m_pad / (g.ln_threads / 32);
     }
@@ -1091,9 +1098,12 @@ ee_status gemm_run(const void* storage, cudaStream_t stream) {
                                    g.ln.beta[0], g.ln_eps, g.row_idx, g.m_dev, g.y, p.M, p.d, p.ctrl); break;
         case 2: err = launch_pdl(layer_norm_rows_kernel<2>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
         case 4: err = launch_pdl(layer_norm_rows_kernel<4>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
-        case -2: err = launch_pdl(layer_norm_wide_rows_kernel<2>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
-        case -3: err = launch_pdl(layer_norm_wide_rows_kernel<3>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
-        case -4: err = launch_pdl(layer_norm_wide_rows_kernel<4>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -2: err = launch_pdl(layer_norm_wide_rows_kernel<2, false>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -3: err = launch_pdl(layer_norm_wide_rows_kernel<3, false>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -4: err = launch_pdl(layer_norm_wide_rows_kernel<4, false>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -12: err = launch_pdl(layer_norm_wide_rows_kernel<2, true>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -13: err = launch_pdl(layer_norm_wide_rows_kernel<3, true>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
+        case -14: err = launch_pdl(layer_norm_wide_rows_kernel<4, true>, ln_grid, 128, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
         default: err = launch_pdl(layer_norm_rows_kernel<0>, ln_grid, g.ln_threads, 0, stream, g.ln, g.ln_eps, g.y, p.M, p.d, p.ctrl); break;
     }
     if (err != cudaSuccess) return EE_ERR_CUDA;

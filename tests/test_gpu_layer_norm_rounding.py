@@ -45,9 +45,12 @@ def _rows(rng, M, d):
     ("tcgen05", 4096, 64),        # rows in registers, two vectors per lane
     ("tcgen05", 4096, 520),       # four vectors per lane, ragged
     ("tcgen05", 2048, 1024),
-    ("tcgen05", 2048, 1536),      # wide rows: four warps per row, two vectors per thread
-    ("tcgen05", 2048, 2560),      # ... three vectors per thread
+    ("tcgen05", 1024, 1536),      # wide rows: four warps per row, two vectors per thread
+    ("tcgen05", 1024, 2560),      # ... three vectors per thread
     ("tcgen05", 1024, 3080),      # ... four
+    ("tcgen05", 2048, 1536),      # from 2048 rows on: the same with the parameters read where they are used
+    ("tcgen05", 2048, 2560),
+    ("tcgen05", 2304, 3080),
     ("tcgen05", 600, 4104),       # rows re-read from global memory
     ("stream", 512, 64), ("stream", 512, 520), ("stream", 256, 1536),
     ("skinny", 64, 64), ("skinny", 64, 1024),
