@@ -17,6 +17,7 @@
 #include "kernels.h"
 #include "layer_norm.cuh"
 #include "sm100_ptx.cuh"
+#include "gemm_roles.cuh"
 #include "tensor_map.h"
 
 namespace ee {
@@ -24,9 +25,8 @@ namespace ee {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BK = 64;
+constexpr int BK = kRoleBK;
 constexpr int kGemmThreads = 320;           // producer warp, MMA warp, eight epilogue warps
-constexpr int kGroupM = 16;                 // m-tiles per super-row of the tile order
 constexpr int kATileBytes = BM * BK * 2;    // 16 KB
 
 constexpr int kBarBytes = 512 + 2048 + 1024;   // barriers and flags (512 B), then 128 states and 128 (max, second) pairs
@@ -132,23 +132,6 @@ struct GemmParams {
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
     MergeHeads mg;
 };
-
-__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
-    const int per_group = kGroupM * n_tiles;
-    const int grp = tile / per_group;
-    const int within = tile - grp * per_group;
-    const int rows_in_group = min(kGroupM, m_tiles - grp * kGroupM);
-    n_tile = within / rows_in_group;
-    m_tile = grp * kGroupM + (within - n_tile * rows_in_group);
-}
-
-__device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abort_flag, unsigned role, unsigned stage,
-                                               unsigned tile) {
-    if (atomicCAS(&ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
-        ctrl->error_info = (role << 24) | ((stage & 0xffu) << 16) | (tile & 0xffffu);
-    *abort_flag = 1;
-    __threadfence_block();
-}
 
 // Fold 32 consecutive logits of one row (columns col0 .. col0+31, the first `nvalid` of them real).
 template <bool kFull>
@@ -354,20 +337,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (*abort_flag) {
-                // Let the copies still in flight land before the CTA gives its shared memory back.  (Rank 1 of a
-                // pair cannot poll the barrier its copies report to: it waits out a fixed time instead.)
-                if (rank != 0) {
-                    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
-                } else {
-                    for (int s = 0; s < S; ++s)
-                        if (armed & (1u << s)) {
-                            const uint32_t par = (armed_parity >> s) & 1u;
-                            for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i)
-                                __nanosleep(100);
-                        }
-                }
-            }
+            if (*abort_flag) producer_drain(rank, S, full_bar(0), armed, armed_parity);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
@@ -387,35 +357,17 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
+                    if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * a_tile_bytes,
+                                            b_base + stage * b_tile_bytes, d_tmem, idesc, kb == 0, abort_flag)) {
                         record_failure(p.ctrl, abort_flag, 2, stage, tile);
                         ok = false;
                         break;
                     }
-                    ptx::tc_fence_after_sync();
-                    const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * a_tile_bytes);
-                    const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {   // 16 bf16 = 32 bytes = 2 descriptor units per step
-                        if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                        else ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    // frees the smem stage (in both CTAs of a pair) when these MMAs are done
-                    if (kPair) ptx::mma_commit_pair(empty_bar(stage), 3);
-                    else ptx::mma_commit(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) {                                 // accumulator complete
-                    if (kPair) ptx::mma_commit_pair(tfull_bar(buf), 3);
-                    else ptx::mma_commit(tfull_bar(buf));
-                }
+                if (ok) mma_commit_all<kPair>(tfull_bar(buf));    // accumulator complete
             }
-            if (*abort_flag) {
-                // Make sure no MMA is still writing TMEM when it is released.
-                if (kPair) ptx::mma_commit_pair(drain_bar, 1);
-                else ptx::mma_commit(drain_bar);
-                for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
-            }
+            if (*abort_flag) mma_drain<kPair>(drain_bar);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)

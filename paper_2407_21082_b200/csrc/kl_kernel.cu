@@ -22,6 +22,7 @@
 #include "layer_norm.cuh"
 #include "kernels.h"
 #include "sm100_ptx.cuh"
+#include "gemm_roles.cuh"
 #include "tensor_map.h"
 
 namespace ee {
@@ -29,9 +30,8 @@ namespace ee {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BK = 64;
+constexpr int BK = kRoleBK;
 constexpr int kThreads = 320;                   // producer warp, MMA warp, eight epilogue warps
-constexpr int kGroupM = 16;
 constexpr int kATileBytes = BM * BK * 2;
 constexpr int kBarBytes = 512 + 2048 + 2048;    // barriers, then 128 head states and 128 teacher/cross states exchanged
 constexpr size_t kSmemBudget = 226 * 1024;
@@ -61,23 +61,6 @@ struct KlParams {
     Control* ctrl;
     const int* labels;     // [M] or NULL (no cross-entropy asked for)
 };
-
-__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& m_tile, int& n_tile) {
-    const int per_group = kGroupM * n_tiles;
-    const int grp = tile / per_group;
-    const int within = tile - grp * per_group;
-    const int rows_in_group = min(kGroupM, m_tiles - grp * kGroupM);
-    n_tile = within / rows_in_group;
-    m_tile = grp * kGroupM + (within - n_tile * rows_in_group);
-}
-
-__device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abort_flag, unsigned role, unsigned stage,
-                                               unsigned tile) {
-    if (atomicCAS(&ctrl->error, 0u, (unsigned)EE_ERR_TIMEOUT) == 0u)
-        ctrl->error_info = (role << 24) | ((stage & 0xffu) << 16) | (tile & 0xffffu);
-    *abort_flag = 1;
-    __threadfence_block();
-}
 
 // Fold 32 consecutive head logits of one row (the first `nvalid` real) into (m, s, t, idx); the logit at the
 // row's label is picked up on the way.
@@ -294,19 +277,7 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     }
                 }
             }
-            if (*abort_flag) {
-                // copies in flight land before the shared memory is given back (rank 1 of a pair cannot poll the
-                // barrier its copies report to and waits out a fixed time)
-                if (rank != 0) {
-                    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
-                } else {
-                    for (int s = 0; s < S; ++s)
-                        if (armed & (1u << s)) {
-                            const uint32_t par = (armed_parity >> s) & 1u;
-                            for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(full_bar(s), par); ++i) __nanosleep(100);
-                        }
-                }
-            }
+            if (*abort_flag) producer_drain(rank, S, full_bar(0), armed, armed_parity);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer: buffer 0 = head, 1 = teacher
@@ -327,34 +298,18 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     ptx::tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(which * kAccStride);
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!ptx::mbar_wait(full_bar(stage), phase, abort_flag)) {
+                        if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * kATileBytes,
+                                                b_base + stage * b_tile_bytes, d_tmem, idesc, kb == 0, abort_flag)) {
                             record_failure(p.ctrl, abort_flag, 2, stage, tile);
                             ok = false;
                             break;
                         }
-                        ptx::tc_fence_after_sync();
-                        const uint64_t adesc = ptx::smem_desc_k128(a_base + stage * kATileBytes);
-                        const uint64_t bdesc = ptx::smem_desc_k128(b_base + stage * b_tile_bytes);
-#pragma unroll
-                        for (int k = 0; k < BK / 16; ++k) {
-                            if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                            else ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                        }
-                        if (kPair) ptx::mma_commit_pair(empty_bar(stage), 3);
-                        else ptx::mma_commit(empty_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok) {
-                        if (kPair) ptx::mma_commit_pair(tfull_bar(which), 3);
-                        else ptx::mma_commit(tfull_bar(which));
-                    }
+                    if (ok) mma_commit_all<kPair>(tfull_bar(which));
                 }
             }
-            if (*abort_flag) {
-                if (kPair) ptx::mma_commit_pair(drain_bar, 1);
-                else ptx::mma_commit(drain_bar);
-                for (uint32_t i = 0; i < (1u << 16) && !ptx::mbar_try_wait(drain_bar, 0); ++i) __nanosleep(100);
-            }
+            if (*abort_flag) mma_drain<kPair>(drain_bar);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
