@@ -130,6 +130,7 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
+    int merge_looks;       // how often a row group's owner looks at the ticket before it leaves its rows to the last arriver
     MergeHeads mg;
 };
 
@@ -484,7 +485,7 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             // The barrier orders the epilogue threads' stores before one thread's acquire-release ticket, which is
             // cumulative: whoever sees the full count sees every CTA's states.  A CTA whose roles gave up still
             // takes its ticket (its tiles' states are missing, the error word says so).
-            constexpr int kMergeLooks = 96;
+            const int kMergeLooks = p.merge_looks;
             const int et = (warp - 2) * 32 + lane;
             const int grid = (int)gridDim.x;
             const int n_groups = min(grid, (total_rows + 7) >> 3);
@@ -860,6 +861,16 @@ int resident_pairs(int device) {
 
 // Pairs of CTAs work on 256-row tiles when a head has an even number of 128-row tiles; EE_GEMM_PAIRS=0 in the
 // environment keeps every CTA on its own 128-row tiles (for comparisons).
+// Looks an owner of the in-kernel merge takes at the ticket before it hands its rows to the last arriver: 96
+// (some hundred microseconds with the back-off) unless EE_MERGE_LOOKS says otherwise -- 0 makes every owner give
+// up at once, which is how the tests drive the hand-over paths that otherwise need contention to occur.
+int merge_looks() {
+    const char* e = getenv("EE_MERGE_LOOKS");
+    if (!e || !*e) return 96;
+    const int v = atoi(e);
+    return v < 0 ? 0 : (v > 4096 ? 4096 : v);
+}
+
 bool pairs_enabled() {
     static int enabled = -1;
     if (enabled < 0) {
@@ -1018,6 +1029,7 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     p.bn = bn;
     p.mma_m = mma_m;
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
+    p.merge_looks = merge_looks();
     p.mg = mg;
     p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
     g.pair = pair ? 1 : 0;

@@ -387,6 +387,49 @@ def test_calls_in_flight_on_several_streams(ee, M, d, V, n_heads, n_streams):
             assert_head_matches(outs[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"{n_streams} streams head {k}")
 
 
+@pytest.mark.parametrize("looks", [0, 1, 3])
+@pytest.mark.parametrize("M,d,V,n_heads", [(64, 256, 6000, 3), (512, 128, 9000, 1), (130, 64, 40000, 3), (5, 512, 50304, 1)])
+def test_merge_hand_over_paths_give_the_same_results(ee, monkeypatch, looks, M, d, V, n_heads):
+    """The in-kernel merge with owners that give up after 0, 1 or 3 looks at the ticket (EE_MERGE_LOOKS, read when a call
+    is planned): their row groups then go to the last CTA to arrive, or are claimed back by an owner whose final look
+    finds the count full.  Whoever merges a group, the results are the same bits as with patient owners, run after
+    run, also with several calls in flight, and nothing is reported as a time-out."""
+    cfg = gen.make_config("c1", seed=71, planted=True, M=M, d=d, V=V, heads=n_heads)
+    hds = [head_to_dev(hd) for hd in cfg["heads"]]
+    h = dev_bf16(cfg["h"])
+    heads = [dict(h=h, gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=1.0) for hd in hds]
+    monkeypatch.delenv("EE_MERGE_LOOKS", raising=False)
+    ref = [{k: v.clone() for k, v in o.items()} for o in ee.ee_exit_head_multi(heads, 1e-5)]
+    torch.cuda.synchronize()
+    monkeypatch.setenv("EE_MERGE_LOOKS", str(looks))
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    prepared = []
+    for stream in streams:
+        with torch.cuda.stream(stream):
+            ws = torch.empty(ee.ee_exit_head_multi_workspace_bytes(n_heads, M, d, V), dtype=torch.uint8, device="cuda")
+            ee.ee_workspace_init(ws)
+            outs = [ee.new_outputs(M) for _ in range(n_heads)]
+            prepared.append((ee.PreparedMulti([dict(hd, out=o) for hd, o in zip(heads, outs)], 1e-5, ws), outs, ws))
+    monkeypatch.delenv("EE_MERGE_LOOKS")
+    torch.cuda.synchronize()
+    for rep in range(25):
+        for call, outs, _ in prepared:
+            call()
+        if rep % 8 == 0:                                             # look at intermediate runs too, not only the last
+            torch.cuda.synchronize()
+            for _, outs, _ in prepared:
+                for k in range(n_heads):
+                    for key in ref[k]:
+                        assert torch.equal(outs[k][key], ref[k][key]), (rep, k, key)
+    torch.cuda.synchronize()
+    for _, outs, ws in prepared:
+        assert ee.ee_query_async_error(ws) == 0
+        for k in range(n_heads):
+            for key in ref[k]:
+                assert torch.equal(outs[k][key], ref[k][key]), (k, key)
+            assert_head_matches(outs[k], oracle_head(cfg["h"], cfg["heads"][k], 1.0), label=f"looks={looks} head {k}")
+
+
 def test_plan_runs_equal_the_one_step_call_and_follow_the_buffers_contents(ee):
     """ee_exit_head_plan_init / ee_exit_head_plan_run: the same results as ee_exit_head_multi, bit for bit, run after
     run; the plan captures pointers, not contents, so new rows written into the same buffer give the new rows' results."""
