@@ -749,7 +749,7 @@ def measure_kl(peaks: dict, src: str, M: int, calls: int = 100) -> dict:
     roof.update(peak_source=f"of {src}", traffic=None, algorithmic_bytes=nbytes, flops=flops)
     if not hbm_bound:
         roof.update(peak_source=f"of {src} (burst)", frac_of_sustained=round(tfs / peaks["bf16_tflops_sustained"], 4))
-    return dict(M=M, d=d, V=V, us_per_call=round(us, 2), launches=4, tokens_per_s=M / (us * 1e-6), roofline=roof,
+    return dict(M=M, d=d, V=V, us_per_call=round(us, 2), launches=3, tokens_per_s=M / (us * 1e-6), roofline=roof,
                 max_abs_error_vs_oracle=float(np.abs(got[:rows] - ref["kl"]).max()), loss=float(prepared[(calls - 1) % 2].out["loss"][0].item()),
                 cpu_baseline=dict(value=rows / cpu_s, unit="tokens/s", seconds=round(cpu_s, 2), kind="oracle", cores=oracle_threads(),
                                   sample=f"the first {rows} tokens"))

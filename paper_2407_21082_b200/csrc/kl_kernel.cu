@@ -17,7 +17,8 @@
 //   sum the teacher's exponentials out of buffer 1 while the next tile's head MMAs run (only the second pass
 //   does not overlap MMAs; the roles and the bounded waits are those of the inference kernel); with an even number of 128-row tiles two CTAs of a cluster share 256-row tiles, each
 //   staging half of every W tile (cta_group::2 MMAs), as in the inference kernel;
-//   a merge kernel (warp per row) that combines the per-tile states and writes kl, and a one-CTA mean.
+//   a merge kernel (warp per row) that combines the per-tile states and writes kl; its last CTA to finish adds the
+//   means in a fixed order.
 #include "common.cuh"
 #include "layer_norm.cuh"
 #include "kernels.h"
@@ -464,14 +465,33 @@ __global__ void __launch_bounds__(256) kl_layer_norm_kernel(const __grid_constan
     for (int c = lane; c < nvec; c += 32) yrow[c] = layer_norm_vec8(ld_dep(hrow + c), st, a.gamma[which], a.beta[which], c);
 }
 
-// One warp per row: the tiles' states in vocabulary order -> kl.
+// Sum of src[0 .. M) by the 256 threads of a CTA in a fixed order (bit-identical from run to run), divided by M.
+__device__ __forceinline__ float cta_mean_fixed_order(const float* src, int M, float* part) {
+    float s = 0.f;
+    for (int i = threadIdx.x; i < M; i += 256) s += ld_dep(src + i);
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    const float mean = part[0] / (float)M;
+    __syncthreads();
+    return mean;
+}
+
+// One warp per row: the tiles' states in vocabulary order -> kl (and ce).  With `loss`, the CTA that finishes last
+// (a ticket in the control block, taken after the CTA's rows are stored) also writes the means: loss[0] = mean of kl,
+// loss[1] = mean of ce if there is one -- summed in a fixed order whichever CTA that is.
 __global__ void __launch_bounds__(256) kl_merge_kernel(const State* head_part, const Cross* cross_part,
-                                                       int n_tiles, int M, float* kl, float* ce) {
+                                                       int n_tiles, int M, float* kl, float* ce, float* loss, Control* ctrl) {
+    __shared__ float part[256];
+    __shared__ int is_last;
     launch_dependents();
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (row >= M) return;
     grid_dependency_wait();
+    if (row < M) {
     State st = state_empty();
     Cross cr = {-CUDART_INF_F, 0.f, 0.f, -CUDART_INF_F};
     for (int n = lane; n < n_tiles; n += 32) {
@@ -500,25 +520,19 @@ __global__ void __launch_bounds__(256) kl_merge_kernel(const State* head_part, c
         kl[row] = -entropy + log_z_teacher - cr.u / st.s;
         if (ce) ce[row] = st.m + logf(st.s) - cr.zl;                    // -log p_head(label)
     }
-}
-
-// loss[0] = mean of kl, loss[1] = mean of ce (if there is one); CTA b sums array b in a fixed order
-// (bit-identical from run to run).
-__global__ void __launch_bounds__(256) kl_mean_kernel(const float* kl, const float* ce, int M,
-                                                      float* loss) {
-    __shared__ float part[256];
-    launch_dependents();
-    grid_dependency_wait();
-    const float* src = blockIdx.x == 0 ? kl : ce;
-    float s = 0.f;
-    for (int i = threadIdx.x; i < M; i += 256) s += ld_dep(src + i);
-    part[threadIdx.x] = s;
-    __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) {
-        if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
-        __syncthreads();
     }
-    if (threadIdx.x == 0) loss[blockIdx.x] = part[0] / (float)M;
+    if (!loss) return;
+    __syncthreads();                                                    // the CTA's rows are stored
+    if (threadIdx.x == 0) is_last = ticket_arrive_is_last(&ctrl->head_ticket[0], gridDim.x) ? 1 : 0;
+    __syncthreads();
+    if (!is_last) return;
+    const float mean_kl = cta_mean_fixed_order(kl, M, part);
+    const float mean_ce = ce ? cta_mean_fixed_order(ce, M, part) : 0.f;
+    if (threadIdx.x == 0) {
+        loss[0] = mean_kl;
+        if (ce) loss[1] = mean_ce;
+        ctrl->head_ticket[0] = 0;                                       // ready for the next call
+    }
 }
 
 int stages_for(int b_rows) {
@@ -635,10 +649,7 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
         if (launch_pdl(kl_pair_gemm_kernel<false>, grid, kThreads, smem, head.stream, maps, p) != cudaSuccess) return EE_ERR_CUDA;
     }
     if (launch_pdl(kl_merge_kernel, (M + 7) / 8, 256, 0, head.stream, (const State*)head_part, (const Cross*)cross_part, p.n_tiles,
-                   M, kl, ce) != cudaSuccess)
-        return EE_ERR_CUDA;
-    if (loss && launch_pdl(kl_mean_kernel, ce ? 2 : 1, 256, 0, head.stream, (const float*)kl, (const float*)ce, M, loss) !=
-                    cudaSuccess)
+                   M, kl, ce, loss, p.ctrl) != cudaSuccess)
         return EE_ERR_CUDA;
     return EE_OK;
 }
