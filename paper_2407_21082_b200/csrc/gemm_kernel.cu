@@ -130,6 +130,7 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
+    int k2;                // a stage holds two k-blocks, fetched by one request per operand (pairs, runtime width; d % 64 == 0)
     int merge_looks;       // how often a row group's owner looks at the ticket before it leaves its rows to the last arriver
     MergeHeads mg;
 };
@@ -210,13 +211,21 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     // 128-row MMA whose lower half would be padding, and an 8 KB instead of a 16 KB y tile per stage.
     const int mma_m = BN_T ? BM : p.mma_m;
     const int a_tile_bytes = mma_m * BK * 2;
-    const int stage_bytes = a_tile_bytes + b_tile_bytes;
+    // A stage of the ring holds one k-block of both operands, or -- CTA pairs with a runtime width -- two: a pair's
+    // CTAs each stage half a W tile, boxes of at most 128 rows, and requests that small stream from HBM at 5.4 TB/s
+    // where one request for two k-blocks (256 bytes of every row) reaches the rate of a contiguous copy; it also
+    // halves the barrier traffic per k-block.
+    constexpr bool kCanK2 = kPair && BN_T == 0;
+    const int kbs = (kCanK2 && p.k2) ? 2 : 1;                     // k-blocks per stage
+    const int n_steps = (p.k_blocks + kbs - 1) / kbs;             // stages per tile
+    const int a_stage_bytes = kbs * a_tile_bytes, b_stage_bytes = kbs * b_tile_bytes;
+    const int stage_bytes = a_stage_bytes + b_stage_bytes;
     constexpr int kAccStride = 256;                               // TMEM columns between the two accumulators
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
     const uint32_t a_base = ptx::smem_addr(smem);
-    const uint32_t b_base = a_base + S * a_tile_bytes;
+    const uint32_t b_base = a_base + S * a_stage_bytes;
     unsigned char* bar_mem = smem + S * stage_bytes;
     const uint32_t bar_base = ptx::smem_addr(bar_mem);
     // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], drain
@@ -285,9 +294,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     };
     // Where a stage's loads report their bytes (rank 0's barrier) and how they are issued.
     auto load_full_bar = [&](int s) { return kPair ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s); };
-    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
-        if (kPair) ptx::tma_load_2d_pair(dst, m, c0, c1, bar);
-        else ptx::tma_load_2d(dst, m, c0, c1, bar);
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int step, int row, uint32_t bar) {   // the k-block(s) of stage `step`
+        if (kCanK2 && kbs == 2) ptx::tma_load_3d_pair(dst, m, 0, row, 2 * step, bar);
+        else if (kPair) ptx::tma_load_2d_pair(dst, m, step * BK, row, bar);
+        else ptx::tma_load_2d(dst, m, step * BK, row, bar);
     };
     const uint32_t arm_bytes = (uint32_t)stage_bytes * (kPair ? 2u : 1u);
 
@@ -303,11 +313,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
             if (worker < total_tiles) {
                 int head, m_tile, n_tile;
                 locate(worker, head, m_tile, n_tile);
-                n_pre = min(S, p.k_blocks);
+                n_pre = min(S, n_steps);
                 for (int kb = 0; kb < n_pre; ++kb) {
                     if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(kb), arm_bytes);
-                    load_tile(b_base + kb * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
-                              load_full_bar(kb));
+                    load_tile(b_base + kb * b_stage_bytes, &maps.w[head], kb, n_tile * BN + (int)rank * b_rows, load_full_bar(kb));
                     armed |= 1u << kb;
                 }
             }
@@ -318,9 +327,9 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 locate(tile, head, m_tile, n_tile);
                 const int y_row = (head * p.m_tiles + m_tile) * BM;   // each head's rows are padded to whole tiles
                 if (BN_T != 0 && tile + n_workers >= total_tiles) launch_dependents();
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
+                for (int kb = 0; kb < n_steps; ++kb, ++issued) {
                     if (issued < n_pre) {                 // stage `issued`, armed above, W tile on its way
-                        load_tile(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
+                        load_tile(a_base + stage * a_stage_bytes, &maps.y, kb, y_row, load_full_bar(stage));
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                         continue;
                     }
@@ -330,9 +339,8 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                         break;
                     }
                     if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), arm_bytes);
-                    load_tile(a_base + stage * a_tile_bytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
-                    load_tile(b_base + stage * b_tile_bytes, &maps.w[head], kb * BK, n_tile * BN + (int)rank * b_rows,
-                              load_full_bar(stage));
+                    load_tile(a_base + stage * a_stage_bytes, &maps.y, kb, y_row, load_full_bar(stage));
+                    load_tile(b_base + stage * b_stage_bytes, &maps.w[head], kb, n_tile * BN + (int)rank * b_rows, load_full_bar(stage));
                     armed |= 1u << stage;
                     armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -357,9 +365,12 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
                 }
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kAccStride);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * a_tile_bytes,
-                                            b_base + stage * b_tile_bytes, d_tmem, idesc, kb == 0, abort_flag)) {
+                for (int kb = 0; kb < n_steps; ++kb) {
+                    // with two k-blocks in a stage the second one is absent at the end of an odd number of them
+                    const bool two = kCanK2 && kbs == 2 && 2 * kb + 1 < p.k_blocks;
+                    if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * a_stage_bytes,
+                                            b_base + stage * b_stage_bytes, d_tmem, idesc, kb == 0, abort_flag,
+                                            two ? (uint32_t)a_tile_bytes : 0u, (uint32_t)b_tile_bytes)) {
                         record_failure(p.ctrl, abort_flag, 2, stage, tile);
                         ok = false;
                         break;
@@ -808,8 +819,8 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const State* partials_a
 constexpr int kMinTileN = 64;
 constexpr int kFusedMergeMaxRows = 512;    // rows (over all heads of a launch) up to which the GEMM kernel merges itself
 // Ring depth for a runtime tile width; b_rows = rows of W one CTA stages per k-block.
-int stages_for(int b_rows, int mma_m) {
-    const size_t stage = (size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2;
+int stages_for(int b_rows, int mma_m, int kbs) {
+    const size_t stage = (size_t)kbs * ((size_t)mma_m * BK * 2 + (size_t)b_rows * BK * 2);
     const size_t n = (kGemmSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxGemmStages ? n : (size_t)kMaxGemmStages);
 }
@@ -831,7 +842,7 @@ ee_status launch_gemm(const GemmMaps& maps, const GemmParams& p, int grid, int d
     if (configure_gemm<BN_T, kTop2, kPair>(device) != EE_OK) return EE_ERR_CUDA;
     const int b_rows = kPair ? p.bn / 2 : p.bn;
     const size_t smem = BN_T ? (size_t)Cfg<BN_T>::kSmemBytes
-                             : (size_t)p.n_stages * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
+                             : (size_t)p.n_stages * (p.k2 ? 2 : 1) * ((size_t)p.mma_m * BK * 2 + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
     const cudaError_t err = kPair ? launch_pdl_pairs(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p)
                                   : launch_pdl(exit_head_gemm_kernel<BN_T, kTop2, kPair>, grid, kGemmThreads, smem, stream, maps, p);
     return err == cudaSuccess ? EE_OK : EE_ERR_CUDA;
@@ -869,6 +880,15 @@ int merge_looks() {
     if (!e || !*e) return 96;
     const int v = atoi(e);
     return v < 0 ? 0 : (v > 4096 ? 4096 : v);
+}
+
+bool k2_enabled() {
+    static int enabled = -1;
+    if (enabled < 0) {
+        const char* e = getenv("EE_GEMM_K2");
+        enabled = (e && e[0] == '0') ? 0 : 1;
+    }
+    return enabled != 0;
 }
 
 bool pairs_enabled() {
@@ -1006,9 +1026,16 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     GemmMaps maps;
     const int mma_m = a.M <= 64 ? 64 : BM;
-    if (!make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)) return EE_ERR_CUDA;
-    for (int k = 0; k < kGemmMaxHeads; ++k)
-        if (!make_tile_map(&maps.w[k], heads[k < n_heads ? k : 0].W, a.V, a.d, pair ? bn / 2 : bn, promo)) return EE_ERR_CUDA;
+    // pairs with a runtime width fetch two k-blocks per request (see the kernel); EE_GEMM_K2=0 switches it off for comparisons
+    const int k2 = (pair && a.M <= 1024 && a.d % 64 == 0 && k2_enabled()) ? 1 : 0;
+    if (!(k2 ? make_tile_map_k2(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)
+             : make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)))
+        return EE_ERR_CUDA;
+    for (int k = 0; k < kGemmMaxHeads; ++k) {
+        const void* W = heads[k < n_heads ? k : 0].W;
+        if (!(k2 ? make_tile_map_k2(&maps.w[k], W, a.V, a.d, bn / 2, promo) : make_tile_map(&maps.w[k], W, a.V, a.d, pair ? bn / 2 : bn, promo)))
+            return EE_ERR_CUDA;
+    }
     memcpy(g.maps, &maps, sizeof(maps));
 
     GemmParams& p = g.p;
@@ -1031,7 +1058,8 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     p.fused_merge = (n_heads * a.M <= kFusedMergeMaxRows) ? 1 : 0;
     p.merge_looks = merge_looks();
     p.mg = mg;
-    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m);
+    p.k2 = k2;
+    p.n_stages = stages_for(pair ? bn / 2 : bn, mma_m, k2 ? 2 : 1);
     g.pair = pair ? 1 : 0;
     g.wide = a.M > 1024 ? 1 : 0;
     g.top2 = p.second ? 1 : 0;

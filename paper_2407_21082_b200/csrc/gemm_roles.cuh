@@ -34,13 +34,15 @@ __device__ __forceinline__ void record_failure(Control* ctrl, volatile int* abor
     __threadfence_block();
 }
 
-// One k-block by the MMA-issuing thread: wait until the stage's operands have landed, four MMAs of K = 16 on the
+// One stage by the MMA-issuing thread: wait until the stage's operands have landed, four MMAs of K = 16 on the
 // 128-byte-swizzled tiles at a_addr / b_addr into the accumulator at d_tmem (the first MMA of a tile overwrites
-// it), then a commit that frees the stage -- in both CTAs of a pair -- once the tensor core has read it.  False if
-// the wait gave up.
+// it) -- and, if the stage holds a second k-block (a_second != 0: its tiles lie a_second / b_second bytes further
+// on), four more --, then a commit that frees the stage, in both CTAs of a pair, once the tensor core has read it.
+// False if the wait gave up.
 template <bool kPair>
 __device__ __forceinline__ bool mma_k_block(uint32_t full_bar, uint32_t phase, uint32_t empty_bar, uint32_t a_addr, uint32_t b_addr,
-                                            uint32_t d_tmem, uint32_t idesc, bool first_of_tile, const volatile int* abort_flag) {
+                                            uint32_t d_tmem, uint32_t idesc, bool first_of_tile, const volatile int* abort_flag,
+                                            uint32_t a_second = 0, uint32_t b_second = 0) {
     if (!ptx::mbar_wait(full_bar, phase, abort_flag)) return false;
     ptx::tc_fence_after_sync();
     const uint64_t adesc = ptx::smem_desc_k128(a_addr);
@@ -50,6 +52,15 @@ __device__ __forceinline__ bool mma_k_block(uint32_t full_bar, uint32_t phase, u
         const uint32_t accumulate = (first_of_tile && k == 0) ? 0u : 1u;
         if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accumulate);
         else ptx::mma_bf16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accumulate);
+    }
+    if (a_second != 0) {
+        const uint64_t adesc2 = ptx::smem_desc_k128(a_addr + a_second);
+        const uint64_t bdesc2 = ptx::smem_desc_k128(b_addr + b_second);
+#pragma unroll
+        for (int k = 0; k < kRoleBK / 16; ++k) {
+            if (kPair) ptx::mma_bf16_ss_pair(d_tmem, adesc2 + 2u * k, bdesc2 + 2u * k, idesc, 1u);
+            else ptx::mma_bf16_ss(d_tmem, adesc2 + 2u * k, bdesc2 + 2u * k, idesc, 1u);
+        }
     }
     if (kPair) ptx::mma_commit_pair(empty_bar, 3);
     else ptx::mma_commit(empty_bar);

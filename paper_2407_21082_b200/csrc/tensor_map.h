@@ -38,4 +38,21 @@ inline bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen as [cols / 64 chunks][rows][64 columns], box = [2 chunks x box_rows x 64 columns]: one request
+// fetches two neighbouring k-blocks of box_rows rows (256 bytes of each row) and lays them down as two
+// consecutive [box_rows x 64] swizzled tiles.  cols must be a multiple of 64 (a partial last chunk would read
+// into the next row instead of being filled with zeros); a chunk index beyond the last is filled with zeros.
+inline bool make_tile_map_k2(CUtensorMap* map, const void* base, int rows, int cols, int box_rows,
+                             CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_128B) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || cols % 64 != 0) return false;
+    const cuuint64_t dims[3] = {64u, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128u};
+    const cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 2u};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace ee

@@ -234,6 +234,10 @@ def test_device_side_argument_errors(ee):
     ("one_row", 1, 512, 777, 4),
     ("paired_tiles", 256, 256, 3000, 3),          # 256-row tiles shared by two CTAs, merge kernel (768 rows)
     ("paired_fused", 160, 128, 1200, 2),          # the same with the merge inside the GEMM kernel (320 rows)
+    ("paired_odd_k_blocks", 256, 320, 2500, 2),   # pairs fetch two k-blocks per request: five of them, the last stage half empty
+    ("paired_one_k_block", 200, 64, 1800, 1),     # ... a single k-block: every stage half empty
+    ("paired_ragged_k", 256, 328, 2000, 1),       # d % 64 != 0: pairs fall back to one k-block per request
+    ("paired_long_k", 512, 1536, 1500, 1),        # 24 k-blocks, four row tiles, several trips round the three-stage ring
 ])
 @pytest.mark.parametrize("kernel", ["auto", "stream", "skinny", "gemm", "none"])
 def test_multi_head_call_matches_oracle(ee, monkeypatch, name, M, d, V, n_heads, kernel):
