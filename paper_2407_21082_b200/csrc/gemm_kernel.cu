@@ -130,7 +130,7 @@ struct GemmParams {
     int n_stages;          // smem ring depth
     int mma_m;             // rows of one MMA: 128, or 64 when no head has more than 64 rows (runtime width only)
     int fused_merge;       // the kernel merges the partial states itself (few rows; runtime width only)
-    int k2;                // a stage holds two k-blocks, fetched by one request per operand (pairs, runtime width; d % 64 == 0)
+    int k2;                // a stage holds two k-blocks, fetched by one request per operand (runtime width; d % 64 == 0)
     int merge_looks;       // how often a row group's owner looks at the ticket before it leaves its rows to the last arriver
     MergeHeads mg;
 };
@@ -211,11 +211,12 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     // 128-row MMA whose lower half would be padding, and an 8 KB instead of a 16 KB y tile per stage.
     const int mma_m = BN_T ? BM : p.mma_m;
     const int a_tile_bytes = mma_m * BK * 2;
-    // A stage of the ring holds one k-block of both operands, or -- CTA pairs with a runtime width -- two: a pair's
-    // CTAs each stage half a W tile, boxes of at most 128 rows, and requests that small stream from HBM at 5.4 TB/s
-    // where one request for two k-blocks (256 bytes of every row) reaches the rate of a contiguous copy; it also
-    // halves the barrier traffic per k-block.
-    constexpr bool kCanK2 = kPair && BN_T == 0;
+    // A stage of the ring holds one k-block of both operands, or -- with a runtime width, when three such stages
+    // fit -- two.  A pair's CTAs each stage half a W tile, boxes of at most 128 rows, and requests that small stream
+    // from HBM at 5.4 TB/s where one request for two k-blocks (256 bytes of every row) reaches the rate of a
+    // contiguous copy; it also halves the requests and the barrier traffic per k-block, which is what a small head
+    // gains from it (d = 512, 8 rows: 17.5 -> 16.8 us per call).
+    constexpr bool kCanK2 = BN_T == 0;
     const int kbs = (kCanK2 && p.k2) ? 2 : 1;                     // k-blocks per stage
     const int n_steps = (p.k_blocks + kbs - 1) / kbs;             // stages per tile
     const int a_stage_bytes = kbs * a_tile_bytes, b_stage_bytes = kbs * b_tile_bytes;
@@ -295,7 +296,10 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     // Where a stage's loads report their bytes (rank 0's barrier) and how they are issued.
     auto load_full_bar = [&](int s) { return kPair ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s); };
     auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int step, int row, uint32_t bar) {   // the k-block(s) of stage `step`
-        if (kCanK2 && kbs == 2) ptx::tma_load_3d_pair(dst, m, 0, row, 2 * step, bar);
+        if (kCanK2 && kbs == 2) {
+            if (kPair) ptx::tma_load_3d_pair(dst, m, 0, row, 2 * step, bar);
+            else ptx::tma_load_3d(dst, m, 0, row, 2 * step, bar);
+        }
         else if (kPair) ptx::tma_load_2d_pair(dst, m, step * BK, row, bar);
         else ptx::tma_load_2d(dst, m, step * BK, row, bar);
     };
@@ -1026,14 +1030,15 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     GemmMaps maps;
     const int mma_m = a.M <= 64 ? 64 : BM;
-    // pairs with a runtime width fetch two k-blocks per request (see the kernel); EE_GEMM_K2=0 switches it off for comparisons
-    const int k2 = (pair && a.M <= 1024 && a.d % 64 == 0 && k2_enabled()) ? 1 : 0;
+    // With a runtime width a ring slot holds two k-blocks fetched by one request per operand (see the kernel) whenever
+    // three such slots fit; EE_GEMM_K2=0 switches it off for comparisons.
+    const int k2 = (a.M <= 1024 && a.d % 64 == 0 && k2_enabled() && stages_for(pair ? bn / 2 : bn, mma_m, 2) >= 3) ? 1 : 0;
     if (!(k2 ? make_tile_map_k2(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)
              : make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)))
         return EE_ERR_CUDA;
     for (int k = 0; k < kGemmMaxHeads; ++k) {
         const void* W = heads[k < n_heads ? k : 0].W;
-        if (!(k2 ? make_tile_map_k2(&maps.w[k], W, a.V, a.d, bn / 2, promo) : make_tile_map(&maps.w[k], W, a.V, a.d, pair ? bn / 2 : bn, promo)))
+        if (!(k2 ? make_tile_map_k2(&maps.w[k], W, a.V, a.d, pair ? bn / 2 : bn, promo) : make_tile_map(&maps.w[k], W, a.V, a.d, pair ? bn / 2 : bn, promo)))
             return EE_ERR_CUDA;
     }
     memcpy(g.maps, &maps, sizeof(maps));
