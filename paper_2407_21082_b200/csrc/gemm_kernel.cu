@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p) {
     using C = Cfg<BN_T>;
     const int BN = BN_T ? BN_T : p.bn;
-    const int S = BN_T ? (kPair ? C::kPairStages : C::kStages) : p.n_stages;
+    const int S = BN_T ? (kPair ? (p.k2 ? C::kPairStages / 2 : C::kPairStages) : C::kStages) : p.n_stages;
     const uint32_t rank = kPair ? ptx::cluster_cta_rank() : 0u;
     const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;        // tiles go round the CTAs / the pairs
     const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -211,12 +211,12 @@ exit_head_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmParams p)
     // 128-row MMA whose lower half would be padding, and an 8 KB instead of a 16 KB y tile per stage.
     const int mma_m = BN_T ? BM : p.mma_m;
     const int a_tile_bytes = mma_m * BK * 2;
-    // A stage of the ring holds one k-block of both operands, or -- with a runtime width, when three such stages
-    // fit -- two.  A pair's CTAs each stage half a W tile, boxes of at most 128 rows, and requests that small stream
+    // A stage of the ring holds one k-block of both operands, or -- when three such stages fit: narrow tiles, and
+    // pairs at any width -- two.  A pair's CTAs each stage half a W tile, boxes of at most 128 rows, and requests that small stream
     // from HBM at 5.4 TB/s where one request for two k-blocks (256 bytes of every row) reaches the rate of a
     // contiguous copy; it also halves the requests and the barrier traffic per k-block, which is what a small head
     // gains from it (d = 512, 8 rows: 17.5 -> 16.8 us per call).
-    constexpr bool kCanK2 = BN_T == 0;
+    constexpr bool kCanK2 = BN_T == 0 || kPair;
     const int kbs = (kCanK2 && p.k2) ? 2 : 1;                     // k-blocks per stage
     const int n_steps = (p.k_blocks + kbs - 1) / kbs;             // stages per tile
     const int a_stage_bytes = kbs * a_tile_bytes, b_stage_bytes = kbs * b_tile_bytes;
@@ -1030,9 +1030,9 @@ ee_status gemm_plan(const HeadArgs* heads, int n_heads, void* storage) {
     const CUtensorMapL2promotion promo = a.M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     GemmMaps maps;
     const int mma_m = a.M <= 64 ? 64 : BM;
-    // With a runtime width a ring slot holds two k-blocks fetched by one request per operand (see the kernel) whenever
-    // three such slots fit; EE_GEMM_K2=0 switches it off for comparisons.
-    const int k2 = (a.M <= 1024 && a.d % 64 == 0 && k2_enabled() && stages_for(pair ? bn / 2 : bn, mma_m, 2) >= 3) ? 1 : 0;
+    // A ring slot holds two k-blocks fetched by one request per operand (see the kernel) whenever three such slots
+    // fit (with the 256-wide tiles of large batches: pairs); EE_GEMM_K2=0 switches it off for comparisons.
+    const int k2 = (a.d % 64 == 0 && k2_enabled() && (a.M > 1024 ? pair : stages_for(pair ? bn / 2 : bn, mma_m, 2) >= 3)) ? 1 : 0;
     if (!(k2 ? make_tile_map_k2(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)
              : make_tile_map(&maps.y, y, (int)y_rows(a.M, n_heads), a.d, mma_m)))
         return EE_ERR_CUDA;

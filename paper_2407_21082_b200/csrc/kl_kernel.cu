@@ -57,6 +57,7 @@ struct KlParams {
     int M, V, d;
     int m_tiles, n_tiles, k_blocks, m_pad;
     int bn, n_stages;
+    int k2;                // a ring slot holds two k-blocks, fetched by one request per operand (d % 64 == 0)
     State* head_part;      // [M][n_tiles]
     Cross* cross_part;     // [M][n_tiles]
     Control* ctrl;
@@ -166,12 +167,16 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
     const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int b_rows = kPair ? BN / 2 : BN;
     const int b_tile_bytes = b_rows * BK * 2;
-    const int stage_bytes = kATileBytes + b_tile_bytes;
+    // one k-block per ring slot, or two fetched by one request per operand (as in the inference kernel)
+    const int kbs = p.k2 ? 2 : 1;
+    const int n_steps = (p.k_blocks + kbs - 1) / kbs;
+    const int a_stage_bytes = kbs * kATileBytes, b_stage_bytes = kbs * b_tile_bytes;
+    const int stage_bytes = a_stage_bytes + b_stage_bytes;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
     const uint32_t a_base = ptx::smem_addr(smem);
-    const uint32_t b_base = a_base + S * kATileBytes;
+    const uint32_t b_base = a_base + S * a_stage_bytes;
     unsigned char* bar_mem = smem + S * stage_bytes;
     const uint32_t bar_base = ptx::smem_addr(bar_mem);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
@@ -227,9 +232,12 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
         if (kPair) m_tile = 2 * m_tile + (int)rank;
     };
     auto load_full_bar = [&](int s) { return kPair ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s); };
-    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int c0, int c1, uint32_t bar) {
-        if (kPair) ptx::tma_load_2d_pair(dst, m, c0, c1, bar);
-        else ptx::tma_load_2d(dst, m, c0, c1, bar);
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* m, int step, int row, uint32_t bar) {   // the k-block(s) of stage `step`
+        if (kbs == 2) {
+            if (kPair) ptx::tma_load_3d_pair(dst, m, 0, row, 2 * step, bar);
+            else ptx::tma_load_3d(dst, m, 0, row, 2 * step, bar);
+        } else if (kPair) ptx::tma_load_2d_pair(dst, m, step * BK, row, bar);
+        else ptx::tma_load_2d(dst, m, step * BK, row, bar);
     };
     const uint32_t arm_bytes = (uint32_t)stage_bytes * (kPair ? 2u : 1u);
 
@@ -243,10 +251,10 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
             if (worker < total_tiles) {                       // head weights of the first stages before the wait
                 int m_tile, n_tile;
                 locate(worker, m_tile, n_tile);
-                n_pre = min(S, p.k_blocks);
+                n_pre = min(S, n_steps);
                 for (int kb = 0; kb < n_pre; ++kb) {
                     if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(kb), arm_bytes);
-                    load_tile(b_base + kb * b_tile_bytes, &maps.w[0], kb * BK, n_tile * BN + (int)rank * b_rows, load_full_bar(kb));
+                    load_tile(b_base + kb * b_stage_bytes, &maps.w[0], kb, n_tile * BN + (int)rank * b_rows, load_full_bar(kb));
                     armed |= 1u << kb;
                 }
             }
@@ -257,9 +265,9 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                 locate(tile, m_tile, n_tile);
                 for (int which = 0; ok && which < 2; ++which) {
                     const int y_row = which * p.m_pad + m_tile * BM;
-                    for (int kb = 0; kb < p.k_blocks; ++kb, ++issued) {
+                    for (int kb = 0; kb < n_steps; ++kb, ++issued) {
                         if (issued < n_pre) {
-                            load_tile(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
+                            load_tile(a_base + stage * a_stage_bytes, &maps.y, kb, y_row, load_full_bar(stage));
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                             continue;
                         }
@@ -269,8 +277,8 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                             break;
                         }
                         if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), arm_bytes);
-                        load_tile(a_base + stage * kATileBytes, &maps.y, kb * BK, y_row, load_full_bar(stage));
-                        load_tile(b_base + stage * b_tile_bytes, &maps.w[which], kb * BK, n_tile * BN + (int)rank * b_rows,
+                        load_tile(a_base + stage * a_stage_bytes, &maps.y, kb, y_row, load_full_bar(stage));
+                        load_tile(b_base + stage * b_stage_bytes, &maps.w[which], kb, n_tile * BN + (int)rank * b_rows,
                                   load_full_bar(stage));
                         armed |= 1u << stage;
                         armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
@@ -298,9 +306,11 @@ kl_pair_gemm_kernel(const __grid_constant__ KlMaps maps, const KlParams p) {
                     }
                     ptx::tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + (uint32_t)(which * kAccStride);
-                    for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * kATileBytes,
-                                                b_base + stage * b_tile_bytes, d_tmem, idesc, kb == 0, abort_flag)) {
+                    for (int kb = 0; kb < n_steps; ++kb) {
+                        const bool two = kbs == 2 && 2 * kb + 1 < p.k_blocks;        // the second k-block of the slot exists
+                        if (!mma_k_block<kPair>(full_bar(stage), phase, empty_bar(stage), a_base + stage * a_stage_bytes,
+                                                b_base + stage * b_stage_bytes, d_tmem, idesc, kb == 0, abort_flag,
+                                                two ? (uint32_t)kATileBytes : 0u, (uint32_t)b_tile_bytes)) {
                             record_failure(p.ctrl, abort_flag, 2, stage, tile);
                             ok = false;
                             break;
@@ -535,8 +545,8 @@ __global__ void __launch_bounds__(256) kl_merge_kernel(const State* head_part, c
     }
 }
 
-int stages_for(int b_rows) {
-    const size_t stage = kATileBytes + (size_t)b_rows * BK * 2;
+int stages_for(int b_rows, int kbs) {
+    const size_t stage = (size_t)kbs * (kATileBytes + (size_t)b_rows * BK * 2);
     const size_t n = (kSmemBudget - kBarBytes - 1024) / stage;
     return (int)(n < (size_t)kMaxStages ? n : (size_t)kMaxStages);
 }
@@ -616,8 +626,13 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
 
     KlMaps maps;
     const CUtensorMapL2promotion promo = M <= 1024 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
-    if (!make_tile_map(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map(&maps.w[0], head.W, V, d, b_rows, promo) ||
-        !make_tile_map(&maps.w[1], teacher.W, V, d, b_rows, promo))
+    // two k-blocks per request whenever three such ring slots fit (M = 4096: 686 -> 618 us, M = 1024: 194 -> 174)
+    static const bool k2_on = !(getenv("EE_GEMM_K2") && getenv("EE_GEMM_K2")[0] == '0');
+    const int k2 = (d % 64 == 0 && k2_on && stages_for(b_rows, 2) >= 3) ? 1 : 0;
+    if (k2 ? (!make_tile_map_k2(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map_k2(&maps.w[0], head.W, V, d, b_rows, promo) ||
+              !make_tile_map_k2(&maps.w[1], teacher.W, V, d, b_rows, promo))
+           : (!make_tile_map(&maps.y, y, 2 * m_pad, d, BM) || !make_tile_map(&maps.w[0], head.W, V, d, b_rows, promo) ||
+              !make_tile_map(&maps.w[1], teacher.W, V, d, b_rows, promo)))
         return EE_ERR_CUDA;
     KlParams p;
     p.M = M; p.V = V; p.d = d;
@@ -626,7 +641,8 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
     p.k_blocks = (d + BK - 1) / BK;
     p.m_pad = m_pad;
     p.bn = bn;
-    p.n_stages = stages_for(b_rows);
+    p.k2 = k2;
+    p.n_stages = stages_for(b_rows, k2 ? 2 : 1);
     p.head_part = head_part;
     p.cross_part = cross_part;
     p.ctrl = reinterpret_cast<Control*>(ws);
@@ -638,7 +654,7 @@ ee_status kl_launch(const HeadArgs& head, const HeadArgs& teacher, const int* la
             return EE_ERR_CUDA;
         configured[head.device] = true;
     }
-    const size_t smem = (size_t)p.n_stages * (kATileBytes + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
+    const size_t smem = (size_t)p.n_stages * (k2 ? 2 : 1) * (kATileBytes + (size_t)b_rows * BK * 2) + kBarBytes + 1024;
     if (pair) {
         const long long total = (long long)(p.m_tiles / 2) * p.n_tiles;
         const int grid = 2 * (int)(total < n_pairs ? total : n_pairs);
