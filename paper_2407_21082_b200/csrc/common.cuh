@@ -308,7 +308,18 @@ __device__ __forceinline__ void merge_token_batches(const State* src, bool src_i
 __device__ __forceinline__ void merge_tokens(const State* src, bool src_is_smem, int n_cta, int np, int M, int warp,
                                              int n_warps, int lane, const float* tau_per_row, float tau, int* argmax,
                                              float* entropy, float* maxprob, unsigned char* exit_mask) {
-    if (n_cta <= 160)
+    // as few tokens per warp and batch as keeps every warp busy: a batch's tokens are reduced one after the other
+    const int per_warp = (M + n_warps - 1) / n_warps;
+    if (n_cta <= 160 && per_warp <= 1)
+        merge_token_batches<1, 5>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
+                                  maxprob, exit_mask);
+    else if (n_cta <= 160 && per_warp <= 2)
+        merge_token_batches<2, 5>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
+                                  maxprob, exit_mask);
+    else if (n_cta <= 160 && per_warp <= 4)
+        merge_token_batches<4, 5>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
+                                  maxprob, exit_mask);
+    else if (n_cta <= 160)
         merge_token_batches<8, 5>(src, src_is_smem, n_cta, np, M, warp, n_warps, lane, tau_per_row, tau, argmax, entropy,
                                   maxprob, exit_mask);
     else

@@ -84,19 +84,26 @@ __device__ __forceinline__ uint4* y_vec(unsigned char* y_tiles, int r, int c) {
 
 // LayerNorm of one head's M rows into the swizzled tiles at y_tiles, by `n_warps` whole warps (this one being
 // number `w`).  `sync` is a barrier over exactly those warps; it returns false if the barrier gave up.
+// A head's LayerNorm parameters into shared memory (asynchronous copies, completed by the wait in fill_activations).
+// They are weights: for the first head of a launch this runs before the dependency wait.
+__device__ __forceinline__ void fill_params(const SkinnyParams& p, const SkinnyHead& hd, float* gamma_s, float* beta_s, int t, int nt) {
+    for (int i = t; i < (p.d >> 2); i += nt) {
+        sk_cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(hd.gamma) + i);
+        sk_cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(hd.beta) + i);
+    }
+}
+
 template <int N, class Sync>
 __device__ __forceinline__ bool fill_activations(const SkinnyParams& p, const SkinnyHead& hd, unsigned char* y_tiles,
-                                                 float* gamma_s, float* beta_s, int w, int n_warps, int lane, Sync sync) {
+                                                 float* gamma_s, float* beta_s, int w, int n_warps, int lane, Sync sync,
+                                                 bool params_on_their_way = false) {
     const int nvec = p.d >> 3;
     const int t = w * 32 + lane, nt = n_warps * 32;
     for (int i = t; i < p.M * nvec; i += nt) {
         const int r = i / nvec, c = i - r * nvec;
         sk_cp_async_16(y_vec<N>(y_tiles, r, c), reinterpret_cast<const uint4*>(hd.h + (size_t)r * hd.ld_h) + c);
     }
-    for (int i = t; i < (p.d >> 2); i += nt) {
-        sk_cp_async_16(reinterpret_cast<float4*>(gamma_s) + i, reinterpret_cast<const float4*>(hd.gamma) + i);
-        sk_cp_async_16(reinterpret_cast<float4*>(beta_s) + i, reinterpret_cast<const float4*>(hd.beta) + i);
-    }
+    if (!params_on_their_way) fill_params(p, hd, gamma_s, beta_s, t, nt);
     sk_cp_async_wait_all();
     if (!sync()) return false;
     auto vec = [&](int r, int c) { return y_vec<N>(y_tiles, r, c); };
@@ -194,9 +201,10 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
     if (threadIdx.x == 0)
         for (; preloaded < total_loads && preloaded < S; ++preloaded) issue_load(preloaded);
 
-    // Activations of the first head: all warps.
+    // Activations of the first head: all warps (its LayerNorm parameters are requested before the wait).
+    fill_params(p, p.head[0], gamma_s, beta_s, (int)threadIdx.x, kSkThreads);
     sk_grid_dependency_wait();
-    fill_activations<N>(p, p.head[0], y_all, gamma_s, beta_s, warp, kSkWarps, lane, [] { __syncthreads(); return true; });
+    fill_activations<N>(p, p.head[0], y_all, gamma_s, beta_s, warp, kSkWarps, lane, [] { __syncthreads(); return true; }, true);
     __syncthreads();
 
     if (warp == 0) {
@@ -344,6 +352,7 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
             // Cross-lane reduction of this warp's states: per token a warp maximum, then sums of rescaled terms.
 #pragma unroll
             for (int c = 0; c < TOK; ++c) {
+                if (group * 32 + c >= p.M) break;                 // padding tokens: nobody reads their states
                 const State a = state_reduce_lanes<1, 16>(own[c]);
                 if (lane == 0) qpart[quarter * N + group * 32 + c] = a;
             }
@@ -358,7 +367,7 @@ exit_head_skinny_kernel(const __grid_constant__ SkinnyMaps maps, const __grid_co
             if (!(ok = epi_sync())) break;
             // Merge the four quarters; publish the CTA partial of head k.
             State* part_k = p.partials + (size_t)k * gridDim.x * N;
-            if (et < N) {
+            if (et < p.M) {
                 const State four[4] = {qpart[et], qpart[N + et], qpart[2 * N + et], qpart[3 * N + et]};
                 part_k[(size_t)blockIdx.x * N + et] = state_combine<4>(four);
             }
