@@ -16,6 +16,13 @@
  * the next call.  Everything else -- hidden states, thresholds, masks, tokens -- may be produced by
  * earlier work of the same stream, by ordinary or by programmatic dependent launches.
  *
+ * Environment switches, read by the library for comparisons and tests (none is needed in normal use):
+ * EE_MULTI_KERNEL=stream|skinny|gemm|none forces the kernel of multi-head calls (read per call);
+ * EE_GEMM_PAIRS=0 keeps every CTA on its own 128-row tiles and EE_GEMM_K2=0 keeps one k-block per ring slot
+ * (both read once per process); EE_MERGE_LOOKS=n sets how often a row group's owner looks for the launch's
+ * other CTAs before it hands its rows over (read when a call is planned); EE_CASCADE_ALL_ROWS_MAX=m moves
+ * the batch size at which ee_cascade changes path (read once).  None of them changes a result.
+ *
  * Notation follows the paper: a head h_k maps the hidden features of a transformer block to a
  * distribution p_k over the vocabulary V (section 3.1 "Early exit heads", section 3.2); the confidence
  * is the entropy of p_k (section 3.4.1); tau_k is the calibrated threshold of head k (section 3.4.1);
