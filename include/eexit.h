@@ -21,7 +21,9 @@
  * EE_GEMM_PAIRS=0 keeps every CTA on its own 128-row tiles and EE_GEMM_K2=0 keeps one k-block per ring slot
  * (both read once per process); EE_MERGE_LOOKS=n sets how often a row group's owner looks for the launch's
  * other CTAs before it hands its rows over (read when a call is planned); EE_CASCADE_ALL_ROWS_MAX=m moves
- * the batch size at which ee_cascade changes path (read once).  None of them changes a result.
+ * the batch size at which ee_cascade changes path (read once).  They change which kernel or tile width runs, so
+ * entropy and max-probability may differ in their last bits (sums taken in another order); decisions away from
+ * the tolerance band do not change.
  *
  * Notation follows the paper: a head h_k maps the hidden features of a transformer block to a
  * distribution p_k over the vocabulary V (section 3.1 "Early exit heads", section 3.2); the confidence
