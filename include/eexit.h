@@ -316,7 +316,9 @@ ee_status dssd_commit(const int* draft_tok, const unsigned char* draft_exit_mask
  * h'S LAYER are wanted) and once for the verification pass (which = K: n_rows = S * (k + 1) tokens, row (s, j) =
  * the token before draft position j, j = k being the bonus position; the full model's final hidden states); it
  * must enqueue on `stream` work that writes the hidden states bf16 [n_rows, d] (dense) of the positions FOLLOWING
- * those tokens to h_out, and return 0.
+ * those tokens to h_out, and return 0.  A real model produces the states of all its exit layers in one forward
+ * pass: with hidden_all_layers != 0 the drafting steps call `hidden` ONCE per step, with which = -1, and it must
+ * write layer h's states to h_out + h * n_rows * d elements for every h < K (the verification call is unchanged).
  * Both pointers it receives are device buffers inside `workspace`.  The work it enqueues may be ordinary stream
  * work, or kernels launched with programmatic stream serialization that trigger their dependents early -- the
  * round's own kernels are chained that way -- provided every such kernel executes griddepcontrol.wait before it
@@ -365,6 +367,7 @@ typedef struct {
     int n_draft_heads;
     const ee_head* draft_heads;
     long long* head_use;
+    int hidden_all_layers;              /* non-zero: one call of `hidden` per drafting step fills every draft head's layer */
 } ee_dssd_round_args;
 size_t    dssd_round_workspace_bytes(int S, int k, int d, int V);     /* host-only, pure; 0 if a size is invalid */
 size_t    dssd_round_multi_workspace_bytes(int S, int k, int d, int V, int n_draft_heads);
@@ -374,7 +377,8 @@ ee_status dssd_round(const ee_dssd_round_args* args);
  * A ready-made ee_hidden_fn for tests and benchmarks (no counterpart in the paper; the transformer is the
  * caller's): the hidden state of a row is row `token` of table[which] -- table[h] for draft head h's layer,
  * table[K] for the verification pass -- each bf16 [V, d] on the device, contiguous, 16-byte aligned; a token
- * outside [0, V) gives a zero row.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a pointer to an
+ * outside [0, V) gives a zero row; which = -1 (hidden_all_layers) fills the layers of all draft tables -- every
+ * non-NULL table but the last -- with one launch.  Give dssd_round `ee_hidden_from_tables` as `hidden` and a pointer to an
  * ee_hidden_tables (host memory that outlives the call) as `hidden_user`.  One kernel launch on `stream` per call;
  * returns 0, or 1 if an argument is unusable or the launch failed.  chained = 0: an ordinary launch; chained != 0:
  * the kernel is launched with programmatic stream serialization, lets its dependents start at once and waits for

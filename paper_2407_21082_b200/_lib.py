@@ -27,7 +27,8 @@ class EEDssdRoundArgs(C.Structure):
                 ("draft_head", EEHead), ("verify_head", EEHead), ("hidden", HIDDEN_FN), ("hidden_user", _p),
                 ("last_tok", _p), ("out_tok", _p), ("capacity", C.c_int), ("seq_len", _p), ("finished", _p), ("stats", _p),
                 ("draft_len", _p), ("accept_len", _p), ("next_tok", _p), ("workspace", _p), ("workspace_bytes", C.c_size_t),
-                ("stream", _p), ("n_draft_heads", C.c_int), ("draft_heads", C.POINTER(EEHead)), ("head_use", _p)]
+                ("stream", _p), ("n_draft_heads", C.c_int), ("draft_heads", C.POINTER(EEHead)), ("head_use", _p),
+                ("hidden_all_layers", C.c_int)]
 
 
 EE_PLAN_MAX_HEADS = 16

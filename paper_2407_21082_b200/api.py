@@ -611,10 +611,12 @@ class DssdRound:
     first confident one supplies the token); verify_head: dict with gamma, beta, W.  hidden_fn(tokens, which, h_out) is
     the caller's model: `tokens` int32 [n_rows] and `h_out` bf16 [n_rows, d] are device tensors (views into the
     workspace); it must fill h_out on the current stream with the hidden states at draft head `which`'s layer
-    (which < K) or the full model's (which = K).  `state`: last_tok, out_tok, seq_len, finished, stats.  With a list
+    (which < K) or the full model's (which = K).  all_layers=True asks for ONE call per drafting step instead of K:
+    which = -1 and h_out bf16 [K, n_rows, d], layer by layer (the library's TableModel is always driven that way).
+    `state`: last_tok, out_tok, seq_len, finished, stats.  With a list
     of heads, self.head_use (int64 [K]) accumulates the positions each head supplied."""
 
-    def __init__(self, draft_head, verify_head, ln_eps, k, eos_token, hidden_fn, state, workspace=None):
+    def __init__(self, draft_head, verify_head, ln_eps, k, eos_token, hidden_fn, state, workspace=None, all_layers=None):
         import ctypes as C
         S = state["last_tok"].numel()
         multi = isinstance(draft_head, (list, tuple))
@@ -635,7 +637,9 @@ class DssdRound:
         def trampoline(user, tokens_ptr, n_rows, which, h_ptr, stream):
             try:
                 tokens = workspace[tokens_ptr - base:tokens_ptr - base + 4 * n_rows].view(torch.int32)
-                h_out = workspace[h_ptr - base:h_ptr - base + 2 * n_rows * d].view(torch.bfloat16).view(n_rows, d)
+                layers = K if which < 0 else 1
+                h_out = workspace[h_ptr - base:h_ptr - base + 2 * layers * n_rows * d].view(torch.bfloat16)
+                h_out = h_out.view(K, n_rows, d) if which < 0 else h_out.view(n_rows, d)
                 hidden_fn(tokens, which, h_out)
                 return 0
             except Exception:                    # an exception must not cross the C boundary
@@ -655,6 +659,7 @@ class DssdRound:
         if multi:
             a.n_draft_heads, a.draft_heads, a.head_use = K, arr, _ptr(self.head_use)
         a.hidden, a.hidden_user = self._cb, (C.cast(C.pointer(hidden_fn.struct), C.c_void_p) if native else None)
+        a.hidden_all_layers = int(native if all_layers is None else bool(all_layers))
         a.last_tok, a.out_tok, a.capacity = _ptr(state["last_tok"]), _ptr(state["out_tok"]), state["out_tok"].shape[1]
         a.seq_len, a.finished, a.stats = _ptr(state["seq_len"]), _ptr(state["finished"]), _ptr(state["stats"])
         a.draft_len, a.accept_len, a.next_tok = (_ptr(self.out[n]) for n in ("draft_len", "accept_len", "next_tok"))

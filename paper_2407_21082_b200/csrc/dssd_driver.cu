@@ -155,8 +155,12 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, const ee_head* draft_heads
                    cur_tok) != cudaSuccess)
         return EE_ERR_CUDA;
     for (int j = 0; j < k; ++j) {
-        for (int hd = 0; hd < K; ++hd)
-            if (a.hidden(a.hidden_user, cur_tok, S, hd, h + (size_t)hd * S * d * 2, a.stream) != 0) return EE_ERR_CUDA;
+        if (a.hidden_all_layers) {                        // one forward pass of the caller's model for all K layers
+            if (a.hidden(a.hidden_user, cur_tok, S, -1, h, a.stream) != 0) return EE_ERR_CUDA;
+        } else {
+            for (int hd = 0; hd < K; ++hd)
+                if (a.hidden(a.hidden_user, cur_tok, S, hd, h + (size_t)hd * S * d * 2, a.stream) != 0) return EE_ERR_CUDA;
+        }
         ee_status st = ee_exit_head_multi(step_heads, K, a.ln_eps, S, d, V, ws + L.head_ws, head_ws_bytes, a.stream);
         if (st != EE_OK) return st;
         if (launch_pdl(record_draft_kernel, gs, 256, 0, s, (const unsigned char*)(ws + L.outs),
@@ -189,30 +193,49 @@ ee_status dssd_round_run(const ee_dssd_round_args& a, const ee_head* draft_heads
 // programmatic dependent launches like the library's own kernels: it lets its dependents start at once and waits
 // for its predecessors before it reads the tokens or writes a hidden state.
 namespace {
-__global__ void __launch_bounds__(256) hidden_from_table_kernel(const uint4* __restrict__ table, int V, int nvec,
+struct TableList {
+    const uint4* table[EE_ROUND_MAX_DRAFT_HEADS];
+};
+// blockIdx.y = table: layer y's rows go to h_out + y * n_rows rows (one table: the plain lookup).
+__global__ void __launch_bounds__(256) hidden_from_table_kernel(const __grid_constant__ TableList tl, int V, int nvec,
                                                                 const int* tokens, int n_rows, uint4* h_out, int chained) {
     if (chained) launch_dependents();
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= n_rows) return;
     if (chained) grid_dependency_wait();
+    const uint4* table = tl.table[blockIdx.y];
+    uint4* out = h_out + ((size_t)blockIdx.y * n_rows + r) * nvec;
     const int t = ld_dep(tokens + r);
     const bool in = t >= 0 && t < V;
-    for (int c = lane; c < nvec; c += 32) h_out[(size_t)r * nvec + c] = in ? __ldg(table + (size_t)t * nvec + c) : make_uint4(0, 0, 0, 0);
+    for (int c = lane; c < nvec; c += 32) out[c] = in ? __ldg(table + (size_t)t * nvec + c) : make_uint4(0, 0, 0, 0);
 }
 }  // namespace
 
 int hidden_from_tables(const ee_hidden_tables* m, const int* tokens, int n_rows, int which, void* h_out, cudaStream_t stream) {
-    if (!m || !tokens || !h_out || which < 0 || which > EE_ROUND_MAX_DRAFT_HEADS || !m->table[which]) return 1;
+    if (!m || !tokens || !h_out || which < -1 || which > EE_ROUND_MAX_DRAFT_HEADS) return 1;
     if (m->d < 8 || (m->d % 8) != 0 || m->V < 1 || n_rows < 0) return 1;
-    if ((reinterpret_cast<uintptr_t>(m->table[which]) & 15) != 0) return 1;
+    TableList tl = {};
+    int n_tables = 1;
+    if (which >= 0) {
+        tl.table[0] = static_cast<const uint4*>(m->table[which]);
+    } else {
+        // all draft tables: every non-NULL entry but the last (the verification pass's)
+        int filled = 0;
+        while (filled <= EE_ROUND_MAX_DRAFT_HEADS && m->table[filled]) ++filled;
+        n_tables = filled - 1;
+        if (n_tables < 1) return 1;
+        for (int i = 0; i < n_tables; ++i) tl.table[i] = static_cast<const uint4*>(m->table[i]);
+    }
+    for (int i = 0; i < n_tables; ++i)
+        if (!tl.table[i] || (reinterpret_cast<uintptr_t>(tl.table[i]) & 15) != 0) return 1;
     if (n_rows == 0) return 0;
+    const dim3 grid((n_rows + 7) / 8, n_tables);
     if (m->chained)
-        return launch_pdl(hidden_from_table_kernel, (n_rows + 7) / 8, 256, 0, stream, static_cast<const uint4*>(m->table[which]),
-                          m->V, m->d / 8, tokens, n_rows, static_cast<uint4*>(h_out), 1) == cudaSuccess ? 0 : 1;
+        return launch_pdl(hidden_from_table_kernel, grid, 256, 0, stream, tl, m->V, m->d / 8, tokens, n_rows,
+                          static_cast<uint4*>(h_out), 1) == cudaSuccess ? 0 : 1;
     // An ordinary launch, like any kernel of a caller's model: it starts when everything before it in the stream
     // has finished and what follows starts when it has.
-    hidden_from_table_kernel<<<(n_rows + 7) / 8, 256, 0, stream>>>(static_cast<const uint4*>(m->table[which]), m->V, m->d / 8,
-                                                                  tokens, n_rows, static_cast<uint4*>(h_out), 0);
+    hidden_from_table_kernel<<<grid, 256, 0, stream>>>(tl, m->V, m->d / 8, tokens, n_rows, static_cast<uint4*>(h_out), 0);
     return cudaGetLastError() == cudaSuccess ? 0 : 1;
 }
 

@@ -107,7 +107,8 @@ def test_whole_rounds_match_oracle(ee, S, k, V, d, tau, eos, model):
 @pytest.mark.parametrize("S,k,V,d,taus,eos", [(12, 4, 400, 64, (1.0,), -1), (40, 8, 1000, 128, (0.4, 0.8, 1.5), 5),
                                                (3, 1, 300, 64, (0.5, 5.0, 5.0), -1), (70, 6, 640, 256, (0.6, 1.0, 2.0), 17),
                                                (33, 5, 500, 64, (0.5, 1.0, 1.0, 1.5, 2.0), -1)])
-@pytest.mark.parametrize("model", ["python callback", "chained table model"])
+@pytest.mark.parametrize("model", ["python callback", "python callback, one call per step", "chained table model",
+                                   "chained table model, one call per layer"])
 def test_whole_rounds_with_several_draft_heads_match_oracle(ee, S, k, V, d, taus, eos, model):
     """K draft heads, shallowest first, each on its own layer's hidden states: per position the first confident head
     supplies the token (section 4.3.1).  State, outputs and the per-head usage counts against oracle.dssd_round_multi
@@ -134,12 +135,20 @@ def test_whole_rounds_with_several_draft_heads_match_oracle(ee, S, k, V, d, taus
 
     def hidden(tokens, which, h_out):
         calls.append((which, tokens.numel()))
-        torch.index_select(E[which], 0, tokens.long(), out=h_out)
+        if which < 0:                                                   # one forward pass: every drafting layer's states
+            for layer in range(K):
+                torch.index_select(E[layer], 0, tokens.long(), out=h_out[layer])
+        else:
+            torch.index_select(E[which], 0, tokens.long(), out=h_out)
 
     devs = [head_to_dev(hd) for hd in cfg["heads"]]
     drafts = [dict(gamma=hd["gamma"], beta=hd["beta"], W=hd["W"], tau=float(t)) for hd, t in zip(devs[:K], taus)]
     verify = dict(gamma=devs[K]["gamma"], beta=devs[K]["beta"], W=devs[K]["W"])
-    rnd = ee.DssdRound(drafts, verify, 1e-5, k, eos, hidden if model == "python callback" else ee.TableModel(E[:K], E[K], chained=True), state)
+    if model.startswith("python callback"):
+        rnd = ee.DssdRound(drafts, verify, 1e-5, k, eos, hidden, state, all_layers=model.endswith("one call per step"))
+    else:
+        rnd = ee.DssdRound(drafts, verify, 1e-5, k, eos, ee.TableModel(E[:K], E[K], chained=True), state,
+                           all_layers=not model.endswith("one call per layer"))
     clean = np.ones(S, bool)
     for r in range(3):
         ref = oracle.dssd_round_multi(E_drafts, E_verify, cfg["heads"][:K], cfg["heads"][K], list(taus), eos, k, ref_last, *ref_state, ref_use)
@@ -163,6 +172,8 @@ def test_whole_rounds_with_several_draft_heads_match_oracle(ee, S, k, V, d, taus
             assert rnd.head_use.cpu().numpy().tolist() == ref_use.tolist(), r
     if model == "python callback":
         assert calls[:K * k + 1] == [(h, S) for _ in range(k) for h in range(K)] + [(K, S * (k + 1))]
+    if model == "python callback, one call per step":
+        assert calls[:k + 1] == [(-1, S)] * k + [(K, S * (k + 1))]
     assert clean.sum() >= S // 2
     if K > 1 and clean.all():
         assert ref_use.sum() == ref_state[3][0]                         # every drafted position has its head
