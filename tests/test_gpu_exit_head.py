@@ -161,6 +161,31 @@ def test_c4_full_size_on_a_stratified_row_sample(ee):
     assert np.array_equal(out["exit_mask"].cpu().numpy()[decided], other["exit_mask"].cpu().numpy()[decided])
 
 
+@pytest.mark.parametrize("path_name", ["tcgen05", "stream", "skinny"])
+@pytest.mark.parametrize("M,d,V", [(8, 512, 3000), (40, 64, 700)])
+def test_rows_with_nan_or_infinite_hidden_states_never_exit(ee, path_name, M, d, V):
+    """A NaN or an infinity in a row's hidden state makes that row's entropy NaN (LayerNorm of such a row has no
+    value) and a NaN entropy never exits, whatever the threshold; the other rows of the batch are not touched."""
+    if ee.ee_exit_head_launches(M, d, V, PATHS[path_name]) == 0:
+        pytest.skip(f"{path_name} kernel does not take M={M}")
+    cfg = gen.make_config("c0", seed=5, planted=True, M=M, d=d, V=V)
+    h = cfg["h"].copy()
+    bad = {1: 0x7FC0, 3: 0x7F80, M - 1: 0xFF80}                      # bf16 NaN, +inf, -inf in one element of the row
+    for row, bits in bad.items():
+        h[row, (7 * row) % d] = bits
+    good = np.array([r for r in range(M) if r not in bad])
+    hd = head_to_dev(cfg["heads"][0])
+    out = ee.ee_exit_head(dev_bf16(h), hd["gamma"], hd["beta"], 1e-5, hd["W"], float("inf"), path=PATHS[path_name])
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    for row in bad:
+        assert np.isnan(got["entropy"][row]), (row, got["entropy"][row])
+        assert got["exit_mask"][row] == 0                              # even with tau = +inf
+    ref = oracle_head(cfg["h"][good], cfg["heads"][0], float("inf"))
+    assert_head_matches({k: v[torch.from_numpy(good).to(v.device)] for k, v in out.items()}, ref, label=f"{path_name} rows without NaN")
+    assert (got["exit_mask"][good] == 1).all()
+
+
 def test_both_kernels_agree_and_runs_are_bit_identical(ee):
     cfg = gen.make_config("c1", seed=5, planted=True, M=32, V=20000)
     a = _run(ee, cfg, 0, 1.0, ee.EE_PATH_STREAM)
