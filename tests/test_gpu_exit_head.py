@@ -464,7 +464,8 @@ def test_plan_runs_equal_the_one_step_call_and_follow_the_buffers_contents(ee):
     run; the plan captures pointers, not contents, so new rows written into the same buffer give the new rows' results."""
     import ctypes as C
     from paper_2407_21082_b200 import _lib
-    for M, d, V, n_heads in ((64, 256, 5000, 3), (300, 136, 3001, 5), (8, 512, 50304, 1), (256, 2048, 4000, 2)):
+    # (the last shape: sixteen heads, the most a plan holds -- four launch groups)
+    for M, d, V, n_heads in ((64, 256, 5000, 3), (300, 136, 3001, 5), (8, 512, 50304, 1), (256, 2048, 4000, 2), (12, 64, 900, 16)):
         cfg = gen.make_config("c1", seed=61, planted=True, M=M, d=d, V=V, heads=n_heads)
         other = gen.make_config("c1", seed=62, planted=True, M=M, d=d, V=V, heads=n_heads)
         hds = [head_to_dev(hd) for hd in cfg["heads"]]
